@@ -1,0 +1,26 @@
+"""CPU oracle for the layout-lowered named-dimension einsum and the Transformer blocks built on it.
+
+THIS PACKAGE IS TEST INFRASTRUCTURE.  It is a plain, slow, fp64 restatement of what the paper says
+the method computes, used to check the CUDA library.  Only the tests, the smoke check and the
+bench's CPU-baseline leg may import it; the product library never does, and the two share no code.
+
+Contents
+  einsum_loops.c  the einsum definition as one fp64 loop nest (the only native part)
+  named.py        named tensors, dense einsum / reductions / component-wise ops
+  mesh.py         mesh, computation layout, legality, per-processor slice boxes
+  lowering.py     per-processor simulation: local op on slices, then the group sum (Allreduce)
+  blocks.py       feed-forward, attention, layer norm, decoder layer - forward and backward
+  cost.py         per-processor cost counts (Table 1, Appendix B)
+
+Pins (tests that tie each part to something other than itself) are listed in the test files named
+test_oracle_*.py.  Parts without an external pin: the bf16 rounding behaviour of the GPU path is
+compared by tolerance only ("parity unpinned" beyond the stated tolerances).
+"""
+from .named import (NT, DenseOps, DuplicateDim, IllegalLayout, NotDivisible, OracleError, SizeMismatch,
+                    UnknownDim, einsum_arrays)
+from .mesh import Layout, Mesh
+from .lowering import LT, LoweredOps
+from . import blocks, cost
+
+__all__ = ["NT", "DenseOps", "LoweredOps", "LT", "Mesh", "Layout", "blocks", "cost", "einsum_arrays",
+           "OracleError", "DuplicateDim", "UnknownDim", "SizeMismatch", "IllegalLayout", "NotDivisible"]
