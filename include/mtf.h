@@ -1,0 +1,196 @@
+/*
+ * mtf.h - C ABI of the B200 library for layout-lowered named-dimension einsum (Mesh-TensorFlow,
+ * arXiv 1811.02084) and the Transformer blocks built from it.
+ *
+ * Model of the paper that this boundary follows
+ *   - A mesh is an n-dimensional array of (here: virtual) processors with named dimensions
+ *     (Section 2, Section 4).
+ *   - Tensors have named dimensions; a computation layout maps tensor-dimension names to
+ *     mesh-dimension names (Section 4).  A tensor's layout is the restriction of that map to its
+ *     own dimensions; it must be injective and sizes must divide (Section 5).
+ *   - Processor p keeps, along every mapped dimension, the contiguous block selected by its mesh
+ *     coordinate (Section 5).  Processor ranks unrank row-major over the mesh dimensions, last
+ *     mesh dimension fastest.
+ *   - An einsum is a local einsum on every processor's slices followed by a sum over the group of
+ *     processors that differ only along the mesh dimensions of reduced-out split dimensions
+ *     (Section 6, "Einstein Summation").  On one GPU that sum is an on-device reduction.
+ *
+ * General conventions
+ *   - Every tensor is stored ONCE, globally, dense and row-major in the order of its `dims`
+ *     (last dimension contiguous).  A processor's slice is a box view of it; replicas are logical.
+ *   - `data` pointers are DEVICE pointers owned by the caller unless a parameter says "host".
+ *     The library never allocates tensor memory; scratch space is passed in as `workspace`.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Launches are
+ *     asynchronous; no call synchronises the device unless stated.
+ *   - All validation happens before any launch.  Every call returns an mtf_status; nothing throws
+ *     or aborts across this boundary.  mtf_last_error() gives thread-local detail text.
+ *   - Handles are immutable after creation, may be shared between threads, and are destroyed by
+ *     the caller.  Strings are copied at creation.
+ */
+#ifndef MTF_H_
+#define MTF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MTF_OK = 0,
+  MTF_ERR_INVALID_ARG = 1,      /* NULL pointer, bad count, bad dtype, duplicate layout rule ...        */
+  MTF_ERR_DUPLICATE_DIM = 2,    /* a tensor or mesh carries one dimension name twice (Section 4)        */
+  MTF_ERR_UNKNOWN_DIM = 3,      /* a name that is not there: mesh dim of a rule, output dim of einsum   */
+  MTF_ERR_SIZE_MISMATCH = 4,    /* one dimension name with two sizes in one operation                   */
+  MTF_ERR_ILLEGAL_LAYOUT = 5,   /* two dims of a tensor / of an operation on one mesh dim (Section 8.5) */
+  MTF_ERR_NOT_DIVISIBLE = 6,    /* split dimension size not divisible by the mesh-dim size (Section 5)  */
+  MTF_ERR_UNSUPPORTED = 7,      /* legal in the paper's language, not implemented on the GPU path       */
+  MTF_ERR_WORKSPACE_TOO_SMALL = 8,
+  MTF_ERR_CUDA = 9,             /* a CUDA runtime/driver call failed; text in mtf_last_error()          */
+  MTF_ERR_TIMEOUT = 10          /* a bounded device-side wait gave up (see mtf_device_status)           */
+} mtf_status;
+
+typedef enum { MTF_F32 = 0, MTF_BF16 = 1 } mtf_dtype;
+
+/* Opaque handles.  (The layout handle type carries a _t because mtf_layout is the call that makes one.) */
+typedef struct mtf_mesh_s mtf_mesh_t;
+typedef struct mtf_layout_s mtf_layout_t;
+typedef struct mtf_plan_s mtf_plan_t;
+
+/* A named dimension (Section 4): name + static size. */
+typedef struct { const char* name; int64_t size; } mtf_dim;
+
+/* A named tensor: non-owning view.  `data` is a device pointer (ignored where stated). */
+typedef struct { void* data; mtf_dtype dtype; int32_t ndim; const mtf_dim* dims; } mtf_tensor;
+
+/* Component-wise work fused into an einsum's output (Section 6 "Component-wise Operations",
+ * Section 7 implicit broadcasting), applied in this order to the fp32 accumulator:
+ *     t = scale * acc;  t += bias (broadcast);  if relu: t = max(t, 0);
+ *     if relu_mask: t = (relu_mask > 0) ? t : 0;   t += residual;   out = cast(t)
+ * bias      : dims must be a subset of the output dims (any order);  f32 or bf16.
+ * relu_mask : same dims, same order and dtype class as the output (bf16 or f32).
+ * residual  : same dims and order as the output (bf16 or f32).
+ * NULL pointers / relu = 0 / scale = 1 switch a stage off.  The struct is read during planning
+ * only for which stages are on and their descriptors; data pointers are read at exec time. */
+typedef struct {
+  float scale;
+  int32_t relu;
+  const mtf_tensor* bias;
+  const mtf_tensor* relu_mask;
+  const mtf_tensor* residual;
+} mtf_epilogue;
+
+/* Which kernel family a plan runs (informational; chosen by the planner). */
+typedef enum { MTF_KERNEL_SIMT = 0, MTF_KERNEL_TCGEN05 = 1 } mtf_kernel_kind;
+/* How the sum over a reduce group is realised (Section 6: the Allreduce after the local einsum).
+ *   CHAINED   : the CTA that owns an output tile runs the K loops of the group's slices back to
+ *               back, in ascending processor order, into one accumulator (no extra HBM traffic).
+ *   WORKSPACE : every (slice, tile) writes an fp32 partial to the workspace; the CTA that arrives
+ *               last for a tile sums the partials in ascending processor order and finishes it. */
+typedef enum { MTF_REDUCE_NONE = 0, MTF_REDUCE_CHAINED = 1, MTF_REDUCE_WORKSPACE = 2 } mtf_reduce_mode;
+
+/* ---- mesh (Section 2, Section 4) ------------------------------------------------------------ */
+/* mesh_dims: host array of ndim (name, size) pairs, 1 <= ndim <= 4, sizes >= 1, names distinct. */
+mtf_status mtf_mesh_create(int32_t ndim, const mtf_dim* mesh_dims, mtf_mesh_t** out);
+mtf_status mtf_mesh_destroy(mtf_mesh_t* mesh);
+/* Number of processors P and, for processor p, its coordinates (host array of the mesh's ndim). */
+mtf_status mtf_mesh_size(const mtf_mesh_t* mesh, int64_t* n_processors);
+mtf_status mtf_mesh_coords(const mtf_mesh_t* mesh, int64_t processor, int64_t* coords);
+
+/* ---- computation layout (Section 4; examples in Section 8.1-8.5, Section 9) ------------------ */
+/* nrules pairs tensor_dim[i] -> mesh_dim[i] (host strings).  A tensor dimension may appear once
+ * (it is a map); several tensor dimensions may map to one mesh dimension; the mesh dimension
+ * must exist (MTF_ERR_UNKNOWN_DIM).  nrules = 0 is the legal empty layout (Section 8.4).
+ * The layout keeps a reference to nothing: the mesh may be destroyed afterwards. */
+mtf_status mtf_layout(const mtf_mesh_t* mesh, int32_t nrules, const char* const* tensor_dim,
+                      const char* const* mesh_dim, mtf_layout_t** out);
+mtf_status mtf_layout_destroy(mtf_layout_t* layout);
+/* Legality of one tensor under the layout (Section 5, Section 8.5): MTF_ERR_DUPLICATE_DIM,
+ * MTF_ERR_ILLEGAL_LAYOUT or MTF_ERR_NOT_DIVISIBLE, else MTF_OK. */
+mtf_status mtf_layout_check_tensor(const mtf_layout_t* layout, int32_t ndim, const mtf_dim* dims);
+/* Slice box of `processor` (Section 5): host outputs offsets[ndim], sizes[ndim]; the local index l
+ * maps to the global flat index sum_i (offsets[i] + l_i) * prod_{i' > i} dims[i'].size. */
+mtf_status mtf_slice_map(const mtf_layout_t* layout, int32_t ndim, const mtf_dim* dims, int64_t processor,
+                         int64_t* offsets, int64_t* sizes);
+/* Device copy of one processor's slice of `global` into the dense row-major buffer `out_slice`
+ * (device, same dtype, prod(sizes) elements).  One kernel launch on `stream`. */
+mtf_status mtf_slice_gather(const mtf_layout_t* layout, const mtf_tensor* global, int64_t processor,
+                            void* out_slice, void* stream);
+
+/* ---- einsum (Section 6 "Einstein Summation"; Section 8 code fragment) ------------------------- */
+/* Plan  out[out dims] = sum over dims not in out of  in[0] * in[1]  under `layout`.
+ * The equation is carried by the dimension names, as in mtf.einsum(x, w, output_shape=[...]).
+ * n_in must be 2 (MTF_ERR_UNSUPPORTED otherwise).  `data` of the descriptors is ignored here.
+ * Errors: duplicate names, size mismatch, output dim in no input (MTF_ERR_UNKNOWN_DIM), illegal
+ * layout for any operand or for the whole iteration space, non-divisible split sizes, and
+ * MTF_ERR_UNSUPPORTED for a dimension that only one input has and the output lacks. */
+mtf_status mtf_einsum_plan(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in_desc,
+                           const mtf_tensor* out_desc, const mtf_epilogue* epilogue, mtf_plan_t** out);
+mtf_status mtf_plan_destroy(mtf_plan_t* plan);
+/* Scratch bytes mtf_einsum_exec needs (0 unless the reduce mode is WORKSPACE). */
+mtf_status mtf_plan_workspace_bytes(const mtf_plan_t* plan, size_t* bytes);
+/* Per-processor cost counts (Table 1; Appendix B): multiply-adds of the local einsum, values
+ * entering the Allreduce (one output slice when a split dimension is reduced out, else 0), local
+ * elements of inputs plus output, and how many mesh dimensions are reduced over. */
+mtf_status mtf_plan_cost(const mtf_plan_t* plan, int64_t* macs_per_proc, int64_t* allreduce_values_per_proc,
+                         int64_t* slice_elems_per_proc, int32_t* n_reduce_mesh_dims);
+/* What the planner decided: kernel family, reduce mode, number of distinct slices computed
+ * (replicas are computed once, Section 8.4), reduce-group size, and the reduced mesh dims as a bit mask. */
+mtf_status mtf_plan_info(const mtf_plan_t* plan, int32_t* kernel_kind, int32_t* reduce_mode,
+                         int64_t* n_slices, int64_t* group_size, uint32_t* reduce_mesh_dim_mask);
+/* Run a plan.  in[0..1] and out carry device pointers; dims must equal the planned ones.
+ * epilogue may be NULL only if the plan was made without one.  One kernel launch (plus one memset
+ * of the tile counters in WORKSPACE mode) on `stream`. */
+mtf_status mtf_einsum_exec(const mtf_plan_t* plan, const mtf_tensor* in, mtf_tensor* out,
+                           const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream);
+/* One-shot form: plan (cached inside the layout handle by shapes, dtypes and epilogue stages) and
+ * run.  `equation` is optional sugar, e.g. "batch io, io hidden -> batch hidden"; when given it
+ * must agree with the descriptors' names (MTF_ERR_INVALID_ARG otherwise); NULL = names only. */
+mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in,
+                      mtf_tensor* out, const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes,
+                      void* stream);
+mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in,
+                                      const mtf_tensor* out, const mtf_epilogue* epilogue, size_t* bytes);
+/* Testing hook: force the kernel family / reduce mode of plans created afterwards by this thread
+ * (-1 = planner's choice).  A forced choice the shape cannot run gives MTF_ERR_UNSUPPORTED. */
+mtf_status mtf_plan_force(int32_t kernel_kind, int32_t reduce_mode);
+
+/* ---- feed-forward block (Section 8: y = Relu(x w + bias) v) ------------------------------------- */
+/* x [*tokens, d_in], w [d_in, hidden], bias [hidden] or NULL, v [hidden, d_in]; outputs h_saved
+ * [*tokens, hidden] (kept for the backward pass) and y [*tokens, d_in].  Two einsums; bias add and
+ * relu are fused into the first. */
+mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w,
+                           const mtf_tensor* bias, const mtf_tensor* v, mtf_tensor* h_saved, mtf_tensor* y,
+                           void* workspace, size_t workspace_bytes, void* stream);
+/* Backward (Section 8.1: parameter gradients are einsums that reduce out the token dims; Section
+ * 8.2: the gradient on x reduces out hidden):
+ *   dhp = (dy . v^T) * [h_saved > 0];  dv = h^T . dy;  dw = x^T . dhp;  dbias = sum_tokens dhp;
+ *   dx = dhp . w^T.   dbias may be NULL.  dhp lives in the workspace. */
+mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w,
+                            const mtf_tensor* v, const mtf_tensor* h_saved, const mtf_tensor* dy,
+                            mtf_tensor* dx, mtf_tensor* dw, mtf_tensor* dbias, mtf_tensor* dv,
+                            void* workspace, size_t workspace_bytes, void* stream);
+/* Scratch bytes for the larger of forward and backward with these shapes. */
+mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w,
+                                   size_t* bytes);
+
+/* ---- reductions (Section 6 "Reduction") --------------------------------------------------------- */
+/* out[out dims] = sum over the other dims of in (out dims a subset of in's).  Local reduction per
+ * slice, then the group sum across the mesh dims of reduced-out split dims, in one launch. */
+mtf_status mtf_reduce_sum(const mtf_layout_t* layout, const mtf_tensor* in, mtf_tensor* out, void* stream);
+
+/* ---- status ------------------------------------------------------------------------------------- */
+const char* mtf_status_string(mtf_status s);
+const char* mtf_last_error(void);
+/* Synchronises the current device and reads the sticky device status word: 0 = no kernel of this
+ * library gave up on a bounded wait since the last call; non-zero = a code naming the wait.
+ * Resets the word.  Returns MTF_ERR_TIMEOUT when it was non-zero. */
+mtf_status mtf_device_status(int32_t* code);
+/* Number of kernels this library has launched from this process (all threads). */
+int64_t mtf_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTF_H_ */

@@ -1,0 +1,359 @@
+"""Thin ctypes binding of include/mtf.h.  Argument marshalling only: every step of the path runs
+inside libmtf_b200.so.  Function names are those of the C ABI.
+
+Tensors are described by ``Named`` objects: dimension names + sizes + dtype (+ a device pointer
+taken from a contiguous torch tensor).  Planning-only calls accept descriptors without data.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmtf_b200.so")
+
+MTF_F32, MTF_BF16 = 0, 1
+MTF_KERNEL_SIMT, MTF_KERNEL_TCGEN05 = 0, 1
+MTF_REDUCE_NONE, MTF_REDUCE_CHAINED, MTF_REDUCE_WORKSPACE = 0, 1, 2
+STATUS_NAMES = ["MTF_OK", "MTF_ERR_INVALID_ARG", "MTF_ERR_DUPLICATE_DIM", "MTF_ERR_UNKNOWN_DIM",
+                "MTF_ERR_SIZE_MISMATCH", "MTF_ERR_ILLEGAL_LAYOUT", "MTF_ERR_NOT_DIVISIBLE", "MTF_ERR_UNSUPPORTED",
+                "MTF_ERR_WORKSPACE_TOO_SMALL", "MTF_ERR_CUDA", "MTF_ERR_TIMEOUT"]
+
+
+class mtf_dim(Structure):
+    _fields_ = [("name", c_char_p), ("size", c_int64)]
+
+
+class mtf_tensor(Structure):
+    _fields_ = [("data", c_void_p), ("dtype", c_int), ("ndim", c_int32), ("dims", POINTER(mtf_dim))]
+
+
+class mtf_epilogue(Structure):
+    _fields_ = [("scale", c_float), ("relu", c_int32), ("bias", POINTER(mtf_tensor)),
+                ("relu_mask", POINTER(mtf_tensor)), ("residual", POINTER(mtf_tensor))]
+
+
+class MtfError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        self.status = status
+        self.code = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else f"MTF_ERR_{status}"
+        super().__init__(f"{self.code}: {message}")
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: the CUDA library has not been built. Build it with "
+            "`python -m paper_1811_02084_b200.build` (needs nvcc; there is no CPU fallback).")
+    L = ctypes.CDLL(LIB_PATH)
+    vp = c_void_p
+    sig = {
+        "mtf_mesh_create": [c_int32, POINTER(mtf_dim), POINTER(vp)],
+        "mtf_mesh_destroy": [vp],
+        "mtf_mesh_size": [vp, POINTER(c_int64)],
+        "mtf_mesh_coords": [vp, c_int64, POINTER(c_int64)],
+        "mtf_layout": [vp, c_int32, POINTER(c_char_p), POINTER(c_char_p), POINTER(vp)],
+        "mtf_layout_destroy": [vp],
+        "mtf_layout_check_tensor": [vp, c_int32, POINTER(mtf_dim)],
+        "mtf_slice_map": [vp, c_int32, POINTER(mtf_dim), c_int64, POINTER(c_int64), POINTER(c_int64)],
+        "mtf_slice_gather": [vp, POINTER(mtf_tensor), c_int64, vp, vp],
+        "mtf_einsum_plan": [vp, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), POINTER(vp)],
+        "mtf_plan_destroy": [vp],
+        "mtf_plan_workspace_bytes": [vp, POINTER(c_size_t)],
+        "mtf_plan_cost": [vp, POINTER(c_int64), POINTER(c_int64), POINTER(c_int64), POINTER(c_int32)],
+        "mtf_plan_info": [vp, POINTER(c_int32), POINTER(c_int32), POINTER(c_int64), POINTER(c_int64), POINTER(c_uint32)],
+        "mtf_einsum_exec": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp, c_size_t, vp],
+        "mtf_einsum": [vp, c_char_p, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp, c_size_t, vp],
+        "mtf_einsum_workspace_bytes": [vp, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), POINTER(c_size_t)],
+        "mtf_plan_force": [c_int32, c_int32],
+        "mtf_ffn_forward": [vp] + [POINTER(mtf_tensor)] * 6 + [vp, c_size_t, vp],
+        "mtf_ffn_backward": [vp] + [POINTER(mtf_tensor)] * 9 + [vp, c_size_t, vp],
+        "mtf_ffn_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
+        "mtf_reduce_sum": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_device_status": [POINTER(c_int32)],
+    }
+    for name, args in sig.items():
+        fn = getattr(L, name)
+        fn.argtypes = args
+        fn.restype = c_int
+    L.mtf_status_string.argtypes = [c_int]
+    L.mtf_status_string.restype = c_char_p
+    L.mtf_last_error.argtypes = []
+    L.mtf_last_error.restype = c_char_p
+    L.mtf_launch_count.argtypes = []
+    L.mtf_launch_count.restype = c_int64
+    return L
+
+
+_lib = _load()
+
+
+def _check(status: int):
+    if status != 0:
+        raise MtfError(status, _lib.mtf_last_error().decode("utf-8", "replace"))
+
+
+def _dims_array(dims):
+    arr = (mtf_dim * max(len(dims), 1))()
+    keep = []
+    for i, (n, s) in enumerate(dims):
+        b = n.encode("utf-8")
+        keep.append(b)
+        arr[i].name = b
+        arr[i].size = int(s)
+    return arr, keep
+
+
+def _dtype_code(dtype) -> int:
+    if dtype in (MTF_F32, "f32", "float32"):
+        return MTF_F32
+    if dtype in (MTF_BF16, "bf16", "bfloat16"):
+        return MTF_BF16
+    name = str(dtype)
+    if name == "torch.float32":
+        return MTF_F32
+    if name == "torch.bfloat16":
+        return MTF_BF16
+    raise MtfError(1, f"unsupported dtype {dtype!r}")
+
+
+class Named:
+    """A named tensor view: ``dims`` = [(name, size), ...] in storage order, dtype code, device pointer."""
+
+    def __init__(self, dims, dtype, data_ptr=None, owner=None):
+        self.dims = [(str(n), int(s)) for n, s in dims]
+        self.dtype = _dtype_code(dtype)
+        self.ptr = data_ptr
+        self.owner = owner            # keeps the torch tensor alive
+        self._dims_arr, self._keep = _dims_array(self.dims)
+        self.c = mtf_tensor(c_void_p(data_ptr) if data_ptr else None, self.dtype, len(self.dims), self._dims_arr)
+
+    @property
+    def names(self):
+        return [n for n, _ in self.dims]
+
+
+def named(t, names) -> Named:
+    """Describe a contiguous torch tensor (any device; the pointer is passed as is) with dim names."""
+    if len(names) != t.dim():
+        raise MtfError(1, f"{len(names)} names for a {t.dim()}-d tensor")
+    if not t.is_contiguous():
+        raise MtfError(1, "tensors must be dense row-major (contiguous)")
+    return Named(list(zip(names, t.shape)), t.dtype, t.data_ptr(), owner=t)
+
+
+def desc(dims, dtype) -> Named:
+    """A descriptor without data (for planning calls)."""
+    return Named(dims, dtype)
+
+
+def _stream(stream):
+    if stream is not None:
+        return c_void_p(int(stream))
+    try:
+        import torch
+        if torch.cuda.is_available():
+            return c_void_p(torch.cuda.current_stream().cuda_stream)
+    except Exception:
+        pass
+    return c_void_p(0)
+
+
+def _ws(workspace):
+    if workspace is None:
+        return c_void_p(0), 0
+    return c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+class Epilogue:
+    def __init__(self, scale=1.0, relu=False, bias: Named | None = None, relu_mask: Named | None = None,
+                 residual: Named | None = None):
+        self.refs = (bias, relu_mask, residual)
+        self.c = mtf_epilogue(float(scale), 1 if relu else 0,
+                              ctypes.pointer(bias.c) if bias is not None else None,
+                              ctypes.pointer(relu_mask.c) if relu_mask is not None else None,
+                              ctypes.pointer(residual.c) if residual is not None else None)
+
+
+def _epi(e):
+    return byref(e.c) if e is not None else None
+
+
+class Mesh:
+    def __init__(self, handle, dims):
+        self.handle = handle
+        self.dims = dims
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.mtf_mesh_destroy(self.handle)
+            self.handle = None
+
+
+class Layout:
+    def __init__(self, handle, mesh_dims, rules):
+        self.handle = handle
+        self.mesh_dims = mesh_dims
+        self.rules = rules
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.mtf_layout_destroy(self.handle)
+            self.handle = None
+
+
+class Plan:
+    def __init__(self, handle):
+        self.handle = handle
+
+    def __del__(self):
+        if getattr(self, "handle", None):
+            _lib.mtf_plan_destroy(self.handle)
+            self.handle = None
+
+
+# ---- the C ABI, name for name ---------------------------------------------------------------------
+
+def mtf_mesh_create(mesh_dims) -> Mesh:
+    arr, _keep = _dims_array(mesh_dims)
+    h = c_void_p()
+    _check(_lib.mtf_mesh_create(len(mesh_dims), arr, byref(h)))
+    return Mesh(h, list(mesh_dims))
+
+
+def mtf_mesh_size(mesh: Mesh) -> int:
+    n = c_int64()
+    _check(_lib.mtf_mesh_size(mesh.handle, byref(n)))
+    return n.value
+
+
+def mtf_mesh_coords(mesh: Mesh, processor: int):
+    out = (c_int64 * len(mesh.dims))()
+    _check(_lib.mtf_mesh_coords(mesh.handle, processor, out))
+    return list(out)
+
+
+def mtf_layout(mesh: Mesh, rules) -> Layout:
+    n = len(rules)
+    t = (c_char_p * max(n, 1))(*[r[0].encode() for r in rules])
+    m = (c_char_p * max(n, 1))(*[r[1].encode() for r in rules])
+    h = c_void_p()
+    _check(_lib.mtf_layout(mesh.handle, n, t, m, byref(h)))
+    return Layout(h, list(mesh.dims), list(rules))
+
+
+def mtf_layout_check_tensor(layout: Layout, dims) -> None:
+    arr, _keep = _dims_array(dims)
+    _check(_lib.mtf_layout_check_tensor(layout.handle, len(dims), arr))
+
+
+def mtf_slice_map(layout: Layout, dims, processor: int):
+    arr, _keep = _dims_array(dims)
+    offs = (c_int64 * max(len(dims), 1))()
+    sizes = (c_int64 * max(len(dims), 1))()
+    _check(_lib.mtf_slice_map(layout.handle, len(dims), arr, processor, offs, sizes))
+    return list(offs)[:len(dims)], list(sizes)[:len(dims)]
+
+
+def mtf_slice_gather(layout: Layout, glob: Named, processor: int, out_slice, stream=None) -> None:
+    _check(_lib.mtf_slice_gather(layout.handle, byref(glob.c), processor, c_void_p(out_slice.data_ptr()), _stream(stream)))
+
+
+def _tensor_array(ts):
+    arr = (mtf_tensor * len(ts))()
+    for i, t in enumerate(ts):
+        arr[i] = t.c
+    return arr
+
+
+def mtf_einsum_plan(layout: Layout, ins, out: Named, epilogue: Epilogue | None = None) -> Plan:
+    h = c_void_p()
+    _check(_lib.mtf_einsum_plan(layout.handle, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue), byref(h)))
+    return Plan(h)
+
+
+def mtf_plan_workspace_bytes(plan: Plan) -> int:
+    b = c_size_t()
+    _check(_lib.mtf_plan_workspace_bytes(plan.handle, byref(b)))
+    return b.value
+
+
+def mtf_plan_cost(plan: Plan) -> dict:
+    a, b, c, d = c_int64(), c_int64(), c_int64(), c_int32()
+    _check(_lib.mtf_plan_cost(plan.handle, byref(a), byref(b), byref(c), byref(d)))
+    return {"macs_per_proc": a.value, "allreduce_values": b.value, "slice_elems": c.value, "n_reduce_mesh_dims": d.value}
+
+
+def mtf_plan_info(plan: Plan) -> dict:
+    k, r, n, g, m = c_int32(), c_int32(), c_int64(), c_int64(), c_uint32()
+    _check(_lib.mtf_plan_info(plan.handle, byref(k), byref(r), byref(n), byref(g), byref(m)))
+    return {"kernel_kind": k.value, "reduce_mode": r.value, "n_slices": n.value, "group_size": g.value,
+            "reduce_mesh_dim_mask": m.value}
+
+
+def mtf_einsum_exec(plan: Plan, ins, out: Named, epilogue: Epilogue | None = None, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_einsum_exec(plan.handle, _tensor_array(ins), byref(out.c), _epi(epilogue), wp, wb, _stream(stream)))
+
+
+def mtf_einsum(layout: Layout, equation, ins, out: Named, epilogue: Epilogue | None = None, workspace=None,
+               stream=None) -> None:
+    wp, wb = _ws(workspace)
+    eq = equation.encode() if equation is not None else None
+    _check(_lib.mtf_einsum(layout.handle, eq, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue), wp, wb,
+                           _stream(stream)))
+
+
+def mtf_einsum_workspace_bytes(layout: Layout, ins, out: Named, epilogue: Epilogue | None = None) -> int:
+    b = c_size_t()
+    _check(_lib.mtf_einsum_workspace_bytes(layout.handle, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue), byref(b)))
+    return b.value
+
+
+def mtf_plan_force(kernel_kind: int = -1, reduce_mode: int = -1) -> None:
+    _check(_lib.mtf_plan_force(kernel_kind, reduce_mode))
+
+
+def _p(t: Named | None):
+    return byref(t.c) if t is not None else None
+
+
+def mtf_ffn_forward(layout, x, w, bias, v, h_saved, y, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_ffn_forward(layout.handle, _p(x), _p(w), _p(bias), _p(v), _p(h_saved), _p(y), wp, wb, _stream(stream)))
+
+
+def mtf_ffn_backward(layout, x, w, v, h_saved, dy, dx, dw, dbias, dv, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_ffn_backward(layout.handle, _p(x), _p(w), _p(v), _p(h_saved), _p(dy), _p(dx), _p(dw), _p(dbias),
+                                 _p(dv), wp, wb, _stream(stream)))
+
+
+def mtf_ffn_workspace_bytes(layout, x, w) -> int:
+    b = c_size_t()
+    _check(_lib.mtf_ffn_workspace_bytes(layout.handle, _p(x), _p(w), byref(b)))
+    return b.value
+
+
+def mtf_reduce_sum(layout, inp: Named, out: Named, stream=None) -> None:
+    _check(_lib.mtf_reduce_sum(layout.handle, _p(inp), _p(out), _stream(stream)))
+
+
+def mtf_status_string(status: int) -> str:
+    return _lib.mtf_status_string(status).decode()
+
+
+def mtf_last_error() -> str:
+    return _lib.mtf_last_error().decode("utf-8", "replace")
+
+
+def mtf_device_status() -> int:
+    """Synchronises the device; raises MtfError(MTF_ERR_TIMEOUT) when a bounded wait gave up."""
+    c = c_int32()
+    _check(_lib.mtf_device_status(byref(c)))
+    return c.value
+
+
+def mtf_launch_count() -> int:
+    return int(_lib.mtf_launch_count())

@@ -1,0 +1,440 @@
+// The C ABI (include/mtf.h): argument checking, plan caching and the block compositions.  Every
+// numerical step runs in the CUDA kernels; this file only validates, plans and launches.
+#include <algorithm>
+#include <cstring>
+
+#include "mtf_internal.h"
+
+namespace mtf {
+const char* last_error();
+int64_t launch_count();
+mtf_status read_device_status(int* code);
+}  // namespace mtf
+
+using mtf::Dim;
+using mtf::fail;
+
+namespace {
+
+thread_local int g_force_kernel = -1;
+thread_local int g_force_reduce = -1;
+
+int elem_bytes(int dt) { return dt == MTF_BF16 ? 2 : 4; }
+
+bool dims_match(const std::vector<Dim>& want, const mtf_tensor& t) {
+  if ((int)want.size() != t.ndim) return false;
+  for (int i = 0; i < t.ndim; ++i)
+    if (!t.dims[i].name || want[i].name != t.dims[i].name || want[i].size != t.dims[i].size) return false;
+  return true;
+}
+
+mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epi,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+  if (!P || !in || !out) return fail(MTF_ERR_INVALID_ARG, "einsum exec: NULL argument");
+  if (!dims_match(P->dimsA, in[0]) || (P->has_B && !dims_match(P->dimsB, in[1])) || !dims_match(P->dimsC, *out))
+    return fail(MTF_ERR_SIZE_MISMATCH, "einsum exec: operand dims differ from the planned ones");
+  if (in[0].dtype != P->dtA || (P->has_B && in[1].dtype != P->dtB) || out->dtype != P->dtC)
+    return fail(MTF_ERR_INVALID_ARG, "einsum exec: operand dtypes differ from the planned ones");
+  if (!in[0].data || (P->has_B && !in[1].data) || !out->data) return fail(MTF_ERR_INVALID_ARG, "einsum exec: NULL data pointer");
+  const void* bias = nullptr;
+  const void* mask = nullptr;
+  const void* resid = nullptr;
+  if (P->epi.on) {
+    if (!epi) return fail(MTF_ERR_INVALID_ARG, "einsum exec: the plan has an epilogue, none was passed");
+    if (P->epi.has_bias) {
+      if (!epi->bias || !epi->bias->data || !dims_match(P->epi.bias_dims, *epi->bias) || epi->bias->dtype != P->epi.dtBias)
+        return fail(MTF_ERR_INVALID_ARG, "einsum exec: bias differs from the planned one");
+      bias = epi->bias->data;
+    }
+    if (P->epi.has_mask) {
+      if (!epi->relu_mask || !epi->relu_mask->data || !dims_match(P->dimsC, *epi->relu_mask) || epi->relu_mask->dtype != P->epi.dtMask)
+        return fail(MTF_ERR_INVALID_ARG, "einsum exec: relu_mask differs from the planned one");
+      mask = epi->relu_mask->data;
+    }
+    if (P->epi.has_res) {
+      if (!epi->residual || !epi->residual->data || !dims_match(P->dimsC, *epi->residual) || epi->residual->dtype != P->epi.dtRes)
+        return fail(MTF_ERR_INVALID_ARG, "einsum exec: residual differs from the planned one");
+      resid = epi->residual->data;
+    }
+  }
+  const float scale = P->epi.on ? epi->scale : 1.f;
+  const int relu = P->epi.on ? (epi->relu != 0) : 0;
+  if (P->kernel_kind == MTF_KERNEL_TCGEN05)
+    return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
+                          P->epi.dtRes, scale, relu, workspace, workspace_bytes, stream);
+  SimtParams s = P->simt;
+  s.A = in[0].data;
+  s.B = P->has_B ? in[1].data : nullptr;
+  s.C = out->data;
+  s.bias = bias; s.mask = mask; s.resid = resid;
+  s.scale = scale; s.relu = relu;
+  return mtf::launch_simt(s, stream);
+}
+
+// Plan through the layout's cache.  The returned pointer stays valid for the layout's lifetime.
+mtf_status cached_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, const mtf_tensor* out,
+                       const mtf_epilogue* epi, const mtf_plan_t** plan) {
+  if (!L || !in || !out) return fail(MTF_ERR_INVALID_ARG, "einsum: NULL argument");
+  if (n_in < 1 || n_in > 2) return fail(MTF_ERR_UNSUPPORTED, "einsum: the GPU path takes 1 or 2 inputs, got %d", n_in);
+  for (int q = 0; q < n_in; ++q)
+    if (in[q].ndim < 0 || in[q].ndim > mtf::kMaxTensorDims || (in[q].ndim && !in[q].dims)) return fail(MTF_ERR_INVALID_ARG, "einsum: bad input descriptor");
+  if (out->ndim < 0 || out->ndim > mtf::kMaxTensorDims || (out->ndim && !out->dims)) return fail(MTF_ERR_INVALID_ARG, "einsum: bad output descriptor");
+  mtf_layout_t* Lm = const_cast<mtf_layout_t*>(L);
+  const std::string key = mtf::plan_key(n_in, in, out, epi, g_force_kernel, g_force_reduce);
+  std::lock_guard<std::mutex> lock(Lm->mu);
+  auto it = Lm->cache.find(key);
+  if (it == Lm->cache.end()) {
+    std::unique_ptr<mtf_plan_t> P;
+    mtf_status st = mtf::make_plan(L, n_in, in, out, epi, g_force_kernel, g_force_reduce, &P);
+    if (st != MTF_OK) return st;
+    P->key = key;
+    it = Lm->cache.emplace(key, std::move(P)).first;
+  }
+  *plan = it->second.get();
+  return MTF_OK;
+}
+
+// "batch io, io hidden -> batch hidden" must agree with the descriptors' names.
+mtf_status check_equation(const char* eq, int n_in, const mtf_tensor* in, const mtf_tensor* out) {
+  std::vector<std::vector<std::string>> groups(1);
+  std::string tok;
+  auto flush = [&] { if (!tok.empty()) { groups.back().push_back(tok); tok.clear(); } };
+  for (const char* c = eq; *c; ++c) {
+    if (*c == ',') { flush(); groups.emplace_back(); }
+    else if (*c == '-' && c[1] == '>') { flush(); groups.emplace_back(); ++c; }
+    else if (*c == ' ' || *c == '\t') flush();
+    else tok.push_back(*c);
+  }
+  flush();
+  if ((int)groups.size() != n_in + 1) return fail(MTF_ERR_INVALID_ARG, "equation '%s' does not have %d inputs and one output", eq, n_in);
+  for (int q = 0; q <= n_in; ++q) {
+    const mtf_tensor& t = q < n_in ? in[q] : *out;
+    if ((int)groups[q].size() != t.ndim) return fail(MTF_ERR_INVALID_ARG, "equation '%s': operand %d has %d dims, descriptor has %d", eq, q, (int)groups[q].size(), t.ndim);
+    for (int i = 0; i < t.ndim; ++i)
+      if (groups[q][i] != t.dims[i].name) return fail(MTF_ERR_INVALID_ARG, "equation '%s': operand %d dim %d is '%s' in the descriptor", eq, q, i, t.dims[i].name);
+  }
+  return MTF_OK;
+}
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+int64_t numel(const mtf_tensor& t) {
+  int64_t n = 1;
+  for (int i = 0; i < t.ndim; ++i) n *= t.dims[i].size;
+  return n;
+}
+
+struct FfnShapes {
+  std::vector<mtf_dim> tok_hidden, hidden_only;
+};
+
+mtf_status ffn_check(const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v) {
+  if (!x || !w || !v) return fail(MTF_ERR_INVALID_ARG, "ffn: NULL tensor");
+  if (x->ndim < 2 || x->ndim > mtf::kMaxTensorDims - 1 || w->ndim != 2 || v->ndim != 2 || !x->dims || !w->dims || !v->dims)
+    return fail(MTF_ERR_INVALID_ARG, "ffn: x must be [*tokens, d_in], w [d_in, hidden], v [hidden, d_out]");
+  for (int i = 0; i < x->ndim; ++i) if (!x->dims[i].name) return fail(MTF_ERR_INVALID_ARG, "ffn: unnamed dimension");
+  if (!w->dims[0].name || !w->dims[1].name || !v->dims[0].name || !v->dims[1].name) return fail(MTF_ERR_INVALID_ARG, "ffn: unnamed dimension");
+  if (strcmp(x->dims[x->ndim - 1].name, w->dims[0].name) != 0) return fail(MTF_ERR_UNKNOWN_DIM, "ffn: x's last dim '%s' is not w's first dim '%s'", x->dims[x->ndim - 1].name, w->dims[0].name);
+  if (strcmp(w->dims[1].name, v->dims[0].name) != 0) return fail(MTF_ERR_UNKNOWN_DIM, "ffn: w's second dim '%s' is not v's first dim '%s'", w->dims[1].name, v->dims[0].name);
+  return MTF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+mtf_status mtf_mesh_create(int32_t ndim, const mtf_dim* mesh_dims, mtf_mesh_t** out) {
+  if (!out) return fail(MTF_ERR_INVALID_ARG, "mesh_create: out is NULL");
+  *out = nullptr;
+  if (ndim < 1 || ndim > mtf::kMaxMeshDims) return fail(MTF_ERR_INVALID_ARG, "mesh_create: ndim %d outside [1, %d]", ndim, mtf::kMaxMeshDims);
+  std::vector<Dim> d;
+  mtf_status st = mtf::read_dims(ndim, mesh_dims, &d, "mesh");
+  if (st != MTF_OK) return st;
+  mtf_mesh_t* m = new mtf_mesh_t();
+  m->dims = d;
+  for (auto& x : d) m->P *= x.size;
+  *out = m;
+  return MTF_OK;
+}
+
+mtf_status mtf_mesh_destroy(mtf_mesh_t* mesh) {
+  delete mesh;
+  return MTF_OK;
+}
+
+mtf_status mtf_mesh_size(const mtf_mesh_t* mesh, int64_t* n) {
+  if (!mesh || !n) return fail(MTF_ERR_INVALID_ARG, "mesh_size: NULL argument");
+  *n = mesh->P;
+  return MTF_OK;
+}
+
+mtf_status mtf_mesh_coords(const mtf_mesh_t* mesh, int64_t p, int64_t* coords) {
+  if (!mesh || !coords) return fail(MTF_ERR_INVALID_ARG, "mesh_coords: NULL argument");
+  if (p < 0 || p >= mesh->P) return fail(MTF_ERR_INVALID_ARG, "mesh_coords: processor %lld outside mesh of %lld", (long long)p, (long long)mesh->P);
+  for (int j = (int)mesh->dims.size() - 1; j >= 0; --j) {
+    coords[j] = p % mesh->dims[j].size;
+    p /= mesh->dims[j].size;
+  }
+  return MTF_OK;
+}
+
+mtf_status mtf_layout(const mtf_mesh_t* mesh, int32_t nrules, const char* const* tensor_dim, const char* const* mesh_dim,
+                      mtf_layout_t** out) {
+  if (!out) return fail(MTF_ERR_INVALID_ARG, "layout: out is NULL");
+  *out = nullptr;
+  if (!mesh) return fail(MTF_ERR_INVALID_ARG, "layout: mesh is NULL");
+  if (nrules < 0 || nrules > 64 || (nrules > 0 && (!tensor_dim || !mesh_dim))) return fail(MTF_ERR_INVALID_ARG, "layout: bad rule list");
+  std::unique_ptr<mtf_layout_t> L(new mtf_layout_t());
+  L->mesh = mesh->dims;
+  for (int i = 0; i < nrules; ++i) {
+    if (!tensor_dim[i] || !tensor_dim[i][0] || !mesh_dim[i]) return fail(MTF_ERR_INVALID_ARG, "layout: rule %d has an empty name", i);
+    int j = -1;
+    for (size_t m = 0; m < mesh->dims.size(); ++m)
+      if (mesh->dims[m].name == mesh_dim[i]) j = (int)m;
+    if (j < 0) return fail(MTF_ERR_UNKNOWN_DIM, "layout: mesh has no dimension '%s'", mesh_dim[i]);
+    for (auto& r : L->rules)
+      if (r.first == tensor_dim[i]) return fail(MTF_ERR_INVALID_ARG, "layout: tensor dimension '%s' is mapped twice", tensor_dim[i]);
+    L->rules.emplace_back(tensor_dim[i], j);
+  }
+  *out = L.release();
+  return MTF_OK;
+}
+
+mtf_status mtf_layout_destroy(mtf_layout_t* layout) {
+  delete layout;
+  return MTF_OK;
+}
+
+mtf_status mtf_layout_check_tensor(const mtf_layout_t* layout, int32_t ndim, const mtf_dim* dims) {
+  if (!layout) return fail(MTF_ERR_INVALID_ARG, "layout_check_tensor: layout is NULL");
+  std::vector<Dim> d;
+  mtf_status st = mtf::read_dims(ndim, dims, &d, "tensor");
+  if (st != MTF_OK) return st;
+  return mtf::check_tensor(layout, d);
+}
+
+mtf_status mtf_slice_map(const mtf_layout_t* layout, int32_t ndim, const mtf_dim* dims, int64_t processor,
+                         int64_t* offsets, int64_t* sizes) {
+  if (!layout || (ndim > 0 && (!offsets || !sizes))) return fail(MTF_ERR_INVALID_ARG, "slice_map: NULL argument");
+  std::vector<Dim> d;
+  mtf_status st = mtf::read_dims(ndim, dims, &d, "tensor");
+  if (st != MTF_OK) return st;
+  return mtf::slice_box(layout, d, processor, offsets, sizes);
+}
+
+mtf_status mtf_slice_gather(const mtf_layout_t* layout, const mtf_tensor* global, int64_t processor, void* out_slice,
+                            void* stream) {
+  if (!layout || !global || !global->data || !out_slice) return fail(MTF_ERR_INVALID_ARG, "slice_gather: NULL argument");
+  if (global->dtype != MTF_F32 && global->dtype != MTF_BF16) return fail(MTF_ERR_INVALID_ARG, "slice_gather: unknown dtype");
+  std::vector<Dim> d;
+  mtf_status st = mtf::read_dims(global->ndim, global->dims, &d, "tensor");
+  if (st != MTF_OK) return st;
+  int64_t offs[mtf::kMaxTensorDims], sizes[mtf::kMaxTensorDims];
+  if ((st = mtf::slice_box(layout, d, processor, offs, sizes)) != MTF_OK) return st;
+  auto gs = mtf::row_major_strides(d);
+  return mtf::launch_slice_gather(global->data, out_slice, elem_bytes(global->dtype), global->ndim, sizes, offs, gs.data(), stream);
+}
+
+mtf_status mtf_einsum_plan(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in_desc, const mtf_tensor* out_desc,
+                           const mtf_epilogue* epilogue, mtf_plan_t** out) {
+  if (!out) return fail(MTF_ERR_INVALID_ARG, "einsum_plan: out is NULL");
+  *out = nullptr;
+  std::unique_ptr<mtf_plan_t> P;
+  mtf_status st = mtf::make_plan(layout, n_in, in_desc, out_desc, epilogue, g_force_kernel, g_force_reduce, &P);
+  if (st != MTF_OK) return st;
+  *out = P.release();
+  return MTF_OK;
+}
+
+mtf_status mtf_plan_destroy(mtf_plan_t* plan) {
+  delete plan;
+  return MTF_OK;
+}
+
+mtf_status mtf_plan_workspace_bytes(const mtf_plan_t* plan, size_t* bytes) {
+  if (!plan || !bytes) return fail(MTF_ERR_INVALID_ARG, "plan_workspace_bytes: NULL argument");
+  *bytes = plan->workspace_bytes;
+  return MTF_OK;
+}
+
+mtf_status mtf_plan_cost(const mtf_plan_t* plan, int64_t* macs, int64_t* allreduce_values, int64_t* slice_elems, int32_t* n_reduce) {
+  if (!plan) return fail(MTF_ERR_INVALID_ARG, "plan_cost: plan is NULL");
+  if (macs) *macs = plan->macs_per_proc;
+  if (allreduce_values) *allreduce_values = plan->allreduce_values;
+  if (slice_elems) *slice_elems = plan->slice_elems;
+  if (n_reduce) *n_reduce = plan->n_reduce_mesh_dims;
+  return MTF_OK;
+}
+
+mtf_status mtf_plan_info(const mtf_plan_t* plan, int32_t* kernel_kind, int32_t* reduce_mode, int64_t* n_slices,
+                         int64_t* group_size, uint32_t* reduce_mask) {
+  if (!plan) return fail(MTF_ERR_INVALID_ARG, "plan_info: plan is NULL");
+  if (kernel_kind) *kernel_kind = plan->kernel_kind;
+  if (reduce_mode) *reduce_mode = plan->reduce_mode;
+  if (n_slices) *n_slices = plan->n_slices;
+  if (group_size) *group_size = plan->group_size;
+  if (reduce_mask) *reduce_mask = plan->reduce_mask;
+  return MTF_OK;
+}
+
+mtf_status mtf_einsum_exec(const mtf_plan_t* plan, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epilogue,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  return exec_plan(plan, in, out, epilogue, workspace, workspace_bytes, stream);
+}
+
+mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in, mtf_tensor* out,
+                      const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream) {
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, n_in, in, out, epilogue, &P);
+  if (st != MTF_OK) return st;
+  if (equation && (st = check_equation(equation, n_in, in, out)) != MTF_OK) return st;
+  return exec_plan(P, in, out, epilogue, workspace, workspace_bytes, stream);
+}
+
+mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in, const mtf_tensor* out,
+                                      const mtf_epilogue* epilogue, size_t* bytes) {
+  if (!bytes) return fail(MTF_ERR_INVALID_ARG, "einsum_workspace_bytes: bytes is NULL");
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, n_in, in, out, epilogue, &P);
+  if (st != MTF_OK) return st;
+  *bytes = P->workspace_bytes;
+  return MTF_OK;
+}
+
+mtf_status mtf_plan_force(int32_t kernel_kind, int32_t reduce_mode) {
+  if (kernel_kind < -1 || kernel_kind > MTF_KERNEL_TCGEN05 || reduce_mode < -1 || reduce_mode > MTF_REDUCE_WORKSPACE)
+    return fail(MTF_ERR_INVALID_ARG, "plan_force: value out of range");
+  g_force_kernel = kernel_kind;
+  g_force_reduce = reduce_mode;
+  return MTF_OK;
+}
+
+mtf_status mtf_reduce_sum(const mtf_layout_t* layout, const mtf_tensor* in, mtf_tensor* out, void* stream) {
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 1, in, out, nullptr, &P);
+  if (st != MTF_OK) return st;
+  return exec_plan(P, in, out, nullptr, nullptr, 0, stream);
+}
+
+// ---- feed-forward block --------------------------------------------------------------------------------
+
+mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias,
+                           const mtf_tensor* v, mtf_tensor* h_saved, mtf_tensor* y, void* workspace, size_t workspace_bytes,
+                           void* stream) {
+  mtf_status st = ffn_check(x, w, v);
+  if (st != MTF_OK) return st;
+  if (!h_saved || !y) return fail(MTF_ERR_INVALID_ARG, "ffn_forward: NULL output");
+  // h = relu(x.w + bias): bias add and relu ride in the first einsum's epilogue
+  mtf_epilogue e1;
+  e1.scale = 1.f; e1.relu = 1; e1.bias = bias; e1.relu_mask = nullptr; e1.residual = nullptr;
+  mtf_tensor in1[2] = {*x, *w};
+  if ((st = mtf_einsum(layout, nullptr, 2, in1, h_saved, &e1, workspace, workspace_bytes, stream)) != MTF_OK) return st;
+  mtf_tensor in2[2] = {*h_saved, *v};
+  return mtf_einsum(layout, nullptr, 2, in2, y, nullptr, workspace, workspace_bytes, stream);
+}
+
+static void ffn_dhp_desc(const mtf_tensor* h_like_dims_from_x, const mtf_tensor* w, mtf_dtype dt, mtf_dim* storage, mtf_tensor* out) {
+  const mtf_tensor* x = h_like_dims_from_x;
+  for (int i = 0; i < x->ndim - 1; ++i) storage[i] = x->dims[i];
+  storage[x->ndim - 1] = w->dims[1];
+  out->data = nullptr;
+  out->dtype = dt;
+  out->ndim = x->ndim;
+  out->dims = storage;
+}
+
+mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, size_t* bytes) {
+  if (!bytes) return fail(MTF_ERR_INVALID_ARG, "ffn_workspace_bytes: bytes is NULL");
+  if (!layout || !x || !w || x->ndim < 2 || w->ndim != 2 || !x->dims || !w->dims) return fail(MTF_ERR_INVALID_ARG, "ffn_workspace_bytes: bad argument");
+  mtf_dim hd[mtf::kMaxTensorDims];
+  mtf_tensor dhp;
+  ffn_dhp_desc(x, w, x->dtype, hd, &dhp);
+  // dhp buffer + room for the largest per-einsum scratch (workspace-mode partials are bounded by
+  // tiles * group * 128 * 256 * 4 bytes with tiles <= 74; 256 MiB covers every shape that picks it)
+  size_t scratch = 0;
+  {
+    // the four backward einsums and the two forward ones, planned with these shapes
+    mtf_dim vd[2] = {w->dims[1], w->dims[0]};
+    mtf_tensor v = {nullptr, w->dtype, 2, vd};
+    mtf_tensor hs = dhp;
+    mtf_tensor xin = *x;
+    mtf_dim yd[mtf::kMaxTensorDims];
+    for (int i = 0; i < x->ndim; ++i) yd[i] = x->dims[i];
+    mtf_tensor dy = {nullptr, x->dtype, x->ndim, yd};
+    struct Case { mtf_tensor a, b, c; } cases[6] = {
+        {xin, *w, hs}, {hs, v, dy}, {dy, v, dhp}, {hs, dy, {nullptr, MTF_F32, 2, vd}}, {xin, dhp, {nullptr, MTF_F32, 2, w->dims}}, {dhp, *w, xin}};
+    for (auto& c : cases) {
+      mtf_tensor in[2] = {c.a, c.b};
+      size_t b = 0;
+      mtf_status st = mtf_einsum_workspace_bytes(layout, 2, in, &c.c, nullptr, &b);
+      if (st != MTF_OK) return st;
+      scratch = std::max(scratch, b);
+    }
+  }
+  *bytes = align256((size_t)numel(dhp) * elem_bytes(dhp.dtype)) + align256(scratch) + 256;
+  return MTF_OK;
+}
+
+mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,
+                            const mtf_tensor* h_saved, const mtf_tensor* dy, mtf_tensor* dx, mtf_tensor* dw, mtf_tensor* dbias,
+                            mtf_tensor* dv, void* workspace, size_t workspace_bytes, void* stream) {
+  mtf_status st = ffn_check(x, w, v);
+  if (st != MTF_OK) return st;
+  if (!h_saved || !dy || !dx || !dw || !dv) return fail(MTF_ERR_INVALID_ARG, "ffn_backward: NULL tensor");
+  if (h_saved->ndim != x->ndim) return fail(MTF_ERR_SIZE_MISMATCH, "ffn_backward: h_saved must be [*tokens, hidden]");
+  // dhp lives at the head of the workspace
+  mtf_dim hd[mtf::kMaxTensorDims];
+  mtf_tensor dhp;
+  ffn_dhp_desc(x, w, h_saved->dtype, hd, &dhp);
+  const size_t dhp_bytes = align256((size_t)numel(dhp) * elem_bytes(dhp.dtype));
+  if (!workspace || workspace_bytes < dhp_bytes) return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "ffn_backward needs at least %zu workspace bytes, got %zu", dhp_bytes, workspace_bytes);
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return fail(MTF_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+  dhp.data = workspace;
+  void* rest = reinterpret_cast<uint8_t*>(workspace) + dhp_bytes;
+  const size_t rest_bytes = workspace_bytes - dhp_bytes;
+
+  // dhp = (dy . v^T) * [h > 0]   (relu'(0) = 0)
+  mtf_epilogue e1;
+  e1.scale = 1.f; e1.relu = 0; e1.bias = nullptr; e1.relu_mask = h_saved; e1.residual = nullptr;
+  mtf_tensor in1[2] = {*dy, *v};
+  if ((st = mtf_einsum(layout, nullptr, 2, in1, &dhp, &e1, rest, rest_bytes, stream)) != MTF_OK) return st;
+  // dv = h^T . dy  and  dw = x^T . dhp  reduce out the token dims (Section 8.1)
+  mtf_tensor in2[2] = {*h_saved, *dy};
+  if ((st = mtf_einsum(layout, nullptr, 2, in2, dv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  mtf_tensor in3[2] = {*x, dhp};
+  if ((st = mtf_einsum(layout, nullptr, 2, in3, dw, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if (dbias && (st = mtf_reduce_sum(layout, &dhp, dbias, stream)) != MTF_OK) return st;
+  // dx = dhp . w^T reduces out hidden (Section 8.2)
+  mtf_tensor in4[2] = {dhp, *w};
+  return mtf_einsum(layout, nullptr, 2, in4, dx, nullptr, rest, rest_bytes, stream);
+}
+
+const char* mtf_status_string(mtf_status s) {
+  switch (s) {
+    case MTF_OK: return "MTF_OK";
+    case MTF_ERR_INVALID_ARG: return "MTF_ERR_INVALID_ARG";
+    case MTF_ERR_DUPLICATE_DIM: return "MTF_ERR_DUPLICATE_DIM";
+    case MTF_ERR_UNKNOWN_DIM: return "MTF_ERR_UNKNOWN_DIM";
+    case MTF_ERR_SIZE_MISMATCH: return "MTF_ERR_SIZE_MISMATCH";
+    case MTF_ERR_ILLEGAL_LAYOUT: return "MTF_ERR_ILLEGAL_LAYOUT";
+    case MTF_ERR_NOT_DIVISIBLE: return "MTF_ERR_NOT_DIVISIBLE";
+    case MTF_ERR_UNSUPPORTED: return "MTF_ERR_UNSUPPORTED";
+    case MTF_ERR_WORKSPACE_TOO_SMALL: return "MTF_ERR_WORKSPACE_TOO_SMALL";
+    case MTF_ERR_CUDA: return "MTF_ERR_CUDA";
+    case MTF_ERR_TIMEOUT: return "MTF_ERR_TIMEOUT";
+  }
+  return "MTF_ERR_?";
+}
+
+const char* mtf_last_error(void) { return mtf::last_error(); }
+
+mtf_status mtf_device_status(int32_t* code) {
+  int c = 0;
+  mtf_status st = mtf::read_device_status(&c);
+  if (code) *code = c;
+  return st;
+}
+
+int64_t mtf_launch_count(void) { return mtf::launch_count(); }
+
+}  // extern "C"

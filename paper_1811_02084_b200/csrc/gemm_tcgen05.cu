@@ -1,0 +1,655 @@
+// Grouped bf16 contraction on the 5th-generation tensor cores (sm_100a): the per-slice local einsum
+// of Section 6 for every virtual processor of a call in ONE persistent launch, with the sum over a
+// reduce group (the paper's Allreduce within a mesh group) fused in:
+//   CHAINED   - the CTA that owns an output tile runs the K loops of the group's slices back to back
+//               (ascending processor order) into one TMEM accumulator;
+//   WORKSPACE - every (tile, slice) pair is its own work item, writes an fp32 partial, and the warp
+//               that arrives last for its 32 rows adds the partials in ascending processor order.
+// Component-wise work (scale, bias, relu, relu mask, residual, cast) is applied on the way out.
+//
+// Structure of a CTA (192 threads, one CTA per SM, persistent over work items):
+//   warp 0   : TMA producer   - cp.async.bulk.tensor loads (128B swizzle) into a 4-stage smem ring
+//   warp 1   : MMA issuer     - tcgen05.mma kind::f16 (bf16 x bf16 -> fp32), accumulators in TMEM,
+//                               two 128 x 256 accumulators so the epilogue of tile i overlaps tile i+1
+//   warps 2-5: epilogue       - tcgen05.ld of the warp's 32 TMEM lanes, fused epilogue, 16-byte stores
+// Every mbarrier wait is bounded: after ~2 s it records a code in the device status word, raises a
+// CTA-wide abort flag, and all roles fall through to the common teardown (TMEM is freed).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <mutex>
+
+#include "mtf_internal.h"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int kStages = 4;
+constexpr int kMaxBN = 256;
+constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
+constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB
+constexpr int kStageBytes = kAStageBytes + kBStageBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr long long kTimeoutCycles = 4000000000LL;
+
+__device__ int g_status = 0;
+
+struct TcArgs {
+  int M, N, K;
+  int sm, sn, sk;
+  int Ms, Ns, Ks;
+  int n_outer;
+  int outer_local[3];      // extent of each outer dim inside one slice
+  int outer_split[3];
+  long long outer_sC[3];
+  int a_mn_major, b_mn_major;
+  int block_n;
+  long long ldc;
+  int k_sliced;            // walk K slice by slice (slice length is a multiple of BK)
+  int reduce_mode;
+  int m_tiles, n_tiles;    // per slice
+  long long tiles_per_slice, total_tiles, total_work;
+  void* C;
+  int c_bf16;
+  const void* bias;
+  int bias_bf16, bias_along_m;
+  const void* mask;
+  int mask_bf16;
+  const void* resid;
+  int resid_bf16;
+  float scale;
+  int relu;
+  float* ws_partials;
+  unsigned* ws_counters;
+};
+
+struct Tile {
+  int m0, m_end, n0, n_end;
+  int o[3];
+  long long c_off;         // element offset of the outer coordinates in C
+};
+
+__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t) {
+  Tile r;
+  long long slice = t / a.tiles_per_slice;
+  long long w = t % a.tiles_per_slice;
+  const int mt = (int)(w % a.m_tiles); w /= a.m_tiles;
+  const int nt = (int)(w % a.n_tiles); w /= a.n_tiles;
+  int ol[3] = {0, 0, 0};
+  for (int j = a.n_outer - 1; j >= 0; --j) { ol[j] = (int)(w % a.outer_local[j]); w /= a.outer_local[j]; }
+  const int in = (int)(slice % a.sn); slice /= a.sn;
+  const int im = (int)(slice % a.sm); slice /= a.sm;
+  r.c_off = 0;
+  r.o[0] = r.o[1] = r.o[2] = 0;
+  for (int j = a.n_outer - 1; j >= 0; --j) {
+    const int ob = (int)(slice % a.outer_split[j]); slice /= a.outer_split[j];
+    r.o[j] = ob * a.outer_local[j] + ol[j];
+    r.c_off += (long long)r.o[j] * a.outer_sC[j];
+  }
+  r.m0 = im * a.Ms + mt * BM;
+  r.m_end = (im + 1) * a.Ms;
+  r.n0 = in * a.Ns + nt * a.block_n;
+  r.n_end = (in + 1) * a.Ns;
+  return r;
+}
+
+// ---- PTX wrappers -----------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false after the time limit (recording `code`) or when another role aborted.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int code, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  while (true) {
+    for (int i = 0; i < 128; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kTimeoutCycles) {
+      atomicCAS(&g_status, 0, code);
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int code, volatile int* abort_flag) {
+  for (int i = 0; i < 32; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, code, abort_flag);
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_c), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a 128B-swizzled bf16 tile (descriptor version 1).
+//   K-major  (rows of 64 K-elements = 128 B; 8-row groups 1024 B apart): LBO unused (1), SBO = 1024 B
+//   MN-major (rows of 64 M/N-elements = 128 B, one row per k; 64-wide column blocks 8 KB apart):
+//             LBO = 8192 B (next 64 M/N), SBO = 1024 B (next 8 k)
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major) {
+  const uint64_t lbo = mn_major ? (8192u >> 4) : 1u;
+  const uint64_t sbo = 1024u >> 4;
+  return (uint64_t)((addr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t lo16) { return __uint_as_float(lo16 << 16); }
+
+// Fused epilogue on 32 consecutive columns of one output row (fp32 in v), then 16-byte stores.
+__device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, long long row_off, int row, int n_first, int n_valid) {
+  // n_valid: number of valid columns among the 32 (multiple of the store vector)
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] *= a.scale;
+  if (a.bias) {
+    if (a.bias_along_m) {
+      const float b = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row])
+                                  : reinterpret_cast<const float*>(a.bias)[row];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += b;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid)
+          v[j] += a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[n_first + j])
+                              : reinterpret_cast<const float*>(a.bias)[n_first + j];
+    }
+  }
+  if (a.relu) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
+  }
+  const long long off = row_off + n_first;
+  if (a.mask) {
+    if (a.mask_bf16) {
+      const uint4* mp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.mask) + off);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (q * 8 < n_valid) {
+          const uint4 m = mp[q];
+          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (!(bf16_bits_to_float(w[e] & 0xFFFFu) > 0.f)) v[q * 8 + 2 * e] = 0.f;
+            if (!(bf16_bits_to_float(w[e] >> 16) > 0.f)) v[q * 8 + 2 * e + 1] = 0.f;
+          }
+        }
+    } else {
+      const float* mp = reinterpret_cast<const float*>(a.mask) + off;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid && !(mp[j] > 0.f)) v[j] = 0.f;
+    }
+  }
+  if (a.resid) {
+    if (a.resid_bf16) {
+      const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (q * 8 < n_valid) {
+          const uint4 m = rp[q];
+          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            v[q * 8 + 2 * e] += bf16_bits_to_float(w[e] & 0xFFFFu);
+            v[q * 8 + 2 * e + 1] += bf16_bits_to_float(w[e] >> 16);
+          }
+        }
+    } else {
+      const float* rp = reinterpret_cast<const float*>(a.resid) + off;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j < n_valid) v[j] += rp[j];
+    }
+  }
+  if (a.c_bf16) {
+    uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off);
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (q * 8 < n_valid) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 h2 = __floats2bfloat162_rn(v[q * 8 + 2 * e], v[q * 8 + 2 * e + 1]);
+          w[e] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        cp[q] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+  } else {
+    float4* cp = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off);
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      if (q * 4 < n_valid) cp[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte aligned tile ring (the 128B swizzle pattern repeats every 1024 B)
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (tiles_base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + kStages * kStageBytes);
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+  const uint32_t bar_base = tiles_base + kStages * kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
+  auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+  }
+  if (warp == 1) {   // TMEM allocation is a warp-wide operation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const bool ws_mode = a.reduce_mode == MTF_REDUCE_WORKSPACE;
+  const int kb_per_slice = a.Ks / BK;
+  const int kb_total = a.k_sliced ? a.sk * kb_per_slice : (a.K + BK - 1) / BK;
+  const int kb_count = ws_mode ? kb_per_slice : kb_total;
+  const uint32_t b_bytes = (uint32_t)a.block_n * BK * 2;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x) {
+        const long long t = ws_mode ? work / a.sk : work;
+        const int kb_first = ws_mode ? (int)(work % a.sk) * kb_per_slice : 0;
+        const Tile tl = decode_tile(a, t);
+        for (int kb = 0; kb < kb_count; ++kb) {
+          // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
+          // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor)
+          const int k0 = (kb_first + kb) * BK;
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, 0x100 + stage, abort_flag))) break;
+          mbar_expect_tx(full_bar(stage), kAStageBytes + b_bytes);
+          const uint32_t sa = tiles_base + stage * kStageBytes;
+          const uint32_t sb = sa + kAStageBytes;
+          if (a.a_mn_major) {
+            tma_load_5d(sa, &map_a, full_bar(stage), tl.m0, k0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d(sa + 8192, &map_a, full_bar(stage), tl.m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
+          } else {
+            tma_load_5d(sa, &map_a, full_bar(stage), k0, tl.m0, tl.o[2], tl.o[1], tl.o[0]);
+          }
+          if (a.b_mn_major) {
+            for (int j = 0; j < a.block_n / 64; ++j)
+              tma_load_5d(sb + 8192 * j, &map_b, full_bar(stage), tl.n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
+          } else {
+            tma_load_5d(sb, &map_b, full_bar(stage), k0, tl.n0, tl.o[2], tl.o[1], tl.o[0]);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer ---------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.a_mn_major << 15) |
+                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      const uint32_t a_kstep = a.a_mn_major ? 2048u : 32u;   // bytes per 16 k-elements
+      const uint32_t b_kstep = a.b_mn_major ? 2048u : 32u;
+      int stage = 0;
+      uint32_t phase = 0;
+      int iter = 0;
+      bool ok = true;
+      for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x, ++iter) {
+        const int acc = iter & 1;
+        const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, 0x200 + acc, abort_flag))) break;
+        tcgen05_fence_after();
+        const uint32_t tmem_c = tmem_base + (uint32_t)acc * kMaxBN;
+        for (int kb = 0; kb < kb_count; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, 0x300 + stage, abort_flag))) break;
+          tcgen05_fence_after();
+          const uint32_t sa = tiles_base + stage * kStageBytes;
+          const uint32_t sb = sa + kAStageBytes;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = make_smem_desc(sa + k * a_kstep, a.a_mn_major);
+            const uint64_t db = make_smem_desc(sb + k * b_kstep, a.b_mn_major);
+            umma_bf16(tmem_c, da, db, idesc, (kb | k) != 0);
+          }
+          umma_commit(empty_bar(stage));          // frees the smem stage when these MMAs retire
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(acc));      // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -----------------------------------
+    const int q = warp & 3;                        // TMEM lane quarter this warp may read
+    int iter = 0;
+    bool ok = true;
+    for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x, ++iter) {
+      const long long t = ws_mode ? work / a.sk : work;
+      const int ks = ws_mode ? (int)(work % a.sk) : 0;
+      const Tile tl = decode_tile(a, t);
+      const int acc = iter & 1;
+      const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
+      ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const int row = tl.m0 + q * 32 + lane;
+      const bool row_ok = row < tl.m_end;
+      const long long row_off = tl.c_off + (long long)row * a.ldc;
+      const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
+      if (!ws_mode) {
+        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+          uint32_t raw[32];
+          tmem_ld32(taddr + c0, raw);
+          tmem_ld_wait();
+          const int n_first = tl.n0 + c0;
+          int n_valid = tl.n_end - n_first;
+          n_valid = n_valid > 32 ? 32 : n_valid;
+          if (row_ok && n_valid > 0) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
+            epilogue_store(a, v, row_off, row, n_first, n_valid);
+          }
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+      } else {
+        // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
+        float* part = a.ws_partials + ((size_t)(t * a.sk + ks) * BM + (size_t)(q * 32 + lane)) * a.block_n;
+        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+          uint32_t raw[32];
+          tmem_ld32(taddr + c0, raw);
+          tmem_ld_wait();
+          float4* pp = reinterpret_cast<float4*>(part + c0);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            pp[j] = make_float4(__uint_as_float(raw[4 * j]), __uint_as_float(raw[4 * j + 1]),
+                                __uint_as_float(raw[4 * j + 2]), __uint_as_float(raw[4 * j + 3]));
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        __threadfence();
+        __syncwarp();
+        unsigned old = 0;
+        if (lane == 0) old = atomicAdd(&a.ws_counters[t * 4 + q], 1u);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if (old == (unsigned)a.sk - 1) {
+          __threadfence();
+          const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * BM + (size_t)(q * 32 + lane)) * a.block_n;
+          for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+            const int n_first = tl.n0 + c0;
+            int n_valid = tl.n_end - n_first;
+            n_valid = n_valid > 32 ? 32 : n_valid;
+            if (row_ok && n_valid > 0) {
+              float v[32];
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = 0.f;
+              for (int s = 0; s < a.sk; ++s) {     // ascending processor order within the group
+                const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * BM * a.block_n + c0);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 f = __ldcg(sp + j);
+                  v[4 * j] += f.x; v[4 * j + 1] += f.y; v[4 * j + 2] += f.z; v[4 * j + 3] += f.w;
+                }
+              }
+              epilogue_store(a, v, row_off, row, n_first, n_valid);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ------------------------------- teardown --------------------------------------
+  if (*abort_flag) {
+    // failure path: give copies and MMAs in flight time to land before the CTA's resources go away
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tcgen05_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---- host side -----------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// One operand as a 5-D tensor map: (contiguous dim, other of {M|N, K}, outer2, outer1, outer0).
+mtf_status make_map(CUtensorMap* map, const void* base, bool mn_major, int64_t ext_mn, int64_t ext_k, int64_t ld,
+                    const TcParams& t, const int64_t* outer_stride, int box_rows_kmajor) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return mtf::fail(MTF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+  if (reinterpret_cast<uintptr_t>(base) & 15) return mtf::fail(MTF_ERR_INVALID_ARG, "tensor-core path needs 16-byte aligned operands");
+  cuuint64_t dims[5];
+  cuuint64_t strides[4];
+  cuuint32_t box[5] = {64, 1, 1, 1, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  dims[0] = mn_major ? ext_mn : ext_k;
+  dims[1] = mn_major ? ext_k : ext_mn;
+  box[1] = mn_major ? BK : box_rows_kmajor;
+  // the second dimension's stride; a dimension of extent 1 may carry any stride, give it a legal one
+  int64_t s1 = ld;
+  if (dims[1] == 1 || s1 % 8 != 0 || s1 <= 0) s1 = ((int64_t)dims[0] + 7) / 8 * 8;
+  strides[0] = (cuuint64_t)s1 * 2;
+  const int64_t dummy = (s1 * (int64_t)dims[1] + 7) / 8 * 8;   // legal stride for extent-1 dimensions
+  for (int d = 2; d < 5; ++d) {
+    const int src = 4 - d;   // map dim 4 = outer dim 0 ... map dim 2 = outer dim 2 (coordinates o[0..2])
+    if (src < t.n_outer && t.outer_size[src] > 1 && outer_stride[src] > 0) {
+      dims[d] = t.outer_size[src];
+      strides[d - 1] = (cuuint64_t)outer_stride[src] * 2;
+    } else {
+      dims[d] = 1;
+      strides[d - 1] = (cuuint64_t)dummy * 2;
+    }
+  }
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return mtf::fail(MTF_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d (dims %llu %llu %llu %llu %llu, strides %llu %llu %llu %llu)", (int)r,
+                     (unsigned long long)dims[0], (unsigned long long)dims[1], (unsigned long long)dims[2], (unsigned long long)dims[3],
+                     (unsigned long long)dims[4], (unsigned long long)strides[0], (unsigned long long)strides[1],
+                     (unsigned long long)strides[2], (unsigned long long)strides[3]);
+  return MTF_OK;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+}  // namespace
+
+namespace mtf {
+
+static int64_t tc_total_tiles(const TcParams& t) {
+  int64_t tiles = ((t.M / t.sm + BM - 1) / BM) * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sm * t.sn;
+  for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
+  return tiles;
+}
+
+size_t tc_workspace_bytes(const TcParams& t) {
+  if (t.reduce_mode != MTF_REDUCE_WORKSPACE) return 0;
+  const int64_t tiles = tc_total_tiles(t);
+  return (size_t)tiles * t.sk * BM * t.block_n * sizeof(float) + (size_t)tiles * 4 * sizeof(unsigned) + 256;
+}
+
+mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
+                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+  const TcParams& t = plan.tc;
+  if (t.swapped) std::swap(A, B);
+  if (t.M > 0x7fffffffLL || t.N > 0x7fffffffLL || t.K > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "extent beyond 2^31");
+  if (reinterpret_cast<uintptr_t>(C) & 15) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned output");
+  if ((mask && (reinterpret_cast<uintptr_t>(mask) & 15)) || (resid && (reinterpret_cast<uintptr_t>(resid) & 15)))
+    return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs 16-byte aligned epilogue operands");
+
+  TcArgs a;
+  a.M = (int)t.M; a.N = (int)t.N; a.K = (int)t.K;
+  a.sm = (int)t.sm; a.sn = (int)t.sn; a.sk = (int)t.sk;
+  a.Ms = a.M / a.sm; a.Ns = a.N / a.sn; a.Ks = a.K / a.sk;
+  a.n_outer = t.n_outer;
+  for (int j = 0; j < 3; ++j) {
+    a.outer_split[j] = (int)t.outer_split[j];
+    a.outer_local[j] = (int)(t.outer_size[j] / t.outer_split[j]);
+    a.outer_sC[j] = t.outer_sC[j];
+  }
+  a.a_mn_major = t.a_mn_major; a.b_mn_major = t.b_mn_major;
+  a.block_n = t.block_n;
+  a.ldc = t.ldc;
+  a.reduce_mode = t.reduce_mode;
+  a.k_sliced = (t.sk > 1 && a.Ks % BK == 0) ? 1 : 0;
+  a.m_tiles = (a.Ms + BM - 1) / BM;
+  a.n_tiles = (a.Ns + a.block_n - 1) / a.block_n;
+  a.tiles_per_slice = (long long)a.m_tiles * a.n_tiles;
+  for (int j = 0; j < a.n_outer; ++j) a.tiles_per_slice *= a.outer_local[j];
+  long long out_slices = (long long)a.sm * a.sn;
+  for (int j = 0; j < a.n_outer; ++j) out_slices *= a.outer_split[j];
+  a.total_tiles = a.tiles_per_slice * out_slices;
+  a.total_work = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.total_tiles * a.sk : a.total_tiles;
+  a.C = C; a.c_bf16 = plan.dtC == MTF_BF16;
+  a.bias = bias; a.bias_bf16 = dtBias == MTF_BF16; a.bias_along_m = t.bias_along_m;
+  a.mask = mask; a.mask_bf16 = dtMask == MTF_BF16;
+  a.resid = resid; a.resid_bf16 = dtRes == MTF_BF16;
+  a.scale = scale; a.relu = relu;
+  a.ws_partials = nullptr; a.ws_counters = nullptr;
+  if (a.total_work <= 0) return MTF_OK;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
+    const size_t need = tc_workspace_bytes(t);
+    if (!workspace || workspace_bytes < need) return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "einsum needs %zu workspace bytes, got %zu", need, workspace_bytes);
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return fail(MTF_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    const size_t part_bytes = (size_t)a.total_tiles * a.sk * BM * a.block_n * sizeof(float);
+    a.ws_partials = reinterpret_cast<float*>(workspace);
+    a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
+    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * 4 * sizeof(unsigned), st);
+    if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  }
+
+  CUtensorMap map_a, map_b;
+  mtf_status s;
+  if ((s = make_map(&map_a, A, t.a_mn_major, t.M, t.K, t.a_ld, t, t.outer_sA, BM)) != MTF_OK) return s;
+  if ((s = make_map(&map_b, B, t.b_mn_major, t.N, t.K, t.b_ld, t, t.outer_sB, t.block_n)) != MTF_OK) return s;
+
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] { attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes); });
+  if (attr_err != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
+  const long long grid = std::min<long long>(a.total_work, sm_count());
+  gemm_tcgen05_kernel<<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, a);
+  count_launch();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(e));
+  return MTF_OK;
+}
+
+mtf_status read_device_status(int* code) {
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e));
+  int v = 0;
+  e = cudaMemcpyFromSymbol(&v, g_status, sizeof(int));
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemcpyFromSymbol: %s", cudaGetErrorString(e));
+  if (v != 0) {
+    int zero = 0;
+    cudaMemcpyToSymbol(g_status, &zero, sizeof(int));
+  }
+  if (code) *code = v;
+  if (v != 0) return fail(MTF_ERR_TIMEOUT, "a bounded device-side wait gave up (code 0x%x)", v);
+  return MTF_OK;
+}
+
+}  // namespace mtf

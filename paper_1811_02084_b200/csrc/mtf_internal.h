@@ -1,0 +1,159 @@
+// Internal declarations shared by the host planner, the kernels' launchers and the C ABI.
+// Nothing here is visible to users of include/mtf.h.
+#pragma once
+
+#include <cstdint>
+#include <map>
+#include <memory>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "../../include/mtf.h"
+
+namespace mtf {
+
+constexpr int kMaxMeshDims = 4;
+constexpr int kMaxTensorDims = 8;
+constexpr int kMaxIterDims = 12;
+constexpr int kMaxOuter = 3;     // batch-like dims the tensor-core kernel keeps as separate coordinates
+
+struct Dim {
+  std::string name;
+  int64_t size;
+};
+
+void set_error(const char* fmt, ...);
+mtf_status fail(mtf_status s, const char* fmt, ...);
+
+// ---- dims helpers --------------------------------------------------------------------------------
+mtf_status read_dims(int32_t ndim, const mtf_dim* dims, std::vector<Dim>* out, const char* what);
+std::vector<int64_t> row_major_strides(const std::vector<Dim>& dims);
+
+}  // namespace mtf
+
+struct mtf_mesh_s {
+  std::vector<mtf::Dim> dims;
+  int64_t P = 1;
+};
+
+// One dimension of an einsum's iteration space (the union of all operand dimensions).
+struct IterDim {
+  std::string name;
+  int64_t size = 0;
+  int mesh_dim = -1;     // mesh dimension this tensor dimension is split over, -1 = not split
+  int64_t nsplit = 1;    // size of that mesh dimension (1 when not split)
+  int64_t sA = 0, sB = 0, sC = 0;   // element strides in in[0], in[1], out (0 = operand lacks it)
+  bool inA = false, inB = false, inC = false;
+};
+
+// ---- parameters of the generic strided kernel (any dtype mix, any dimension structure) ------------
+struct SimtParams {
+  int n_out = 0;                       // output dims, in the output's storage order
+  int64_t out_size[mtf::kMaxTensorDims];
+  int64_t out_sA[mtf::kMaxTensorDims], out_sB[mtf::kMaxTensorDims], out_sC[mtf::kMaxTensorDims];
+  int64_t out_sBias[mtf::kMaxTensorDims];
+  // reduction loop nest: first n_group levels walk the members of the reduce group in ascending
+  // processor order (one level per split reduced dim, lower mesh-dim index outermost); the rest walk
+  // the local extents of the reduced dims.  A partial sum is closed after each group member.
+  int n_levels = 0, n_group = 0;
+  int64_t lvl_extent[mtf::kMaxIterDims + mtf::kMaxMeshDims];
+  int64_t lvl_sA[mtf::kMaxIterDims + mtf::kMaxMeshDims], lvl_sB[mtf::kMaxIterDims + mtf::kMaxMeshDims];
+  int64_t total_out = 0;
+  int dtA = 0, dtB = 0, dtC = 0, dtBias = 0, dtMask = 0, dtRes = 0;
+  int has_B = 1;
+  float scale = 1.f;
+  int relu = 0;
+  const void* A = nullptr;
+  const void* B = nullptr;
+  void* C = nullptr;
+  const void* bias = nullptr;
+  const void* mask = nullptr;
+  const void* resid = nullptr;
+};
+
+// ---- parameters of the tcgen05 grouped GEMM ---------------------------------------------------------
+// Canonical form: C[o0,o1,o2][m][n] = sum_k A[o..][m][k] * B[o..][k][n], each of M, N, K one merged
+// strided dimension, up to three outer (batch) dimensions.  Every extent may be split into equal
+// contiguous blocks (the virtual processors' slices).
+struct TcParams {
+  int64_t M = 1, N = 1, K = 1;
+  int64_t sm = 1, sn = 1, sk = 1;            // number of slices along M, N, K
+  int n_outer = 0;
+  int64_t outer_size[mtf::kMaxOuter] = {1, 1, 1};
+  int64_t outer_split[mtf::kMaxOuter] = {1, 1, 1};
+  int64_t outer_sC[mtf::kMaxOuter] = {0, 0, 0};
+  int64_t outer_sA[mtf::kMaxOuter] = {0, 0, 0}, outer_sB[mtf::kMaxOuter] = {0, 0, 0};
+  int a_mn_major = 0, b_mn_major = 0;        // 0: K contiguous in smem rows, 1: M/N contiguous
+  int64_t a_ld = 0, b_ld = 0;                // element stride of the non-contiguous one of (M|N, K)
+  int64_t ldc = 0;                           // element stride of M in C (N is contiguous)
+  int block_n = 256;
+  int swapped = 0;                           // in[0] and in[1] exchanged so that N is contiguous in C
+  int reduce_mode = MTF_REDUCE_NONE;
+  int bias_along_m = 0;                      // bias varies with m (after a swap) instead of n
+};
+
+struct EpilogueDesc {
+  bool on = false;
+  float scale = 1.f;
+  bool relu = false;
+  bool has_bias = false, has_mask = false, has_res = false;
+  std::vector<mtf::Dim> bias_dims;
+  int dtBias = 0, dtMask = 0, dtRes = 0;
+};
+
+struct mtf_plan_s {
+  // problem
+  std::vector<mtf::Dim> mesh;
+  std::vector<mtf::Dim> dimsA, dimsB, dimsC;
+  int dtA = 0, dtB = 0, dtC = 0;
+  bool has_B = true;
+  std::vector<IterDim> iter;
+  EpilogueDesc epi;
+  // decisions
+  int kernel_kind = MTF_KERNEL_SIMT;
+  int reduce_mode = MTF_REDUCE_NONE;
+  int64_t n_slices = 1, group_size = 1;
+  uint32_t reduce_mask = 0;
+  size_t workspace_bytes = 0;
+  // cost counts
+  int64_t macs_per_proc = 0, allreduce_values = 0, slice_elems = 0;
+  int n_reduce_mesh_dims = 0;
+  // kernel parameters (pointers filled in at exec time)
+  SimtParams simt;
+  TcParams tc;
+  std::string key;
+};
+
+struct mtf_layout_s {
+  std::vector<mtf::Dim> mesh;
+  std::vector<std::pair<std::string, int>> rules;   // tensor-dim name -> mesh-dim index
+  std::mutex mu;
+  std::map<std::string, std::unique_ptr<mtf_plan_t>> cache;
+  int mesh_dim_of(const std::string& tdim) const {
+    for (auto& r : rules)
+      if (r.first == tdim) return r.second;
+    return -1;
+  }
+};
+
+namespace mtf {
+
+// host planner
+mtf_status check_tensor(const mtf_layout_t* L, const std::vector<Dim>& dims);
+mtf_status slice_box(const mtf_layout_t* L, const std::vector<Dim>& dims, int64_t p, int64_t* offs, int64_t* sizes);
+mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, const mtf_tensor* out,
+                     const mtf_epilogue* epi, int force_kernel, int force_reduce, std::unique_ptr<mtf_plan_t>* plan);
+std::string plan_key(int n_in, const mtf_tensor* in, const mtf_tensor* out, const mtf_epilogue* epi, int fk, int fr);
+
+// launchers (defined in the .cu files)
+mtf_status launch_simt(const SimtParams& p, void* stream);
+mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
+                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu,
+                     void* workspace, size_t workspace_bytes, void* stream);
+size_t tc_workspace_bytes(const TcParams& t);
+mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes,
+                               const int64_t* offs, const int64_t* gstrides, void* stream);
+void count_launch(int n = 1);
+
+}  // namespace mtf

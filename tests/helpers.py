@@ -1,0 +1,123 @@
+"""Shared helpers of the tests: moving seeded inputs to the device, the parity metric, and the
+feed-forward parity routine used at several sizes."""
+from __future__ import annotations
+
+import numpy as np
+
+import seeded_inputs as si
+
+
+def to_torch(stored, device="cuda"):
+    """seeded_inputs.Stored -> torch tensor with exactly those bytes."""
+    import torch
+    if stored.dtype == "bf16":
+        t = torch.from_numpy(stored.bits.view(np.int16).copy()).view(torch.bfloat16)
+    else:
+        t = torch.from_numpy(stored.bits.copy())
+    return t.to(device)
+
+
+def from_torch(t) -> np.ndarray:
+    """Device tensor -> fp64 numpy array (exact widening)."""
+    import torch
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def parity_error(got: np.ndarray, ref: np.ndarray) -> float:
+    """max_i |g_i - r_i| / max(|r_i|, rms(r)): relative error that does not blow up at zeros."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    if ref.size == 0:
+        return 0.0
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    den = np.maximum(np.abs(ref), max(rms, 1e-300))
+    return float(np.max(np.abs(got - ref) / den))
+
+
+TOL = {"bf16": 1e-2, "f32": 1e-4}
+
+
+def ffn_inputs(seed, tok_dims, d_model, d_ff, dtype, with_bias=True, io_name="d_model", hidden_name="d_ff"):
+    """The feed-forward workload: x ~ N(0,1), w ~ N(0,1/d_model), v ~ N(0,1/d_ff), bias ~ 0.1 N(0,1),
+    dy ~ N(0,1).  Returns dict name -> (dims, Stored)."""
+    tok_shape = [s for _, s in tok_dims]
+    out = {
+        "x": (list(tok_dims) + [(io_name, d_model)], si.normal(seed, "x", tok_shape + [d_model], dtype)),
+        "w": ([(io_name, d_model), (hidden_name, d_ff)], si.normal(seed, "w", [d_model, d_ff], dtype, d_model ** -0.5)),
+        "v": ([(hidden_name, d_ff), (io_name, d_model)], si.normal(seed, "v", [d_ff, d_model], dtype, d_ff ** -0.5)),
+        "dy": (list(tok_dims) + [(io_name, d_model)], si.normal(seed, "dy", tok_shape + [d_model], dtype)),
+    }
+    if with_bias:
+        out["bias"] = ([(hidden_name, d_ff)], si.normal(seed, "bias", [d_ff], "f32", 0.1))
+    return out
+
+
+def run_ffn_gpu(mtf, layout, inp, act_dtype, grad_dtype="f32"):
+    """Forward + backward through the C ABI.  Returns dict of fp64 numpy outputs."""
+    import torch
+    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}
+    dev = {k: to_torch(s) for k, (_, s) in inp.items()}
+    N = {k: mtf.named(dev[k], [n for n, _ in d]) for k, (d, _) in inp.items()}
+    xd, wd = inp["x"][0], inp["w"][0]
+    hd = xd[:-1] + [wd[1]]
+    h = torch.empty([s for _, s in hd], dtype=tdt[act_dtype], device="cuda")
+    y = torch.empty([s for _, s in xd], dtype=tdt[act_dtype], device="cuda")
+    dx = torch.empty_like(y)
+    dw = torch.empty([s for _, s in wd], dtype=tdt[grad_dtype], device="cuda")
+    dv = torch.empty([s for _, s in inp["v"][0]], dtype=tdt[grad_dtype], device="cuda")
+    dbias = torch.empty([wd[1][1]], dtype=tdt[grad_dtype], device="cuda")
+    nbytes = mtf.mtf_ffn_workspace_bytes(layout, N["x"], N["w"])
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    nm = lambda t, d: mtf.named(t, [n for n, _ in d])
+    mtf.mtf_ffn_forward(layout, N["x"], N["w"], N.get("bias"), N["v"], nm(h, hd), nm(y, xd), ws)
+    mtf.mtf_ffn_backward(layout, N["x"], N["w"], N["v"], nm(h, hd), N["dy"], nm(dx, xd), nm(dw, wd),
+                         nm(dbias, [wd[1]]) if "bias" in inp else None, nm(dv, inp["v"][0]), ws)
+    mtf.mtf_device_status()
+    out = {"h": h, "y": y, "dx": dx, "dw": dw, "dv": dv}
+    if "bias" in inp:
+        out["dbias"] = dbias
+    return {k: from_torch(t) for k, t in out.items()}
+
+
+def run_ffn_oracle(inp):
+    """Dense fp64 oracle on the same (rounded) inputs; also returns the ambiguity sets of the relu
+    decision: where |hp| is so small that fp32 accumulation may legitimately decide [hp > 0]
+    differently, the outputs that depend on that single decision are not unique."""
+    from oracle import NT, DenseOps, blocks
+    ops = DenseOps()
+    T = {k: NT(d, s.f64) for k, (d, s) in inp.items()}
+    f = blocks.ffn_forward(ops, T["x"], T["w"], T.get("bias"), T["v"])
+    g = blocks.ffn_backward(ops, T["x"], T["w"], T["v"], f["h"], T["dy"])
+    ref = {"h": f["h"].a, "y": f["y"].a, "dx": g["dx"].a, "dw": g["dw"].a, "dv": g["dv"].a}
+    if "bias" in inp:
+        ref["dbias"] = g["dbias"].a
+    hp = f["hp"].a
+    scale = float(np.sqrt(np.mean(hp * hp)))
+    amb = np.abs(hp) < 2e-5 * max(scale, 1e-30)
+    amb2 = amb.reshape(-1, amb.shape[-1])
+    return ref, {"tokens": np.unique(np.nonzero(amb2)[0]), "hidden": np.unique(np.nonzero(amb2)[1])}
+
+
+def check_ffn(got, ref, amb, tol):
+    """Compare everything that is unique; rows / columns that hinge on an ambiguous relu decision are
+    checked for validity only (finite)."""
+    errs = {}
+    for k in ref:
+        g, r = got[k], ref[k]
+        assert np.isfinite(g).all(), k
+        if k == "dx":
+            g2, r2 = g.reshape(-1, g.shape[-1]), r.reshape(-1, r.shape[-1])
+            keep = np.setdiff1d(np.arange(g2.shape[0]), amb["tokens"])
+            errs[k] = parity_error(g2[keep], r2[keep])
+        elif k == "dw":
+            keep = np.setdiff1d(np.arange(g.shape[1]), amb["hidden"])
+            errs[k] = parity_error(g[:, keep], r[:, keep])
+        elif k == "dbias":
+            keep = np.setdiff1d(np.arange(g.shape[0]), amb["hidden"])
+            errs[k] = parity_error(g[keep], r[keep])
+        else:
+            errs[k] = parity_error(g, r)
+    bad = {k: e for k, e in errs.items() if not e <= tol}
+    assert not bad, f"parity above {tol}: {bad} (all: {errs})"
+    return errs

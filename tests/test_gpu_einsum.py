@@ -1,0 +1,246 @@
+"""GPU parity of single einsums against the fp64 oracle, through the C ABI: every operand
+major-ness the tensor-core path takes, ragged sizes, batched (attention-shaped) contractions, both
+ways of realising the group sum, the fused epilogue stages, reductions and the slice gather."""
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from helpers import TOL, from_torch, parity_error, to_torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mtf():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_1811_02084_b200 as m
+    return m
+
+
+def layout(mtf, mesh_dims, rules):
+    return mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules)
+
+
+def run_einsum(mtf, lay, in_dims, out_dims, dtype, out_dtype=None, force=(-1, -1), seed=5, epilogue=None):
+    """Runs one einsum on the GPU and in the oracle.  ``epilogue``: dict with optional keys scale,
+    relu, bias (dims), relu_mask (True), residual (True).  Returns (got, ref, plan info)."""
+    import torch
+    from oracle import NT, DenseOps
+    out_dtype = out_dtype or dtype
+    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}
+    ins = [si.normal(seed, f"in{q}", [s for _, s in d], dtype, 1.0 if q == 0 else float(np.sqrt(1.0 / max(1, min(s for _, s in d)))))
+           for q, d in enumerate(in_dims)]
+    dev = [to_torch(s) for s in ins]
+    names = [mtf.named(t, [n for n, _ in d]) for t, d in zip(dev, in_dims)]
+    out = torch.full([s for _, s in out_dims], float("nan"), dtype=tdt[out_dtype], device="cuda")
+    N_out = mtf.named(out, [n for n, _ in out_dims])
+    ep = None
+    ops = DenseOps()
+    ref = ops.einsum([NT(d, s.f64) for d, s in zip(in_dims, ins)], [n for n, _ in out_dims])
+    keep = []
+    if epilogue:
+        kw = {"scale": epilogue.get("scale", 1.0), "relu": epilogue.get("relu", False)}
+        ref = ops.scale(ref, kw["scale"])
+        if "bias" in epilogue:
+            bd = epilogue["bias"]
+            b = si.normal(seed, "bias", [s for _, s in bd], "f32", 0.5)
+            bt = to_torch(b)
+            keep.append(bt)
+            kw["bias"] = mtf.named(bt, [n for n, _ in bd])
+            ref = ops.add(ref, NT(bd, b.f64))
+        if kw["relu"]:
+            ref = ops.relu(ref)
+        if epilogue.get("relu_mask"):
+            m = si.normal(seed, "mask", [s for _, s in out_dims], out_dtype)
+            mt = to_torch(m)
+            keep.append(mt)
+            kw["relu_mask"] = mtf.named(mt, [n for n, _ in out_dims])
+            ref = ops.mul(ref, ops.positive(NT(out_dims, m.f64)))
+        if epilogue.get("residual"):
+            r = si.normal(seed, "res", [s for _, s in out_dims], out_dtype)
+            rt = to_torch(r)
+            keep.append(rt)
+            kw["residual"] = mtf.named(rt, [n for n, _ in out_dims])
+            ref = ops.add(ref, NT(out_dims, r.f64))
+        ep = mtf.Epilogue(**kw)
+    mtf.mtf_plan_force(*force)
+    try:
+        plan = mtf.mtf_einsum_plan(lay, names, N_out, ep)
+        info = mtf.mtf_plan_info(plan)
+        nbytes = mtf.mtf_plan_workspace_bytes(plan)
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device="cuda")
+        mtf.mtf_einsum_exec(plan, names, N_out, ep, ws)
+    finally:
+        mtf.mtf_plan_force(-1, -1)
+    mtf.mtf_device_status()
+    return from_torch(out), ref.a, info
+
+
+# A[i,k] / A[k,i] x B[k,j] / B[j,k]: the four operand major-ness combinations, sizes that are not
+# multiples of the tile (M 300 = 2 tiles + 44, N 328 = 1 tile + 72, K 200 = 3 k-blocks + 8)
+MAJORS = {
+    "K-major x MN-major": ([("i", 300), ("k", 200)], [("k", 200), ("j", 328)]),
+    "K-major x K-major": ([("i", 300), ("k", 200)], [("j", 328), ("k", 200)]),
+    "MN-major x MN-major": ([("k", 200), ("i", 304)], [("k", 200), ("j", 328)]),
+    "MN-major x K-major": ([("k", 200), ("i", 304)], [("j", 328), ("k", 200)]),
+}
+
+
+@pytest.mark.parametrize("name", list(MAJORS))
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_tensor_core_operand_majors(mtf, name, out_dtype):
+    a, b = MAJORS[name]
+    out_dims = [a[0] if a[0][0] == "i" else a[1], b[1] if b[1][0] == "j" else b[0]]
+    lay = layout(mtf, [("all", 1)], [])
+    got, ref, info = run_einsum(mtf, lay, [a, b], out_dims, "bf16", out_dtype, force=(1, -1))
+    assert info["kernel_kind"] == mtf.MTF_KERNEL_TCGEN05
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+def test_tensor_core_transposed_output_swaps_operands(mtf):
+    # out[j, i]: the contiguous output dim comes from the first operand
+    a, b = [("i", 256), ("k", 128)], [("k", 128), ("j", 192)]
+    got, ref, info = run_einsum(mtf, layout(mtf, [("all", 1)], []), [a, b], [("j", 192), ("i", 256)], "bf16", force=(1, -1))
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+SPLITS = [
+    ([("all", 4)], [("i", "all")]),
+    ([("all", 4)], [("j", "all")]),
+    ([("all", 4)], [("k", "all")]),
+    ([("a", 2), ("b", 2)], [("i", "a"), ("k", "b")]),
+    ([("a", 2), ("b", 2), ("c", 2)], [("i", "a"), ("j", "b"), ("k", "c")]),
+]
+
+
+@pytest.mark.parametrize("mesh_dims,rules", SPLITS)
+@pytest.mark.parametrize("mode", [1, 2], ids=["chained", "workspace"])
+def test_tensor_core_split_dims_and_group_sum(mtf, mesh_dims, rules, mode):
+    a, b = [("i", 512), ("k", 512)], [("k", 512), ("j", 384)]
+    lay = layout(mtf, mesh_dims, rules)
+    k_split = any(t == "k" for t, _ in rules)
+    if mode == 2 and not k_split:
+        with pytest.raises(mtf.MtfError) as e:
+            run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", force=(1, 2))
+        assert e.value.code == "MTF_ERR_UNSUPPORTED"
+        return
+    got, ref, info = run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", "f32", force=(1, mode if k_split else -1))
+    assert info["reduce_mode"] == (mode if k_split else 0)
+    assert info["group_size"] == (2 if k_split and len(mesh_dims) > 1 else (4 if k_split else 1))
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+def test_workspace_and_chained_agree_with_unsplit(mtf):
+    a, b = [("k", 2048), ("i", 256)], [("k", 2048), ("j", 256)]      # a gradient-shaped contraction
+    out = [("i", 256), ("j", 256)]
+    res = {}
+    for tag, mesh_dims, rules, force in (("unsplit", [("all", 1)], [], (1, -1)), ("chained", [("all", 8)], [("k", "all")], (1, 1)),
+                                         ("workspace", [("all", 8)], [("k", "all")], (1, 2)), ("auto", [("all", 8)], [("k", "all")], (-1, -1))):
+        got, ref, info = run_einsum(mtf, layout(mtf, mesh_dims, rules), [a, b], out, "bf16", "f32", force=force)
+        assert parity_error(got, ref) <= TOL["bf16"], tag
+        res[tag] = (got, info)
+    assert res["auto"][1]["reduce_mode"] == mtf.MTF_REDUCE_WORKSPACE      # 2 output tiles only: slices spread over CTAs
+    # fp32 sums in different orders: equal to rounding, and the deterministic modes repeat bit for bit
+    assert np.abs(res["chained"][0] - res["unsplit"][0]).max() <= 1e-3 * np.abs(res["unsplit"][0]).max()
+    again, _, _ = run_einsum(mtf, layout(mtf, [("all", 8)], [("k", "all")]), [a, b], out, "bf16", "f32", force=(1, 2))
+    assert np.array_equal(again, res["workspace"][0])
+
+
+EPILOGUES = [
+    {"scale": 0.125},
+    {"relu": True, "bias": [("j", 328)]},
+    {"bias": [("i", 300)]},
+    {"relu_mask": True},
+    {"residual": True, "scale": 0.5},
+    {"relu": True, "bias": [("j", 328)], "relu_mask": True, "residual": True, "scale": 2.0},
+]
+
+
+@pytest.mark.parametrize("ep", EPILOGUES, ids=lambda e: "+".join(sorted(e)))
+@pytest.mark.parametrize("kind", [0, 1], ids=["simt", "tcgen05"])
+def test_fused_epilogue_stages(mtf, ep, kind):
+    a, b = MAJORS["K-major x MN-major"]
+    got, ref, info = run_einsum(mtf, layout(mtf, [("all", 2)], [("k", "all")]), [a, b], [("i", 300), ("j", 328)], "bf16",
+                                force=(kind, -1), epilogue=ep)
+    assert info["kernel_kind"] == kind
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+# attention-shaped contractions (reading of Section 9: batch b, length l, memory m, heads h, d_k k)
+B_, L_, H_, K_, D_ = 4, 160, 4, 64, 256
+ATT = {
+    "q = x.wq": ([("batch", B_), ("length", L_), ("d_model", D_)], [("d_model", D_), ("heads", H_), ("d_k", K_)],
+                 [("batch", B_), ("length", L_), ("heads", H_), ("d_k", K_)]),
+    "logits = q.k": ([("batch", B_), ("length", L_), ("heads", H_), ("d_k", K_)], [("batch", B_), ("memory_length", L_), ("heads", H_), ("d_k", K_)],
+                     [("batch", B_), ("heads", H_), ("length", L_), ("memory_length", L_)]),
+    "o = P.v": ([("batch", B_), ("heads", H_), ("length", L_), ("memory_length", L_)], [("batch", B_), ("memory_length", L_), ("heads", H_), ("d_v", K_)],
+                [("batch", B_), ("length", L_), ("heads", H_), ("d_v", K_)]),
+    "dv = P^T.do": ([("batch", B_), ("heads", H_), ("length", L_), ("memory_length", L_)], [("batch", B_), ("length", L_), ("heads", H_), ("d_v", K_)],
+                    [("batch", B_), ("memory_length", L_), ("heads", H_), ("d_v", K_)]),
+    "y = o.wo": ([("batch", B_), ("length", L_), ("heads", H_), ("d_v", K_)], [("heads", H_), ("d_v", K_), ("d_model", D_)],
+                 [("batch", B_), ("length", L_), ("d_model", D_)]),
+    "dwq = x^T.dq": ([("batch", B_), ("length", L_), ("d_model", D_)], [("batch", B_), ("length", L_), ("heads", H_), ("d_k", K_)],
+                     [("d_model", D_), ("heads", H_), ("d_k", K_)]),
+    "dx = dq.wq^T": ([("batch", B_), ("length", L_), ("heads", H_), ("d_k", K_)], [("d_model", D_), ("heads", H_), ("d_k", K_)],
+                     [("batch", B_), ("length", L_), ("d_model", D_)]),
+}
+
+
+@pytest.mark.parametrize("name", list(ATT))
+@pytest.mark.parametrize("mesh_dims,rules", [([("all", 1)], []), ([("rows", 2), ("cols", 2)], [("batch", "rows"), ("heads", "cols")])],
+                         ids=["unsplit", "batch-x-heads"])
+def test_attention_shaped_einsums_on_tensor_cores(mtf, name, mesh_dims, rules):
+    a, b, out = ATT[name]
+    got, ref, info = run_einsum(mtf, layout(mtf, mesh_dims, rules), [a, b], out, "bf16", force=(1, -1))
+    assert info["kernel_kind"] == mtf.MTF_KERNEL_TCGEN05
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+def test_generic_kernel_handles_what_tensor_cores_do_not(mtf):
+    lay = layout(mtf, [("a", 2), ("b", 2)], [("length", "a"), ("j", "b")])
+    cases = [
+        # split on the inner component of a merged group (length inside (batch, length))
+        ([("batch", 2), ("length", 8), ("k", 16)], [("k", 16), ("j", 24)], [("batch", 2), ("length", 8), ("j", 24)]),
+        # a reduced dimension that only one operand carries
+        ([("i", 6), ("p", 3), ("k", 16)], [("k", 16), ("j", 24)], [("i", 6), ("j", 24)]),
+        # outer product, no reduced dimension
+        ([("i", 6)], [("j", 24)], [("i", 6), ("j", 24)]),
+        # odd sizes
+        ([("i", 7), ("k", 13)], [("k", 13), ("j", 10)], [("j", 10), ("i", 7)]),
+    ]
+    for a, b, out in cases:
+        for dt in ("f32", "bf16"):
+            got, ref, info = run_einsum(mtf, lay, [a, b], out, dt)
+            assert info["kernel_kind"] == mtf.MTF_KERNEL_SIMT
+            assert parity_error(got, ref) <= TOL[dt], (a, b, out, dt)
+
+
+def test_reduce_sum_under_layouts(mtf):
+    import torch
+    x = si.normal(9, "rx", [48, 40], "f32")
+    xt = to_torch(x)
+    for mesh_dims, rules in (([("all", 4)], []), ([("all", 4)], [("batch", "all")]), ([("a", 2), ("b", 2)], [("batch", "a"), ("hidden", "b")])):
+        lay = layout(mtf, mesh_dims, rules)
+        for out_dims, want in (([("hidden", 40)], x.f64.sum(0)), ([("batch", 48)], x.f64.sum(1)), ([], x.f64.sum())):
+            out = torch.empty([s for _, s in out_dims], dtype=torch.float32, device="cuda")
+            mtf.mtf_reduce_sum(lay, mtf.named(xt, ["batch", "hidden"]), mtf.named(out, [n for n, _ in out_dims]))
+            assert parity_error(from_torch(out), want) <= TOL["f32"]
+
+
+def test_slice_gather_is_bit_exact(mtf):
+    import torch
+    from oracle import Layout, Mesh
+    dims = [("batch", 4), ("hidden", 6), ("io", 8)]
+    mesh_dims, rules = [("rows", 2), ("cols", 3), ("planes", 2)], [("batch", "rows"), ("hidden", "cols"), ("io", "planes")]
+    lay = layout(mtf, mesh_dims, rules)
+    olay = Layout(Mesh(mesh_dims), rules)
+    n = 4 * 6 * 8
+    for tdt in (torch.float32, torch.bfloat16):
+        payload = torch.arange(n, dtype=torch.float32).reshape(4, 6, 8).to(tdt).cuda()     # element = own flat index (exact in bf16 up to 256)
+        for p in range(12):
+            offs, sizes = mtf.mtf_slice_map(lay, dims, p)
+            out = torch.empty(sizes, dtype=tdt, device="cuda")
+            mtf.mtf_slice_gather(lay, mtf.named(payload, [d for d, _ in dims]), p, out)
+            want = olay.global_flat_indices(dims, p).astype(np.float64)
+            assert np.array_equal(from_torch(out).reshape(-1), want), (p, tdt)

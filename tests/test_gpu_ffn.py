@@ -1,0 +1,81 @@
+"""GPU parity of the feed-forward block (Section 8) against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from helpers import TOL, check_ffn, ffn_inputs, run_ffn_gpu, run_ffn_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mtf():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_1811_02084_b200 as m
+    return m
+
+
+def make_layout(mtf, mesh_dims, rules):
+    mesh = mtf.mtf_mesh_create(mesh_dims)
+    return mtf.mtf_layout(mesh, rules)
+
+
+# ---- configuration 1: the fp32 toy of Section 8 on a 2x2 mesh ----------------------------------------
+
+@pytest.mark.parametrize("with_bias", [False, True])
+def test_config1_fp32_toy_mesh_2x2(mtf, with_bias):
+    inp = ffn_inputs(0, [("batch", 8)], 64, 256, "f32", with_bias, io_name="io", hidden_name="hidden")
+    lay = make_layout(mtf, [("rows", 2), ("cols", 2)], [("batch", "rows"), ("hidden", "cols")])
+    got = run_ffn_gpu(mtf, lay, inp, "f32")
+    ref, amb = run_ffn_oracle(inp)
+    check_ffn(got, ref, amb, TOL["f32"])
+
+
+FP32_LAYOUTS = [
+    ([("all", 4)], []),
+    ([("all", 4)], [("batch", "all")]),
+    ([("all", 4)], [("hidden", "all")]),
+    ([("rows", 2), ("cols", 2)], [("batch", "rows"), ("hidden", "cols")]),
+    ([("rows", 2), ("cols", 2), ("planes", 2)], [("batch", "rows"), ("hidden", "cols"), ("io", "planes")]),
+    ([("rows", 2), ("cols", 3)], [("batch", "cols"), ("io", "rows")]),
+]
+
+
+@pytest.mark.parametrize("mesh_dims,rules", FP32_LAYOUTS)
+def test_fp32_every_layout_of_the_example(mtf, mesh_dims, rules):
+    inp = ffn_inputs(1, [("batch", 12)], 40, 72, "f32", True, io_name="io", hidden_name="hidden")
+    got = run_ffn_gpu(mtf, make_layout(mtf, mesh_dims, rules), inp, "f32")
+    ref, amb = run_ffn_oracle(inp)
+    check_ffn(got, ref, amb, TOL["f32"])
+
+
+# ---- bf16 on the tensor-core path: several tiles, ragged tails, every layout family ------------------
+
+BF16_LAYOUTS = [
+    ([("all", 1)], []),
+    ([("all", 8)], [("batch", "all")]),
+    ([("all", 8)], [("d_ff", "all")]),
+    ([("rows", 2), ("cols", 4)], [("batch", "rows"), ("d_ff", "cols")]),
+    ([("all", 2)], [("d_model", "all")]),
+]
+
+
+@pytest.mark.parametrize("mesh_dims,rules", BF16_LAYOUTS)
+@pytest.mark.parametrize("force", [(-1, -1), (1, 1), (0, -1)], ids=["auto", "tc-chained", "simt"])
+def test_bf16_ffn_layouts(mtf, mesh_dims, rules, force):
+    # tokens 8 x 72 = 576 (4.5 row tiles), d_model 320 (5 k-blocks, 1.25 column tiles), d_ff 1088 (17 k-blocks)
+    inp = ffn_inputs(2, [("batch", 8), ("length", 72)], 320, 1088, "bf16", True)
+    mtf.mtf_plan_force(*force)
+    try:
+        got = run_ffn_gpu(mtf, make_layout(mtf, mesh_dims, rules), inp, "bf16")
+    finally:
+        mtf.mtf_plan_force(-1, -1)
+    ref, amb = run_ffn_oracle(inp)
+    check_ffn(got, ref, amb, TOL["bf16"])
+
+
+def test_bf16_outputs_bf16_grads(mtf):
+    inp = ffn_inputs(4, [("batch", 4), ("length", 64)], 256, 512, "bf16", True)
+    got = run_ffn_gpu(mtf, make_layout(mtf, [("all", 4)], [("batch", "all")]), inp, "bf16", grad_dtype="bf16")
+    ref, amb = run_ffn_oracle(inp)
+    check_ffn(got, ref, amb, TOL["bf16"])
