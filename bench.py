@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the hot path: Transformer feed-forward block, forward + backward, as layout-lowered
+named-dimension einsums on one B200 (or N replicas of the batch-split mesh dimension on N GPUs).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--layout mp8|dp8|none] [--impl reference]
+
+One step = mtf_ffn_forward + mtf_ffn_backward through the C ABI on the workload
+tokens 8192 (batch 32 x length 256), d_model 1024, d_ff 8192, bf16 storage / fp32 accumulation
+(six tensor-core contractions, 12 * tokens * d_model * d_ff flop).  Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = {"batch": 32, "length": 256, "d_model": 1024, "d_ff": 8192}
+LAYOUTS = {
+    "none": ([("all", 1)], []),
+    "dp8": ([("all", 8)], [("batch", "all")]),
+    "mp8": ([("all", 8)], [("d_ff", "all")]),
+}
+METRIC = "transformer_ffn_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+
+
+def ffn_flops(tokens, d_model, d_ff):
+    return 12.0 * tokens * d_model * d_ff
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {"bf16_sustained": float(d["bf16_tflops_sustained"]), "bf16_burst": float(d["bf16_tflops"]),
+                    "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+        except Exception:
+            pass
+    return {"bf16_sustained": 1400.0, "bf16_burst": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs (read only)."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self.reasons = set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+
+    def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nvml = None
+            return self
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def _run(self):
+        nv = self._nvml
+        names = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "hw_power_brake_slowdown": 0x80, "sw_power_cap": 0x4}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.005)
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join(timeout=1.0)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------------
+
+def oracle_step_fn(tokens: int, seed: int = 0):
+    import seeded_inputs as si
+    from oracle import NT, DenseOps, blocks
+    d_model, d_ff = WORKLOAD["d_model"], WORKLOAD["d_ff"]
+    ops = DenseOps()
+    x = NT([("batch", 1), ("length", tokens), ("d_model", d_model)], si.normal(seed, "x", [1, tokens, d_model], "bf16").f64)
+    dy = NT(x.dims, si.normal(seed, "dy", [1, tokens, d_model], "bf16").f64)
+    w = NT([("d_model", d_model), ("d_ff", d_ff)], si.normal(seed, "w", [d_model, d_ff], "bf16", d_model ** -0.5).f64)
+    v = NT([("d_ff", d_ff), ("d_model", d_model)], si.normal(seed, "v", [d_ff, d_model], "bf16", d_ff ** -0.5).f64)
+    bias = NT([("d_ff", d_ff)], si.normal(seed, "bias", [d_ff], "f32", 0.1).f64)
+
+    def step():
+        f = blocks.ffn_forward(ops, x, w, bias, v)
+        blocks.ffn_backward(ops, x, w, v, f["h"], dy)
+    return step
+
+
+def time_oracle(tokens: int, steps: int, warmup: int):
+    step = oracle_step_fn(tokens)
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(steps, 1)
+    return dt, ffn_flops(tokens, WORKLOAD["d_model"], WORKLOAD["d_ff"]) / dt / 1e12
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    # size the per-step sample so that the whole run takes about two minutes
+    dt1, _ = time_oracle(1, 1, 1)
+    budget = 120.0 / max(args.steps + args.warmup, 1)
+    tokens = int(max(1, min(256, budget / max(dt1, 1e-6))))
+    dt, tflops = time_oracle(tokens, args.steps, args.warmup)
+    sample = f"ffn fwd+bwd on {tokens} of {WORKLOAD['batch'] * WORKLOAD['length']} tokens (full d_model, d_ff), fp64 loop nest"
+    line = {"impl": "reference", "metric": METRIC, "value": tflops, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "transformer_ffn_fwd_bwd tokens=8192 d_model=1024 d_ff=8192", "sampled_tokens": tokens},
+            "cpu_baseline": {"value": tflops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tflops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import seeded_inputs as si
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
+    import paper_1811_02084_b200 as mtf
+
+    B, L, D, F = WORKLOAD["batch"], WORKLOAD["length"], WORKLOAD["d_model"], WORKLOAD["d_ff"]
+    T = B * L
+    seed = 1000 * rank          # every rank owns its own shard of the (replica x batch) global batch
+    host = {
+        "x": si.normal(seed, "x", [B, L, D], "bf16"),
+        "dy": si.normal(seed, "dy", [B, L, D], "bf16"),
+        "w": si.normal(0, "w", [D, F], "bf16", D ** -0.5),
+        "v": si.normal(0, "v", [F, D], "bf16", F ** -0.5),
+        "bias": si.normal(0, "bias", [F], "f32", 0.1),
+    }
+
+    def dev(s):
+        if s.dtype == "bf16":
+            return torch.from_numpy(s.bits.view(np.int16)).view(torch.bfloat16).cuda()
+        return torch.from_numpy(s.bits).cuda()
+
+    t = {k: dev(s) for k, s in host.items()}
+    h = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda")
+    y = torch.empty(B, L, D, dtype=torch.bfloat16, device="cuda")
+    dx = torch.empty_like(y)
+    dw = torch.empty(D, F, dtype=torch.float32, device="cuda")
+    dv = torch.empty(F, D, dtype=torch.float32, device="cuda")
+    dbias = torch.empty(F, dtype=torch.float32, device="cuda")
+    act, wn, vn = ["batch", "length", "d_model"], ["d_model", "d_ff"], ["d_ff", "d_model"]
+    N = {"x": mtf.named(t["x"], act), "dy": mtf.named(t["dy"], act), "w": mtf.named(t["w"], wn), "v": mtf.named(t["v"], vn),
+         "bias": mtf.named(t["bias"], ["d_ff"]), "h": mtf.named(h, ["batch", "length", "d_ff"]), "y": mtf.named(y, act),
+         "dx": mtf.named(dx, act), "dw": mtf.named(dw, wn), "dv": mtf.named(dv, vn), "dbias": mtf.named(dbias, ["d_ff"])}
+
+    layouts = {}
+    for name, (mesh_dims, rules) in LAYOUTS.items():
+        layouts[name] = mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules)
+    ws_bytes = max(mtf.mtf_ffn_workspace_bytes(l, N["x"], N["w"]) for l in layouts.values())
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(lay):
+        mtf.mtf_ffn_forward(lay, N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
+        mtf.mtf_ffn_backward(lay, N["x"], N["w"], N["v"], N["h"], N["dy"], N["dx"], N["dw"], N["dbias"], N["dv"], ws)
+        if dist is not None:
+            # Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs sums the
+            # parameter gradients across ranks
+            dist.all_reduce(dw)
+            dist.all_reduce(dv)
+            dist.all_reduce(dbias)
+
+    def timed(lay, steps, warmup, sampler=None):
+        for _ in range(warmup):
+            step(lay)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n0 = mtf.mtf_launch_count()
+        e0.record(stream)
+        for _ in range(steps):
+            step(lay)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if sampler else None
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        launches = mtf.mtf_launch_count() - n0
+        if dist is not None:
+            tm = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            ms = float(tm.item())
+        return ms / steps, launches, clocks
+
+    flops_step = ffn_flops(T, D, F)
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    ms_step, launches, clocks = timed(layouts[args.layout], args.steps, max(args.warmup, 3), sampler)
+    mtf.mtf_device_status()
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    per_layout = {}
+    if world == 1:
+        for name, lay in layouts.items():
+            if name == args.layout:
+                per_layout[name] = value
+                continue
+            ms_l, _, _ = timed(lay, max(args.steps // 2, 5), 3)
+            per_layout[name] = flops_step / (ms_l * 1e-3) / 1e12
+
+    # end to end: the step's inputs come from pinned host memory and its results go back, every step
+    hx, hdy = t["x"].cpu().pin_memory(), t["dy"].cpu().pin_memory()
+    hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    lay = layouts[args.layout]
+
+    def e2e_step():
+        t["x"].copy_(hx, non_blocking=True)
+        t["dy"].copy_(hdy, non_blocking=True)
+        step(lay)
+        hy.copy_(y, non_blocking=True)
+        hdx.copy_(dx, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    e2e_steps = max(args.steps // 4, 5)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if dist is not None:
+        tm = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tm.item())
+    e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
+    act_bytes = hx.numel() * hx.element_size()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    # dominant kernel: gemm_tcgen05_kernel, six launches per step of equal algorithmic work
+    gemm_launches_per_step = 6
+    flops_per_launch = flops_step / gemm_launches_per_step
+    avg_launch_ms = ms_step / gemm_launches_per_step        # includes launch gaps: a lower bound on the rate
+    achieved = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(tp):
+        try:
+            traffic = json.load(open(tp)).get("gemm_tcgen05_kernel_bytes_per_launch")
+        except Exception:
+            traffic = None
+    roofline = {"bound": "tensor", "kernel": "gemm_tcgen05_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
+                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "frac_of_datasheet_2250": achieved / 2250.0,
+                "frac_of_measured_burst": achieved / peaks["bf16_burst"], "flops_per_launch": flops_per_launch,
+                "avg_launch_ms": avg_launch_ms}
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cores = len(os.sched_getaffinity(0))
+        tokens = 192
+        dt, tf = time_oracle(tokens, 1, 0)
+        cpu = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"ffn fwd+bwd on {tokens} of {T} tokens (full d_model, d_ff), fp64 loop nest, {dt:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"transformer_ffn_fwd_bwd tokens={T} (batch {B} x length {L}) d_model={D} d_ff={F} per GPU",
+                       "layout": args.layout, "mesh": LAYOUTS[args.layout][0], "rules": LAYOUTS[args.layout][1],
+                       "grad_dtype": "f32", "l2": "inputs larger than L2 (working set ~0.6 GB per step), no flush",
+                       "multi_gpu": "batch split over ranks; NCCL all-reduce of dw, dv, dbias each step" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
+                                      "d2h_bytes_per_step": 2 * act_bytes, "ms_per_step": e2e_ms},
+            "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu, "per_layout_tflops": per_layout,
+            "frac_of_datasheet_bf16_peak": value / world / 2250.0}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layout", default="mp8", choices=sorted(LAYOUTS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -71,6 +71,11 @@ typedef struct { void* data; mtf_dtype dtype; int32_t ndim; const mtf_dim* dims;
  * bias      : dims must be a subset of the output dims (any order);  f32 or bf16.
  * relu_mask : same dims, same order and dtype class as the output (bf16 or f32).
  * residual  : same dims and order as the output (bf16 or f32).
+ * reduce_sum_out : optional second output (Section 6 "Reduction" fused into the einsum): an f32
+ *             tensor whose dims are a subset of the output dims; it receives the sum of t (taken
+ *             after the relu_mask stage, before the residual and the cast) over the other output
+ *             dims.  The library zeroes it on the stream before the launch and accumulates with
+ *             fp32 atomics (order not fixed).  Used for dbias = sum over tokens of dhp.
  * NULL pointers / relu = 0 / scale = 1 switch a stage off.  The struct is read during planning
  * only for which stages are on and their descriptors; data pointers are read at exec time. */
 typedef struct {
@@ -79,6 +84,7 @@ typedef struct {
   const mtf_tensor* bias;
   const mtf_tensor* relu_mask;
   const mtf_tensor* residual;
+  const mtf_tensor* reduce_sum_out;
 } mtf_epilogue;
 
 /* Which kernel family a plan runs (informational; chosen by the planner). */

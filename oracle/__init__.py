@@ -11,6 +11,7 @@ Contents
   lowering.py     per-processor simulation: local op on slices, then the group sum (Allreduce)
   blocks.py       feed-forward, attention, layer norm, decoder layer - forward and backward
   cost.py         per-processor cost counts (Table 1, Appendix B)
+  rounding.py     the one rounding step applied where the method stores an intermediate in bf16
 
 Pins (tests that tie each part to something other than itself) are listed in the test files named
 test_oracle_*.py.  Parts without an external pin: the bf16 rounding behaviour of the GPU path is
@@ -20,7 +21,7 @@ from .named import (NT, DenseOps, DuplicateDim, IllegalLayout, NotDivisible, Ora
                     UnknownDim, einsum_arrays)
 from .mesh import Layout, Mesh
 from .lowering import LT, LoweredOps
-from . import blocks, cost
+from . import blocks, cost, rounding
 
 __all__ = ["NT", "DenseOps", "LoweredOps", "LT", "Mesh", "Layout", "blocks", "cost", "einsum_arrays",
            "OracleError", "DuplicateDim", "UnknownDim", "SizeMismatch", "IllegalLayout", "NotDivisible"]

@@ -20,30 +20,37 @@ import numpy as np
 # Feed-forward block (Section 8)
 # --------------------------------------------------------------------------------------------------
 
-def ffn_forward(ops, x, w, bias, v):
+def _identity(t):
+    return t
+
+
+def ffn_forward(ops, x, w, bias, v, store=_identity):
     """hp = x.w (+ bias);  h = relu(hp);  y = h.v.
-    x: [*tokens, io]   w: [io, hidden]   bias: [hidden] or None   v: [hidden, io]."""
+    x: [*tokens, io]   w: [io, hidden]   bias: [hidden] or None   v: [hidden, io].
+    ``store`` is applied where a result is kept between two einsums (h): identity = exact
+    mathematics, a rounding function = the storage precision of that tensor."""
     tok = list(x.names[:-1])
     hidden = w.names[1]
     hp = ops.einsum([x, w], tok + [hidden])
     if bias is not None:
         hp = ops.add(hp, bias)
-    h = ops.relu(hp)
+    h = store(ops.relu(hp))
     y = ops.einsum([h, v], tok + [v.names[1]])
     return {"hp": hp, "h": h, "y": y}
 
 
-def ffn_backward(ops, x, w, v, h, dy):
+def ffn_backward(ops, x, w, v, h, dy, store=_identity):
     """dh = dy.v^T;  dhp = dh * [h > 0]  (relu'(0) = 0; h > 0 exactly where hp > 0);
     dv = h^T.dy and dw = x^T.dhp (reduce the token dims);  dbias = sum over tokens of dhp;
     dx = dhp.w^T (reduces hidden)."""
     tok = list(x.names[:-1])
     hidden = w.names[1]
     dh = ops.einsum([dy, v], tok + [hidden])
-    dhp = ops.mul(dh, ops.positive(h))
+    dhp_exact = ops.mul(dh, ops.positive(h))
+    dhp = store(dhp_exact)                       # kept between einsums
     dv = ops.einsum([h, dy], list(v.names))
     dw = ops.einsum([x, dhp], list(w.names))
-    dbias = ops.reduce_sum(dhp, [hidden])
+    dbias = ops.reduce_sum(dhp_exact, [hidden])    # summed before the value is stored
     dx = ops.einsum([dhp, w], list(x.names))
     return {"dhp": dhp, "dv": dv, "dw": dw, "dbias": dbias, "dx": dx}
 

@@ -31,7 +31,8 @@ class mtf_tensor(Structure):
 
 class mtf_epilogue(Structure):
     _fields_ = [("scale", c_float), ("relu", c_int32), ("bias", POINTER(mtf_tensor)),
-                ("relu_mask", POINTER(mtf_tensor)), ("residual", POINTER(mtf_tensor))]
+                ("relu_mask", POINTER(mtf_tensor)), ("residual", POINTER(mtf_tensor)),
+                ("reduce_sum_out", POINTER(mtf_tensor))]
 
 
 class MtfError(RuntimeError):
@@ -168,12 +169,13 @@ def _ws(workspace):
 
 class Epilogue:
     def __init__(self, scale=1.0, relu=False, bias: Named | None = None, relu_mask: Named | None = None,
-                 residual: Named | None = None):
-        self.refs = (bias, relu_mask, residual)
+                 residual: Named | None = None, reduce_sum_out: Named | None = None):
+        self.refs = (bias, relu_mask, residual, reduce_sum_out)
         self.c = mtf_epilogue(float(scale), 1 if relu else 0,
                               ctypes.pointer(bias.c) if bias is not None else None,
                               ctypes.pointer(relu_mask.c) if relu_mask is not None else None,
-                              ctypes.pointer(residual.c) if residual is not None else None)
+                              ctypes.pointer(residual.c) if residual is not None else None,
+                              ctypes.pointer(reduce_sum_out.c) if reduce_sum_out is not None else None)
 
 
 def _epi(e):

@@ -57,18 +57,27 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
       resid = epi->residual->data;
     }
   }
+  float* rsum = nullptr;
+  int64_t rsum_elems = 1;
+  if (P->epi.on && P->epi.has_rsum) {
+    if (!epi->reduce_sum_out || !epi->reduce_sum_out->data || !dims_match(P->epi.rsum_dims, *epi->reduce_sum_out) || epi->reduce_sum_out->dtype != MTF_F32)
+      return fail(MTF_ERR_INVALID_ARG, "einsum exec: reduce_sum_out differs from the planned one");
+    rsum = reinterpret_cast<float*>(epi->reduce_sum_out->data);
+    for (auto& d : P->epi.rsum_dims) rsum_elems *= d.size;
+  }
   const float scale = P->epi.on ? epi->scale : 1.f;
   const int relu = P->epi.on ? (epi->relu != 0) : 0;
   if (P->kernel_kind == MTF_KERNEL_TCGEN05)
     return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
-                          P->epi.dtRes, scale, relu, workspace, workspace_bytes, stream);
+                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream);
   SimtParams s = P->simt;
   s.A = in[0].data;
   s.B = P->has_B ? in[1].data : nullptr;
   s.C = out->data;
   s.bias = bias; s.mask = mask; s.resid = resid;
   s.scale = scale; s.relu = relu;
-  return mtf::launch_simt(s, stream);
+  s.rsum = rsum;
+  return mtf::launch_simt(s, rsum_elems, stream);
 }
 
 // Plan through the layout's cache.  The returned pointer stays valid for the layout's lifetime.
@@ -326,7 +335,7 @@ mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, cons
   if (!h_saved || !y) return fail(MTF_ERR_INVALID_ARG, "ffn_forward: NULL output");
   // h = relu(x.w + bias): bias add and relu ride in the first einsum's epilogue
   mtf_epilogue e1;
-  e1.scale = 1.f; e1.relu = 1; e1.bias = bias; e1.relu_mask = nullptr; e1.residual = nullptr;
+  e1.scale = 1.f; e1.relu = 1; e1.bias = bias; e1.relu_mask = nullptr; e1.residual = nullptr; e1.reduce_sum_out = nullptr;
   mtf_tensor in1[2] = {*x, *w};
   if ((st = mtf_einsum(layout, nullptr, 2, in1, h_saved, &e1, workspace, workspace_bytes, stream)) != MTF_OK) return st;
   mtf_tensor in2[2] = {*h_saved, *v};
@@ -395,7 +404,10 @@ mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, con
 
   // dhp = (dy . v^T) * [h > 0]   (relu'(0) = 0)
   mtf_epilogue e1;
+  // dbias = sum over tokens of dhp rides in the same launch when it is an f32 tensor
+  const bool fuse_dbias = dbias && dbias->dtype == MTF_F32;
   e1.scale = 1.f; e1.relu = 0; e1.bias = nullptr; e1.relu_mask = h_saved; e1.residual = nullptr;
+  e1.reduce_sum_out = fuse_dbias ? dbias : nullptr;
   mtf_tensor in1[2] = {*dy, *v};
   if ((st = mtf_einsum(layout, nullptr, 2, in1, &dhp, &e1, rest, rest_bytes, stream)) != MTF_OK) return st;
   // dv = h^T . dy  and  dw = x^T . dhp  reduce out the token dims (Section 8.1)
@@ -403,7 +415,7 @@ mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, con
   if ((st = mtf_einsum(layout, nullptr, 2, in2, dv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   mtf_tensor in3[2] = {*x, dhp};
   if ((st = mtf_einsum(layout, nullptr, 2, in3, dw, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if (dbias && (st = mtf_reduce_sum(layout, &dhp, dbias, stream)) != MTF_OK) return st;
+  if (dbias && !fuse_dbias && (st = mtf_reduce_sum(layout, &dhp, dbias, stream)) != MTF_OK) return st;
   // dx = dhp . w^T reduces out hidden (Section 8.2)
   mtf_tensor in4[2] = {dhp, *w};
   return mtf_einsum(layout, nullptr, 2, in4, dx, nullptr, rest, rest_bytes, stream);

@@ -24,7 +24,7 @@ __device__ __forceinline__ float ld_as_float(const void* p, int dt, int64_t off)
 __global__ void __launch_bounds__(256) einsum_simt_kernel(const SimtParams p) {
   const int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (o >= p.total_out) return;
-  int64_t offA = 0, offB = 0, offC = 0, offBias = 0, rem = o;
+  int64_t offA = 0, offB = 0, offC = 0, offBias = 0, offRsum = 0, rem = o;
   for (int d = p.n_out - 1; d >= 0; --d) {
     const int64_t i = rem % p.out_size[d];
     rem /= p.out_size[d];
@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(256) einsum_simt_kernel(const SimtParams p) {
     offB += i * p.out_sB[d];
     offC += i * p.out_sC[d];
     offBias += i * p.out_sBias[d];
+    offRsum += i * p.out_sRsum[d];
   }
   int64_t n_group = 1, n_local = 1;
   for (int l = 0; l < p.n_group; ++l) n_group *= p.lvl_extent[l];
@@ -70,6 +71,7 @@ __global__ void __launch_bounds__(256) einsum_simt_kernel(const SimtParams p) {
   if (p.bias) t += ld_as_float(p.bias, p.dtBias, offBias);
   if (p.relu) t = fmaxf(t, 0.f);
   if (p.mask && !(ld_as_float(p.mask, p.dtMask, offC) > 0.f)) t = 0.f;
+  if (p.rsum) atomicAdd(p.rsum + offRsum, t);      // fused reduction output (Section 6 "Reduction")
   if (p.resid) t += ld_as_float(p.resid, p.dtRes, offC);
   if (p.dtC == MTF_BF16) reinterpret_cast<__nv_bfloat16*>(p.C)[offC] = __float2bfloat16_rn(t);
   else reinterpret_cast<float*>(p.C)[offC] = t;
@@ -110,8 +112,12 @@ static mtf_status check_launch(const char* what) {
   return MTF_OK;
 }
 
-mtf_status launch_simt(const SimtParams& p, void* stream) {
+mtf_status launch_simt(const SimtParams& p, int64_t rsum_elems, void* stream) {
   if (p.total_out <= 0) return MTF_OK;
+  if (p.rsum) {
+    cudaError_t e = cudaMemsetAsync(p.rsum, 0, (size_t)rsum_elems * sizeof(float), (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  }
   const int64_t blocks = (p.total_out + 255) / 256;
   if (blocks > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "output too large for the generic kernel's grid");
   einsum_simt_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(p);

@@ -64,6 +64,7 @@ struct TcArgs {
   int resid_bf16;
   float scale;
   int relu;
+  float* rsum;             // fused reduce_sum over M of the epilogue value (fp32, pre-zeroed), indexed by n
   float* ws_partials;
   unsigned* ws_counters;
 };
@@ -187,8 +188,25 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, int mn_major) 
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t lo16) { return __uint_as_float(lo16 << 16); }
 
+// Sum over the 32 lanes (rows) of each of 32 columns: lane j ends with column j's total.  Each step
+// halves the number of values a lane holds and exchanges the other half with its partner.
+__device__ __forceinline__ float warp_column_sums(float* v, int lane) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int i = 0; i < off; ++i) {
+      const float send = upper ? v[i] : v[i + off];
+      const float keep = upper ? v[i + off] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+  return v[0];
+}
+
 // Fused epilogue on 32 consecutive columns of one output row (fp32 in v), then 16-byte stores.
-__device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, long long row_off, int row, int n_first, int n_valid) {
+// With a fused reduce_sum the value before the residual stage is left in `r` for the caller.
+__device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, float* r, long long row_off, int row, int n_first, int n_valid) {
   // n_valid: number of valid columns among the 32 (multiple of the store vector)
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] *= a.scale;
@@ -231,6 +249,10 @@ __device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, long l
       for (int j = 0; j < 32; ++j)
         if (j < n_valid && !(mp[j] > 0.f)) v[j] = 0.f;
     }
+  }
+  if (a.rsum) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) r[j] = j < n_valid ? v[j] : 0.f;
   }
   if (a.resid) {
     if (a.resid_bf16) {
@@ -412,11 +434,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const int n_first = tl.n0 + c0;
           int n_valid = tl.n_end - n_first;
           n_valid = n_valid > 32 ? 32 : n_valid;
+          float r[32];
+          if (a.rsum) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = 0.f;
+          }
           if (row_ok && n_valid > 0) {
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
-            epilogue_store(a, v, row_off, row, n_first, n_valid);
+            epilogue_store(a, v, r, row_off, row, n_first, n_valid);
+          }
+          if (a.rsum && n_valid > 0) {      // warp-uniform: every lane takes part in the shuffles
+            const float col = warp_column_sums(r, lane);
+            if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
           }
         }
         tcgen05_fence_before();
@@ -450,6 +481,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const int n_first = tl.n0 + c0;
             int n_valid = tl.n_end - n_first;
             n_valid = n_valid > 32 ? 32 : n_valid;
+            float r[32];
+            if (a.rsum) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = 0.f;
+            }
             if (row_ok && n_valid > 0) {
               float v[32];
 #pragma unroll
@@ -462,7 +498,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                   v[4 * j] += f.x; v[4 * j + 1] += f.y; v[4 * j + 2] += f.z; v[4 * j + 3] += f.w;
                 }
               }
-              epilogue_store(a, v, row_off, row, n_first, n_valid);
+              epilogue_store(a, v, r, row_off, row, n_first, n_valid);
+            }
+            if (a.rsum && n_valid > 0) {
+              const float col = warp_column_sums(r, lane);
+              if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
             }
           }
         }
@@ -568,7 +608,7 @@ size_t tc_workspace_bytes(const TcParams& t) {
 }
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
-                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu,
+                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream) {
   const TcParams& t = plan.tc;
   if (t.swapped) std::swap(A, B);
@@ -605,6 +645,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.mask = mask; a.mask_bf16 = dtMask == MTF_BF16;
   a.resid = resid; a.resid_bf16 = dtRes == MTF_BF16;
   a.scale = scale; a.relu = relu;
+  a.rsum = rsum;
   a.ws_partials = nullptr; a.ws_counters = nullptr;
   if (a.total_work <= 0) return MTF_OK;
 
@@ -620,6 +661,10 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
   }
 
+  if (rsum) {
+    cudaError_t e = cudaMemsetAsync(rsum, 0, (size_t)t.N * sizeof(float), st);
+    if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  }
   CUtensorMap map_a, map_b;
   mtf_status s;
   if ((s = make_map(&map_a, A, t.a_mn_major, t.M, t.K, t.a_ld, t, t.outer_sA, BM)) != MTF_OK) return s;

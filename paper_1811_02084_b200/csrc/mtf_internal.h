@@ -53,6 +53,7 @@ struct SimtParams {
   int64_t out_size[mtf::kMaxTensorDims];
   int64_t out_sA[mtf::kMaxTensorDims], out_sB[mtf::kMaxTensorDims], out_sC[mtf::kMaxTensorDims];
   int64_t out_sBias[mtf::kMaxTensorDims];
+  int64_t out_sRsum[mtf::kMaxTensorDims];
   // reduction loop nest: first n_group levels walk the members of the reduce group in ascending
   // processor order (one level per split reduced dim, lower mesh-dim index outermost); the rest walk
   // the local extents of the reduced dims.  A partial sum is closed after each group member.
@@ -70,6 +71,7 @@ struct SimtParams {
   const void* bias = nullptr;
   const void* mask = nullptr;
   const void* resid = nullptr;
+  float* rsum = nullptr;                // fused reduce_sum output (fp32, pre-zeroed)
 };
 
 // ---- parameters of the tcgen05 grouped GEMM ---------------------------------------------------------
@@ -97,8 +99,8 @@ struct EpilogueDesc {
   bool on = false;
   float scale = 1.f;
   bool relu = false;
-  bool has_bias = false, has_mask = false, has_res = false;
-  std::vector<mtf::Dim> bias_dims;
+  bool has_bias = false, has_mask = false, has_res = false, has_rsum = false;
+  std::vector<mtf::Dim> bias_dims, rsum_dims;
   int dtBias = 0, dtMask = 0, dtRes = 0;
 };
 
@@ -147,9 +149,9 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
 std::string plan_key(int n_in, const mtf_tensor* in, const mtf_tensor* out, const mtf_epilogue* epi, int fk, int fr);
 
 // launchers (defined in the .cu files)
-mtf_status launch_simt(const SimtParams& p, void* stream);
+mtf_status launch_simt(const SimtParams& p, int64_t rsum_elems, void* stream);
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
-                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu,
+                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream);
 size_t tc_workspace_bytes(const TcParams& t);
 mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes,

@@ -127,6 +127,7 @@ std::string plan_key(int n_in, const mtf_tensor* in, const mtf_tensor* out, cons
     if (epi->bias) { k += 'b'; add_t(epi->bias); }
     if (epi->relu_mask) { k += 'm'; k += dt_name(epi->relu_mask->dtype); }
     if (epi->residual) { k += 'a'; k += dt_name(epi->residual->dtype); }
+    if (epi->reduce_sum_out) { k += 'S'; add_t(epi->reduce_sum_out); }
   }
   k += "|f" + std::to_string(fk) + "," + std::to_string(fr);
   return k;
@@ -260,6 +261,14 @@ static bool plan_tc(mtf_plan_t* P, std::string* why) {
     else if (covers(other)) t.bias_along_m = 1;
     else { *why = "bias dims are not exactly the N (or M) group in storage order"; return false; }
   }
+  if (P->epi.has_rsum) {
+    const auto& rd = P->epi.rsum_dims;
+    std::vector<int> g = swap ? cm : cn;              // the kernel's N group
+    std::sort(g.begin(), g.end(), [&](int a, int b) { return it[a].sC > it[b].sC; });
+    bool same = rd.size() == g.size();
+    for (size_t j = 0; same && j < g.size(); ++j) same = rd[j].name == it[g[j]].name;
+    if (!same) { *why = "reduce_sum_out dims are not exactly the contiguous output group"; return false; }
+  }
   int64_t Ns = t.N / t.sn;
   t.block_n = Ns > 128 ? 256 : (Ns > 64 ? 128 : 64);
   P->tc = t;
@@ -340,6 +349,16 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
         if (e->size != b.size) return fail(MTF_ERR_SIZE_MISMATCH, "bias dimension '%s' has size %lld, output has %lld", b.name.c_str(), (long long)b.size, (long long)e->size);
       }
     }
+    if (epi->reduce_sum_out) {
+      P->epi.has_rsum = true;
+      if (epi->reduce_sum_out->dtype != MTF_F32) return fail(MTF_ERR_UNSUPPORTED, "reduce_sum_out must be f32");
+      if ((st = read_dims(epi->reduce_sum_out->ndim, epi->reduce_sum_out->dims, &P->epi.rsum_dims, "reduce_sum_out")) != MTF_OK) return st;
+      for (auto& b : P->epi.rsum_dims) {
+        IterDim* e = find(b.name);
+        if (!e || !e->inC) return fail(MTF_ERR_UNKNOWN_DIM, "reduce_sum_out dimension '%s' is not an output dimension", b.name.c_str());
+        if (e->size != b.size) return fail(MTF_ERR_SIZE_MISMATCH, "reduce_sum_out dimension '%s' has size %lld, output has %lld", b.name.c_str(), (long long)b.size, (long long)e->size);
+      }
+    }
     for (int which = 0; which < 2; ++which) {
       const mtf_tensor* t = which == 0 ? epi->relu_mask : epi->residual;
       if (!t) continue;
@@ -395,6 +414,13 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
     s.out_size[i] = e->size;
     s.out_sA[i] = e->sA; s.out_sB[i] = e->sB; s.out_sC[i] = e->sC;
     s.out_sBias[i] = 0;
+    s.out_sRsum[i] = 0;
+  }
+  if (P->epi.has_rsum) {
+    auto rs = row_major_strides(P->epi.rsum_dims);
+    for (size_t b = 0; b < P->epi.rsum_dims.size(); ++b)
+      for (int i = 0; i < s.n_out; ++i)
+        if (P->dimsC[i].name == P->epi.rsum_dims[b].name) s.out_sRsum[i] = rs[b];
   }
   if (P->epi.has_bias) {
     auto bs = row_major_strides(P->epi.bias_dims);
@@ -432,6 +458,8 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
   // ---- kernel family and reduce mode ----
   std::string why;
   bool tc_ok = plan_tc(P.get(), &why);
+  if (!P->has_B && force_kernel == MTF_KERNEL_TCGEN05) force_kernel = -1;   // forcing concerns contractions only
+  if (!P->has_B && force_reduce == MTF_REDUCE_WORKSPACE) force_reduce = -1;
   if (force_kernel == MTF_KERNEL_TCGEN05 && !tc_ok) return fail(MTF_ERR_UNSUPPORTED, "tensor-core path cannot run this einsum: %s", why.c_str());
   P->kernel_kind = (tc_ok && force_kernel != MTF_KERNEL_SIMT) ? MTF_KERNEL_TCGEN05 : MTF_KERNEL_SIMT;
   P->reduce_mode = P->group_size > 1 ? MTF_REDUCE_CHAINED : MTF_REDUCE_NONE;

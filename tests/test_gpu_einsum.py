@@ -167,6 +167,31 @@ def test_fused_epilogue_stages(mtf, ep, kind):
     assert parity_error(got, ref) <= TOL["bf16"]
 
 
+def test_fused_reduce_sum_output(mtf):
+    """dbias-style second output: sum over the rows of the masked value, fused into the einsum."""
+    import torch
+    from oracle import NT, DenseOps
+    ops = DenseOps()
+    a_d, b_d, o_d = [("t", 300), ("d", 200)], [("f", 328), ("d", 200)], [("t", 300), ("f", 328)]
+    a, b, m = si.normal(6, "a", [300, 200], "bf16"), si.normal(6, "b", [328, 200], "bf16", 200 ** -0.5), si.normal(6, "m", [300, 328], "bf16")
+    val = ops.mul(ops.einsum([NT(a_d, a.f64), NT(b_d, b.f64)], ["t", "f"]), ops.positive(NT(o_d, m.f64)))
+    want = ops.reduce_sum(val, ["f"]).a
+    at, bt, mt = to_torch(a), to_torch(b), to_torch(m)
+    for kind, mesh_dims, rules in ((0, [("all", 1)], []), (1, [("all", 1)], []), (1, [("all", 4)], [("t", "all")]), (1, [("all", 4)], [("d", "all")])):
+        out = torch.empty(300, 328, dtype=torch.bfloat16, device="cuda")
+        rs = torch.full((328,), 7.0, dtype=torch.float32, device="cuda")          # the library zeroes it
+        ep = mtf.Epilogue(relu_mask=mtf.named(mt, ["t", "f"]), reduce_sum_out=mtf.named(rs, ["f"]))
+        mtf.mtf_plan_force(kind, -1)
+        try:
+            mtf.mtf_einsum(layout(mtf, mesh_dims, rules), "t d, f d -> t f", [mtf.named(at, ["t", "d"]), mtf.named(bt, ["f", "d"])],
+                           mtf.named(out, ["t", "f"]), ep)
+        finally:
+            mtf.mtf_plan_force(-1, -1)
+        mtf.mtf_device_status()
+        assert parity_error(from_torch(rs), want) <= 1e-3, (kind, rules)
+        assert parity_error(from_torch(out), val.a) <= TOL["bf16"]
+
+
 # attention-shaped contractions (reading of Section 9: batch b, length l, memory m, heads h, d_k k)
 B_, L_, H_, K_, D_ = 4, 160, 4, 64, 256
 ATT = {

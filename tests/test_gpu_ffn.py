@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from helpers import TOL, check_ffn, ffn_inputs, run_ffn_gpu, run_ffn_oracle
+from helpers import TOL, check_ffn, check_ffn_block, ffn_inputs, run_ffn_gpu, run_ffn_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -70,12 +70,10 @@ def test_bf16_ffn_layouts(mtf, mesh_dims, rules, force):
         got = run_ffn_gpu(mtf, make_layout(mtf, mesh_dims, rules), inp, "bf16")
     finally:
         mtf.mtf_plan_force(-1, -1)
-    ref, amb = run_ffn_oracle(inp)
-    check_ffn(got, ref, amb, TOL["bf16"])
+    check_ffn_block(got, inp, "bf16")
 
 
 def test_bf16_outputs_bf16_grads(mtf):
     inp = ffn_inputs(4, [("batch", 4), ("length", 64)], 256, 512, "bf16", True)
     got = run_ffn_gpu(mtf, make_layout(mtf, [("all", 4)], [("batch", "all")]), inp, "bf16", grad_dtype="bf16")
-    ref, amb = run_ffn_oracle(inp)
-    check_ffn(got, ref, amb, TOL["bf16"])
+    check_ffn_block(got, inp, "bf16")
