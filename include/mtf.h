@@ -159,7 +159,9 @@ mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t 
 mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in,
                                       const mtf_tensor* out, const mtf_epilogue* epilogue, size_t* bytes);
 /* Testing hook: force the kernel family / reduce mode of plans created afterwards by this thread
- * (-1 = planner's choice).  A forced choice the shape cannot run gives MTF_ERR_UNSUPPORTED. */
+ * (-1 = planner's choice; kernel_kind 2 = tensor cores with one CTA per tile, i.e. without the
+ * two-CTA pairs the planner prefers on tall slices).  A forced choice the shape cannot run gives
+ * MTF_ERR_UNSUPPORTED. */
 mtf_status mtf_plan_force(int32_t kernel_kind, int32_t reduce_mode);
 
 /* ---- feed-forward block (Section 8: y = Relu(x w + bias) v) ------------------------------------- */

@@ -27,12 +27,11 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kStages = 4;
 constexpr int kMaxBN = 256;
 constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
-constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB
-constexpr int kStageBytes = kAStageBytes + kBStageBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stages half of it)
+constexpr int kRingBytes = 4 * (kAStageBytes + kBStageBytes);   // = 6 * (16 KB + 16 KB) = 192 KB
+constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
@@ -75,7 +74,7 @@ struct Tile {
   long long c_off;         // element offset of the outer coordinates in C
 };
 
-__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t) {
+__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int tile_rows) {
   Tile r;
   long long slice = t / a.tiles_per_slice;
   long long w = t % a.tiles_per_slice;
@@ -92,7 +91,7 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t) {
     r.o[j] = ob * a.outer_local[j] + ol[j];
     r.c_off += (long long)r.o[j] * a.outer_sC[j];
   }
-  r.m0 = im * a.Ms + mt * BM;
+  r.m0 = im * a.Ms + mt * tile_rows;
   r.m_end = (im + 1) * a.Ms;
   r.n0 = in * a.Ns + nt * a.block_n;
   r.n_end = (in + 1) * a.Ns;
@@ -140,27 +139,71 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int cod
   return mbar_wait_slow(bar, parity, code, abort_flag);
 }
 
+// kPair: the completion may count on the partner CTA's barrier (cta_group::2 form); never multicast.
+template <bool kPair>
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
                                             int c3, int c4) {
-  asm volatile(
-      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-      : "memory");
+  if (kPair)
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+  else
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Arrive on the barrier at the same offset in the even CTA of the pair (own barrier when !kPair).
+template <bool kPair>
+__device__ __forceinline__ void mbar_arrive_pair(uint32_t bar) {
+  if (kPair)
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+        ::"r"(bar) : "memory");
+  else
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+template <bool kPair>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_c), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (kPair)
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_c), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+  else
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_c), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
+// Arrives on `bar` when every MMA issued so far has retired; for a pair, on the barrier at that
+// offset in both CTAs (completion multicast, not a load).
+template <bool kPair>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (kPair) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(both) : "memory");
+  } else {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
   asm volatile(
@@ -216,12 +259,28 @@ __device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, float*
                                   : reinterpret_cast<const float*>(a.bias)[row];
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += b;
-    } else {
+    } else if (a.bias_bf16) {
+      // bias[n_first .. n_first+31]: same addresses for every lane (broadcast), 16-byte loads
+      const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.bias) + n_first);
 #pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (j < n_valid)
-          v[j] += a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[n_first + j])
-                              : reinterpret_cast<const float*>(a.bias)[n_first + j];
+      for (int q = 0; q < 4; ++q)
+        if (q * 8 < n_valid) {
+          const uint4 m = __ldg(bp + q);
+          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            v[q * 8 + 2 * e] += bf16_bits_to_float(w[e] & 0xFFFFu);
+            v[q * 8 + 2 * e + 1] += bf16_bits_to_float(w[e] >> 16);
+          }
+        }
+    } else {
+      const float4* bp = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.bias) + n_first);
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (q * 4 < n_valid) {
+          const float4 b = __ldg(bp + q);
+          v[q * 4] += b.x; v[q * 4 + 1] += b.y; v[q * 4 + 2] += b.z; v[q * 4 + 3] += b.w;
+        }
     }
   }
   if (a.relu) {
@@ -296,8 +355,21 @@ __device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, float*
   }
 }
 
+// kPair = false: one CTA owns a 128 x block_n tile (tcgen05 cta_group::1), 4-stage ring of 48 KB.
+// kPair = true : a cluster of two CTAs owns a 256 x block_n tile (tcgen05 cta_group::2).  Each CTA
+//   stages its own 128 rows of A and its own half of the N columns of B (32 KB per stage, 6 stages),
+//   the even CTA of the pair issues every MMA for both, each CTA's TMEM receives its own 128 rows of
+//   the result, and each CTA runs the epilogue on its own rows.  Compared with kPair = false a CTA
+//   pulls 2/3 of the bytes through L2 per flop and holds 1.5x as many k-blocks in flight.
+//   The loads of both CTAs report to the even CTA's "full" barrier; MMA completion is multicast to
+//   both CTAs' "empty" and "accumulator full" barriers; the epilogue warps of both CTAs report to
+//   the even CTA's "accumulator empty" barrier.  No load uses cluster multicast.
+template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+  constexpr int kStages = kPair ? 6 : 4;
+  constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
+  constexpr int kTileRows = kPair ? 2 * BM : BM;       // rows of C owned by a work item
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned tile ring (the 128B swizzle pattern repeats every 1024 B)
   const uint32_t raw = smem_u32(smem_raw);
@@ -315,21 +387,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const int cta_rank = kPair ? (int)(blockIdx.x & 1u) : 0;     // position in the CTA pair
+  const bool leader = cta_rank == 0;
+  const long long work_first = kPair ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
+  const long long work_step = kPair ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kPair ? 8 : 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
   }
-  if (warp == 1) {   // TMEM allocation is a warp-wide operation
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 1) {   // TMEM allocation is a warp-wide operation (the same warp of both CTAs of a pair)
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tcgen05_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync();      // the partner's barriers must exist before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -337,7 +419,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int kb_per_slice = a.Ks / BK;
   const int kb_total = a.k_sliced ? a.sk * kb_per_slice : (a.K + BK - 1) / BK;
   const int kb_count = ws_mode ? kb_per_slice : kb_total;
-  const uint32_t b_bytes = (uint32_t)a.block_n * BK * 2;
+  const int n_local = kPair ? a.block_n / 2 : a.block_n;       // N columns of B this CTA stages
+  const uint32_t b_bytes = (uint32_t)n_local * BK * 2;
 
   if (warp == 0) {
     // ------------------------------- TMA producer -------------------------------
@@ -345,46 +428,51 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x) {
+      for (long long work = work_first; ok && work < a.total_work; work += work_step) {
         const long long t = ws_mode ? work / a.sk : work;
         const int kb_first = ws_mode ? (int)(work % a.sk) * kb_per_slice : 0;
-        const Tile tl = decode_tile(a, t);
+        const Tile tl = decode_tile(a, t, kTileRows);
+        const int m0 = tl.m0 + cta_rank * BM;
+        const int n0 = tl.n0 + cta_rank * n_local;
         for (int kb = 0; kb < kb_count; ++kb) {
           // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
           // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor)
           const int k0 = (kb_first + kb) * BK;
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, 0x100 + stage, abort_flag))) break;
-          mbar_expect_tx(full_bar(stage), kAStageBytes + b_bytes);
+          // a pair's loads all count on the even CTA's barrier, which expects both CTAs' bytes
+          if (!kPair) mbar_expect_tx(full_bar(stage), kAStageBytes + b_bytes);
+          else if (leader) mbar_expect_tx(full_bar(stage), 2u * (kAStageBytes + b_bytes));
+          const uint32_t fb = kPair ? (full_bar(stage) & 0xFEFFFFFFu) : full_bar(stage);
           const uint32_t sa = tiles_base + stage * kStageBytes;
           const uint32_t sb = sa + kAStageBytes;
           if (a.a_mn_major) {
-            tma_load_5d(sa, &map_a, full_bar(stage), tl.m0, k0, tl.o[2], tl.o[1], tl.o[0]);
-            tma_load_5d(sa + 8192, &map_a, full_bar(stage), tl.m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa, &map_a, fb, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa + 8192, &map_a, fb, m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
-            tma_load_5d(sa, &map_a, full_bar(stage), k0, tl.m0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa, &map_a, fb, k0, m0, tl.o[2], tl.o[1], tl.o[0]);
           }
           if (a.b_mn_major) {
-            for (int j = 0; j < a.block_n / 64; ++j)
-              tma_load_5d(sb + 8192 * j, &map_b, full_bar(stage), tl.n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
+            for (int j = 0; j < n_local / 64; ++j)
+              tma_load_5d<kPair>(sb + 8192 * j, &map_b, fb, n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
-            tma_load_5d(sb, &map_b, full_bar(stage), k0, tl.n0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sb, &map_b, fb, k0, n0, tl.o[2], tl.o[1], tl.o[0]);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------- MMA issuer ---------------------------------
-    if (lane == 0) {
+    // ------------------------------- MMA issuer (even CTA of a pair only) -------
+    if (lane == 0 && leader) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.a_mn_major << 15) |
-                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
       const uint32_t a_kstep = a.a_mn_major ? 2048u : 32u;   // bytes per 16 k-elements
       const uint32_t b_kstep = a.b_mn_major ? 2048u : 32u;
       int stage = 0;
       uint32_t phase = 0;
       int iter = 0;
       bool ok = true;
-      for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x, ++iter) {
+      for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
         const int acc = iter & 1;
         const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
         if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, 0x200 + acc, abort_flag))) break;
@@ -399,12 +487,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t da = make_smem_desc(sa + k * a_kstep, a.a_mn_major);
             const uint64_t db = make_smem_desc(sb + k * b_kstep, a.b_mn_major);
-            umma_bf16(tmem_c, da, db, idesc, (kb | k) != 0);
+            umma_bf16<kPair>(tmem_c, da, db, idesc, (kb | k) != 0);
           }
-          umma_commit(empty_bar(stage));          // frees the smem stage when these MMAs retire
+          umma_commit<kPair>(empty_bar(stage));    // frees the smem stage (of both CTAs) when these MMAs retire
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(tfull_bar(acc));      // accumulator complete
+        if (ok) umma_commit<kPair>(tfull_bar(acc)); // accumulator complete (in both CTAs)
       }
     }
   } else {
@@ -412,17 +500,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     int iter = 0;
     bool ok = true;
-    for (long long work = blockIdx.x; ok && work < a.total_work; work += gridDim.x, ++iter) {
+    for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
       const long long t = ws_mode ? work / a.sk : work;
       const int ks = ws_mode ? (int)(work % a.sk) : 0;
-      const Tile tl = decode_tile(a, t);
+      const Tile tl = decode_tile(a, t, kTileRows);
       const int acc = iter & 1;
       const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
       ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
-      const int row = tl.m0 + q * 32 + lane;
+      const int tile_row = cta_rank * BM + q * 32 + lane;       // row inside the work item's tile
+      const int row = tl.m0 + tile_row;
       const bool row_ok = row < tl.m_end;
       const long long row_off = tl.c_off + (long long)row * a.ldc;
       const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
@@ -452,10 +541,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc));
       } else {
         // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
-        float* part = a.ws_partials + ((size_t)(t * a.sk + ks) * BM + (size_t)(q * 32 + lane)) * a.block_n;
+        float* part = a.ws_partials + ((size_t)(t * a.sk + ks) * kTileRows + (size_t)tile_row) * a.block_n;
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
@@ -468,15 +557,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc));
         __threadfence();
         __syncwarp();
         unsigned old = 0;
-        if (lane == 0) old = atomicAdd(&a.ws_counters[t * 4 + q], 1u);
+        if (lane == 0) old = atomicAdd(&a.ws_counters[t * (kTileRows / 32) + cta_rank * 4 + q], 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old == (unsigned)a.sk - 1) {
           __threadfence();
-          const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * BM + (size_t)(q * 32 + lane)) * a.block_n;
+          const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * kTileRows + (size_t)tile_row) * a.block_n;
           for (int c0 = 0; c0 < a.block_n; c0 += 32) {
             const int n_first = tl.n0 + c0;
             int n_valid = tl.n_end - n_first;
@@ -491,7 +580,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
               for (int j = 0; j < 32; ++j) v[j] = 0.f;
               for (int s = 0; s < a.sk; ++s) {     // ascending processor order within the group
-                const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * BM * a.block_n + c0);
+                const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * kTileRows * a.block_n + c0);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                   const float4 f = __ldcg(sp + j);
@@ -517,10 +606,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   }
   tcgen05_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync();      // the partner may still signal this CTA's barriers or read its tiles
   if (warp == 1) {
     __syncwarp();
     tcgen05_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -595,8 +686,11 @@ int sm_count() {
 
 namespace mtf {
 
+static int tc_tile_rows(const TcParams& t) { return t.cta_pair ? 2 * BM : BM; }
+
 static int64_t tc_total_tiles(const TcParams& t) {
-  int64_t tiles = ((t.M / t.sm + BM - 1) / BM) * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sm * t.sn;
+  const int rows = tc_tile_rows(t);
+  int64_t tiles = ((t.M / t.sm + rows - 1) / rows) * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sm * t.sn;
   for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
   return tiles;
 }
@@ -604,7 +698,7 @@ static int64_t tc_total_tiles(const TcParams& t) {
 size_t tc_workspace_bytes(const TcParams& t) {
   if (t.reduce_mode != MTF_REDUCE_WORKSPACE) return 0;
   const int64_t tiles = tc_total_tiles(t);
-  return (size_t)tiles * t.sk * BM * t.block_n * sizeof(float) + (size_t)tiles * 4 * sizeof(unsigned) + 256;
+  return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * sizeof(unsigned) + 256;
 }
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
@@ -614,6 +708,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (t.swapped) std::swap(A, B);
   if (t.M > 0x7fffffffLL || t.N > 0x7fffffffLL || t.K > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "extent beyond 2^31");
   if (reinterpret_cast<uintptr_t>(C) & 15) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned output");
+  if (bias && !t.bias_along_m && (reinterpret_cast<uintptr_t>(bias) & 15)) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned bias");
   if ((mask && (reinterpret_cast<uintptr_t>(mask) & 15)) || (resid && (reinterpret_cast<uintptr_t>(resid) & 15)))
     return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs 16-byte aligned epilogue operands");
 
@@ -632,7 +727,8 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.ldc = t.ldc;
   a.reduce_mode = t.reduce_mode;
   a.k_sliced = (t.sk > 1 && a.Ks % BK == 0) ? 1 : 0;
-  a.m_tiles = (a.Ms + BM - 1) / BM;
+  const int tile_rows = tc_tile_rows(t);
+  a.m_tiles = (a.Ms + tile_rows - 1) / tile_rows;
   a.n_tiles = (a.Ns + a.block_n - 1) / a.block_n;
   a.tiles_per_slice = (long long)a.m_tiles * a.n_tiles;
   for (int j = 0; j < a.n_outer; ++j) a.tiles_per_slice *= a.outer_local[j];
@@ -654,10 +750,10 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     const size_t need = tc_workspace_bytes(t);
     if (!workspace || workspace_bytes < need) return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "einsum needs %zu workspace bytes, got %zu", need, workspace_bytes);
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return fail(MTF_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
-    const size_t part_bytes = (size_t)a.total_tiles * a.sk * BM * a.block_n * sizeof(float);
+    const size_t part_bytes = (size_t)a.total_tiles * a.sk * tile_rows * a.block_n * sizeof(float);
     a.ws_partials = reinterpret_cast<float*>(workspace);
     a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
-    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * 4 * sizeof(unsigned), st);
+    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * (tile_rows / 32) * sizeof(unsigned), st);
     if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
   }
 
@@ -668,14 +764,41 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   CUtensorMap map_a, map_b;
   mtf_status s;
   if ((s = make_map(&map_a, A, t.a_mn_major, t.M, t.K, t.a_ld, t, t.outer_sA, BM)) != MTF_OK) return s;
-  if ((s = make_map(&map_b, B, t.b_mn_major, t.N, t.K, t.b_ld, t, t.outer_sB, t.block_n)) != MTF_OK) return s;
+  if ((s = make_map(&map_b, B, t.b_mn_major, t.N, t.K, t.b_ld, t, t.outer_sB, t.cta_pair ? t.block_n / 2 : t.block_n)) != MTF_OK) return s;
 
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] { attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes); });
+  static int max_pairs = 0;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (attr_err != cudaSuccess) return;
+    // how many CTA pairs can be resident at once (one CTA per SM; a pair shares a TPC)
+    cudaLaunchConfig_t q = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    q.gridDim = dim3(2 * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
+    q.attrs = at; q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<true>, &q) == cudaSuccess && n > 0) max_pairs = n;
+    else { max_pairs = sm_count() / 2; (void)cudaGetLastError(); }
+  });
   if (attr_err != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
-  const long long grid = std::min<long long>(a.total_work, sm_count());
-  gemm_tcgen05_kernel<<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, a);
+  if (t.cta_pair) {
+    const long long pairs = std::min<long long>(a.total_work, max_pairs);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<true>, map_a, map_b, a);
+    if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<pair>: %s", cudaGetErrorString(le));
+  } else {
+    const long long grid = std::min<long long>(a.total_work, sm_count());
+    gemm_tcgen05_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, a);
+  }
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(e));

@@ -179,7 +179,7 @@ static Merged merge_category(const std::vector<IterDim>& it, std::vector<int> id
   return m;
 }
 
-static bool plan_tc(mtf_plan_t* P, std::string* why) {
+static bool plan_tc(mtf_plan_t* P, std::string* why, int force_single_cta) {
   const auto& it = P->iter;
   if (!P->has_B) { *why = "one operand"; return false; }
   if (P->dtA != MTF_BF16 || P->dtB != MTF_BF16) { *why = "operands are not bf16"; return false; }
@@ -271,6 +271,8 @@ static bool plan_tc(mtf_plan_t* P, std::string* why) {
   }
   int64_t Ns = t.N / t.sn;
   t.block_n = Ns > 128 ? 256 : (Ns > 64 ? 128 : 64);
+  // CTA pairs need a B half of at least one 64-wide swizzle block and pay off on tall slices
+  t.cta_pair = (t.block_n >= 128 && t.M / t.sm > 128 && force_single_cta == 0) ? 1 : 0;
   P->tc = t;
   return true;
 }
@@ -457,7 +459,9 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
 
   // ---- kernel family and reduce mode ----
   std::string why;
-  bool tc_ok = plan_tc(P.get(), &why);
+  const int force_single_cta = force_kernel == 2 ? 1 : 0;     // testing hook: tensor cores without CTA pairs
+  if (force_kernel == 2) force_kernel = MTF_KERNEL_TCGEN05;
+  bool tc_ok = plan_tc(P.get(), &why, force_single_cta);
   if (!P->has_B && force_kernel == MTF_KERNEL_TCGEN05) force_kernel = -1;   // forcing concerns contractions only
   if (!P->has_B && force_reduce == MTF_REDUCE_WORKSPACE) force_reduce = -1;
   if (force_kernel == MTF_KERNEL_TCGEN05 && !tc_ok) return fail(MTF_ERR_UNSUPPORTED, "tensor-core path cannot run this einsum: %s", why.c_str());
@@ -473,9 +477,10 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
       mode = MTF_REDUCE_WORKSPACE;
     } else if (force_reduce < 0 && ws_possible) {
       // few output tiles and a long, split K: spread the group's slices over CTAs instead
-      int64_t tiles = ((t.M / t.sm + 127) / 128) * t.sm * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sn;
+      const int64_t rows = t.cta_pair ? 256 : 128;
+      int64_t tiles = ((t.M / t.sm + rows - 1) / rows) * t.sm * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sn;
       for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
-      if (tiles * 2 <= 148 && t.K / t.sk >= 256) mode = MTF_REDUCE_WORKSPACE;
+      if (tiles * (t.cta_pair ? 4 : 2) <= 148 && t.K / t.sk >= 256) mode = MTF_REDUCE_WORKSPACE;
     }
     t.reduce_mode = mode;
     P->reduce_mode = mode;

@@ -89,11 +89,12 @@ MAJORS = {
 
 @pytest.mark.parametrize("name", list(MAJORS))
 @pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
-def test_tensor_core_operand_majors(mtf, name, out_dtype):
+@pytest.mark.parametrize("kind", [1, 2], ids=["cta-pairs", "single-cta"])
+def test_tensor_core_operand_majors(mtf, name, out_dtype, kind):
     a, b = MAJORS[name]
     out_dims = [a[0] if a[0][0] == "i" else a[1], b[1] if b[1][0] == "j" else b[0]]
     lay = layout(mtf, [("all", 1)], [])
-    got, ref, info = run_einsum(mtf, lay, [a, b], out_dims, "bf16", out_dtype, force=(1, -1))
+    got, ref, info = run_einsum(mtf, lay, [a, b], out_dims, "bf16", out_dtype, force=(kind, -1))
     assert info["kernel_kind"] == mtf.MTF_KERNEL_TCGEN05
     assert parity_error(got, ref) <= TOL["bf16"]
 
@@ -116,16 +117,17 @@ SPLITS = [
 
 @pytest.mark.parametrize("mesh_dims,rules", SPLITS)
 @pytest.mark.parametrize("mode", [1, 2], ids=["chained", "workspace"])
-def test_tensor_core_split_dims_and_group_sum(mtf, mesh_dims, rules, mode):
+@pytest.mark.parametrize("kind", [1, 2], ids=["cta-pairs", "single-cta"])
+def test_tensor_core_split_dims_and_group_sum(mtf, mesh_dims, rules, mode, kind):
     a, b = [("i", 512), ("k", 512)], [("k", 512), ("j", 384)]
     lay = layout(mtf, mesh_dims, rules)
     k_split = any(t == "k" for t, _ in rules)
     if mode == 2 and not k_split:
         with pytest.raises(mtf.MtfError) as e:
-            run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", force=(1, 2))
+            run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", force=(kind, 2))
         assert e.value.code == "MTF_ERR_UNSUPPORTED"
         return
-    got, ref, info = run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", "f32", force=(1, mode if k_split else -1))
+    got, ref, info = run_einsum(mtf, lay, [a, b], [("i", 512), ("j", 384)], "bf16", "f32", force=(kind, mode if k_split else -1))
     assert info["reduce_mode"] == (mode if k_split else 0)
     assert info["group_size"] == (2 if k_split and len(mesh_dims) > 1 else (4 if k_split else 1))
     assert parity_error(got, ref) <= TOL["bf16"]

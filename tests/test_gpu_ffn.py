@@ -61,7 +61,7 @@ BF16_LAYOUTS = [
 
 
 @pytest.mark.parametrize("mesh_dims,rules", BF16_LAYOUTS)
-@pytest.mark.parametrize("force", [(-1, -1), (1, 1), (0, -1)], ids=["auto", "tc-chained", "simt"])
+@pytest.mark.parametrize("force", [(-1, -1), (1, 1), (2, 1), (0, -1)], ids=["auto", "tc-chained", "tc-single-cta", "simt"])
 def test_bf16_ffn_layouts(mtf, mesh_dims, rules, force):
     # tokens 8 x 72 = 576 (4.5 row tiles), d_model 320 (5 k-blocks, 1.25 column tiles), d_ff 1088 (17 k-blocks)
     inp = ffn_inputs(2, [("batch", 8), ("length", 72)], 320, 1088, "bf16", True)
