@@ -31,7 +31,8 @@ constexpr int kMaxBN = 256;
 constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
 constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stages half of it)
 constexpr int kRingBytes = 4 * (kAStageBytes + kBStageBytes);   // = 6 * (16 KB + 16 KB) = 192 KB
-constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kStagingBytes = 4 * 2 * 4096;      // per epilogue warp: two 32-row x 128-byte boxes for TMA stores
+constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
@@ -59,6 +60,7 @@ struct TcArgs {
   int bias_bf16, bias_along_m;
   const void* mask;
   int mask_bf16;
+  int mask_tma;            // bf16 mask boxes are loaded by TMA into the output staging buffers (bf16 output only)
   const void* resid;
   int resid_bf16;
   float scale;
@@ -106,9 +108,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -247,112 +246,144 @@ __device__ __forceinline__ float warp_column_sums(float* v, int lane) {
   return v[0];
 }
 
-// Fused epilogue on 32 consecutive columns of one output row (fp32 in v), then 16-byte stores.
-// With a fused reduce_sum the value before the residual stage is left in `r` for the caller.
-__device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, float* r, long long row_off, int row, int n_first, int n_valid) {
-  // n_valid: number of valid columns among the 32 (multiple of the store vector)
+__device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
+  const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    f[2 * e] = bf16_bits_to_float(w[e] & 0xFFFFu);
+    f[2 * e + 1] = bf16_bits_to_float(w[e] >> 16);
+  }
+}
+
+// Fetch the relu mask of one 32-column chunk of this thread's row (bf16 mask: four 16-byte loads).
+__device__ __forceinline__ void mask_fetch(const TcArgs& a, long long off, bool on, int n_valid, uint4* mk) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    mk[q] = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);   // 1.0: keeps the value
+    if (on && q * 8 < n_valid) mk[q] = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.mask) + off + q * 8);
+  }
+}
+
+// The component-wise stages on one 32-column chunk of one row, in registers (Section 6, Section 7):
+// scale, bias (broadcast), relu, relu mask; the value then feeds the fused reduce_sum; residual last.
+//   bias_lane : bias of column (n_first + lane), handed to every lane by shuffle (bias along n)
+//   bias_row  : bias of this thread's row (bias along m)
+__device__ __forceinline__ void epilogue_math(const TcArgs& a, float* v, float bias_lane, float bias_row, const uint4* mk,
+                                              long long off, bool live, int n_valid) {
 #pragma unroll
   for (int j = 0; j < 32; ++j) v[j] *= a.scale;
   if (a.bias) {
     if (a.bias_along_m) {
-      const float b = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row])
-                                  : reinterpret_cast<const float*>(a.bias)[row];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] += b;
-    } else if (a.bias_bf16) {
-      // bias[n_first .. n_first+31]: same addresses for every lane (broadcast), 16-byte loads
-      const uint4* bp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.bias) + n_first);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (q * 8 < n_valid) {
-          const uint4 m = __ldg(bp + q);
-          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            v[q * 8 + 2 * e] += bf16_bits_to_float(w[e] & 0xFFFFu);
-            v[q * 8 + 2 * e + 1] += bf16_bits_to_float(w[e] >> 16);
-          }
-        }
+      for (int j = 0; j < 32; ++j) v[j] += bias_row;
     } else {
-      const float4* bp = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.bias) + n_first);
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        if (q * 4 < n_valid) {
-          const float4 b = __ldg(bp + q);
-          v[q * 4] += b.x; v[q * 4 + 1] += b.y; v[q * 4 + 2] += b.z; v[q * 4 + 3] += b.w;
-        }
+      for (int j = 0; j < 32; ++j) v[j] += __shfl_sync(0xffffffffu, bias_lane, j);
     }
   }
   if (a.relu) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
   }
-  const long long off = row_off + n_first;
   if (a.mask) {
     if (a.mask_bf16) {
-      const uint4* mp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.mask) + off);
 #pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (q * 8 < n_valid) {
-          const uint4 m = mp[q];
-          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+      for (int q = 0; q < 4; ++q) {
+        float f[8];
+        unpack_bf16x8(mk[q], f);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            if (!(bf16_bits_to_float(w[e] & 0xFFFFu) > 0.f)) v[q * 8 + 2 * e] = 0.f;
-            if (!(bf16_bits_to_float(w[e] >> 16) > 0.f)) v[q * 8 + 2 * e + 1] = 0.f;
-          }
-        }
-    } else {
+        for (int e = 0; e < 8; ++e)
+          if (!(f[e] > 0.f)) v[q * 8 + e] = 0.f;
+      }
+    } else if (live) {
       const float* mp = reinterpret_cast<const float*>(a.mask) + off;
 #pragma unroll
       for (int j = 0; j < 32; ++j)
         if (j < n_valid && !(mp[j] > 0.f)) v[j] = 0.f;
     }
   }
-  if (a.rsum) {
+}
+
+__device__ __forceinline__ void epilogue_residual(const TcArgs& a, float* v, long long off, bool live, int n_valid) {
+  if (!a.resid || !live) return;
+  if (a.resid_bf16) {
+    const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
 #pragma unroll
-    for (int j = 0; j < 32; ++j) r[j] = j < n_valid ? v[j] : 0.f;
+    for (int q = 0; q < 4; ++q)
+      if (q * 8 < n_valid) {
+        float f[8];
+        unpack_bf16x8(rp[q], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[q * 8 + e] += f[e];
+      }
+  } else {
+    const float* rp = reinterpret_cast<const float*>(a.resid) + off;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < n_valid) v[j] += rp[j];
   }
-  if (a.resid) {
-    if (a.resid_bf16) {
-      const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (q * 8 < n_valid) {
-          const uint4 m = rp[q];
-          const uint32_t w[4] = {m.x, m.y, m.z, m.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            v[q * 8 + 2 * e] += bf16_bits_to_float(w[e] & 0xFFFFu);
-            v[q * 8 + 2 * e + 1] += bf16_bits_to_float(w[e] >> 16);
-          }
-        }
-    } else {
-      const float* rp = reinterpret_cast<const float*>(a.resid) + off;
-#pragma unroll
-      for (int j = 0; j < 32; ++j)
-        if (j < n_valid) v[j] += rp[j];
-    }
-  }
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h2);
+}
+
+// 16-byte stores of one chunk straight from registers (ragged tiles and the workspace mode).
+__device__ __forceinline__ void store_direct(const TcArgs& a, const float* v, long long off, int n_valid) {
   if (a.c_bf16) {
     uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-      if (q * 8 < n_valid) {
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          __nv_bfloat162 h2 = __floats2bfloat162_rn(v[q * 8 + 2 * e], v[q * 8 + 2 * e + 1]);
-          w[e] = *reinterpret_cast<uint32_t*>(&h2);
-        }
-        cp[q] = make_uint4(w[0], w[1], w[2], w[3]);
-      }
+      if (q * 8 < n_valid)
+        cp[q] = make_uint4(pack_bf16x2(v[q * 8], v[q * 8 + 1]), pack_bf16x2(v[q * 8 + 2], v[q * 8 + 3]),
+                           pack_bf16x2(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16x2(v[q * 8 + 6], v[q * 8 + 7]));
   } else {
     float4* cp = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off);
 #pragma unroll
     for (int q = 0; q < 8; ++q)
       if (q * 4 < n_valid) cp[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
   }
+}
+
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 r;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr) : "memory");
+  return r;
+}
+
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global [%0, {%1, %2, %3, %4, %5}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+// One chunk of this thread's row into the warp's staging box (32 rows x 128 B, 128B-swizzled as
+// the output tensor map expects): 16-byte piece p of row r lives at r*128 + ((p ^ (r & 7)) * 16).
+__device__ __forceinline__ void store_staged(const TcArgs& a, const float* v, uint32_t box, int lane, int half) {
+  const uint32_t row = box + (uint32_t)lane * 128u;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  if (a.c_bf16) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      st_shared_v4(row + ((((uint32_t)(half * 4 + q)) ^ sw) << 4), pack_bf16x2(v[q * 8], v[q * 8 + 1]),
+                   pack_bf16x2(v[q * 8 + 2], v[q * 8 + 3]), pack_bf16x2(v[q * 8 + 4], v[q * 8 + 5]),
+                   pack_bf16x2(v[q * 8 + 6], v[q * 8 + 7]));
+  } else {
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      st_shared_v4(row + (((uint32_t)q ^ sw) << 4), __float_as_uint(v[q * 4]), __float_as_uint(v[q * 4 + 1]),
+                   __float_as_uint(v[q * 4 + 2]), __float_as_uint(v[q * 4 + 3]));
+  }
+}
+
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
 // kPair = false: one CTA owns a 128 x block_n tile (tcgen05 cta_group::1), 4-stage ring of 48 KB.
@@ -366,7 +397,8 @@ __device__ __forceinline__ void epilogue_store(const TcArgs& a, float* v, float*
 //   the even CTA's "accumulator empty" barrier.  No load uses cluster multicast.
 template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcArgs a) {
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m, const TcArgs a) {
   constexpr int kStages = kPair ? 6 : 4;
   constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kTileRows = kPair ? 2 * BM : BM;       // rows of C owned by a work item
@@ -375,14 +407,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (tiles_base - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + kStages * kStageBytes);
+  // after the ring: per epilogue warp two 4 KB staging boxes for the output stores, then the barriers
+  const uint32_t staging_base = tiles_base + kRingBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + kRingBytes + kStagingBytes);
   // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
-  const uint32_t bar_base = tiles_base + kStages * kStageBytes;
+  const uint32_t bar_base = staging_base + kStagingBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
   auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  // then [2S+4..2S+12): per epilogue warp two barriers for relu-mask boxes loaded into the staging buffers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -395,10 +430,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kPair ? 8 : 4); }
+    for (int i = 0; i < 8; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
   }
   if (warp == 1) {   // TMEM allocation is a warp-wide operation (the same warp of both CTAs of a pair)
     if (kPair) {
@@ -498,6 +535,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else {
     // ------------------------------- epilogue -----------------------------------
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
+    const uint32_t stg = staging_base + (uint32_t)(warp - 2) * 8192u;
+    uint32_t stg_buf = 0;
+    uint32_t mask_phase = 0;                       // bit b: phase of this warp's mask barrier b
+    auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
     int iter = 0;
     bool ok = true;
     for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
@@ -506,36 +547,102 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const Tile tl = decode_tile(a, t, kTileRows);
       const int acc = iter & 1;
       const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
-      ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tcgen05_fence_after();
       const int tile_row = cta_rank * BM + q * 32 + lane;       // row inside the work item's tile
       const int row = tl.m0 + tile_row;
       const bool row_ok = row < tl.m_end;
       const long long row_off = tl.c_off + (long long)row * a.ldc;
+      // what the epilogue needs from memory is requested before the accumulator is waited for:
+      // the tile's bias (lane l keeps columns l, l+32, ...) and the first chunk's relu mask
+      const bool bias_n = a.bias != nullptr && !a.bias_along_m;
+      auto bias_at = [&](int col) -> float {       // bias of one column, 0 outside the slice
+        if (!bias_n || col >= tl.n_end) return 0.f;
+        return a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[col]) : reinterpret_cast<const float*>(a.bias)[col];
+      };
+      float bias_cur = bias_at(tl.n0 + lane);      // lane l keeps column l of the current chunk
+      float bias_row = 0.f;
+      if (a.bias && a.bias_along_m && row_ok)
+        bias_row = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row]) : reinterpret_cast<const float*>(a.bias)[row];
+      const int row0 = tl.m0 + cta_rank * BM + q * 32;           // first row of this warp
+      const bool rows_full = row0 + 32 <= tl.m_end;
+      const bool mask_tma = a.mask_tma != 0 && !ws_mode && rows_full;
+      if (mask_tma && lane == 0) {
+        // pull the warp's part of the mask tile towards L2 and request its first box
+        for (int b = 0; b < a.block_n; b += 64)
+          if (tl.n0 + b + 64 <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
+        if (tl.n0 + 64 <= tl.n_end) {
+          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          mbar_expect_tx(mfull_bar(stg_buf), 4096u);
+          tma_load_5d<false>(stg + stg_buf * 4096u, &map_m, mfull_bar(stg_buf), tl.n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+        }
+      }
+      ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
       if (!ws_mode) {
-        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+        // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
+        // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
+        // ragged edges are read and stored from registers
+        const int box_cols = a.c_bf16 ? 64 : 32;
+#pragma unroll 1
+        for (int c = 0; c < kMaxBN / 32; ++c) {
+          if (c * 32 >= a.block_n) break;
+          const int c0 = c * 32;
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
-          tmem_ld_wait();
           const int n_first = tl.n0 + c0;
           int n_valid = tl.n_end - n_first;
           n_valid = n_valid > 32 ? 32 : n_valid;
-          float r[32];
-          if (a.rsum) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) r[j] = 0.f;
+          const bool live = row_ok && n_valid > 0;
+          const int box_n0 = tl.n0 + (c0 & ~(box_cols - 1));
+          const bool staged = rows_full && box_n0 + box_cols <= tl.n_end;
+          const uint32_t box = stg + stg_buf * 4096u;
+          const int half = (c0 >> 5) & 1;
+          if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box
+            if (mask_tma) {
+              // request the next box's mask into the other buffer (free once its last store was
+              // read out), then wait for this box's mask
+              const int next_n0 = box_n0 + 64;
+              if (lane == 0 && next_n0 < tl.n0 + a.block_n && next_n0 + 64 <= tl.n_end) {
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_expect_tx(mfull_bar(stg_buf ^ 1u), 4096u);
+                tma_load_5d<false>(stg + (stg_buf ^ 1u) * 4096u, &map_m, mfull_bar(stg_buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+              }
+              mbar_wait(mfull_bar(stg_buf), (mask_phase >> stg_buf) & 1u, 0x500 + (int)stg_buf, abort_flag);
+              mask_phase ^= 1u << stg_buf;
+            } else {
+              if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+              __syncwarp();
+            }
           }
-          if (row_ok && n_valid > 0) {
-            float v[32];
+          uint4 mk[4];
+          if (a.mask && a.mask_bf16) {
+            if (staged && mask_tma) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]);
-            epilogue_store(a, v, r, row_off, row, n_first, n_valid);
+              for (int i = 0; i < 4; ++i) mk[i] = ld_shared_v4(box + (uint32_t)lane * 128u + ((((uint32_t)(half * 4 + i)) ^ (uint32_t)(lane & 7)) << 4));
+            } else {
+              mask_fetch(a, row_off + n_first, row_ok, n_valid, mk);
+            }
           }
-          if (a.rsum && n_valid > 0) {      // warp-uniform: every lane takes part in the shuffles
-            const float col = warp_column_sums(r, lane);
+          const float bias_next = bias_at(n_first + 32 + lane);   // travels while this chunk is processed
+          tmem_ld_wait();
+          float* v = reinterpret_cast<float*>(raw);
+          epilogue_math(a, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
+          bias_cur = bias_next;
+          epilogue_residual(a, v, row_off + n_first, live, n_valid);
+          if (staged) store_staged(a, v, box, lane, half);
+          else if (live) store_direct(a, v, row_off + n_first, n_valid);
+          if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+            stg_buf ^= 1u;
+          }
+          if (a.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (live && j < n_valid) ? v[j] : 0.f;
+            const float col = warp_column_sums(v, lane);
             if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
           }
         }
@@ -566,19 +673,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (old == (unsigned)a.sk - 1) {
           __threadfence();
           const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * kTileRows + (size_t)tile_row) * a.block_n;
-          for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+#pragma unroll
+          for (int c0 = 0; c0 < kMaxBN; c0 += 32) {
+            if (c0 >= a.block_n) break;
             const int n_first = tl.n0 + c0;
             int n_valid = tl.n_end - n_first;
             n_valid = n_valid > 32 ? 32 : n_valid;
-            float r[32];
-            if (a.rsum) {
+            const bool live = row_ok && n_valid > 0;
+            float v[32];
 #pragma unroll
-              for (int j = 0; j < 32; ++j) r[j] = 0.f;
-            }
-            if (row_ok && n_valid > 0) {
-              float v[32];
-#pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = 0.f;
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+            if (live) {
               for (int s = 0; s < a.sk; ++s) {     // ascending processor order within the group
                 const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * kTileRows * a.block_n + c0);
 #pragma unroll
@@ -587,17 +692,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                   v[4 * j] += f.x; v[4 * j + 1] += f.y; v[4 * j + 2] += f.z; v[4 * j + 3] += f.w;
                 }
               }
-              epilogue_store(a, v, r, row_off, row, n_first, n_valid);
             }
-            if (a.rsum && n_valid > 0) {
-              const float col = warp_column_sums(r, lane);
-              if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
+            if (n_valid > 0) {                     // warp-uniform: the bias hand-out and the column sums use shuffles
+              uint4 mkw[4];
+              if (a.mask && a.mask_bf16) mask_fetch(a, row_off + n_first, row_ok, n_valid, mkw);
+              epilogue_math(a, v, bias_at(n_first + lane), bias_row, mkw, row_off + n_first, live, n_valid);
+              float col = 0.f;
+              if (a.rsum) {
+                float r[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = (live && j < n_valid) ? v[j] : 0.f;
+                col = warp_column_sums(r, lane);
+                if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
+              }
+              epilogue_residual(a, v, row_off + n_first, live, n_valid);
+              if (live) store_direct(a, v, row_off + n_first, n_valid);
             }
           }
         }
       }
     }
   }
+
+  if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // staged output stores have landed
 
   // ------------------------------- teardown --------------------------------------
   if (*abort_flag) {
@@ -632,37 +749,39 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
-// One operand as a 5-D tensor map: (contiguous dim, other of {M|N, K}, outer2, outer1, outer0).
-mtf_status make_map(CUtensorMap* map, const void* base, bool mn_major, int64_t ext_mn, int64_t ext_k, int64_t ld,
-                    const TcParams& t, const int64_t* outer_stride, int box_rows_kmajor) {
+// One tensor as a 5-D tensor map: (contiguous dim, second dim, outer2, outer1, outer0), 128B swizzle.
+//   dim0 / dim1 : extents of the contiguous and of the strided dimension; ld = element stride of dim1
+//   box0 / box1 : box extents in elements (box0 * elem_bytes = 128)
+mtf_status make_map(CUtensorMap* map, const void* base, int elem_bytes, int64_t dim0, int64_t dim1, int64_t ld,
+                    int box0, int box1, const TcParams& t, const int64_t* outer_stride) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return mtf::fail(MTF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-  if (reinterpret_cast<uintptr_t>(base) & 15) return mtf::fail(MTF_ERR_INVALID_ARG, "tensor-core path needs 16-byte aligned operands");
+  if (reinterpret_cast<uintptr_t>(base) & 15) return mtf::fail(MTF_ERR_INVALID_ARG, "tensor-core path needs 16-byte aligned tensors");
+  const int64_t align = 16 / elem_bytes;     // strides must be multiples of 16 bytes
   cuuint64_t dims[5];
   cuuint64_t strides[4];
-  cuuint32_t box[5] = {64, 1, 1, 1, 1};
+  cuuint32_t box[5] = {(cuuint32_t)box0, (cuuint32_t)box1, 1, 1, 1};
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-  dims[0] = mn_major ? ext_mn : ext_k;
-  dims[1] = mn_major ? ext_k : ext_mn;
-  box[1] = mn_major ? BK : box_rows_kmajor;
-  // the second dimension's stride; a dimension of extent 1 may carry any stride, give it a legal one
+  dims[0] = dim0;
+  dims[1] = dim1;
+  // a dimension of extent 1 may carry any stride, give it a legal one
   int64_t s1 = ld;
-  if (dims[1] == 1 || s1 % 8 != 0 || s1 <= 0) s1 = ((int64_t)dims[0] + 7) / 8 * 8;
-  strides[0] = (cuuint64_t)s1 * 2;
-  const int64_t dummy = (s1 * (int64_t)dims[1] + 7) / 8 * 8;   // legal stride for extent-1 dimensions
+  if (dims[1] == 1 || s1 % align != 0 || s1 <= 0) s1 = (dim0 + align - 1) / align * align;
+  strides[0] = (cuuint64_t)s1 * elem_bytes;
+  const int64_t dummy = (s1 * dim1 + align - 1) / align * align;   // legal stride for extent-1 dimensions
   for (int d = 2; d < 5; ++d) {
     const int src = 4 - d;   // map dim 4 = outer dim 0 ... map dim 2 = outer dim 2 (coordinates o[0..2])
     if (src < t.n_outer && t.outer_size[src] > 1 && outer_stride[src] > 0) {
       dims[d] = t.outer_size[src];
-      strides[d - 1] = (cuuint64_t)outer_stride[src] * 2;
+      strides[d - 1] = (cuuint64_t)outer_stride[src] * elem_bytes;
     } else {
       dims[d] = 1;
-      strides[d - 1] = (cuuint64_t)dummy * 2;
+      strides[d - 1] = (cuuint64_t)dummy * elem_bytes;
     }
   }
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = enc(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 5, const_cast<void*>(base),
+                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS)
     return mtf::fail(MTF_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d (dims %llu %llu %llu %llu %llu, strides %llu %llu %llu %llu)", (int)r,
                      (unsigned long long)dims[0], (unsigned long long)dims[1], (unsigned long long)dims[2], (unsigned long long)dims[3],
@@ -739,6 +858,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.C = C; a.c_bf16 = plan.dtC == MTF_BF16;
   a.bias = bias; a.bias_bf16 = dtBias == MTF_BF16; a.bias_along_m = t.bias_along_m;
   a.mask = mask; a.mask_bf16 = dtMask == MTF_BF16;
+  a.mask_tma = (mask && a.mask_bf16 && a.c_bf16) ? 1 : 0;
   a.resid = resid; a.resid_bf16 = dtRes == MTF_BF16;
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
@@ -761,10 +881,19 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     cudaError_t e = cudaMemsetAsync(rsum, 0, (size_t)t.N * sizeof(float), st);
     if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
   }
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_c, map_m;
   mtf_status s;
-  if ((s = make_map(&map_a, A, t.a_mn_major, t.M, t.K, t.a_ld, t, t.outer_sA, BM)) != MTF_OK) return s;
-  if ((s = make_map(&map_b, B, t.b_mn_major, t.N, t.K, t.b_ld, t, t.outer_sB, t.cta_pair ? t.block_n / 2 : t.block_n)) != MTF_OK) return s;
+  // operands: K-major = (K contiguous, M|N rows), box 64 x rows;  MN-major = (M|N contiguous, K rows), box 64 x 64
+  const int b_rows = t.cta_pair ? t.block_n / 2 : t.block_n;
+  s = t.a_mn_major ? make_map(&map_a, A, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&map_a, A, 2, t.K, t.M, t.a_ld, 64, BM, t, t.outer_sA);
+  if (s != MTF_OK) return s;
+  s = t.b_mn_major ? make_map(&map_b, B, 2, t.N, t.K, t.b_ld, 64, BK, t, t.outer_sB) : make_map(&map_b, B, 2, t.K, t.N, t.b_ld, 64, b_rows, t, t.outer_sB);
+  if (s != MTF_OK) return s;
+  // output: (N contiguous, M rows), boxes of 32 rows x 128 bytes for the staged stores
+  const int c_bytes = plan.dtC == MTF_BF16 ? 2 : 4;
+  if ((s = make_map(&map_c, C, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
+  map_m = map_c;
+  if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
 
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -793,11 +922,11 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<true>, map_a, map_b, a);
+    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<true>, map_a, map_b, map_c, map_m, a);
     if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<pair>: %s", cudaGetErrorString(le));
   } else {
     const long long grid = std::min<long long>(a.total_work, sm_count());
-    gemm_tcgen05_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, a);
+    gemm_tcgen05_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, map_c, map_m, a);
   }
   count_launch();
   cudaError_t e = cudaGetLastError();

@@ -261,6 +261,7 @@ static bool plan_tc(mtf_plan_t* P, std::string* why, int force_single_cta) {
     else if (covers(other)) t.bias_along_m = 1;
     else { *why = "bias dims are not exactly the N (or M) group in storage order"; return false; }
   }
+  if (P->epi.has_rsum && P->epi.has_res) { *why = "reduce_sum_out together with a residual"; return false; }
   if (P->epi.has_rsum) {
     const auto& rd = P->epi.rsum_dims;
     std::vector<int> g = swap ? cm : cn;              // the kernel's N group
