@@ -26,14 +26,15 @@
 namespace {
 
 constexpr int BM = 128;
+constexpr int kEpilogueWarps = 8;                  // two per TMEM lane quarter, interleaved over the column boxes
 constexpr int BK = 64;
 constexpr int kMaxBN = 256;
 constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
 constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stages half of it)
 constexpr int kRingBytes = 4 * (kAStageBytes + kBStageBytes);   // = 6 * (16 KB + 16 KB) = 192 KB
-constexpr int kStagingBytes = 4 * 2 * 4096;      // per epilogue warp: two 32-row x 128-byte boxes for TMA stores
+constexpr int kStagingBytes = kEpilogueWarps * 4096;   // per epilogue warp: one 32-row x 128-byte box for TMA stores
 constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kThreads = 192;
+constexpr int kThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
 
@@ -416,7 +417,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
   auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
-  // then [2S+4..2S+12): per epilogue warp two barriers for relu-mask boxes loaded into the staging buffers
+  // then [2S+4..2S+12): per epilogue warp one barrier for relu-mask boxes loaded into its staging buffer
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -429,8 +430,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), kPair ? 8 : 4); }
-    for (int i = 0; i < 8; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), (kPair ? 2 : 1) * kEpilogueWarps); }
+    for (int i = 0; i < kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -535,10 +536,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else {
     // ------------------------------- epilogue -----------------------------------
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
-    const uint32_t stg = staging_base + (uint32_t)(warp - 2) * 8192u;
-    uint32_t stg_buf = 0;
-    uint32_t mask_phase = 0;                       // bit b: phase of this warp's mask barrier b
-    auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
+    const int col_half = (warp - 2) >> 2;          // which of the two warps of this lane quarter
+    const uint32_t box = staging_base + (uint32_t)(warp - 2) * 4096u;
+    uint32_t mask_phase = 0;                       // phase of this warp's mask barrier
+    const uint32_t mfull_bar = bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2));
     int iter = 0;
     bool ok = true;
     for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
@@ -558,7 +559,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (!bias_n || col >= tl.n_end) return 0.f;
         return a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[col]) : reinterpret_cast<const float*>(a.bias)[col];
       };
-      float bias_cur = bias_at(tl.n0 + lane);      // lane l keeps column l of the current chunk
       float bias_row = 0.f;
       if (a.bias && a.bias_along_m && row_ok)
         bias_row = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row]) : reinterpret_cast<const float*>(a.bias)[row];
@@ -566,14 +566,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const bool rows_full = row0 + 32 <= tl.m_end;
       const bool mask_tma = a.mask_tma != 0 && !ws_mode && rows_full;
       if (mask_tma && lane == 0) {
-        // pull the warp's part of the mask tile towards L2 and request its first box
-        for (int b = 0; b < a.block_n; b += 64)
+        // pull this warp's boxes of the mask tile towards L2
+        for (int b = col_half * 64; b < a.block_n; b += 128)
           if (tl.n0 + b + 64 <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
-        if (tl.n0 + 64 <= tl.n_end) {
-          asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-          mbar_expect_tx(mfull_bar(stg_buf), 4096u);
-          tma_load_5d<false>(stg + stg_buf * 4096u, &map_m, mfull_bar(stg_buf), tl.n0, row0, tl.o[2], tl.o[1], tl.o[0]);
-        }
       }
       ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -585,10 +580,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
         const int box_cols = a.c_bf16 ? 64 : 32;
+        float bias_cur = bias_at(tl.n0 + col_half * box_cols + lane);      // lane l keeps column l of the current chunk
 #pragma unroll 1
-        for (int c = 0; c < kMaxBN / 32; ++c) {
-          if (c * 32 >= a.block_n) break;
-          const int c0 = c * 32;
+        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+          if (((c0 / box_cols) & 1) != col_half) continue;    // the other warp of this lane quarter owns that box
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
           const int n_first = tl.n0 + c0;
@@ -597,23 +592,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const bool live = row_ok && n_valid > 0;
           const int box_n0 = tl.n0 + (c0 & ~(box_cols - 1));
           const bool staged = rows_full && box_n0 + box_cols <= tl.n_end;
-          const uint32_t box = stg + stg_buf * 4096u;
           const int half = (c0 >> 5) & 1;
-          if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box
-            if (mask_tma) {
-              // request the next box's mask into the other buffer (free once its last store was
-              // read out), then wait for this box's mask
-              const int next_n0 = box_n0 + 64;
-              if (lane == 0 && next_n0 < tl.n0 + a.block_n && next_n0 + 64 <= tl.n_end) {
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                mbar_expect_tx(mfull_bar(stg_buf ^ 1u), 4096u);
-                tma_load_5d<false>(stg + (stg_buf ^ 1u) * 4096u, &map_m, mfull_bar(stg_buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+          if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box: the buffer must be free
+            if (lane == 0) {
+              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+              if (mask_tma) {                                   // the box's relu mask arrives in place
+                mbar_expect_tx(mfull_bar, 4096u);
+                tma_load_5d<false>(box, &map_m, mfull_bar, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
               }
-              mbar_wait(mfull_bar(stg_buf), (mask_phase >> stg_buf) & 1u, 0x500 + (int)stg_buf, abort_flag);
-              mask_phase ^= 1u << stg_buf;
-            } else {
-              if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-              __syncwarp();
+            }
+            __syncwarp();
+            if (mask_tma) {
+              mbar_wait(mfull_bar, mask_phase, 0x500, abort_flag);
+              mask_phase ^= 1u;
             }
           }
           uint4 mk[4];
@@ -625,7 +616,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               mask_fetch(a, row_off + n_first, row_ok, n_valid, mk);
             }
           }
-          const float bias_next = bias_at(n_first + 32 + lane);   // travels while this chunk is processed
+          // bias of the chunk this warp handles next (the next chunk of the box, or two boxes on)
+          const int next_c0 = (half == 0 && box_cols == 64) ? c0 + 32 : c0 + 32 + box_cols;
+          const float bias_next = bias_at(tl.n0 + next_c0 + lane);
           tmem_ld_wait();
           float* v = reinterpret_cast<float*>(raw);
           epilogue_math(a, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
@@ -637,7 +630,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
-            stg_buf ^= 1u;
           }
           if (a.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
 #pragma unroll
@@ -651,8 +643,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc));
       } else {
         // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
+        // (the two warps of a lane quarter split the columns in halves, each with its own counter)
+        const int ws_c_begin = col_half * (a.block_n / 2), ws_c_end = ws_c_begin + a.block_n / 2;
         float* part = a.ws_partials + ((size_t)(t * a.sk + ks) * kTileRows + (size_t)tile_row) * a.block_n;
-        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+        for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
           tmem_ld_wait();
@@ -668,14 +662,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __threadfence();
         __syncwarp();
         unsigned old = 0;
-        if (lane == 0) old = atomicAdd(&a.ws_counters[t * (kTileRows / 32) + cta_rank * 4 + q], 1u);
+        if (lane == 0) old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + cta_rank * 4 + q) * 2 + col_half], 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old == (unsigned)a.sk - 1) {
           __threadfence();
           const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * kTileRows + (size_t)tile_row) * a.block_n;
-#pragma unroll
-          for (int c0 = 0; c0 < kMaxBN; c0 += 32) {
-            if (c0 >= a.block_n) break;
+#pragma unroll 1
+          for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
             const int n_first = tl.n0 + c0;
             int n_valid = tl.n_end - n_first;
             n_valid = n_valid > 32 ? 32 : n_valid;
@@ -817,7 +810,7 @@ static int64_t tc_total_tiles(const TcParams& t) {
 size_t tc_workspace_bytes(const TcParams& t) {
   if (t.reduce_mode != MTF_REDUCE_WORKSPACE) return 0;
   const int64_t tiles = tc_total_tiles(t);
-  return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * sizeof(unsigned) + 256;
+  return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * 2 * sizeof(unsigned) + 256;
 }
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
@@ -873,7 +866,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     const size_t part_bytes = (size_t)a.total_tiles * a.sk * tile_rows * a.block_n * sizeof(float);
     a.ws_partials = reinterpret_cast<float*>(workspace);
     a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
-    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * (tile_rows / 32) * sizeof(unsigned), st);
+    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * (tile_rows / 32) * 2 * sizeof(unsigned), st);
     if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
   }
 
