@@ -54,6 +54,7 @@ struct TcArgs {
   int k_sliced;            // walk K slice by slice (slice length is a multiple of BK)
   int reduce_mode;
   int m_tiles, n_tiles;    // per slice
+  int n_fastest;           // tile order inside a slice: 1 = walk the n tiles of one m tile first
   long long tiles_per_slice, total_tiles, total_work;
   void* C;
   int c_bf16;
@@ -81,8 +82,9 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int ti
   Tile r;
   long long slice = t / a.tiles_per_slice;
   long long w = t % a.tiles_per_slice;
-  const int mt = (int)(w % a.m_tiles); w /= a.m_tiles;
-  const int nt = (int)(w % a.n_tiles); w /= a.n_tiles;
+  int mt, nt;
+  if (a.n_fastest) { nt = (int)(w % a.n_tiles); w /= a.n_tiles; mt = (int)(w % a.m_tiles); w /= a.m_tiles; }
+  else { mt = (int)(w % a.m_tiles); w /= a.m_tiles; nt = (int)(w % a.n_tiles); w /= a.n_tiles; }
   int ol[3] = {0, 0, 0};
   for (int j = a.n_outer - 1; j >= 0; --j) { ol[j] = (int)(w % a.outer_local[j]); w /= a.outer_local[j]; }
   const int in = (int)(slice % a.sn); slice /= a.sn;
@@ -137,6 +139,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int cod
   for (int i = 0; i < 32; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, code, abort_flag);
+}
+
+// Warp-wide wait for the epilogue warps: lane 0 polls with a pause between polls (so that eight
+// waiting warps do not take issue slots from the MMA and TMA threads), the others sleep at the
+// warp barrier and then confirm the phase themselves.  Same time limit and abort rule as mbar_wait.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int code, volatile int* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) {
+    if (!mbar_try_wait(bar, parity)) {
+      const long long t0 = clock64();
+      while (true) {
+        __nanosleep(100);
+        if (mbar_try_wait(bar, parity)) break;
+        if (*abort_flag) { ok = 0; break; }
+        if (clock64() - t0 > kTimeoutCycles) {
+          atomicCAS(&g_status, 0, code);
+          *abort_flag = 1;
+          ok = 0;
+          break;
+        }
+      }
+    }
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (!ok) return false;
+  return mbar_wait(bar, parity, code, abort_flag);
 }
 
 // kPair: the completion may count on the partner CTA's barrier (cta_group::2 form); never multicast.
@@ -570,7 +598,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int b = col_half * 64; b < a.block_n; b += 128)
           if (tl.n0 + b + 64 <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
       }
-      ok = mbar_wait(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag);
+      ok = mbar_wait_warp(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag, lane);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tcgen05_fence_after();
@@ -842,6 +870,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   const int tile_rows = tc_tile_rows(t);
   a.m_tiles = (a.Ms + tile_rows - 1) / tile_rows;
   a.n_tiles = (a.Ns + a.block_n - 1) / a.block_n;
+  a.n_fastest = 0;   // m tiles of one n tile run together: they share the B tile, which measured fastest
   a.tiles_per_slice = (long long)a.m_tiles * a.n_tiles;
   for (int j = 0; j < a.n_outer; ++j) a.tiles_per_slice *= a.outer_local[j];
   long long out_slices = (long long)a.sm * a.sn;
