@@ -1,4 +1,6 @@
-"""Builds the CUDA library (sm_100a only) next to this file:  python -m paper_1811_02084_b200.build"""
+"""Builds the CUDA library (sm_100a only) next to this file:  python paper_1811_02084_b200/build.py
+
+Run it by path (not with -m): importing the package loads the library, which may not exist yet."""
 from __future__ import annotations
 
 import os
