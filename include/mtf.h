@@ -158,6 +158,30 @@ mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t 
                       void* stream);
 mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in,
                                       const mtf_tensor* out, const mtf_epilogue* epilogue, size_t* bytes);
+/* mtf_einsum for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * is a property of the library, not of the method.)  Who needs it: code that runs where a device
+ * allocation is not allowed or not possible - a host that hands the library tensors but owns the
+ * allocator and will not lend it, a loop that must never trigger the implicit device-wide
+ * synchronisation an allocation or a free can cause, a region that is being replayed and may not
+ * create memory.  Such a caller has nowhere to get the `workspace` that mtf_einsum wants when the
+ * planner realises the group sum through partial tiles (MTF_REDUCE_WORKSPACE).  This call takes no
+ * workspace: the partial tiles and tile counters live in a fixed 32 MiB array inside the library
+ * image, which every GPU that loads the library holds until the process exits.
+ *   - Same arguments and results as mtf_einsum, minus the workspace.  The call itself allocates no
+ *     device memory and calls no allocating routine; it launches one memset of the tile counters
+ *     and one kernel on `stream`.
+ *   - An einsum whose plan needs more than 32 MiB of scratch is refused with
+ *     MTF_ERR_WORKSPACE_TOO_SMALL before anything is launched (use mtf_einsum and bring your own).
+ *     Plans that need no scratch run exactly as through mtf_einsum.
+ *   - The first call on each device looks up the array's device address (a one-time query of the
+ *     runtime with that device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left; the
+ *     counters are zeroed on the stream before each launch and partial tiles are written before
+ *     they are read, so calls that follow each other on one stream are fine.  Calls that may
+ *     overlap on the GPU (different streams, different threads) race on it: serialise them. */
+mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* equation, int32_t n_in,
+                                      const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epilogue,
+                                      void* stream);
 /* Testing hook: force the kernel family / reduce mode of plans created afterwards by this thread
  * (-1 = planner's choice; kernel_kind 2 = tensor cores with one CTA per tile, i.e. without the
  * two-CTA pairs the planner prefers on tall slices).  A forced choice the shape cannot run gives

@@ -46,7 +46,7 @@ def _load():
     if not os.path.exists(LIB_PATH):
         raise ImportError(
             f"{LIB_PATH} is missing: the CUDA library has not been built. Build it with "
-            "`python -m paper_1811_02084_b200.build` (needs nvcc; there is no CPU fallback).")
+            "`python paper_1811_02084_b200/build.py` (needs nvcc; there is no CPU fallback).")
     L = ctypes.CDLL(LIB_PATH)
     vp = c_void_p
     sig = {
@@ -66,6 +66,7 @@ def _load():
         "mtf_plan_info": [vp, POINTER(c_int32), POINTER(c_int32), POINTER(c_int64), POINTER(c_int64), POINTER(c_uint32)],
         "mtf_einsum_exec": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp, c_size_t, vp],
         "mtf_einsum": [vp, c_char_p, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp, c_size_t, vp],
+        "mtf_einsum_builtin_scratch": [vp, c_char_p, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp],
         "mtf_einsum_workspace_bytes": [vp, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), POINTER(c_size_t)],
         "mtf_plan_force": [c_int32, c_int32],
         "mtf_ffn_forward": [vp] + [POINTER(mtf_tensor)] * 6 + [vp, c_size_t, vp],
@@ -305,6 +306,14 @@ def mtf_einsum(layout: Layout, equation, ins, out: Named, epilogue: Epilogue | N
     eq = equation.encode() if equation is not None else None
     _check(_lib.mtf_einsum(layout.handle, eq, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue), wp, wb,
                            _stream(stream)))
+
+
+def mtf_einsum_builtin_scratch(layout: Layout, equation, ins, out: Named, epilogue: Epilogue | None = None, stream=None) -> None:
+    """mtf_einsum without a workspace argument, for callers that cannot allocate device memory: the
+    partial tiles of a workspace-mode group sum go to a fixed 32 MiB array inside the library."""
+    eq = equation.encode() if equation is not None else None
+    _check(_lib.mtf_einsum_builtin_scratch(layout.handle, eq, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue),
+                                           _stream(stream)))
 
 
 def mtf_einsum_workspace_bytes(layout: Layout, ins, out: Named, epilogue: Epilogue | None = None) -> int:

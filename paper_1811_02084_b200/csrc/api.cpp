@@ -300,6 +300,36 @@ mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t 
   return exec_plan(P, in, out, epilogue, workspace, workspace_bytes, stream);
 }
 
+mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in,
+                                      mtf_tensor* out, const mtf_epilogue* epilogue, void* stream) {
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, n_in, in, out, epilogue, &P);
+  if (st != MTF_OK) return st;
+  if (equation && (st = check_equation(equation, n_in, in, out)) != MTF_OK) return st;
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->reduce_mode != MTF_REDUCE_WORKSPACE)
+    return exec_plan(P, in, out, epilogue, nullptr, 0, stream);      // this plan needs no scratch at all
+  if (P->workspace_bytes > mtf::builtin_scratch_capacity())
+    return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "this einsum needs %zu scratch bytes, the built-in scratch holds %zu; use mtf_einsum with a caller-provided workspace",
+                P->workspace_bytes, mtf::builtin_scratch_capacity());
+  // same argument checks as the regular path, then the launch on the library's own scratch
+  if (!in || !out || !in[0].data || !in[1].data || !out->data) return fail(MTF_ERR_INVALID_ARG, "einsum: NULL data pointer");
+  if (!dims_match(P->dimsA, in[0]) || !dims_match(P->dimsB, in[1]) || !dims_match(P->dimsC, *out))
+    return fail(MTF_ERR_SIZE_MISMATCH, "einsum: operand dims differ from the planned ones");
+  const void* bias = nullptr;
+  const void* mask = nullptr;
+  const void* resid = nullptr;
+  float* rsum = nullptr;
+  if (P->epi.on) {
+    if (!epilogue) return fail(MTF_ERR_INVALID_ARG, "einsum: the plan has an epilogue, none was passed");
+    if (P->epi.has_bias) { if (!epilogue->bias || !epilogue->bias->data) return fail(MTF_ERR_INVALID_ARG, "einsum: bias has no data"); bias = epilogue->bias->data; }
+    if (P->epi.has_mask) { if (!epilogue->relu_mask || !epilogue->relu_mask->data) return fail(MTF_ERR_INVALID_ARG, "einsum: relu_mask has no data"); mask = epilogue->relu_mask->data; }
+    if (P->epi.has_res) { if (!epilogue->residual || !epilogue->residual->data) return fail(MTF_ERR_INVALID_ARG, "einsum: residual has no data"); resid = epilogue->residual->data; }
+    if (P->epi.has_rsum) { if (!epilogue->reduce_sum_out || !epilogue->reduce_sum_out->data) return fail(MTF_ERR_INVALID_ARG, "einsum: reduce_sum_out has no data"); rsum = reinterpret_cast<float*>(epilogue->reduce_sum_out->data); }
+  }
+  return mtf::launch_tc_builtin_scratch(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid, P->epi.dtRes,
+                                        P->epi.on ? epilogue->scale : 1.f, P->epi.on ? (epilogue->relu != 0) : 0, rsum, stream);
+}
+
 mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in, const mtf_tensor* out,
                                       const mtf_epilogue* epilogue, size_t* bytes) {
   if (!bytes) return fail(MTF_ERR_INVALID_ARG, "einsum_workspace_bytes: bytes is NULL");

@@ -956,6 +956,51 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   return MTF_OK;
 }
 
+// ---- built-in scratch for callers that cannot allocate device memory ---------------------------------
+// Some callers run where no device allocation may happen: code replayed inside an already captured
+// stream, plug-ins that are handed tensors but no allocator, real-time loops that forbid anything
+// that may synchronise the device.  For them the workspace-mode contraction can run on scratch that
+// is part of the library image: a fixed array every GPU that loads the library holds until exit.
+constexpr size_t kBuiltinScratchBytes = 32u << 20;     // 32 MiB
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+
+size_t builtin_scratch_capacity() { return kBuiltinScratchBytes; }
+
+// The array's name is only a host-side handle; the device address comes from the runtime, once per
+// device, with that device current.
+static mtf_status builtin_scratch_ptr(void** out) {
+  static std::mutex mu;
+  static void* cached[64] = {nullptr};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= 64) return fail(MTF_ERR_UNSUPPORTED, "device ordinal %d outside [0, 64)", dev);
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_builtin_scratch);
+    if (e != cudaSuccess || !p) return fail(MTF_ERR_CUDA, "cudaGetSymbolAddress(built-in scratch): %s", cudaGetErrorString(e));
+    cached[dev] = p;
+  }
+  *out = cached[dev];
+  return MTF_OK;
+}
+
+mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
+                                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
+                                     void* stream) {
+  const size_t need = tc_workspace_bytes(plan.tc);
+  if (need > kBuiltinScratchBytes)
+    return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "this einsum needs %zu scratch bytes, the built-in scratch holds %zu; use mtf_einsum with a caller-provided workspace",
+                need, kBuiltinScratchBytes);
+  void* ws = nullptr;
+  mtf_status st = builtin_scratch_ptr(&ws);
+  if (st != MTF_OK) return st;
+  // the tile counters inside the scratch are cleared by the launcher on the stream; partial tiles are
+  // overwritten before they are read, so the previous call's contents do not matter
+  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream);
+}
+
 mtf_status read_device_status(int* code) {
   cudaError_t e = cudaDeviceSynchronize();
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaDeviceSynchronize: %s", cudaGetErrorString(e));

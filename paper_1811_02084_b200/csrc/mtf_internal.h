@@ -155,6 +155,10 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream);
 size_t tc_workspace_bytes(const TcParams& t);
+size_t builtin_scratch_capacity();
+mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
+                                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
+                                     void* stream);
 mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes,
                                const int64_t* offs, const int64_t* gstrides, void* stream);
 void count_launch(int n = 1);
