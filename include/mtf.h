@@ -207,6 +207,74 @@ mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, con
 mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w,
                                    size_t* bytes);
 
+/* ---- softmax, layer normalisation, attention, decoder layer ------------------------------------------
+ * Section 9 gives the layout of the Transformer (batch, heads, d_ff split; no tensor carries two of
+ * them) and defers its mathematics to Vaswani et al.; the formulas below are that model's, written
+ * as named-dim einsums (Section 6) plus the "Reduction" lowering for the row statistics.
+ * Activations bf16; logits and their gradient f32 scratch; parameters of layer norm f32. */
+
+/* weights = softmax over the LAST dimension of logits (f32 in, bf16 out, same dims).  causal != 0
+ * excludes entries whose last index exceeds the second-to-last index (their weight is exactly 0). */
+mtf_status mtf_softmax_forward(const mtf_layout_t* layout, const mtf_tensor* logits, int32_t causal,
+                               mtf_tensor* weights, void* stream);
+/* dlogits = weights * (dweights - sum over the last dim of dweights * weights); dweights f32. */
+mtf_status mtf_softmax_backward(const mtf_layout_t* layout, const mtf_tensor* weights, const mtf_tensor* dweights,
+                                mtf_tensor* dlogits, void* stream);
+/* y = gamma * (x - mean) * (var + eps)^-1/2 + beta over the LAST dimension (biased variance).
+ * stats: f32 tensor with two values per row (mean, reciprocal standard deviation), kept for backward. */
+mtf_status mtf_layernorm_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* gamma,
+                                 const mtf_tensor* beta, float eps, mtf_tensor* y, mtf_tensor* stats, void* stream);
+/* dx = rstd * (g - mean(g) - xh * mean(g * xh)) + residual, g = dy * gamma, xh = (x - mean) * rstd;
+ * dgamma = sum over rows of dy * xh, dbeta = sum over rows of dy (both or neither; zeroed by the call;
+ * under a batch split these sums are the gradient Allreduce of Algorithm 1).  residual may be NULL. */
+mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* dy, const mtf_tensor* x,
+                                  const mtf_tensor* stats, const mtf_tensor* gamma, const mtf_tensor* residual,
+                                  mtf_tensor* dx, mtf_tensor* dgamma, mtf_tensor* dbeta, void* stream);
+
+/* Multi-head attention.  x [batch, length, d_model]; wq, wk [d_model, heads, d_k]; wv [d_model, heads,
+ * d_v]; wo [heads, d_v, d_model] (names are taken from the descriptors; the key/value side uses the
+ * dimension name "memory_length" for a renamed copy of `length`).
+ *   q[b,l,h,k] = sum_d x wq;  kk[b,m,h,k] = sum_d x wk;  vv[b,m,h,v] = sum_d x wv;
+ *   logits[b,h,l,m] = d_k^-1/2 sum_k q kk;  weights = softmax over m (causal: m <= l);
+ *   o[b,l,h,v] = sum_m weights vv;  y[b,l,d] = sum_{h,v} o wo  (+ residual, NULL or y's dims).
+ * q, kk, vv, weights [batch, heads, length, memory_length], o are outputs kept for the backward pass. */
+mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq,
+                                 const mtf_tensor* wk, const mtf_tensor* wv, const mtf_tensor* wo, int32_t causal,
+                                 const mtf_tensor* residual, mtf_tensor* q, mtf_tensor* kk, mtf_tensor* vv,
+                                 mtf_tensor* weights, mtf_tensor* o, mtf_tensor* y, void* workspace,
+                                 size_t workspace_bytes, void* stream);
+/* Gradients of the above for upstream dy [batch, length, d_model]: dwq, dwk, dwv, dwo (reduce out the
+ * token dims) and dx (reduces out heads; dx_residual, NULL or dx's dims, is added). */
+mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq,
+                                  const mtf_tensor* wk, const mtf_tensor* wv, const mtf_tensor* wo, const mtf_tensor* q,
+                                  const mtf_tensor* kk, const mtf_tensor* vv, const mtf_tensor* weights,
+                                  const mtf_tensor* o, const mtf_tensor* dy, const mtf_tensor* dx_residual,
+                                  mtf_tensor* dx, mtf_tensor* dwq, mtf_tensor* dwk, mtf_tensor* dwv, mtf_tensor* dwo,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+mtf_status mtf_attention_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq,
+                                         const mtf_tensor* wv, size_t* bytes);
+
+/* Decoder layer (post-layer-norm residual blocks):  a = LN1(x + Attention(x));  out = LN2(a + FFN(a)). */
+typedef struct {
+  const mtf_tensor *wq, *wk, *wv, *wo, *ln1_gamma, *ln1_beta, *w, *bias /* may be NULL */, *v, *ln2_gamma, *ln2_beta;
+} mtf_decoder_params;
+/* Caller-allocated activations the forward pass fills and the backward pass reads:
+ * q, kk, vv, weights, o as in attention; s1 = x + Attention(x); stats1; a; h [*, d_ff]; s2 = a + FFN(a); stats2. */
+typedef struct {
+  mtf_tensor *q, *kk, *vv, *weights, *o, *s1, *stats1, *a, *h, *s2, *stats2;
+} mtf_decoder_saved;
+typedef struct {
+  mtf_tensor *dwq, *dwk, *dwv, *dwo, *dln1_gamma, *dln1_beta, *dw, *dbias /* may be NULL */, *dv, *dln2_gamma, *dln2_beta;
+} mtf_decoder_grads;
+mtf_status mtf_decoder_layer_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* params,
+                                     int32_t causal, float eps, const mtf_decoder_saved* saved, mtf_tensor* out,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* params,
+                                      const mtf_decoder_saved* saved, const mtf_tensor* dout, mtf_tensor* dx,
+                                      const mtf_decoder_grads* grads, void* workspace, size_t workspace_bytes, void* stream);
+mtf_status mtf_decoder_layer_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x,
+                                             const mtf_decoder_params* params, size_t* bytes);
+
 /* ---- reductions (Section 6 "Reduction") --------------------------------------------------------- */
 /* out[out dims] = sum over the other dims of in (out dims a subset of in's).  Local reduction per
  * slice, then the group sum across the mesh dims of reduced-out split dims, in one launch. */

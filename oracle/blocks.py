@@ -67,36 +67,40 @@ def causal_mask(length, memory_length="memory_length", length_name="length"):
     return NT([(length_name, L), (memory_length, L)], m)
 
 
-def attention_forward(ops, x, wq, wk, wv, wo, mask=None):
+def attention_forward(ops, x, wq, wk, wv, wo, mask=None, store=_identity, residual=None):
     """x: [batch, length, d_model]; wq, wk: [d_model, heads, d_k]; wv: [d_model, heads, d_v];
     wo: [heads, d_v, d_model].  xm is x with `length` renamed `memory_length` (same data; a tensor
     cannot carry one name twice).
         q[b,l,h,k] = sum_d x wq      kk[b,m,h,k] = sum_d xm wk      vv[b,m,h,v] = sum_d xm wv
         lg[b,h,l,m] = d_k^-1/2 sum_k q kk  (+ mask[l,m])
         P = exp(lg - max_m lg) / sum_m exp(lg - max_m lg)
-        o[b,l,h,v] = sum_m P vv      y[b,l,d] = sum_{h,v} o wo"""
+        o[b,l,h,v] = sum_m P vv      y[b,l,d] = sum_{h,v} o wo  (+ residual)
+    ``store`` is applied to q, kk, vv, P and o (kept between einsums); the logits are not stored
+    in a narrow type."""
     b, l, d = x.names
     _, h, k = wq.names
     vdim = wv.names[2]
     m = "memory_length"
     s = 1.0 / np.sqrt(float(dict(wq.dims)[k]))
     xm = ops.rename(x, l, m)
-    q = ops.einsum([x, wq], [b, l, h, k])
-    kk = ops.einsum([xm, wk], [b, m, h, k])
-    vv = ops.einsum([xm, wv], [b, m, h, vdim])
+    q = store(ops.einsum([x, wq], [b, l, h, k]))
+    kk = store(ops.einsum([xm, wk], [b, m, h, k]))
+    vv = store(ops.einsum([xm, wv], [b, m, h, vdim]))
     lg = ops.scale(ops.einsum([q, kk], [b, h, l, m]), s)
     if mask is not None:
         lg = ops.add(lg, mask)
     mx = ops.reduce_max(lg, [b, h, l])
     e = ops.exp(ops.sub(lg, mx))
     z = ops.reduce_sum(e, [b, h, l])
-    P = ops.mul(e, ops.unary(z, lambda a: 1.0 / a))
-    o = ops.einsum([P, vv], [b, l, h, vdim])
+    P = store(ops.mul(e, ops.unary(z, lambda a: 1.0 / a)))
+    o = store(ops.einsum([P, vv], [b, l, h, vdim]))
     y = ops.einsum([o, wo], [b, l, d])
+    if residual is not None:
+        y = ops.add(y, residual)
     return {"q": q, "kk": kk, "vv": vv, "P": P, "o": o, "y": y}
 
 
-def attention_backward(ops, x, wq, wk, wv, wo, saved, dy):
+def attention_backward(ops, x, wq, wk, wv, wo, saved, dy, store=_identity):
     """dwo[h,v,d] = sum_{b,l} o dy;  do = sum_d dy wo;  dP = sum_v do vv;  dvv = sum_l P do;
     dlg = P * (dP - sum_m dP*P);  dq = s sum_m dlg kk;  dkk = s sum_l dlg q;
     dwq = sum_{b,l} x dq;  dwk = sum_{b,m} xm dkk;  dwv = sum_{b,m} xm dvv;
@@ -109,13 +113,13 @@ def attention_backward(ops, x, wq, wk, wv, wo, saved, dy):
     q, kk, vv, P, o = saved["q"], saved["kk"], saved["vv"], saved["P"], saved["o"]
     xm = ops.rename(x, l, m)
     dwo = ops.einsum([o, dy], list(wo.names))
-    do = ops.einsum([dy, wo], [b, l, h, vdim])
+    do = store(ops.einsum([dy, wo], [b, l, h, vdim]))
     dP = ops.einsum([do, vv], [b, h, l, m])
-    dvv = ops.einsum([P, do], [b, m, h, vdim])
+    dvv = store(ops.einsum([P, do], [b, m, h, vdim]))
     row = ops.reduce_sum(ops.mul(dP, P), [b, h, l])
-    dlg = ops.mul(P, ops.sub(dP, row))
-    dq = ops.scale(ops.einsum([dlg, kk], [b, l, h, k]), s)
-    dkk = ops.scale(ops.einsum([dlg, q], [b, m, h, k]), s)
+    dlg = store(ops.mul(P, ops.sub(dP, row)))
+    dq = store(ops.scale(ops.einsum([dlg, kk], [b, l, h, k]), s))
+    dkk = store(ops.scale(ops.einsum([dlg, q], [b, m, h, k]), s))
     dwq = ops.einsum([x, dq], list(wq.names))
     dwk = ops.einsum([xm, dkk], list(wk.names))
     dwv = ops.einsum([xm, dvv], list(wv.names))
@@ -162,25 +166,28 @@ def layernorm_backward(ops, gamma, saved, dy):
 # Decoder layer (reading: post-layer-norm residual blocks, a = LN1(x + Att(x)); out = LN2(a + FFN(a)))
 # --------------------------------------------------------------------------------------------------
 
-def decoder_layer_forward(ops, x, p, mask, eps):
-    """p: dict with wq, wk, wv, wo, g1, b1, w, bias, v, g2, b2 (already in ops' representation)."""
-    att = attention_forward(ops, x, p["wq"], p["wk"], p["wv"], p["wo"], mask)
-    ln1 = layernorm_forward(ops, ops.add(x, att["y"]), p["g1"], p["b1"], eps)
-    a = ln1["y"]
-    ffn = ffn_forward(ops, a, p["w"], p["bias"], p["v"])
-    ln2 = layernorm_forward(ops, ops.add(a, ffn["y"]), p["g2"], p["b2"], eps)
+def decoder_layer_forward(ops, x, p, mask, eps, store=_identity):
+    """p: dict with wq, wk, wv, wo, g1, b1, w, bias, v, g2, b2 (already in ops' representation).
+    ``store`` additionally applies to the two residual sums s1, s2 and to a (kept for backward)."""
+    att = attention_forward(ops, x, p["wq"], p["wk"], p["wv"], p["wo"], mask, store)
+    s1 = store(ops.add(x, att["y"]))
+    ln1 = layernorm_forward(ops, s1, p["g1"], p["b1"], eps)
+    a = store(ln1["y"])
+    ffn = ffn_forward(ops, a, p["w"], p["bias"], p["v"], store)
+    s2 = store(ops.add(a, ffn["y"]))
+    ln2 = layernorm_forward(ops, s2, p["g2"], p["b2"], eps)
     return {"att": att, "ln1": ln1, "a": a, "ffn": ffn, "ln2": ln2, "out": ln2["y"]}
 
 
-def decoder_layer_backward(ops, x, p, saved, dout):
-    """Chain rule through the two residual sums."""
+def decoder_layer_backward(ops, x, p, saved, dout, store=_identity):
+    """Chain rule through the two residual sums (the gradient streams ds2, da, ds1 are stored)."""
     l2 = layernorm_backward(ops, p["g2"], saved["ln2"], dout)
-    ds2 = l2["dx"]                                    # gradient on (a + FFN(a))
-    fb = ffn_backward(ops, saved["a"], p["w"], p["v"], saved["ffn"]["h"], ds2)
-    da = ops.add(ds2, fb["dx"])
+    ds2 = store(l2["dx"])                             # gradient on (a + FFN(a))
+    fb = ffn_backward(ops, saved["a"], p["w"], p["v"], saved["ffn"]["h"], ds2, store)
+    da = store(ops.add(ds2, fb["dx"]))
     l1 = layernorm_backward(ops, p["g1"], saved["ln1"], da)
-    ds1 = l1["dx"]                                    # gradient on (x + Att(x))
-    ab = attention_backward(ops, x, p["wq"], p["wk"], p["wv"], p["wo"], saved["att"], ds1)
+    ds1 = store(l1["dx"])                             # gradient on (x + Att(x))
+    ab = attention_backward(ops, x, p["wq"], p["wk"], p["wv"], p["wo"], saved["att"], ds1, store)
     dx = ops.add(ds1, ab["dx"])
     return {"dx": dx, "dg2": l2["dgamma"], "db2": l2["dbeta"], "dg1": l1["dgamma"], "db1": l1["dbeta"],
             "dw": fb["dw"], "dbias": fb["dbias"], "dv": fb["dv"],

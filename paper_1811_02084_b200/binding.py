@@ -35,6 +35,18 @@ class mtf_epilogue(Structure):
                 ("reduce_sum_out", POINTER(mtf_tensor))]
 
 
+class mtf_decoder_params(Structure):
+    _fields_ = [(n, POINTER(mtf_tensor)) for n in ("wq", "wk", "wv", "wo", "ln1_gamma", "ln1_beta", "w", "bias", "v", "ln2_gamma", "ln2_beta")]
+
+
+class mtf_decoder_saved(Structure):
+    _fields_ = [(n, POINTER(mtf_tensor)) for n in ("q", "kk", "vv", "weights", "o", "s1", "stats1", "a", "h", "s2", "stats2")]
+
+
+class mtf_decoder_grads(Structure):
+    _fields_ = [(n, POINTER(mtf_tensor)) for n in ("dwq", "dwk", "dwv", "dwo", "dln1_gamma", "dln1_beta", "dw", "dbias", "dv", "dln2_gamma", "dln2_beta")]
+
+
 class MtfError(RuntimeError):
     def __init__(self, status: int, message: str):
         self.status = status
@@ -73,6 +85,16 @@ def _load():
         "mtf_ffn_backward": [vp] + [POINTER(mtf_tensor)] * 9 + [vp, c_size_t, vp],
         "mtf_ffn_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
         "mtf_reduce_sum": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_softmax_forward": [vp, POINTER(mtf_tensor), c_int32, POINTER(mtf_tensor), vp],
+        "mtf_softmax_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_layernorm_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), c_float, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_layernorm_backward": [vp] + [POINTER(mtf_tensor)] * 8 + [vp],
+        "mtf_attention_forward": [vp] + [POINTER(mtf_tensor)] * 5 + [c_int32] + [POINTER(mtf_tensor)] * 7 + [vp, c_size_t, vp],
+        "mtf_attention_backward": [vp] + [POINTER(mtf_tensor)] * 17 + [vp, c_size_t, vp],
+        "mtf_attention_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
+        "mtf_decoder_layer_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), c_int32, c_float, POINTER(mtf_decoder_saved), POINTER(mtf_tensor), vp, c_size_t, vp],
+        "mtf_decoder_layer_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(mtf_decoder_saved), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_decoder_grads), vp, c_size_t, vp],
+        "mtf_decoder_layer_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(c_size_t)],
         "mtf_device_status": [POINTER(c_int32)],
     }
     for name, args in sig.items():
@@ -349,6 +371,71 @@ def mtf_ffn_workspace_bytes(layout, x, w) -> int:
 
 def mtf_reduce_sum(layout, inp: Named, out: Named, stream=None) -> None:
     _check(_lib.mtf_reduce_sum(layout.handle, _p(inp), _p(out), _stream(stream)))
+
+
+def mtf_softmax_forward(layout, logits: Named, causal: bool, weights: Named, stream=None) -> None:
+    _check(_lib.mtf_softmax_forward(layout.handle, _p(logits), 1 if causal else 0, _p(weights), _stream(stream)))
+
+
+def mtf_softmax_backward(layout, weights: Named, dweights: Named, dlogits: Named, stream=None) -> None:
+    _check(_lib.mtf_softmax_backward(layout.handle, _p(weights), _p(dweights), _p(dlogits), _stream(stream)))
+
+
+def mtf_layernorm_forward(layout, x, gamma, beta, eps, y, stats, stream=None) -> None:
+    _check(_lib.mtf_layernorm_forward(layout.handle, _p(x), _p(gamma), _p(beta), float(eps), _p(y), _p(stats), _stream(stream)))
+
+
+def mtf_layernorm_backward(layout, dy, x, stats, gamma, residual, dx, dgamma, dbeta, stream=None) -> None:
+    _check(_lib.mtf_layernorm_backward(layout.handle, _p(dy), _p(x), _p(stats), _p(gamma), _p(residual), _p(dx), _p(dgamma), _p(dbeta),
+                                       _stream(stream)))
+
+
+def mtf_attention_forward(layout, x, wq, wk, wv, wo, causal, residual, q, kk, vv, weights, o, y, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_attention_forward(layout.handle, _p(x), _p(wq), _p(wk), _p(wv), _p(wo), 1 if causal else 0, _p(residual), _p(q), _p(kk),
+                                      _p(vv), _p(weights), _p(o), _p(y), wp, wb, _stream(stream)))
+
+
+def mtf_attention_backward(layout, x, wq, wk, wv, wo, q, kk, vv, weights, o, dy, dx_residual, dx, dwq, dwk, dwv, dwo, workspace=None,
+                           stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_attention_backward(layout.handle, _p(x), _p(wq), _p(wk), _p(wv), _p(wo), _p(q), _p(kk), _p(vv), _p(weights), _p(o), _p(dy),
+                                       _p(dx_residual), _p(dx), _p(dwq), _p(dwk), _p(dwv), _p(dwo), wp, wb, _stream(stream)))
+
+
+def mtf_attention_workspace_bytes(layout, x, wq, wv) -> int:
+    b = c_size_t()
+    _check(_lib.mtf_attention_workspace_bytes(layout.handle, _p(x), _p(wq), _p(wv), byref(b)))
+    return b.value
+
+
+def _struct_of(cls, tensors: dict):
+    s = cls()
+    for name, _t in cls._fields_:
+        t = tensors.get(name)
+        setattr(s, name, ctypes.pointer(t.c) if t is not None else None)
+    return s
+
+
+def mtf_decoder_layer_forward(layout, x, params: dict, causal, eps, saved: dict, out, workspace=None, stream=None) -> None:
+    """params / saved: dicts of Named keyed by the field names of mtf_decoder_params / mtf_decoder_saved."""
+    wp, wb = _ws(workspace)
+    ps, sv = _struct_of(mtf_decoder_params, params), _struct_of(mtf_decoder_saved, saved)
+    _check(_lib.mtf_decoder_layer_forward(layout.handle, _p(x), byref(ps), 1 if causal else 0, float(eps), byref(sv), _p(out), wp, wb,
+                                          _stream(stream)))
+
+
+def mtf_decoder_layer_backward(layout, x, params: dict, saved: dict, dout, dx, grads: dict, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    ps, sv, gs = _struct_of(mtf_decoder_params, params), _struct_of(mtf_decoder_saved, saved), _struct_of(mtf_decoder_grads, grads)
+    _check(_lib.mtf_decoder_layer_backward(layout.handle, _p(x), byref(ps), byref(sv), _p(dout), _p(dx), byref(gs), wp, wb, _stream(stream)))
+
+
+def mtf_decoder_layer_workspace_bytes(layout, x, params: dict) -> int:
+    b = c_size_t()
+    ps = _struct_of(mtf_decoder_params, params)
+    _check(_lib.mtf_decoder_layer_workspace_bytes(layout.handle, _p(x), byref(ps), byref(b)))
+    return b.value
 
 
 def mtf_status_string(status: int) -> str:

@@ -10,7 +10,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmtf_b200.so")
-SOURCES = ["planner.cpp", "api.cpp", "einsum_simt.cu", "gemm_tcgen05.cu", "rowwise.cu"]
+SOURCES = ["planner.cpp", "api.cpp", "blocks.cpp", "einsum_simt.cu", "gemm_tcgen05.cu", "rowwise.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

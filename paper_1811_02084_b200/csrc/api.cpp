@@ -6,6 +6,11 @@
 #include "mtf_internal.h"
 
 namespace mtf {
+mtf_status ffn_forward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias, const mtf_tensor* v,
+                            mtf_tensor* h_saved, mtf_tensor* y, const mtf_tensor* y_residual, void* workspace, size_t workspace_bytes, void* stream);
+mtf_status ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v, const mtf_tensor* h_saved,
+                             const mtf_tensor* dy, mtf_tensor* dx, const mtf_tensor* dx_residual, mtf_tensor* dw, mtf_tensor* dbias, mtf_tensor* dv,
+                             void* workspace, size_t workspace_bytes, void* stream);
 const char* last_error();
 int64_t launch_count();
 mtf_status read_device_status(int* code);
@@ -360,6 +365,15 @@ mtf_status mtf_reduce_sum(const mtf_layout_t* layout, const mtf_tensor* in, mtf_
 mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias,
                            const mtf_tensor* v, mtf_tensor* h_saved, mtf_tensor* y, void* workspace, size_t workspace_bytes,
                            void* stream) {
+  return mtf::ffn_forward_impl(layout, x, w, bias, v, h_saved, y, nullptr, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+// y_residual (NULL or a tensor with y's dims) is added to y in the second einsum's epilogue.
+mtf_status mtf::ffn_forward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias,
+                                 const mtf_tensor* v, mtf_tensor* h_saved, mtf_tensor* y, const mtf_tensor* y_residual, void* workspace,
+                                 size_t workspace_bytes, void* stream) {
   mtf_status st = ffn_check(x, w, v);
   if (st != MTF_OK) return st;
   if (!h_saved || !y) return fail(MTF_ERR_INVALID_ARG, "ffn_forward: NULL output");
@@ -369,8 +383,12 @@ mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, cons
   mtf_tensor in1[2] = {*x, *w};
   if ((st = mtf_einsum(layout, nullptr, 2, in1, h_saved, &e1, workspace, workspace_bytes, stream)) != MTF_OK) return st;
   mtf_tensor in2[2] = {*h_saved, *v};
-  return mtf_einsum(layout, nullptr, 2, in2, y, nullptr, workspace, workspace_bytes, stream);
+  mtf_epilogue e2;
+  e2.scale = 1.f; e2.relu = 0; e2.bias = nullptr; e2.relu_mask = nullptr; e2.residual = y_residual; e2.reduce_sum_out = nullptr;
+  return mtf_einsum(layout, nullptr, 2, in2, y, y_residual ? &e2 : nullptr, workspace, workspace_bytes, stream);
 }
+
+extern "C" {
 
 static void ffn_dhp_desc(const mtf_tensor* h_like_dims_from_x, const mtf_tensor* w, mtf_dtype dt, mtf_dim* storage, mtf_tensor* out) {
   const mtf_tensor* x = h_like_dims_from_x;
@@ -417,6 +435,15 @@ mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor*
 mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,
                             const mtf_tensor* h_saved, const mtf_tensor* dy, mtf_tensor* dx, mtf_tensor* dw, mtf_tensor* dbias,
                             mtf_tensor* dv, void* workspace, size_t workspace_bytes, void* stream) {
+  return mtf::ffn_backward_impl(layout, x, w, v, h_saved, dy, dx, nullptr, dw, dbias, dv, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"
+
+// dx_residual (NULL or a tensor with dx's dims) is added to dx in the last einsum's epilogue.
+mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,
+                                  const mtf_tensor* h_saved, const mtf_tensor* dy, mtf_tensor* dx, const mtf_tensor* dx_residual,
+                                  mtf_tensor* dw, mtf_tensor* dbias, mtf_tensor* dv, void* workspace, size_t workspace_bytes, void* stream) {
   mtf_status st = ffn_check(x, w, v);
   if (st != MTF_OK) return st;
   if (!h_saved || !dy || !dx || !dw || !dv) return fail(MTF_ERR_INVALID_ARG, "ffn_backward: NULL tensor");
@@ -448,8 +475,12 @@ mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, con
   if (dbias && !fuse_dbias && (st = mtf_reduce_sum(layout, &dhp, dbias, stream)) != MTF_OK) return st;
   // dx = dhp . w^T reduces out hidden (Section 8.2)
   mtf_tensor in4[2] = {dhp, *w};
-  return mtf_einsum(layout, nullptr, 2, in4, dx, nullptr, rest, rest_bytes, stream);
+  mtf_epilogue e4;
+  e4.scale = 1.f; e4.relu = 0; e4.bias = nullptr; e4.relu_mask = nullptr; e4.residual = dx_residual; e4.reduce_sum_out = nullptr;
+  return mtf_einsum(layout, nullptr, 2, in4, dx, dx_residual ? &e4 : nullptr, rest, rest_bytes, stream);
 }
+
+extern "C" {
 
 const char* mtf_status_string(mtf_status s) {
   switch (s) {

@@ -35,7 +35,20 @@ def parity_error(got: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(got - ref) / den))
 
 
+def rms_error(got, ref) -> float:
+    """||g - r||_2 / ||r||_2: insensitive to isolated one-ulp differences, sensitive to anything systematic."""
+    ref = np.asarray(ref, dtype=np.float64)
+    d = np.asarray(got, dtype=np.float64) - ref
+    return float(np.sqrt((d * d).sum()) / max(np.sqrt((ref * ref).sum()), 1e-300))
+
+
 TOL = {"bf16": 1e-2, "f32": 1e-4}
+# Blocks that chain four to six bf16-stored intermediates (attention, decoder layer): a GPU value and
+# the oracle's value of a stored intermediate may round to neighbouring bf16 numbers (one ulp = 0.78 %),
+# and outputs fed by few terms (the first rows under a causal mask) do not average that out.  Gates:
+# element-wise 2e-2 and rms 4e-3 against the oracle that stores the same intermediates in bf16;
+# 5e-2 / 1e-2 against exact mathematics (which that oracle itself misses by ~3.5e-2 element-wise).
+TOL_CHAIN = {"elem": 2e-2, "rms": 4e-3, "elem_exact": 5e-2, "rms_exact": 1e-2}
 
 
 def ffn_inputs(seed, tok_dims, d_model, d_ff, dtype, with_bias=True, io_name="d_model", hidden_name="d_ff"):

@@ -1,0 +1,265 @@
+"""GPU parity of softmax, layer normalisation, the attention block and the decoder layer against the
+fp64 oracle, through the C ABI, under the Transformer layouts of Section 9."""
+import numpy as np
+import pytest
+
+import seeded_inputs as si
+from helpers import TOL, TOL_CHAIN, from_torch, parity_error, rms_error, to_torch
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mtf():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_1811_02084_b200 as m
+    return m
+
+
+def layout(mtf, mesh_dims, rules):
+    return mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules)
+
+
+LAYOUTS = [
+    ([("all", 1)], []),
+    ([("all", 2)], [("batch", "all")]),
+    ([("all", 4)], [("heads", "all"), ("d_ff", "all"), ("vocab", "all")]),
+    ([("rows", 2), ("cols", 2)], [("batch", "rows"), ("heads", "cols"), ("d_ff", "cols")]),
+]
+
+
+def alloc(dims, dtype):
+    import torch
+    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}[dtype]
+    return torch.full([s for _, s in dims], float("nan"), dtype=tdt, device="cuda")
+
+
+def check_chain(got, ref_stored, ref_exact, elem_exact=TOL_CHAIN["elem_exact"], rms_exact=TOL_CHAIN["rms_exact"]):
+    """Gates of a block that chains several bf16-stored intermediates (see helpers.TOL_CHAIN)."""
+    bad = {}
+    for k in ref_stored:
+        assert np.isfinite(got[k]).all(), k
+        e = (parity_error(got[k], ref_stored[k]), rms_error(got[k], ref_stored[k]), parity_error(got[k], ref_exact[k]), rms_error(got[k], ref_exact[k]))
+        if e[0] > TOL_CHAIN["elem"] or e[1] > TOL_CHAIN["rms"] or e[2] > elem_exact or e[3] > rms_exact:
+            bad[k] = tuple(round(x, 4) for x in e)
+    assert not bad, f"(elem, rms, elem vs exact, rms vs exact) above the gates: {bad}"
+
+
+# ---- softmax ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_softmax_forward_backward(mtf, causal):
+    import torch
+    dims = [("batch", 2), ("heads", 3), ("length", 40), ("memory_length", 40)]
+    lg = si.normal(11, "lg", [2, 3, 40, 40], "f32", 2.0)
+    dP = si.normal(11, "dP", [2, 3, 40, 40], "f32")
+    x = lg.f64.copy()
+    if causal:
+        x = np.where(np.triu(np.ones((40, 40)), 1) > 0, -np.inf, x)
+    e = np.exp(x - x.max(-1, keepdims=True))
+    P = e / e.sum(-1, keepdims=True)
+    names = [n for n, _ in dims]
+    lay = layout(mtf, [("a", 2), ("b", 3)], [("batch", "a"), ("heads", "b")])
+    w = alloc(dims, "bf16")
+    mtf.mtf_softmax_forward(lay, mtf.named(to_torch(lg), names), causal, mtf.named(w, names))
+    got = from_torch(w)
+    assert parity_error(got, P) <= TOL["bf16"]
+    if causal:
+        iu = np.triu_indices(40, 1)
+        assert (got[..., iu[0], iu[1]] == 0.0).all()
+    # backward on the GPU's own (bf16) weights
+    dlg = alloc(dims, "bf16")
+    mtf.mtf_softmax_backward(lay, mtf.named(w, names), mtf.named(to_torch(dP), names), mtf.named(dlg, names))
+    mtf.mtf_device_status()
+    want = got * (dP.f64 - (dP.f64 * got).sum(-1, keepdims=True))
+    assert parity_error(from_torch(dlg), want) <= TOL["bf16"]
+
+
+# ---- layer norm --------------------------------------------------------------------------------------------
+
+def test_layernorm_forward_backward(mtf):
+    import torch
+    from oracle import NT, DenseOps, blocks
+    ops = DenseOps()
+    dims = [("batch", 3), ("length", 50), ("d_model", 136)]
+    names = [n for n, _ in dims]
+    x = si.normal(12, "x", [3, 50, 136], "bf16", 2.0, 0.5)
+    dy = si.normal(12, "dy", [3, 50, 136], "bf16")
+    res = si.normal(12, "res", [3, 50, 136], "bf16")
+    gamma = si.normal(12, "g", [136], "f32", 0.1, 1.0)
+    beta = si.normal(12, "b", [136], "f32", 0.1)
+    eps = 1e-6
+    f = blocks.layernorm_forward(ops, NT(dims, x.f64), NT(dims[2:], gamma.f64), NT(dims[2:], beta.f64), eps)
+    g = blocks.layernorm_backward(ops, NT(dims[2:], gamma.f64), f, NT(dims, dy.f64))
+    lay = layout(mtf, [("all", 3)], [("batch", "all")])
+    xt, dyt, rt, gt, bt = to_torch(x), to_torch(dy), to_torch(res), to_torch(gamma), to_torch(beta)
+    y, dx = alloc(dims, "bf16"), alloc(dims, "bf16")
+    stats = torch.empty(3, 50, 2, dtype=torch.float32, device="cuda")
+    dg, db = alloc(dims[2:], "f32"), alloc(dims[2:], "f32")
+    N = mtf.named
+    mtf.mtf_layernorm_forward(lay, N(xt, names), N(gt, names[2:]), N(bt, names[2:]), eps, N(y, names), N(stats, ["batch", "length", "stat"]))
+    mtf.mtf_layernorm_backward(lay, N(dyt, names), N(xt, names), N(stats, ["batch", "length", "stat"]), N(gt, names[2:]), N(rt, names),
+                               N(dx, names), N(dg, names[2:]), N(db, names[2:]))
+    mtf.mtf_device_status()
+    assert parity_error(from_torch(y), f["y"].a) <= TOL["bf16"]
+    assert parity_error(from_torch(dx), g["dx"].a + res.f64) <= TOL["bf16"]
+    assert parity_error(from_torch(dg), g["dgamma"].a) <= 1e-3
+    assert parity_error(from_torch(db), g["dbeta"].a) <= 1e-3
+    st = from_torch(stats)
+    np.testing.assert_allclose(st[..., 0], x.f64.mean(-1), rtol=1e-4, atol=1e-5)
+    np.testing.assert_allclose(st[..., 1], 1.0 / np.sqrt(x.f64.var(-1) + eps), rtol=1e-4)
+
+
+# ---- attention ----------------------------------------------------------------------------------------------
+
+def attention_case(seed, B, L, D, H, K):
+    dims = {"x": [("batch", B), ("length", L), ("d_model", D)], "wq": [("d_model", D), ("heads", H), ("d_k", K)],
+            "wk": [("d_model", D), ("heads", H), ("d_k", K)], "wv": [("d_model", D), ("heads", H), ("d_v", K)],
+            "wo": [("heads", H), ("d_v", K), ("d_model", D)], "dy": [("batch", B), ("length", L), ("d_model", D)]}
+    scale = {"x": 1.0, "dy": 1.0, "wq": D ** -0.5, "wk": D ** -0.5, "wv": D ** -0.5, "wo": (H * K) ** -0.5}
+    return {k: (d, si.normal(seed, k, [s for _, s in d], "bf16", scale[k])) for k, d in dims.items()}
+
+
+def run_attention_oracle(inp, causal, store_dtype):
+    from oracle import NT, DenseOps, blocks, rounding
+    ops = DenseOps()
+    store = rounding.make_store(ops, store_dtype)
+    T = {k: NT(d, s.f64) for k, (d, s) in inp.items()}
+    L = T["x"].dims[1][1]
+    mask = blocks.causal_mask(L) if causal else None
+    f = blocks.attention_forward(ops, T["x"], T["wq"], T["wk"], T["wv"], T["wo"], mask, store)
+    g = blocks.attention_backward(ops, T["x"], T["wq"], T["wk"], T["wv"], T["wo"], f, T["dy"], store)
+    return {"y": f["y"].a, "P": f["P"].a, "o": f["o"].a, "q": f["q"].a, "dx": g["dx"].a, "dwq": g["dwq"].a, "dwk": g["dwk"].a,
+            "dwv": g["dwv"].a, "dwo": g["dwo"].a}
+
+
+def run_attention_gpu(mtf, lay, inp, causal):
+    import torch
+    dev = {k: to_torch(s) for k, (_, s) in inp.items()}
+    N = {k: mtf.named(dev[k], [n for n, _ in d]) for k, (d, _) in inp.items()}
+    (b, B), (l, L), (d, D) = inp["x"][0]
+    (_, _), (h, H), (k, K) = inp["wq"][0]
+    v = inp["wv"][0][2][0]
+    sd = {"q": [(b, B), (l, L), (h, H), (k, K)], "kk": [(b, B), ("memory_length", L), (h, H), (k, K)],
+          "vv": [(b, B), ("memory_length", L), (h, H), (v, K)], "P": [(b, B), (h, H), (l, L), ("memory_length", L)],
+          "o": [(b, B), (l, L), (h, H), (v, K)], "y": inp["x"][0], "dx": inp["x"][0]}
+    out = {n: alloc(dd, "bf16") for n, dd in sd.items()}
+    for n in ("wq", "wk", "wv", "wo"):
+        out["d" + n] = alloc(inp[n][0], "f32")
+        sd["d" + n] = inp[n][0]
+    O = {n: mtf.named(t, [x for x, _ in sd[n]]) for n, t in out.items()}
+    ws = torch.empty(mtf.mtf_attention_workspace_bytes(lay, N["x"], N["wq"], N["wv"]), dtype=torch.uint8, device="cuda")
+    mtf.mtf_attention_forward(lay, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], causal, None, O["q"], O["kk"], O["vv"], O["P"], O["o"], O["y"], ws)
+    mtf.mtf_attention_backward(lay, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], O["q"], O["kk"], O["vv"], O["P"], O["o"], N["dy"], None,
+                               O["dx"], O["dwq"], O["dwk"], O["dwv"], O["dwo"], ws)
+    mtf.mtf_device_status()
+    return {n: from_torch(t) for n, t in out.items()}
+
+
+@pytest.mark.parametrize("mesh_dims,rules", LAYOUTS)
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_block(mtf, mesh_dims, rules, causal):
+    # length 136 = one 128-row tile + 8; d_k = d_v = 64 as in the paper-sized configurations
+    inp = attention_case(13, 4, 136, 256, 4, 64)
+    got = run_attention_gpu(mtf, layout(mtf, mesh_dims, rules), inp, causal)
+    ref_s = run_attention_oracle(inp, causal, "bf16")      # intermediates kept in bf16 where the method stores them
+    ref_e = run_attention_oracle(inp, causal, None)        # exact mathematics
+    check_chain(got, ref_s, ref_e)
+    if causal:
+        iu = np.triu_indices(136, 1)
+        assert (got["P"][..., iu[0], iu[1]] == 0.0).all()
+
+
+def test_attention_small_head_dims(mtf):
+    inp = attention_case(14, 2, 40, 64, 2, 32)            # d_k = 32: half a k-block, N tiles of 64 half used
+    got = run_attention_gpu(mtf, layout(mtf, [("all", 2)], [("heads", "all")]), inp, True)
+    check_chain(got, run_attention_oracle(inp, True, "bf16"), run_attention_oracle(inp, True, None))
+
+
+# ---- decoder layer -------------------------------------------------------------------------------------------
+
+def decoder_case(seed, B, L, D, H, K, F):
+    inp = attention_case(seed, B, L, D, H, K)
+    inp["dout"] = inp.pop("dy")
+    inp["w"] = ([("d_model", D), ("d_ff", F)], si.normal(seed, "w", [D, F], "bf16", D ** -0.5))
+    inp["v"] = ([("d_ff", F), ("d_model", D)], si.normal(seed, "v", [F, D], "bf16", F ** -0.5))
+    inp["bias"] = ([("d_ff", F)], si.normal(seed, "bias", [F], "f32", 0.1))
+    for n, shift in (("ln1_gamma", 1.0), ("ln1_beta", 0.0), ("ln2_gamma", 1.0), ("ln2_beta", 0.0)):
+        inp[n] = ([("d_model", D)], si.normal(seed, n, [D], "f32", 0.1, shift))
+    return inp
+
+
+PARAMS = ["wq", "wk", "wv", "wo", "ln1_gamma", "ln1_beta", "w", "bias", "v", "ln2_gamma", "ln2_beta"]
+ORACLE_NAME = {"ln1_gamma": "g1", "ln1_beta": "b1", "ln2_gamma": "g2", "ln2_beta": "b2"}
+GRAD_OF = {"wq": "dwq", "wk": "dwk", "wv": "dwv", "wo": "dwo", "ln1_gamma": "dg1", "ln1_beta": "db1", "w": "dw", "bias": "dbias", "v": "dv",
+           "ln2_gamma": "dg2", "ln2_beta": "db2"}
+
+
+def run_decoder_oracle(inp, store_dtype):
+    from oracle import NT, DenseOps, blocks, rounding
+    ops = DenseOps()
+    store = rounding.make_store(ops, store_dtype)
+    T = {k: NT(d, s.f64) for k, (d, s) in inp.items()}
+    p = {ORACLE_NAME.get(k, k): T[k] for k in PARAMS}
+    mask = blocks.causal_mask(T["x"].dims[1][1])
+    f = blocks.decoder_layer_forward(ops, T["x"], p, mask, 1e-6, store)
+    g = blocks.decoder_layer_backward(ops, T["x"], p, f, T["dout"], store)
+    out = {"out": f["out"].a, "dx": g["dx"].a}
+    for k in PARAMS:
+        out["d_" + k] = g[GRAD_OF[k]].a
+    hp = f["ffn"]["hp"].a
+    return out, float(np.abs(hp).min() / np.sqrt(np.mean(hp * hp)))
+
+
+def run_decoder_gpu(mtf, lay, inp):
+    import torch
+    dev = {k: to_torch(s) for k, (_, s) in inp.items()}
+    N = {k: mtf.named(dev[k], [n for n, _ in d]) for k, (d, _) in inp.items()}
+    (b, B), (l, L), (d, D) = inp["x"][0]
+    (_, _), (h, H), (k, K) = inp["wq"][0]
+    F = inp["w"][0][1][1]
+    m = "memory_length"
+    sd = {"q": [(b, B), (l, L), (h, H), (k, K)], "kk": [(b, B), (m, L), (h, H), (k, K)], "vv": [(b, B), (m, L), (h, H), ("d_v", K)],
+          "weights": [(b, B), (h, H), (l, L), (m, L)], "o": [(b, B), (l, L), (h, H), ("d_v", K)], "s1": inp["x"][0], "a": inp["x"][0],
+          "h": [(b, B), (l, L), ("d_ff", F)], "s2": inp["x"][0]}
+    saved_t = {n: alloc(dd, "bf16") for n, dd in sd.items()}
+    saved = {n: mtf.named(t, [x for x, _ in sd[n]]) for n, t in saved_t.items()}
+    for n in ("stats1", "stats2"):
+        saved_t[n] = torch.empty(B, L, 2, dtype=torch.float32, device="cuda")
+        saved[n] = mtf.named(saved_t[n], [b, l, "stat"])
+    params = {k: N[k] for k in PARAMS}
+    out, dx = alloc(inp["x"][0], "bf16"), alloc(inp["x"][0], "bf16")
+    grads_t = {k: alloc(inp[k][0], "f32") for k in PARAMS}
+    gname = {"wq": "dwq", "wk": "dwk", "wv": "dwv", "wo": "dwo", "ln1_gamma": "dln1_gamma", "ln1_beta": "dln1_beta", "w": "dw", "bias": "dbias",
+             "v": "dv", "ln2_gamma": "dln2_gamma", "ln2_beta": "dln2_beta"}
+    grads = {gname[k]: mtf.named(t, [n for n, _ in inp[k][0]]) for k, t in grads_t.items()}
+    names = [n for n, _ in inp["x"][0]]
+    ws = torch.empty(mtf.mtf_decoder_layer_workspace_bytes(lay, N["x"], params), dtype=torch.uint8, device="cuda")
+    mtf.mtf_decoder_layer_forward(lay, N["x"], params, True, 1e-6, saved, mtf.named(out, names), ws)
+    mtf.mtf_decoder_layer_backward(lay, N["x"], params, saved, N["dout"], mtf.named(dx, names), grads, ws)
+    mtf.mtf_device_status()
+    res = {"out": from_torch(out), "dx": from_torch(dx)}
+    for k, t in grads_t.items():
+        res["d_" + k] = from_torch(t)
+    return res
+
+
+@pytest.mark.parametrize("mesh_dims,rules", LAYOUTS)
+def test_decoder_layer(mtf, mesh_dims, rules):
+    # pick a seed for which no relu decision is within fp32 accumulation noise of zero, so that every
+    # output is unique
+    for seed in range(15, 40):
+        inp = decoder_case(seed, 4, 72, 128, 4, 32, 320)
+        ref_s, margin = run_decoder_oracle(inp, "bf16")
+        if margin > 2e-5:
+            break
+    else:
+        pytest.fail("no seed with a clear relu margin")
+    got = run_decoder_gpu(mtf, layout(mtf, mesh_dims, rules), inp)
+    # Against exact mathematics only the rms is gated: the relu decisions of the exact and of the
+    # bf16-storing computation differ for a few hidden units (their inputs differ by the storage
+    # rounding of a), which moves single gradient entries by O(1), and the layer-norm backward
+    # amplifies the storage rounding of the gradient streams (the storing oracle itself is ~4e-2 rms away).
+    ref_e, _ = run_decoder_oracle(inp, None)
+    check_chain(got, ref_s, ref_e, elem_exact=float("inf"), rms_exact=6e-2)
