@@ -29,6 +29,7 @@ LAYOUTS = {
     "dp8": ([("all", 8)], [("batch", "all")]),
     "mp8": ([("all", 8)], [("d_ff", "all")]),
 }
+NCU_DRAM_BYTES_PER_LAUNCH = 234.6e6
 METRIC = "transformer_ffn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
@@ -264,7 +265,7 @@ def run_ours(args):
     value = world * flops_step / (ms_step * 1e-3) / 1e12
 
     per_layout = {}
-    if world == 1:
+    if world == 1 and not args.main_only:
         for name, lay in layouts.items():
             if name == args.layout:
                 per_layout[name] = value
@@ -272,6 +273,13 @@ def run_ours(args):
             ms_l, _, _ = timed(lay, max(args.steps // 2, 5), 3)
             per_layout[name] = flops_step / (ms_l * 1e-3) / 1e12
 
+    if args.main_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "ms_per_step": ms_step, "gpu_launches": launches,
+                              "config": {"workload": f"tokens={T} d_model={D} d_ff={F}", "layout": args.layout}, "note": "main-only run"}), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     # end to end: the step's inputs come from pinned host memory and its results go back, every step
     hx, hdy = t["x"].cpu().pin_memory(), t["dy"].cpu().pin_memory()
     hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
@@ -315,13 +323,9 @@ def run_ours(args):
     flops_per_launch = flops_step / gemm_launches_per_step
     avg_launch_ms = ms_step / gemm_launches_per_step        # includes launch gaps: a lower bound on the rate
     achieved = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12
-    traffic = None
-    tp = os.path.join(ROOT, "profiles", "ncu_traffic.json")
-    if os.path.exists(tp):
-        try:
-            traffic = json.load(open(tp)).get("gemm_tcgen05_kernel_bytes_per_launch")
-        except Exception:
-            traffic = None
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the six launches of a step,
+    # from the full-size ncu capture summarised in profiles/gemm_tcgen05_ffn_target_fullsize.md
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH if (T, D, F) == (8192, 1024, 8192) else None
     roofline = {"bound": "tensor", "kernel": "gemm_tcgen05_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
                 "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "frac_of_datasheet_2250": achieved / 2250.0,
@@ -360,7 +364,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="mp8", choices=sorted(LAYOUTS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=WORKLOAD["batch"], help="sequences of 256 tokens per GPU (smaller only for profiler captures)")
+    ap.add_argument("--main-only", action="store_true", help="skip the per-layout table and the end-to-end leg (profiler captures)")
     args = ap.parse_args()
+    WORKLOAD["batch"] = args.batch
     if args.impl == "reference":
         run_reference(args)
     else:
