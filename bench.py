@@ -184,6 +184,7 @@ def run_ours(args):
         dist = dist_mod
         dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
     import paper_1811_02084_b200 as mtf
+    from paper_1811_02084_b200 import multi_gpu
 
     B, L, D, F = WORKLOAD["batch"], WORKLOAD["length"], WORKLOAD["d_model"], WORKLOAD["d_ff"]
     T = B * L
@@ -223,12 +224,9 @@ def run_ours(args):
     def step(lay):
         mtf.mtf_ffn_forward(lay, N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
         mtf.mtf_ffn_backward(lay, N["x"], N["w"], N["v"], N["h"], N["dy"], N["dx"], N["dw"], N["dbias"], N["dv"], ws)
-        if dist is not None:
-            # Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs sums the
-            # parameter gradients across ranks
-            dist.all_reduce(dw)
-            dist.all_reduce(dv)
-            dist.all_reduce(dbias)
+        # Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs sums the
+        # parameter gradients across ranks (no-op on one GPU)
+        multi_gpu.allreduce_gradients(dist, (dw, dv, dbias))
 
     def timed(lay, steps, warmup, sampler=None):
         for _ in range(warmup):
@@ -252,10 +250,7 @@ def run_ours(args):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1)
         launches = mtf.mtf_launch_count() - n0
-        if dist is not None:
-            tm = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            ms = float(tm.item())
+        ms = multi_gpu.max_over_ranks(dist, ms, "cuda")
         return ms / steps, launches, clocks
 
     flops_step = ffn_flops(T, D, F)
@@ -305,10 +300,7 @@ def run_ours(args):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if dist is not None:
-        tm = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tm.item())
+    e2e_ms = multi_gpu.max_over_ranks(dist, e2e_ms, "cuda")
     e2e_value = world * flops_step / (e2e_ms * 1e-3) / 1e12
     act_bytes = hx.numel() * hx.element_size()
 
