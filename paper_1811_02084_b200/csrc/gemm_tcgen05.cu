@@ -480,6 +480,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (kPair) cluster_sync();      // the partner's barriers must exist before anything signals them
   tcgen05_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: everything above (barriers, TMEM, tensor-map prefetch) may overlap
+  // the tail of the previous kernel on the stream; nothing below touches global memory before that
+  // kernel has completed.  The next kernel on the stream may start its own set-up right away.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const bool ws_mode = a.reduce_mode == MTF_REDUCE_WORKSPACE;
   const int kb_per_slice = a.Ks / BK;
@@ -939,16 +944,25 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (t.cta_pair) {
     const long long pairs = std::min<long long>(a.total_work, max_pairs);
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up may overlap the previous kernel's tail
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
+    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 2;
     cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<true>, map_a, map_b, map_c, map_m, a);
     if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<pair>: %s", cudaGetErrorString(le));
   } else {
     const long long grid = std::min<long long>(a.total_work, sm_count());
-    gemm_tcgen05_kernel<false><<<(unsigned)grid, kThreads, kSmemBytes, st>>>(map_a, map_b, map_c, map_m, a);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
+    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<false>, map_a, map_b, map_c, map_m, a);
+    if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(le));
   }
   count_launch();
   cudaError_t e = cudaGetLastError();
