@@ -31,8 +31,8 @@ constexpr int BK = 64;
 constexpr int kMaxBN = 256;
 constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
 constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stages half of it)
-constexpr int kRingBytes = 4 * (kAStageBytes + kBStageBytes);   // = 6 * (16 KB + 16 KB) = 192 KB
-constexpr int kStagingBytes = kEpilogueWarps * 4096;   // per epilogue warp: one 32-row x 128-byte box for TMA stores
+constexpr int kRingBytes = 5 * (kAStageBytes + kBStageBytes / 2);   // pairs: 5 x (16 KB + 16 KB); single CTAs: 3 x 48 KB fit too
+constexpr int kStagingBytes = kEpilogueWarps * 2 * 4096;   // per epilogue warp: two 32-row x 128-byte boxes for TMA stores
 constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr int kThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kTmemCols = 512;
@@ -428,7 +428,7 @@ template <bool kPair>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m, const TcArgs a) {
-  constexpr int kStages = kPair ? 6 : 4;
+  constexpr int kStages = kPair ? 5 : 3;
   constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kTileRows = kPair ? 2 * BM : BM;       // rows of C owned by a work item
   extern __shared__ uint8_t smem_raw[];
@@ -445,8 +445,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
   auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
-  // then [2S+4..2S+12): per epilogue warp one barrier for relu-mask boxes loaded into its staging buffer
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
+  // then [2S+4..2S+20): per epilogue warp two barriers for relu-mask boxes loaded into its staging buffers
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4 + 2 * kEpilogueWarps);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -459,7 +459,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), (kPair ? 2 : 1) * kEpilogueWarps); }
-    for (int i = 0; i < kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
+    for (int i = 0; i < 2 * kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -570,9 +570,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------- epilogue -----------------------------------
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     const int col_half = (warp - 2) >> 2;          // which of the two warps of this lane quarter
-    const uint32_t box = staging_base + (uint32_t)(warp - 2) * 4096u;
-    uint32_t mask_phase = 0;                       // phase of this warp's mask barrier
-    const uint32_t mfull_bar = bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2));
+    const uint32_t stg = staging_base + (uint32_t)(warp - 2) * 8192u;      // this warp's two staging boxes
+    uint32_t buf = 0;                              // staging box the next output box goes through
+    uint32_t mask_phase = 0;                       // bit b: phase of this warp's mask barrier b
+    auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
     int iter = 0;
     bool ok = true;
     for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
@@ -599,9 +600,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const bool rows_full = row0 + 32 <= tl.m_end;
       const bool mask_tma = a.mask_tma != 0 && !ws_mode && rows_full;
       if (mask_tma && lane == 0) {
-        // pull this warp's boxes of the mask tile towards L2
+        // pull this warp's boxes of the mask tile towards L2 and request the first one into the
+        // staging box it will be processed in (free once all but the latest store have been read out)
         for (int b = col_half * 64; b < a.block_n; b += 128)
           if (tl.n0 + b + 64 <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
+        if (col_half * 64 < a.block_n && tl.n0 + col_half * 64 + 64 <= tl.n_end) {
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          mbar_expect_tx(mfull_bar(buf), 4096u);
+          tma_load_5d<false>(stg + buf * 4096u, &map_m, mfull_bar(buf), tl.n0 + col_half * 64, row0, tl.o[2], tl.o[1], tl.o[0]);
+        }
       }
       ok = mbar_wait_warp(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag, lane);
       ok = __all_sync(0xffffffffu, ok);
@@ -626,18 +633,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const int box_n0 = tl.n0 + (c0 & ~(box_cols - 1));
           const bool staged = rows_full && box_n0 + box_cols <= tl.n_end;
           const int half = (c0 >> 5) & 1;
-          if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box: the buffer must be free
-            if (lane == 0) {
-              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-              if (mask_tma) {                                   // the box's relu mask arrives in place
-                mbar_expect_tx(mfull_bar, 4096u);
-                tma_load_5d<false>(box, &map_m, mfull_bar, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
-              }
-            }
-            __syncwarp();
-            if (mask_tma) {
-              mbar_wait(mfull_bar, mask_phase, 0x500, abort_flag);
-              mask_phase ^= 1u;
+          const uint32_t box = stg + buf * 4096u;
+          if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box
+            if (mask_tma) {                                     // its relu mask was requested a box ago, in place
+              mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag);
+              mask_phase ^= 1u << buf;
+            } else {                                            // the box must be free: all but the latest store read out
+              if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+              __syncwarp();
             }
           }
           uint4 mk[4];
@@ -662,7 +665,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+            if (lane == 0) {
+              tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+              // request the mask of this warp's next box of the tile into the other staging box
+              const int next_n0 = box_n0 + 2 * box_cols;
+              if (mask_tma && next_n0 < tl.n0 + a.block_n && next_n0 + box_cols <= tl.n_end) {
+                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
+                tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+              }
+            }
+            buf ^= 1u;
           }
           if (a.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
 #pragma unroll
