@@ -11,7 +11,10 @@ import os
 from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_int64, c_size_t, c_uint32, c_void_p
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmtf_b200.so")
+_BASE_LIB = os.path.join(_HERE, "libmtf_b200.so")
+_MC_LIB = os.path.join(_HERE, "libmtf_b200_mc.so")     # optional single-GPU build with cluster-multicast operand loads
+_multi_rank = int(os.environ.get("WORLD_SIZE", "1")) > 1
+LIB_PATH = _MC_LIB if (os.path.exists(_MC_LIB) and not _multi_rank and not os.environ.get("MTF_NO_MULTICAST")) else _BASE_LIB
 
 MTF_F32, MTF_BF16 = 0, 1
 MTF_KERNEL_SIMT, MTF_KERNEL_TCGEN05 = 0, 1

@@ -23,6 +23,11 @@
 
 #include "mtf_internal.h"
 
+// Cluster-multicast operand loads exist only in the optional single-GPU build (see tma_multicast.cuh).
+#if defined(MTF_TMA_MULTICAST)
+#include "tma_multicast.cuh"
+#endif
+
 namespace {
 
 constexpr int BM = 128;
@@ -78,7 +83,7 @@ struct Tile {
   long long c_off;         // element offset of the outer coordinates in C
 };
 
-__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int tile_rows) {
+__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int tile_rows, int tile_cols) {
   Tile r;
   long long slice = t / a.tiles_per_slice;
   long long w = t % a.tiles_per_slice;
@@ -98,7 +103,7 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int ti
   }
   r.m0 = im * a.Ms + mt * tile_rows;
   r.m_end = (im + 1) * a.Ms;
-  r.n0 = in * a.Ns + nt * a.block_n;
+  r.n0 = in * a.Ns + nt * tile_cols;
   r.n_end = (in + 1) * a.Ns;
   return r;
 }
@@ -190,13 +195,13 @@ __device__ __forceinline__ void cluster_sync() {
 
 // Arrive on the barrier at the same offset in the even CTA of the pair (own barrier when !kPair).
 template <bool kPair>
-__device__ __forceinline__ void mbar_arrive_pair(uint32_t bar) {
+__device__ __forceinline__ void mbar_arrive_pair(uint32_t bar, uint32_t leader_rank) {
   if (kPair)
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
-        "mapa.shared::cluster.u32 ra, %0, 0;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
         "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
-        ::"r"(bar) : "memory");
+        ::"r"(bar), "r"(leader_rank) : "memory");
   else
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -224,11 +229,10 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_c, uint64_t desc_a, uint
 // Arrives on `bar` when every MMA issued so far has retired; for a pair, on the barrier at that
 // offset in both CTAs (completion multicast, not a load).
 template <bool kPair>
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
+__device__ __forceinline__ void umma_commit(uint32_t bar, uint16_t cta_mask) {
   if (kPair) {
-    const uint16_t both = 3;
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(both) : "memory");
+                 ::"r"(bar), "h"(cta_mask) : "memory");
   } else {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
   }
@@ -424,13 +428,24 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 //   The loads of both CTAs report to the even CTA's "full" barrier; MMA completion is multicast to
 //   both CTAs' "empty" and "accumulator full" barriers; the epilogue warps of both CTAs report to
 //   the even CTA's "accumulator empty" barrier.  No load uses cluster multicast.
-template <bool kPair>
+//
+// CM x CN > 1 (optional single-GPU build only): a cluster of CM x CN CTA pairs owns a (CM * 256) x
+// (CN * block_n) super-tile.  Pairs in one row of the cluster need the same rows of A, pairs in one
+// column the same columns of B; each CTA loads only its 1/CN share of its A rows and its 1/CM share
+// of its B columns and the load writes it into every CTA that needs it, so a CTA pulls
+// 16 KB / CN + 16 KB / CM per k-block through L2 instead of 32 KB.  A stage may be refilled when
+// every pair that reads what this CTA writes has retired its MMAs: CM + CN - 1 pair leaders signal
+// each CTA's "empty" barrier.
+template <bool kPair, int CM, int CN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m, const TcArgs a) {
   constexpr int kStages = kPair ? 5 : 3;
   constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
-  constexpr int kTileRows = kPair ? 2 * BM : BM;       // rows of C owned by a work item
+  constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
+  constexpr int kTileRows = kPairRows * CM;            // rows of C owned by a work item
+  constexpr bool kCluster = CM * CN > 1;
+  static_assert(!kCluster || kPair, "clusters of pairs only");
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte aligned tile ring (the 128B swizzle pattern repeats every 1024 B)
   const uint32_t raw = smem_u32(smem_raw);
@@ -451,13 +466,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int cta_rank = kPair ? (int)(blockIdx.x & 1u) : 0;     // position in the CTA pair
+  constexpr int kClusterCtas = (kPair ? 2 : 1) * CM * CN;
+  const int cluster_rank = (int)(blockIdx.x % kClusterCtas);   // 1-D clusters: rank = position in the cluster
+  const int cta_rank = kPair ? (cluster_rank & 1) : 0;         // position in the CTA pair
+  const int pair_idx = cluster_rank >> 1;                      // which pair of the cluster
+  const int pm = pair_idx / CN, pn = pair_idx % CN;            // the pair's row / column in the cluster
   const bool leader = cta_rank == 0;
-  const long long work_first = kPair ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
-  const long long work_step = kPair ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
+  const long long work_first = (long long)(blockIdx.x / kClusterCtas);
+  const long long work_step = (long long)(gridDim.x / kClusterCtas);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), CM + CN - 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), (kPair ? 2 : 1) * kEpilogueWarps); }
     for (int i = 0; i < 2 * kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
     *abort_flag = 0;
@@ -502,9 +521,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       for (long long work = work_first; ok && work < a.total_work; work += work_step) {
         const long long t = ws_mode ? work / a.sk : work;
         const int kb_first = ws_mode ? (int)(work % a.sk) * kb_per_slice : 0;
-        const Tile tl = decode_tile(a, t, kTileRows);
-        const int m0 = tl.m0 + cta_rank * BM;
-        const int n0 = tl.n0 + cta_rank * n_local;
+        const Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
+        const int m0 = tl.m0 + pm * kPairRows + cta_rank * BM;
+        const int n0 = tl.n0 + pn * a.block_n + cta_rank * n_local;
         for (int kb = 0; kb < kb_count; ++kb) {
           // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
           // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor)
@@ -516,12 +535,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const uint32_t fb = kPair ? (full_bar(stage) & 0xFEFFFFFFu) : full_bar(stage);
           const uint32_t sa = tiles_base + stage * kStageBytes;
           const uint32_t sb = sa + kAStageBytes;
+#if defined(MTF_TMA_MULTICAST)
+          if (CN > 1) {
+            // this CTA's 1/CN share of its 128 rows of A goes to the same-position CTA of every pair in its cluster row
+            uint16_t mask = 0;
+            for (int j = 0; j < CN; ++j) mask |= (uint16_t)(1u << (2 * (pm * CN + j) + cta_rank));
+            if (a.a_mn_major) tma_load_5d_multicast(sa + 8192u * pn, &map_a, fb, mask, m0 + 64 * pn, k0, tl.o[2], tl.o[1], tl.o[0]);
+            else tma_load_5d_multicast(sa + (uint32_t)(pn * (BM / CN)) * 128u, &map_a, fb, mask, k0, m0 + pn * (BM / CN), tl.o[2], tl.o[1], tl.o[0]);
+          } else
+#endif
           if (a.a_mn_major) {
             tma_load_5d<kPair>(sa, &map_a, fb, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
             tma_load_5d<kPair>(sa + 8192, &map_a, fb, m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
             tma_load_5d<kPair>(sa, &map_a, fb, k0, m0, tl.o[2], tl.o[1], tl.o[0]);
           }
+#if defined(MTF_TMA_MULTICAST)
+          if (CM > 1) {
+            // this CTA's 1/CM share of its half of B's columns goes to the same-position CTA of every pair in its cluster column
+            uint16_t mask = 0;
+            for (int j = 0; j < CM; ++j) mask |= (uint16_t)(1u << (2 * (j * CN + pn) + cta_rank));
+            if (a.b_mn_major) tma_load_5d_multicast(sb + 8192u * pm, &map_b, fb, mask, n0 + 64 * pm, k0, tl.o[2], tl.o[1], tl.o[0]);
+            else tma_load_5d_multicast(sb + (uint32_t)(pm * (n_local / CM)) * 128u, &map_b, fb, mask, k0, n0 + pm * (n_local / CM), tl.o[2], tl.o[1], tl.o[0]);
+          } else
+#endif
           if (a.b_mn_major) {
             for (int j = 0; j < n_local / 64; ++j)
               tma_load_5d<kPair>(sb + 8192 * j, &map_b, fb, n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
@@ -536,7 +573,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------- MMA issuer (even CTA of a pair only) -------
     if (lane == 0 && leader) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.a_mn_major << 15) |
-                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+      // completion signals: this pair's two CTAs, and every CTA whose loads land in this pair's tiles
+      // (the pairs of this pair's cluster row and column)
+      const uint16_t pair_mask = (uint16_t)(3u << (2 * pair_idx));
+      uint16_t empty_mask = 0;
+      for (int i = 0; i < CM; ++i)
+        for (int j = 0; j < CN; ++j)
+          if (i == pm || j == pn) empty_mask |= (uint16_t)(3u << (2 * (i * CN + j)));
       const uint32_t a_kstep = a.a_mn_major ? 2048u : 32u;   // bytes per 16 k-elements
       const uint32_t b_kstep = a.b_mn_major ? 2048u : 32u;
       int stage = 0;
@@ -560,10 +604,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const uint64_t db = make_smem_desc(sb + k * b_kstep, a.b_mn_major);
             umma_bf16<kPair>(tmem_c, da, db, idesc, (kb | k) != 0);
           }
-          umma_commit<kPair>(empty_bar(stage));    // frees the smem stage (of both CTAs) when these MMAs retire
+          umma_commit<kPair>(empty_bar(stage), empty_mask);   // frees the stage in every CTA that writes into this pair's tiles
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit<kPair>(tfull_bar(acc)); // accumulator complete (in both CTAs)
+        if (ok) umma_commit<kPair>(tfull_bar(acc), pair_mask);   // accumulator complete (in both CTAs of the pair)
       }
     }
   } else {
@@ -579,7 +623,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
       const long long t = ws_mode ? work / a.sk : work;
       const int ks = ws_mode ? (int)(work % a.sk) : 0;
-      const Tile tl = decode_tile(a, t, kTileRows);
+      Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
+      tl.m0 += pm * kPairRows;            // this pair's 256 x block_n part of the cluster's super-tile
+      tl.n0 += pn * a.block_n;
       const int acc = iter & 1;
       const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
       const int tile_row = cta_rank * BM + q * 32 + lane;       // row inside the work item's tile
@@ -686,7 +732,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc));
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
       } else {
         // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
         // (the two warps of a lane quarter split the columns in halves, each with its own counter)
@@ -704,7 +750,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc));
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
         __threadfence();
         __syncwarp();
         unsigned old = 0;
@@ -840,6 +886,46 @@ int sm_count() {
   return n;
 }
 
+// One kernel variant: shared-memory opt-in and the number of clusters that can be resident at once
+// are looked up on first use; the grid is that many clusters (persistent) or fewer.
+template <bool kPair, int CM, int CN>
+mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
+                          const TcArgs& a, cudaStream_t st) {
+  constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  static int max_clusters = 0;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (attr_err != cudaSuccess) return;
+    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (attr_err != cudaSuccess) return;
+    if (kCtas == 1) { max_clusters = sm_count(); return; }
+    cudaLaunchConfig_t q = {};
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kCtas; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    q.gridDim = dim3(kCtas * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
+    q.attrs = at; q.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN>, &q) == cudaSuccess && n > 0) max_clusters = n;
+    else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
+  });
+  if (attr_err != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
+  const long long clusters = std::min<long long>(a.total_work, max_clusters);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up may overlap the previous kernel's tail
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = kCtas; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
+  cfg.gridDim = dim3((unsigned)(kCtas * clusters), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = kCtas > 1 ? 2 : 1;
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN>, map_a, map_b, map_c, map_m, a);
+  if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d>: %s", (int)kPair, CM, CN, cudaGetErrorString(le));
+  return MTF_OK;
+}
+
 }  // namespace
 
 namespace mtf {
@@ -885,9 +971,22 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.ldc = t.ldc;
   a.reduce_mode = t.reduce_mode;
   a.k_sliced = (t.sk > 1 && a.Ks % BK == 0) ? 1 : 0;
-  const int tile_rows = tc_tile_rows(t);
+  // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads
+  int cm = 1, cn = 1;
+#if defined(MTF_TMA_MULTICAST)
+  if (t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
+    // measured on the FFN shapes: sharing B between two pairs that are neighbours along M is worth
+    // 5-10 % on the contractions whose epilogue is light; with a relu mask or a fused reduction in the
+    // epilogue the coupling of the two pairs costs more than the saved traffic; 2 x 2 clusters lose
+    if (!mask && !rsum) {
+      if (a.Ms % 512 == 0) cm = 2;
+      else if (a.Ns % 512 == 0) cn = 2;
+    }
+  }
+#endif
+  const int tile_rows = tc_tile_rows(t) * cm;
   a.m_tiles = (a.Ms + tile_rows - 1) / tile_rows;
-  a.n_tiles = (a.Ns + a.block_n - 1) / a.block_n;
+  a.n_tiles = (a.Ns + a.block_n * cn - 1) / (a.block_n * cn);
   a.n_fastest = 0;   // m tiles of one n tile run together: they share the B tile, which measured fastest
   a.tiles_per_slice = (long long)a.m_tiles * a.n_tiles;
   for (int j = 0; j < a.n_outer; ++j) a.tiles_per_slice *= a.outer_local[j];
@@ -924,8 +1023,9 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   CUtensorMap map_a, map_b, map_c, map_m;
   mtf_status s;
   // operands: K-major = (K contiguous, M|N rows), box 64 x rows;  MN-major = (M|N contiguous, K rows), box 64 x 64
-  const int b_rows = t.cta_pair ? t.block_n / 2 : t.block_n;
-  s = t.a_mn_major ? make_map(&map_a, A, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&map_a, A, 2, t.K, t.M, t.a_ld, 64, BM, t, t.outer_sA);
+  // (a CTA of a multicast cluster loads 1/cn of its A rows and 1/cm of its B columns per box)
+  const int b_rows = (t.cta_pair ? t.block_n / 2 : t.block_n) / cm;
+  s = t.a_mn_major ? make_map(&map_a, A, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&map_a, A, 2, t.K, t.M, t.a_ld, 64, BM / cn, t, t.outer_sA);
   if (s != MTF_OK) return s;
   s = t.b_mn_major ? make_map(&map_b, B, 2, t.N, t.K, t.b_ld, 64, BK, t, t.outer_sB) : make_map(&map_b, B, 2, t.K, t.N, t.b_ld, 64, b_rows, t, t.outer_sB);
   if (s != MTF_OK) return s;
@@ -935,48 +1035,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   map_m = map_c;
   if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
 
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  static int max_pairs = 0;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (attr_err == cudaSuccess) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (attr_err != cudaSuccess) return;
-    // how many CTA pairs can be resident at once (one CTA per SM; a pair shares a TPC)
-    cudaLaunchConfig_t q = {};
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    q.gridDim = dim3(2 * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
-    q.attrs = at; q.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<true>, &q) == cudaSuccess && n > 0) max_pairs = n;
-    else { max_pairs = sm_count() / 2; (void)cudaGetLastError(); }
-  });
-  if (attr_err != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
-  if (t.cta_pair) {
-    const long long pairs = std::min<long long>(a.total_work, max_pairs);
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute at[2];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up may overlap the previous kernel's tail
-    at[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 2;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<true>, map_a, map_b, map_c, map_m, a);
-    if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<pair>: %s", cudaGetErrorString(le));
-  } else {
-    const long long grid = std::min<long long>(a.total_work, sm_count());
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3((unsigned)grid, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
-    cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<false>, map_a, map_b, map_c, map_m, a);
-    if (le != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(le));
-  }
+  mtf_status ls;
+  if (!t.cta_pair) ls = launch_variant<false, 1, 1>(map_a, map_b, map_c, map_m, a, st);
+#if defined(MTF_TMA_MULTICAST)
+  else if (cm == 1 && cn == 2) ls = launch_variant<true, 1, 2>(map_a, map_b, map_c, map_m, a, st);
+  else if (cm == 2 && cn == 1) ls = launch_variant<true, 2, 1>(map_a, map_b, map_c, map_m, a, st);
+#endif
+  else ls = launch_variant<true, 1, 1>(map_a, map_b, map_c, map_m, a, st);
+  if (ls != MTF_OK) return ls;
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(e));
