@@ -61,6 +61,9 @@ struct TcArgs {
   int m_tiles, n_tiles;    // per slice
   int n_fastest;           // tile order inside a slice: 1 = walk the n tiles of one m tile first
   long long tiles_per_slice, total_tiles, total_work;
+  int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
+  int kb_tile;             // k-blocks of one whole tile
+  int slots;               // partial-tile slots per tile in the workspace (sk, or 2 when balanced)
   void* C;
   int c_bf16;
   const void* bias;
@@ -107,6 +110,64 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int ti
   r.n_end = (in + 1) * a.Ns;
   return r;
 }
+
+// One piece of work for a worker (a CTA, a pair, or a cluster of pairs): k-blocks [kb_begin,
+// kb_begin + kb_count) of one output tile.  nfrag > 1: the tile is shared by nfrag workers; this is
+// fragment `frag`, it leaves through the workspace and whoever arrives last adds the fragments in order.
+struct Seg {
+  long long tile;
+  int kb_begin, kb_count, frag, nfrag;
+};
+
+// The sequence of segments of worker `w` of `W`.  Three schedules:
+//   whole tiles, round robin (tile = w, w + W, ...);
+//   WORKSPACE reduce mode: (tile, slice of the reduce group) pairs, round robin;
+//   balanced: the (tile, k-block) units are numbered tile-major and cut into W equal contiguous
+//   ranges, so that a last, partly filled wave of tiles does not leave SMs idle.  A tile that
+//   straddles a range boundary becomes two fragments.
+struct SegIter {
+  const TcArgs& a;
+  long long w, W, work, u, u_end, total_units;
+  int kb_per_slice;
+  __device__ SegIter(const TcArgs& args, long long worker, long long workers) : a(args), w(worker), W(workers), work(worker) {
+    kb_per_slice = a.Ks / BK;
+    total_units = a.total_tiles * a.kb_tile;
+    u = a.balanced ? (w * total_units) / W : 0;
+    u_end = a.balanced ? ((w + 1) * total_units) / W : 0;
+  }
+  __device__ long long owner(long long unit) const { return ((unit + 1) * W - 1) / total_units; }
+  __device__ bool next(Seg& s) {
+    if (a.balanced) {
+      if (u >= u_end) return false;
+      s.tile = u / a.kb_tile;
+      s.kb_begin = (int)(u - s.tile * a.kb_tile);
+      const long long tile_end = (s.tile + 1) * a.kb_tile;
+      const long long e = u_end < tile_end ? u_end : tile_end;
+      s.kb_count = (int)(e - u);
+      const long long first = owner(s.tile * a.kb_tile), last = owner(tile_end - 1);
+      s.nfrag = (int)(last - first + 1);
+      s.frag = (int)(w - first);
+      u = e;
+      return true;
+    }
+    if (work >= a.total_work) return false;
+    if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
+      s.tile = work / a.sk;
+      s.frag = (int)(work % a.sk);
+      s.nfrag = a.sk;
+      s.kb_begin = s.frag * kb_per_slice;
+      s.kb_count = kb_per_slice;
+    } else {
+      s.tile = work;
+      s.frag = 0;
+      s.nfrag = 1;
+      s.kb_begin = 0;
+      s.kb_count = a.kb_tile;
+    }
+    work += W;
+    return true;
+  }
+};
 
 // ---- PTX wrappers -----------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -505,10 +566,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  const bool ws_mode = a.reduce_mode == MTF_REDUCE_WORKSPACE;
-  const int kb_per_slice = a.Ks / BK;
-  const int kb_total = a.k_sliced ? a.sk * kb_per_slice : (a.K + BK - 1) / BK;
-  const int kb_count = ws_mode ? kb_per_slice : kb_total;
   const int n_local = kPair ? a.block_n / 2 : a.block_n;       // N columns of B this CTA stages
   const uint32_t b_bytes = (uint32_t)n_local * BK * 2;
 
@@ -518,10 +575,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (long long work = work_first; ok && work < a.total_work; work += work_step) {
-        const long long t = ws_mode ? work / a.sk : work;
-        const int kb_first = ws_mode ? (int)(work % a.sk) * kb_per_slice : 0;
-        const Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
+      SegIter it(a, work_first, work_step);
+      Seg sg;
+      while (ok && it.next(sg)) {
+        const int kb_first = sg.kb_begin, kb_count = sg.kb_count;
+        const Tile tl = decode_tile(a, sg.tile, kTileRows, a.block_n * CN);
         const int m0 = tl.m0 + pm * kPairRows + cta_rank * BM;
         const int n0 = tl.n0 + pn * a.block_n + cta_rank * n_local;
         for (int kb = 0; kb < kb_count; ++kb) {
@@ -587,7 +645,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t phase = 0;
       int iter = 0;
       bool ok = true;
-      for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
+      SegIter it(a, work_first, work_step);
+      Seg sg;
+      for (; ok && it.next(sg); ++iter) {
+        const int kb_count = sg.kb_count;
         const int acc = iter & 1;
         const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
         if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, 0x200 + acc, abort_flag))) break;
@@ -620,16 +681,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
     int iter = 0;
     bool ok = true;
-    for (long long work = work_first; ok && work < a.total_work; work += work_step, ++iter) {
-      const long long t = ws_mode ? work / a.sk : work;
-      const int ks = ws_mode ? (int)(work % a.sk) : 0;
+    SegIter it(a, work_first, work_step);
+    Seg sg;
+    for (; ok && it.next(sg); ++iter) {
+      const long long t = sg.tile;
+      const int ks = sg.frag;
+      const bool ws_mode = sg.nfrag > 1;       // this tile is assembled from fragments in the workspace
       Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
       tl.m0 += pm * kPairRows;            // this pair's 256 x block_n part of the cluster's super-tile
       tl.n0 += pn * a.block_n;
       const int acc = iter & 1;
       const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
-      const int tile_row = cta_rank * BM + q * 32 + lane;       // row inside the work item's tile
-      const int row = tl.m0 + tile_row;
+      const int pair_row = cta_rank * BM + q * 32 + lane;       // row inside the pair's part of the tile
+      const int tile_row = pm * kPairRows + pair_row;            // row inside the work item's tile
+      const int row = tl.m0 + pair_row;
       const bool row_ok = row < tl.m_end;
       const long long row_off = tl.c_off + (long long)row * a.ldc;
       // what the epilogue needs from memory is requested before the accumulator is waited for:
@@ -737,7 +802,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
         // (the two warps of a lane quarter split the columns in halves, each with its own counter)
         const int ws_c_begin = col_half * (a.block_n / 2), ws_c_end = ws_c_begin + a.block_n / 2;
-        float* part = a.ws_partials + ((size_t)(t * a.sk + ks) * kTileRows + (size_t)tile_row) * a.block_n;
+        float* part = a.ws_partials + ((size_t)(t * a.slots + ks) * kTileRows + (size_t)tile_row) * a.block_n;
         for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
@@ -754,11 +819,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __threadfence();
         __syncwarp();
         unsigned old = 0;
-        if (lane == 0) old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + cta_rank * 4 + q) * 2 + col_half], 1u);
+        if (lane == 0) old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + tile_row / 32) * 2 + col_half], 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
-        if (old == (unsigned)a.sk - 1) {
+        if (old == (unsigned)sg.nfrag - 1) {
           __threadfence();
-          const float* p0 = a.ws_partials + ((size_t)(t * a.sk) * kTileRows + (size_t)tile_row) * a.block_n;
+          const float* p0 = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)tile_row) * a.block_n;
 #pragma unroll 1
           for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
             const int n_first = tl.n0 + c0;
@@ -769,7 +834,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = 0.f;
             if (live) {
-              for (int s = 0; s < a.sk; ++s) {     // ascending processor order within the group
+              for (int s = 0; s < sg.nfrag; ++s) {     // ascending order of the fragments (= of the processors of the group)
                 const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * kTileRows * a.block_n + c0);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -912,7 +977,8 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
   });
   if (attr_err != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
-  const long long clusters = std::min<long long>(a.total_work, max_clusters);
+  // balanced schedule: every resident cluster takes an equal share of the k-block units
+  const long long clusters = a.balanced ? std::min<long long>(a.total_tiles, max_clusters) : std::min<long long>(a.total_work, max_clusters);
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set-up may overlap the previous kernel's tail
@@ -940,7 +1006,13 @@ static int64_t tc_total_tiles(const TcParams& t) {
 }
 
 size_t tc_workspace_bytes(const TcParams& t) {
-  if (t.reduce_mode != MTF_REDUCE_WORKSPACE) return 0;
+  if (t.reduce_mode != MTF_REDUCE_WORKSPACE) {
+    if (!t.balance) return 0;
+    // two fp32 fragments per tile plus counters, for tiles of up to 512 rows (upper bound over the tile shapes)
+    int64_t area = ((t.M / t.sm + 511) / 512 * 512) * t.sm * (((t.N / t.sn + t.block_n - 1) / t.block_n) * t.block_n) * t.sn;
+    for (int j = 0; j < t.n_outer; ++j) area *= t.outer_size[j];
+    return (size_t)area * 2 * sizeof(float) + (size_t)(area / (32 * 64)) * 2 * sizeof(unsigned) + 1024;
+  }
   const int64_t tiles = tc_total_tiles(t);
   return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * 2 * sizeof(unsigned) + 256;
 }
@@ -1002,9 +1074,29 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
   a.ws_partials = nullptr; a.ws_counters = nullptr;
+  a.kb_tile = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
+  a.slots = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.sk : 2;
+  a.balanced = 0;
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
+  if (t.balance && cn == 1 && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+    // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
+    // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
+    // the workspace by whichever worker finishes last (arrive, never wait).
+    const long long workers = sm_count() / ((t.cta_pair ? 2 : 1) * cm);
+    const long long rounds = (a.total_tiles + workers - 1) / workers;
+    const bool worth = a.total_tiles >= workers && (double)a.total_tiles / (double)(rounds * workers) <= 0.92;
+    const size_t part_bytes = (size_t)a.total_tiles * 2 * tile_rows * a.block_n * sizeof(float);
+    const size_t cnt_bytes = (size_t)a.total_tiles * (tile_rows / 32) * 2 * sizeof(unsigned);
+    if (worth && workspace_bytes >= ((part_bytes + 255) / 256) * 256 + cnt_bytes) {
+      a.balanced = 1;
+      a.ws_partials = reinterpret_cast<float*>(workspace);
+      a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
+      cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, cnt_bytes, st);
+      if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
+  }
   if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
     const size_t need = tc_workspace_bytes(t);
     if (!workspace || workspace_bytes < need) return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "einsum needs %zu workspace bytes, got %zu", need, workspace_bytes);

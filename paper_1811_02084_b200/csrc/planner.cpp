@@ -485,6 +485,17 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
     }
     t.reduce_mode = mode;
     P->reduce_mode = mode;
+    // tail balancing: few whole waves of tiles with a large idle remainder and a long K
+    t.balance = 0;
+    if (mode != MTF_REDUCE_WORKSPACE && t.cta_pair && t.K >= 32 * 64) {
+      int64_t tiles = ((t.M / t.sm + 255) / 256) * t.sm * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sn;
+      for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
+      const int64_t workers = 74;     // CTA pairs of a B200; the launcher re-checks with the device's count
+      const int64_t rounds = (tiles + workers - 1) / workers;
+      // Measured on the FFN shapes the fragment traffic costs more than the idle tail it removes,
+      // so the schedule is only taken when asked for (mtf_plan_force reduce_mode 3).
+      if (force_reduce == 3 && tiles >= workers && (double)tiles / (double)(rounds * workers) <= 0.92) t.balance = 1;
+    }
     P->workspace_bytes = tc_workspace_bytes(t);
   } else if (force_reduce == MTF_REDUCE_WORKSPACE) {
     return fail(MTF_ERR_UNSUPPORTED, "workspace reduction exists only on the tensor-core path");
