@@ -348,6 +348,95 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------------
+# secondary workloads (not the headline line): attention block (config 3) and decoder layer (config 5)
+# ------------------------------------------------------------------------------------------------------
+
+def run_block(args):
+    """Times mtf_attention_* (config 3: batch 16, length 512, d_model 1024, 16 heads of 64, mesh [4,4]) or
+    mtf_decoder_layer_* (config 5: batch 64, length 256, d_model 2048, 32 heads, d_ff 8192, mesh [4,8],
+    causal) forward + backward on one GPU and prints one JSON line (random bf16 inputs made on the
+    device: this leg measures time only, parity is the tests' job)."""
+    import torch
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    import paper_1811_02084_b200 as mtf
+    torch.manual_seed(0)
+    bf, f32 = torch.bfloat16, torch.float32
+    dec = args.workload == "decoder"
+    B, L, D, H, K, F = (64, 256, 2048, 32, 64, 8192) if dec else (16, 512, 1024, 16, 64, 0)
+    if args.batch != WORKLOAD["batch"]:
+        B = args.batch
+    mesh, rules = ([("rows", 4), ("cols", 8)], [("batch", "rows"), ("heads", "cols"), ("d_ff", "cols")]) if dec else \
+                  ([("rows", 4), ("cols", 4)], [("batch", "rows"), ("heads", "cols")])
+    lay = mtf.mtf_layout(mtf.mtf_mesh_create(mesh), rules)
+    rn = lambda shape, scale, dt=bf: (torch.randn(*shape, device="cuda") * scale).to(dt)
+    act = ["batch", "length", "d_model"]
+    T = {"x": (rn((B, L, D), 1.0), act), "dout": (rn((B, L, D), 1.0), act),
+         "wq": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_k"]), "wk": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_k"]),
+         "wv": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_v"]), "wo": (rn((H, K, D), (H * K) ** -0.5), ["heads", "d_v", "d_model"])}
+    if dec:
+        T.update({"w": (rn((D, F), D ** -0.5), ["d_model", "d_ff"]), "v": (rn((F, D), F ** -0.5), ["d_ff", "d_model"]),
+                  "bias": (rn((F,), 0.1, f32), ["d_ff"])})
+        for n in ("ln1_gamma", "ln2_gamma"):
+            T[n] = (1.0 + rn((D,), 0.1, f32), ["d_model"])
+        for n in ("ln1_beta", "ln2_beta"):
+            T[n] = (rn((D,), 0.1, f32), ["d_model"])
+    N = {k: mtf.named(t, names) for k, (t, names) in T.items()}
+    m = "memory_length"
+    sd = {"q": ((B, L, H, K), ["batch", "length", "heads", "d_k"]), "kk": ((B, L, H, K), ["batch", m, "heads", "d_k"]),
+          "vv": ((B, L, H, K), ["batch", m, "heads", "d_v"]), "weights": ((B, H, L, L), ["batch", "heads", "length", m]),
+          "o": ((B, L, H, K), ["batch", "length", "heads", "d_v"]), "s1": ((B, L, D), act), "a": ((B, L, D), act), "s2": ((B, L, D), act)}
+    if dec:
+        sd["h"] = ((B, L, F), ["batch", "length", "d_ff"])
+    keep = {n: torch.empty(shape, dtype=bf, device="cuda") for n, (shape, _) in sd.items()}
+    S = {n: mtf.named(keep[n], sd[n][1]) for n in keep}
+    for n in ("stats1", "stats2"):
+        keep[n] = torch.empty(B, L, 2, dtype=f32, device="cuda")
+        S[n] = mtf.named(keep[n], ["batch", "length", "stat"])
+    out, dx = torch.empty(B, L, D, dtype=bf, device="cuda"), torch.empty(B, L, D, dtype=bf, device="cuda")
+    params = [k for k in T if k not in ("x", "dout")]
+    gname = {"wq": "dwq", "wk": "dwk", "wv": "dwv", "wo": "dwo", "ln1_gamma": "dln1_gamma", "ln1_beta": "dln1_beta", "w": "dw", "bias": "dbias",
+             "v": "dv", "ln2_gamma": "dln2_gamma", "ln2_beta": "dln2_beta"}
+    gt = {k: torch.empty_like(T[k][0], dtype=f32) for k in params}
+    G = {gname[k]: mtf.named(gt[k], T[k][1]) for k in params}
+    P = {k: N[k] for k in params}
+    if dec:
+        ws = torch.empty(mtf.mtf_decoder_layer_workspace_bytes(lay, N["x"], P), dtype=torch.uint8, device="cuda")
+        flops = 3 * (8.0 * B * L * D * H * K + 4.0 * B * H * L * L * K + 4.0 * B * L * D * F)
+
+        def step():
+            mtf.mtf_decoder_layer_forward(lay, N["x"], P, True, 1e-6, S, mtf.named(out, act), ws)
+            mtf.mtf_decoder_layer_backward(lay, N["x"], P, S, N["dout"], mtf.named(dx, act), G, ws)
+    else:
+        ws = torch.empty(mtf.mtf_attention_workspace_bytes(lay, N["x"], N["wq"], N["wv"]), dtype=torch.uint8, device="cuda")
+        flops = 3 * (8.0 * B * L * D * H * K + 4.0 * B * H * L * L * K)
+
+        def step():
+            mtf.mtf_attention_forward(lay, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], False, None, S["q"], S["kk"], S["vv"], S["weights"], S["o"],
+                                      mtf.named(out, act), ws)
+            mtf.mtf_attention_backward(lay, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], S["q"], S["kk"], S["vv"], S["weights"], S["o"], N["dout"], None,
+                                       mtf.named(dx, act), G["dwq"], G["dwk"], G["dwv"], G["dwo"], ws)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = mtf.mtf_launch_count()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    mtf.mtf_device_status()
+    ms = e0.elapsed_time(e1) / args.steps
+    print(json.dumps({"metric": f"transformer_{args.workload}_fwd_bwd_tflops", "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16",
+                      "data": "synthetic", "gpu_launches": mtf.mtf_launch_count() - n0,
+                      "config": {"workload": f"{args.workload} batch={B} length={L} d_model={D} heads={H} d_k={K}" + (f" d_ff={F} causal" if dec else ""),
+                                 "mesh": mesh, "rules": rules, "flops_per_step": flops,
+                                 "flops_note": "dense-equivalent contraction flops (projections, attention core, FFN), 2 per multiply-add, forward + backward = 3x forward"}}),
+          flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -358,10 +447,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=WORKLOAD["batch"], help="sequences of 256 tokens per GPU (smaller only for profiler captures)")
     ap.add_argument("--main-only", action="store_true", help="skip the per-layout table and the end-to-end leg (profiler captures)")
+    ap.add_argument("--workload", default="ffn", choices=["ffn", "attention", "decoder"], help="ffn = the headline line; the others print a secondary line")
     args = ap.parse_args()
     WORKLOAD["batch"] = args.batch
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "ffn":
+        run_block(args)
     else:
         run_ours(args)
 
