@@ -45,6 +45,32 @@ constexpr long long kTimeoutCycles = 4000000000LL;
 
 __device__ int g_status = 0;
 
+// Division by a run-time constant as a multiply-high and a shift (exact for dividends below 2^31):
+// the tile decoder runs once per tile in every warp role and 64-bit divisions made it cost more
+// instructions than a tile's whole epilogue.
+struct FastDiv {
+  uint32_t d, mul, shr;
+};
+static FastDiv make_fastdiv(long long divisor) {
+  FastDiv f;
+  f.d = (uint32_t)(divisor < 1 ? 1 : divisor);
+  f.mul = 0; f.shr = 0;
+  if (f.d > 1) {
+    uint32_t l = 0;
+    while ((1ull << l) < f.d) ++l;                    // smallest l with 2^l >= d
+    const unsigned p = 31 + l;
+    f.mul = (uint32_t)(((1ull << p) + f.d - 1) / f.d);
+    f.shr = p - 32;
+  }
+  return f;
+}
+__device__ __forceinline__ uint32_t fd_div(uint32_t n, const FastDiv& f) { return f.d == 1 ? n : (__umulhi(n, f.mul) >> f.shr); }
+__device__ __forceinline__ uint32_t fd_divmod(uint32_t n, const FastDiv& f, uint32_t* rem) {
+  const uint32_t q = fd_div(n, f);
+  *rem = n - q * f.d;
+  return q;
+}
+
 struct TcArgs {
   int M, N, K;
   int sm, sn, sk;
@@ -78,6 +104,7 @@ struct TcArgs {
   float* rsum;             // fused reduce_sum over M of the epilogue value (fp32, pre-zeroed), indexed by n
   float* ws_partials;
   unsigned* ws_counters;
+  FastDiv fd_tiles_per_slice, fd_n_tiles, fd_m_tiles, fd_outer_local[3], fd_sn, fd_sm, fd_outer_split[3], fd_sk;
 };
 
 struct Tile {
@@ -86,28 +113,29 @@ struct Tile {
   long long c_off;         // element offset of the outer coordinates in C
 };
 
-__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long t, int tile_rows, int tile_cols) {
+__device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long tile, int tile_rows, int tile_cols) {
   Tile r;
-  long long slice = t / a.tiles_per_slice;
-  long long w = t % a.tiles_per_slice;
-  int mt, nt;
-  if (a.n_fastest) { nt = (int)(w % a.n_tiles); w /= a.n_tiles; mt = (int)(w % a.m_tiles); w /= a.m_tiles; }
-  else { mt = (int)(w % a.m_tiles); w /= a.m_tiles; nt = (int)(w % a.n_tiles); w /= a.n_tiles; }
+  uint32_t w, rem;
+  uint32_t slice = fd_divmod((uint32_t)tile, a.fd_tiles_per_slice, &w);
+  uint32_t mt, nt;
+  if (a.n_fastest) { w = fd_divmod(w, a.fd_n_tiles, &nt); w = fd_divmod(w, a.fd_m_tiles, &mt); }
+  else { w = fd_divmod(w, a.fd_m_tiles, &mt); w = fd_divmod(w, a.fd_n_tiles, &nt); }
   int ol[3] = {0, 0, 0};
-  for (int j = a.n_outer - 1; j >= 0; --j) { ol[j] = (int)(w % a.outer_local[j]); w /= a.outer_local[j]; }
-  const int in = (int)(slice % a.sn); slice /= a.sn;
-  const int im = (int)(slice % a.sm); slice /= a.sm;
+  for (int j = a.n_outer - 1; j >= 0; --j) { w = fd_divmod(w, a.fd_outer_local[j], &rem); ol[j] = (int)rem; }
+  uint32_t in, im;
+  slice = fd_divmod(slice, a.fd_sn, &in);
+  slice = fd_divmod(slice, a.fd_sm, &im);
   r.c_off = 0;
   r.o[0] = r.o[1] = r.o[2] = 0;
   for (int j = a.n_outer - 1; j >= 0; --j) {
-    const int ob = (int)(slice % a.outer_split[j]); slice /= a.outer_split[j];
-    r.o[j] = ob * a.outer_local[j] + ol[j];
+    slice = fd_divmod(slice, a.fd_outer_split[j], &rem);
+    r.o[j] = (int)rem * a.outer_local[j] + ol[j];
     r.c_off += (long long)r.o[j] * a.outer_sC[j];
   }
-  r.m0 = im * a.Ms + mt * tile_rows;
-  r.m_end = (im + 1) * a.Ms;
-  r.n0 = in * a.Ns + nt * tile_cols;
-  r.n_end = (in + 1) * a.Ns;
+  r.m0 = (int)im * a.Ms + (int)mt * tile_rows;
+  r.m_end = ((int)im + 1) * a.Ms;
+  r.n0 = (int)in * a.Ns + (int)nt * tile_cols;
+  r.n_end = ((int)in + 1) * a.Ns;
   return r;
 }
 
@@ -152,8 +180,9 @@ struct SegIter {
     }
     if (work >= a.total_work) return false;
     if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
-      s.tile = work / a.sk;
-      s.frag = (int)(work % a.sk);
+      uint32_t frag;
+      s.tile = fd_divmod((uint32_t)work, a.fd_sk, &frag);
+      s.frag = (int)frag;
       s.nfrag = a.sk;
       s.kb_begin = s.frag * kb_per_slice;
       s.kb_count = kb_per_slice;
@@ -349,6 +378,28 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
   }
 }
 
+// Which component-wise stages a launch runs.  EPI_GENERIC reads them from the arguments; the other
+// kinds fix them at compile time, so that the common epilogues carry no branches on them and need
+// far fewer registers and instructions per chunk.
+enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_KINDS = 5 };
+struct EpiFlags {
+  bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, rsum, c_bf16, shared_tiles;
+};
+template <int EPI>
+__device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
+  EpiFlags f;
+  if (EPI == EPI_GENERIC) {
+    f.scale = a.scale != 1.f; f.bias = a.bias != nullptr; f.bias_m = a.bias_along_m != 0; f.relu = a.relu != 0;
+    f.mask = a.mask != nullptr; f.mask_bf16 = a.mask_bf16 != 0; f.mask_tma = a.mask_tma != 0; f.resid = a.resid != nullptr;
+    f.rsum = a.rsum != nullptr; f.c_bf16 = a.c_bf16 != 0; f.shared_tiles = true;
+  } else {
+    f.scale = false; f.bias = EPI == EPI_BIAS_RELU_BF16; f.bias_m = false; f.relu = EPI == EPI_BIAS_RELU_BF16;
+    f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = false;
+    f.c_bf16 = EPI != EPI_PLAIN_F32; f.shared_tiles = false;      // tiles assembled from fragments take the generic kind
+  }
+  return f;
+}
+
 // Fetch the relu mask of one 32-column chunk of this thread's row (bf16 mask: four 16-byte loads).
 __device__ __forceinline__ void mask_fetch(const TcArgs& a, long long off, bool on, int n_valid, uint4* mk) {
 #pragma unroll
@@ -362,12 +413,14 @@ __device__ __forceinline__ void mask_fetch(const TcArgs& a, long long off, bool 
 // scale, bias (broadcast), relu, relu mask; the value then feeds the fused reduce_sum; residual last.
 //   bias_lane : bias of column (n_first + lane), handed to every lane by shuffle (bias along n)
 //   bias_row  : bias of this thread's row (bias along m)
-__device__ __forceinline__ void epilogue_math(const TcArgs& a, float* v, float bias_lane, float bias_row, const uint4* mk,
-                                              long long off, bool live, int n_valid) {
+__device__ __forceinline__ void epilogue_math(const TcArgs& a, const EpiFlags& f, float* v, float bias_lane, float bias_row,
+                                              const uint4* mk, long long off, bool live, int n_valid) {
+  if (f.scale) {
 #pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] *= a.scale;
-  if (a.bias) {
-    if (a.bias_along_m) {
+    for (int j = 0; j < 32; ++j) v[j] *= a.scale;
+  }
+  if (f.bias) {
+    if (f.bias_m) {
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += bias_row;
     } else {
@@ -375,12 +428,12 @@ __device__ __forceinline__ void epilogue_math(const TcArgs& a, float* v, float b
       for (int j = 0; j < 32; ++j) v[j] += __shfl_sync(0xffffffffu, bias_lane, j);
     }
   }
-  if (a.relu) {
+  if (f.relu) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
   }
-  if (a.mask) {
-    if (a.mask_bf16) {
+  if (f.mask) {
+    if (f.mask_bf16) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         float f[8];
@@ -398,8 +451,8 @@ __device__ __forceinline__ void epilogue_math(const TcArgs& a, float* v, float b
   }
 }
 
-__device__ __forceinline__ void epilogue_residual(const TcArgs& a, float* v, long long off, bool live, int n_valid) {
-  if (!a.resid || !live) return;
+__device__ __forceinline__ void epilogue_residual(const TcArgs& a, const EpiFlags& f, float* v, long long off, bool live, int n_valid) {
+  if (!f.resid || !live) return;
   if (a.resid_bf16) {
     const uint4* rp = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
 #pragma unroll
@@ -424,8 +477,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 // 16-byte stores of one chunk straight from registers (ragged tiles and the workspace mode).
-__device__ __forceinline__ void store_direct(const TcArgs& a, const float* v, long long off, int n_valid) {
-  if (a.c_bf16) {
+__device__ __forceinline__ void store_direct(const TcArgs& a, const EpiFlags& f, const float* v, long long off, int n_valid) {
+  if (f.c_bf16) {
     uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
@@ -457,10 +510,10 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t
 
 // One chunk of this thread's row into the warp's staging box (32 rows x 128 B, 128B-swizzled as
 // the output tensor map expects): 16-byte piece p of row r lives at r*128 + ((p ^ (r & 7)) * 16).
-__device__ __forceinline__ void store_staged(const TcArgs& a, const float* v, uint32_t box, int lane, int half) {
+__device__ __forceinline__ void store_staged(const EpiFlags& f, const float* v, uint32_t box, int lane, int half) {
   const uint32_t row = box + (uint32_t)lane * 128u;
   const uint32_t sw = (uint32_t)(lane & 7);
-  if (a.c_bf16) {
+  if (f.c_bf16) {
 #pragma unroll
     for (int q = 0; q < 4; ++q)
       st_shared_v4(row + ((((uint32_t)(half * 4 + q)) ^ sw) << 4), pack_bf16x2(v[q * 8], v[q * 8 + 1]),
@@ -497,10 +550,11 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 // 16 KB / CN + 16 KB / CM per k-block through L2 instead of 32 KB.  A stage may be refilled when
 // every pair that reads what this CTA writes has retired its MMAs: CM + CN - 1 pair leaders signal
 // each CTA's "empty" barrier.
-template <bool kPair, int CM, int CN>
+template <bool kPair, int CM, int CN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                    const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m, const TcArgs a) {
+                    const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
+                    const __grid_constant__ CUtensorMap map_w, const TcArgs a) {
   constexpr int kStages = kPair ? 5 : 3;
   constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
@@ -673,6 +727,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
   } else {
     // ------------------------------- epilogue -----------------------------------
+    const EpiFlags f = epi_flags<EPI>(a);
     const int q = warp & 3;                        // TMEM lane quarter this warp may read
     const int col_half = (warp - 2) >> 2;          // which of the two warps of this lane quarter
     const uint32_t stg = staging_base + (uint32_t)(warp - 2) * 8192u;      // this warp's two staging boxes
@@ -686,7 +741,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (; ok && it.next(sg); ++iter) {
       const long long t = sg.tile;
       const int ks = sg.frag;
-      const bool ws_mode = sg.nfrag > 1;       // this tile is assembled from fragments in the workspace
+      const bool ws_mode = f.shared_tiles && sg.nfrag > 1;       // this tile is assembled from fragments in the workspace
       Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
       tl.m0 += pm * kPairRows;            // this pair's 256 x block_n part of the cluster's super-tile
       tl.n0 += pn * a.block_n;
@@ -699,17 +754,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const long long row_off = tl.c_off + (long long)row * a.ldc;
       // what the epilogue needs from memory is requested before the accumulator is waited for:
       // the tile's bias (lane l keeps columns l, l+32, ...) and the first chunk's relu mask
-      const bool bias_n = a.bias != nullptr && !a.bias_along_m;
+      const bool bias_n = f.bias && !f.bias_m;
       auto bias_at = [&](int col) -> float {       // bias of one column, 0 outside the slice
         if (!bias_n || col >= tl.n_end) return 0.f;
         return a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[col]) : reinterpret_cast<const float*>(a.bias)[col];
       };
       float bias_row = 0.f;
-      if (a.bias && a.bias_along_m && row_ok)
+      if (f.bias && f.bias_m && row_ok)
         bias_row = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row]) : reinterpret_cast<const float*>(a.bias)[row];
       const int row0 = tl.m0 + cta_rank * BM + q * 32;           // first row of this warp
       const bool rows_full = row0 + 32 <= tl.m_end;
-      const bool mask_tma = a.mask_tma != 0 && !ws_mode && rows_full;
+      const bool mask_tma = f.mask_tma && !ws_mode && rows_full;
       if (mask_tma && lane == 0) {
         // pull this warp's boxes of the mask tile towards L2 and request the first one into the
         // staging box it will be processed in (free once all but the latest store have been read out)
@@ -730,7 +785,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
-        const int box_cols = a.c_bf16 ? 64 : 32;
+        const int box_cols = f.c_bf16 ? 64 : 32;
         float bias_cur = bias_at(tl.n0 + col_half * box_cols + lane);      // lane l keeps column l of the current chunk
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
@@ -755,7 +810,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
           }
           uint4 mk[4];
-          if (a.mask && a.mask_bf16) {
+          if (f.mask && f.mask_bf16) {
             if (staged && mask_tma) {
 #pragma unroll
               for (int i = 0; i < 4; ++i) mk[i] = ld_shared_v4(box + (uint32_t)lane * 128u + ((((uint32_t)(half * 4 + i)) ^ (uint32_t)(lane & 7)) << 4));
@@ -768,11 +823,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const float bias_next = bias_at(tl.n0 + next_c0 + lane);
           tmem_ld_wait();
           float* v = reinterpret_cast<float*>(raw);
-          epilogue_math(a, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
+          epilogue_math(a, f, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
           bias_cur = bias_next;
-          epilogue_residual(a, v, row_off + n_first, live, n_valid);
-          if (staged) store_staged(a, v, box, lane, half);
-          else if (live) store_direct(a, v, row_off + n_first, n_valid);
+          epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
+          if (staged) store_staged(f, v, box, lane, half);
+          else if (live) store_direct(a, f, v, row_off + n_first, n_valid);
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -788,7 +843,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             buf ^= 1u;
           }
-          if (a.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
+          if (f.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = (live && j < n_valid) ? v[j] : 0.f;
             const float col = warp_column_sums(v, lane);
@@ -799,64 +854,130 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __syncwarp();
         if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
       } else {
-        // partial of slice `ks` -> workspace; last-arriving warp of this row quarter finishes the tile
-        // (the two warps of a lane quarter split the columns in halves, each with its own counter)
+        // fragment `ks` of the tile -> workspace; whichever warp arrives last on this row quarter and
+        // column half adds the fragments in order and finishes the tile.  The fragment leaves the
+        // way a finished tile does: 32-row x 128-byte boxes through the staging buffers and TMA stores.
         const int ws_c_begin = col_half * (a.block_n / 2), ws_c_end = ws_c_begin + a.block_n / 2;
-        float* part = a.ws_partials + ((size_t)(t * a.slots + ks) * kTileRows + (size_t)tile_row) * a.block_n;
+        const int warp_tile_row = pm * kPairRows + cta_rank * BM + q * 32;      // first row of this warp inside the tile
+        const long long part_row0 = (t * a.slots + ks) * (long long)kTileRows + warp_tile_row;
+#pragma unroll 1
         for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          __syncwarp();
+          const uint32_t box = stg + buf * 4096u;
+          const uint32_t srow = box + (uint32_t)lane * 128u;
+          const uint32_t sw = (uint32_t)(lane & 7);
           tmem_ld_wait();
-          float4* pp = reinterpret_cast<float4*>(part + c0);
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            pp[j] = make_float4(__uint_as_float(raw[4 * j]), __uint_as_float(raw[4 * j + 1]),
-                                __uint_as_float(raw[4 * j + 2]), __uint_as_float(raw[4 * j + 3]));
+            st_shared_v4(srow + (((uint32_t)j ^ sw) << 4), raw[4 * j], raw[4 * j + 1], raw[4 * j + 2], raw[4 * j + 3]);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) tma_store_5d(&map_w, box, c0, (int)part_row0, 0, 0, 0);
+          buf ^= 1u;
         }
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
-        __threadfence();
-        __syncwarp();
         unsigned old = 0;
-        if (lane == 0) old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + tile_row / 32) * 2 + col_half], 1u);
+        if (lane == 0) {
+          mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
+          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");       // the fragment has been written, not only read out
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __threadfence();
+          old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + warp_tile_row / 32) * 2 + col_half], 1u);
+          __threadfence();
+        }
         old = __shfl_sync(0xffffffffu, old, 0);
         if (old == (unsigned)sg.nfrag - 1) {
-          __threadfence();
-          const float* p0 = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)tile_row) * a.block_n;
+          // Coalesced pass over this warp's 32 rows x (block_n / 2) columns: lanes_per_row lanes cover
+          // one row with four columns each, so every load, store and epilogue operand access is a run
+          // of whole 16-byte pieces; the row-per-lane layout of the accumulator is not needed here.
+          const int lanes_per_row = a.block_n / 8, rows_per_pass = 32 / lanes_per_row;
+          const int lc = ws_c_begin + (lane % lanes_per_row) * 4;
+          const int lr = lane / lanes_per_row;
+          const int n = tl.n0 + lc;
+          const bool col_ok = n < tl.n_end;                  // slices are whole multiples of four columns
+          const size_t slot_stride = (size_t)kTileRows * a.block_n;
+          const float* p0 = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)warp_tile_row) * a.block_n + lc;
+          float bq[4] = {0.f, 0.f, 0.f, 0.f};
+          if (bias_n && col_ok) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) bq[e] = bias_at(n + e);
+          }
+          float cs[4] = {0.f, 0.f, 0.f, 0.f};                // fused reduce_sum: this lane's four columns over its rows
 #pragma unroll 1
-          for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
-            const int n_first = tl.n0 + c0;
-            int n_valid = tl.n_end - n_first;
-            n_valid = n_valid > 32 ? 32 : n_valid;
-            const bool live = row_ok && n_valid > 0;
-            float v[32];
+          for (int i0 = 0; i0 < lanes_per_row; i0 += 4) {
+            float4 sum[4];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.f;
-            if (live) {
-              for (int s = 0; s < sg.nfrag; ++s) {     // ascending order of the fragments (= of the processors of the group)
-                const float4* sp = reinterpret_cast<const float4*>(p0 + (size_t)s * kTileRows * a.block_n + c0);
+            for (int u = 0; u < 4; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < sg.nfrag; ++s) {             // ascending order of the fragments (= of the processors of the group)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float4 f = __ldcg(sp + j);
-                  v[4 * j] += f.x; v[4 * j + 1] += f.y; v[4 * j + 2] += f.z; v[4 * j + 3] += f.w;
-                }
+              for (int u = 0; u < 4; ++u) {
+                const int r = (i0 + u) * rows_per_pass + lr;
+                const float4 f = __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)s * slot_stride + (size_t)r * a.block_n));
+                sum[u].x += f.x; sum[u].y += f.y; sum[u].z += f.z; sum[u].w += f.w;
               }
             }
-            if (n_valid > 0) {                     // warp-uniform: the bias hand-out and the column sums use shuffles
-              uint4 mkw[4];
-              if (a.mask && a.mask_bf16) mask_fetch(a, row_off + n_first, row_ok, n_valid, mkw);
-              epilogue_math(a, v, bias_at(n_first + lane), bias_row, mkw, row_off + n_first, live, n_valid);
-              float col = 0.f;
-              if (a.rsum) {
-                float r[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = (live && j < n_valid) ? v[j] : 0.f;
-                col = warp_column_sums(r, lane);
-                if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
+            for (int u = 0; u < 4; ++u) {
+              const int r = (i0 + u) * rows_per_pass + lr;
+              const int grow = tl.m0 + cta_rank * BM + q * 32 + r;
+              if (!col_ok || grow >= tl.m_end) continue;
+              const long long off = tl.c_off + (long long)grow * a.ldc + n;
+              float v[4] = {sum[u].x * a.scale, sum[u].y * a.scale, sum[u].z * a.scale, sum[u].w * a.scale};
+              if (f.bias) {
+                float br = 0.f;
+                if (f.bias_m)
+                  br = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[grow]) : reinterpret_cast<const float*>(a.bias)[grow];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e] += f.bias_m ? br : bq[e];
               }
-              epilogue_residual(a, v, row_off + n_first, live, n_valid);
-              if (live) store_direct(a, v, row_off + n_first, n_valid);
+              if (f.relu) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) v[e] = fmaxf(v[e], 0.f);
+              }
+              if (f.mask) {
+                float mf[4];
+                if (f.mask_bf16) {
+                  const uint2 mw = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.mask) + off);
+                  mf[0] = bf16_bits_to_float(mw.x & 0xFFFFu); mf[1] = bf16_bits_to_float(mw.x >> 16);
+                  mf[2] = bf16_bits_to_float(mw.y & 0xFFFFu); mf[3] = bf16_bits_to_float(mw.y >> 16);
+                } else {
+                  const float4 mw = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.mask) + off);
+                  mf[0] = mw.x; mf[1] = mw.y; mf[2] = mw.z; mf[3] = mw.w;
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                  if (!(mf[e] > 0.f)) v[e] = 0.f;
+              }
+#pragma unroll
+              for (int e = 0; e < 4; ++e) cs[e] += v[e];
+              if (f.resid) {
+                if (a.resid_bf16) {
+                  const uint2 rw = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
+                  v[0] += bf16_bits_to_float(rw.x & 0xFFFFu); v[1] += bf16_bits_to_float(rw.x >> 16);
+                  v[2] += bf16_bits_to_float(rw.y & 0xFFFFu); v[3] += bf16_bits_to_float(rw.y >> 16);
+                } else {
+                  const float4 rw = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.resid) + off);
+                  v[0] += rw.x; v[1] += rw.y; v[2] += rw.z; v[3] += rw.w;
+                }
+              }
+              if (f.c_bf16)
+                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off) = make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
+              else
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off) = make_float4(v[0], v[1], v[2], v[3]);
+            }
+          }
+          if (f.rsum) {                                      // lanes that share columns add up, the first of each set reports
+            for (int o = lanes_per_row; o < 32; o <<= 1) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], o);
+            }
+            if (lr == 0 && col_ok) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) atomicAdd(a.rsum + n + e, cs[e]);
             }
           }
         }
@@ -953,17 +1074,17 @@ int sm_count() {
 
 // One kernel variant: shared-memory opt-in and the number of clusters that can be resident at once
 // are looked up on first use; the grid is that many clusters (persistent) or fewer.
-template <bool kPair, int CM, int CN>
+template <bool kPair, int CM, int CN, int EPI>
 mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
-                          const TcArgs& a, cudaStream_t st) {
+                          const CUtensorMap& map_w, const TcArgs& a, cudaStream_t st) {
   constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   static int max_clusters = 0;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (attr_err != cudaSuccess) return;
-    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (attr_err != cudaSuccess) return;
     if (kCtas == 1) { max_clusters = sm_count(); return; }
     cudaLaunchConfig_t q = {};
@@ -973,7 +1094,7 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     q.gridDim = dim3(kCtas * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
     q.attrs = at; q.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN>, &q) == cudaSuccess && n > 0) max_clusters = n;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI>, &q) == cudaSuccess && n > 0) max_clusters = n;
     else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
   });
   if (attr_err != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
@@ -987,9 +1108,24 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   at[1].val.clusterDim.x = kCtas; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   cfg.gridDim = dim3((unsigned)(kCtas * clusters), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = kCtas > 1 ? 2 : 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN>, map_a, map_b, map_c, map_m, a);
-  if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d>: %s", (int)kPair, CM, CN, cudaGetErrorString(le));
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI>, map_a, map_b, map_c, map_m, map_w, a);
+  if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d,%d>: %s", (int)kPair, CM, CN, EPI, cudaGetErrorString(le));
   return MTF_OK;
+}
+
+// Picks the epilogue kind of a launch.  kAllKinds = false leaves out the relu-mask kind (cluster
+// shapes that are never used with a mask).
+template <bool kPair, int CM, int CN, bool kAllKinds>
+mtf_status launch_kind(int epi, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
+                       const CUtensorMap& map_w, const TcArgs& a, cudaStream_t st) {
+  switch (epi) {
+    case EPI_PLAIN_BF16: return launch_variant<kPair, CM, CN, EPI_PLAIN_BF16>(map_a, map_b, map_c, map_m, map_w, a, st);
+    case EPI_PLAIN_F32: return launch_variant<kPair, CM, CN, EPI_PLAIN_F32>(map_a, map_b, map_c, map_m, map_w, a, st);
+    case EPI_BIAS_RELU_BF16: return launch_variant<kPair, CM, CN, EPI_BIAS_RELU_BF16>(map_a, map_b, map_c, map_m, map_w, a, st);
+    case EPI_MASK_RSUM_BF16:
+      if (kAllKinds) return launch_variant<kPair, CM, CN, kAllKinds ? EPI_MASK_RSUM_BF16 : EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, a, st);
+    default: return launch_variant<kPair, CM, CN, EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, a, st);
+  }
 }
 
 }  // namespace
@@ -1066,6 +1202,11 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   for (int j = 0; j < a.n_outer; ++j) out_slices *= a.outer_split[j];
   a.total_tiles = a.tiles_per_slice * out_slices;
   a.total_work = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.total_tiles * a.sk : a.total_tiles;
+  if (a.total_work >= 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "more than 2^31 tiles");
+  a.fd_tiles_per_slice = make_fastdiv(a.tiles_per_slice);
+  a.fd_n_tiles = make_fastdiv(a.n_tiles); a.fd_m_tiles = make_fastdiv(a.m_tiles);
+  a.fd_sn = make_fastdiv(a.sn); a.fd_sm = make_fastdiv(a.sm); a.fd_sk = make_fastdiv(a.sk);
+  for (int j = 0; j < 3; ++j) { a.fd_outer_local[j] = make_fastdiv(a.outer_local[j]); a.fd_outer_split[j] = make_fastdiv(a.outer_split[j]); }
   a.C = C; a.c_bf16 = plan.dtC == MTF_BF16;
   a.bias = bias; a.bias_bf16 = dtBias == MTF_BF16; a.bias_along_m = t.bias_along_m;
   a.mask = mask; a.mask_bf16 = dtMask == MTF_BF16;
@@ -1126,14 +1267,31 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if ((s = make_map(&map_c, C, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
   map_m = map_c;
   if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
+  // fragments of shared tiles: the workspace as one fp32 matrix of block_n columns, a tile slot after the other
+  CUtensorMap map_w = map_c;
+  if (a.ws_partials) {
+    const long long ws_rows = a.total_tiles * a.slots * tile_rows;
+    if (ws_rows > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "workspace of more than 2^31 rows");
+    TcParams flat = t;
+    flat.n_outer = 0;
+    if ((s = make_map(&map_w, a.ws_partials, 4, a.block_n, ws_rows, a.block_n, 32, 32, flat, t.outer_sC)) != MTF_OK) return s;
+  }
 
+  // epilogue kind: the common combinations have kernels of their own, everything else (and every
+  // launch that assembles tiles from fragments) takes the generic one
+  int epi = EPI_GENERIC;
+  if (!a.ws_partials && scale == 1.f && !resid) {
+    if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+    else if (bias && !a.bias_along_m && relu && !mask && !rsum && a.c_bf16) epi = EPI_BIAS_RELU_BF16;
+    else if (a.mask_tma && rsum && !bias && !relu) epi = EPI_MASK_RSUM_BF16;
+  }
   mtf_status ls;
-  if (!t.cta_pair) ls = launch_variant<false, 1, 1>(map_a, map_b, map_c, map_m, a, st);
+  if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
 #if defined(MTF_TMA_MULTICAST)
-  else if (cm == 1 && cn == 2) ls = launch_variant<true, 1, 2>(map_a, map_b, map_c, map_m, a, st);
-  else if (cm == 2 && cn == 1) ls = launch_variant<true, 2, 1>(map_a, map_b, map_c, map_m, a, st);
+  else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
+  else if (cm == 2 && cn == 1) ls = launch_kind<true, 2, 1, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
 #endif
-  else ls = launch_variant<true, 1, 1>(map_a, map_b, map_c, map_m, a, st);
+  else ls = launch_kind<true, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
   if (ls != MTF_OK) return ls;
   count_launch();
   cudaError_t e = cudaGetLastError();
