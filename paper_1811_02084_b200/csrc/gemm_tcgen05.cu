@@ -103,7 +103,8 @@ struct TcArgs {
   int relu;
   float* rsum;             // fused reduce_sum over M of the epilogue value (fp32, pre-zeroed), indexed by n
   float* ws_partials;
-  unsigned* ws_counters;
+  unsigned* ws_counters;     // per (tile, 32-row group, column part): arrivals, then as many again: fragments written
+  long long ws_ncounters;
   FastDiv fd_tiles_per_slice, fd_n_tiles, fd_m_tiles, fd_outer_local[3], fd_sn, fd_sm, fd_outer_split[3], fd_sk;
 };
 
@@ -395,7 +396,8 @@ __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
   } else {
     f.scale = false; f.bias = EPI == EPI_BIAS_RELU_BF16; f.bias_m = false; f.relu = EPI == EPI_BIAS_RELU_BF16;
     f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = false;
-    f.c_bf16 = EPI != EPI_PLAIN_F32; f.shared_tiles = false;      // tiles assembled from fragments take the generic kind
+    f.c_bf16 = EPI != EPI_PLAIN_F32;
+    f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
   }
   return f;
 }
@@ -781,7 +783,36 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (!ok) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
-      if (!ws_mode) {
+      // A tile shared by several workers: every worker but the last to arrive (per 32-row group and
+      // column part) leaves its fragment in the workspace; the last one keeps its own in registers,
+      // adds the others in ascending order of the fragments (= of the processors of the group) and
+      // runs the regular epilogue.  It may have to wait for a fragment that is still being written:
+      // its writer is already running and waits for nobody.
+      const int warp_tile_row = pm * kPairRows + cta_rank * BM + q * 32;      // first row of this warp inside the tile
+      const long long ws_ci = (t * (kTileRows / 32) + warp_tile_row / 32) * 2 + col_half;
+      bool finisher = true;
+      if (ws_mode) {
+        unsigned old = 0;
+        if (lane == 0) old = atomicAdd(&a.ws_counters[ws_ci], 1u);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        finisher = old == (unsigned)sg.nfrag - 1;
+        if (finisher) {
+          int good = 1;
+          if (lane == 0) {
+            const volatile unsigned* written = a.ws_counters + a.ws_ncounters + ws_ci;
+            const long long t0 = clock64();
+            while (*written < (unsigned)sg.nfrag - 1) {
+              __nanosleep(64);
+              if (*abort_flag) { good = 0; break; }
+              if (clock64() - t0 > kTimeoutCycles) { atomicCAS(&g_status, 0, 0x600); *abort_flag = 1; good = 0; break; }
+            }
+            __threadfence();
+          }
+          ok = __shfl_sync(0xffffffffu, good, 0) != 0;
+          if (!ok) break;
+        }
+      }
+      if (finisher) {
         // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
@@ -823,6 +854,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const float bias_next = bias_at(tl.n0 + next_c0 + lane);
           tmem_ld_wait();
           float* v = reinterpret_cast<float*>(raw);
+          if (ws_mode) {
+            const float* prow = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)tile_row) * a.block_n + c0;
+            const size_t slot_stride = (size_t)kTileRows * a.block_n;
+            float pre[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) pre[j] = 0.f;
+            for (int s2 = 0; s2 < sg.nfrag; ++s2) {
+              if (s2 == ks) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) pre[j] += v[j];
+              } else {
+                const float4* sp = reinterpret_cast<const float4*>(prow + (size_t)s2 * slot_stride);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float4 x4 = __ldcg(sp + j);
+                  pre[4 * j] += x4.x; pre[4 * j + 1] += x4.y; pre[4 * j + 2] += x4.z; pre[4 * j + 3] += x4.w;
+                }
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = pre[j];
+          }
           epilogue_math(a, f, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
           bias_cur = bias_next;
           epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
@@ -854,14 +907,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __syncwarp();
         if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
       } else {
-        // fragment `ks` of the tile -> workspace; whichever warp arrives last on this row quarter and
-        // column half adds the fragments in order and finishes the tile.  The fragment leaves the
-        // way a finished tile does: 32-row x 128-byte boxes through the staging buffers and TMA stores.
-        const int ws_c_begin = col_half * (a.block_n / 2), ws_c_end = ws_c_begin + a.block_n / 2;
-        const int warp_tile_row = pm * kPairRows + cta_rank * BM + q * 32;      // first row of this warp inside the tile
+        // fragment `ks` of the tile -> workspace, the way a finished tile leaves: 32-row x 128-byte
+        // boxes through the staging buffers and TMA stores (the chunks this warp owns in the regular
+        // epilogue, so that the finisher finds them under the same counter)
+        const int box_cols = f.c_bf16 ? 64 : 32;
         const long long part_row0 = (t * a.slots + ks) * (long long)kTileRows + warp_tile_row;
 #pragma unroll 1
-        for (int c0 = ws_c_begin; c0 < ws_c_end; c0 += 32) {
+        for (int c0 = 0; c0 < a.block_n; c0 += 32) {
+          if (((c0 / box_cols) & 1) != col_half) continue;
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
           if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
@@ -880,107 +933,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         tcgen05_fence_before();
         __syncwarp();
-        unsigned old = 0;
         if (lane == 0) {
           mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
           asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");       // the fragment has been written, not only read out
           asm volatile("fence.proxy.async;" ::: "memory");
           __threadfence();
-          old = atomicAdd(&a.ws_counters[(t * (kTileRows / 32) + warp_tile_row / 32) * 2 + col_half], 1u);
-          __threadfence();
+          atomicAdd(&a.ws_counters[a.ws_ncounters + ws_ci], 1u);
         }
-        old = __shfl_sync(0xffffffffu, old, 0);
-        if (old == (unsigned)sg.nfrag - 1) {
-          // Coalesced pass over this warp's 32 rows x (block_n / 2) columns: lanes_per_row lanes cover
-          // one row with four columns each, so every load, store and epilogue operand access is a run
-          // of whole 16-byte pieces; the row-per-lane layout of the accumulator is not needed here.
-          const int lanes_per_row = a.block_n / 8, rows_per_pass = 32 / lanes_per_row;
-          const int lc = ws_c_begin + (lane % lanes_per_row) * 4;
-          const int lr = lane / lanes_per_row;
-          const int n = tl.n0 + lc;
-          const bool col_ok = n < tl.n_end;                  // slices are whole multiples of four columns
-          const size_t slot_stride = (size_t)kTileRows * a.block_n;
-          const float* p0 = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)warp_tile_row) * a.block_n + lc;
-          float bq[4] = {0.f, 0.f, 0.f, 0.f};
-          if (bias_n && col_ok) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) bq[e] = bias_at(n + e);
-          }
-          float cs[4] = {0.f, 0.f, 0.f, 0.f};                // fused reduce_sum: this lane's four columns over its rows
-#pragma unroll 1
-          for (int i0 = 0; i0 < lanes_per_row; i0 += 4) {
-            float4 sum[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int s = 0; s < sg.nfrag; ++s) {             // ascending order of the fragments (= of the processors of the group)
-#pragma unroll
-              for (int u = 0; u < 4; ++u) {
-                const int r = (i0 + u) * rows_per_pass + lr;
-                const float4 f = __ldcg(reinterpret_cast<const float4*>(p0 + (size_t)s * slot_stride + (size_t)r * a.block_n));
-                sum[u].x += f.x; sum[u].y += f.y; sum[u].z += f.z; sum[u].w += f.w;
-              }
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int r = (i0 + u) * rows_per_pass + lr;
-              const int grow = tl.m0 + cta_rank * BM + q * 32 + r;
-              if (!col_ok || grow >= tl.m_end) continue;
-              const long long off = tl.c_off + (long long)grow * a.ldc + n;
-              float v[4] = {sum[u].x * a.scale, sum[u].y * a.scale, sum[u].z * a.scale, sum[u].w * a.scale};
-              if (f.bias) {
-                float br = 0.f;
-                if (f.bias_m)
-                  br = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[grow]) : reinterpret_cast<const float*>(a.bias)[grow];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) v[e] += f.bias_m ? br : bq[e];
-              }
-              if (f.relu) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) v[e] = fmaxf(v[e], 0.f);
-              }
-              if (f.mask) {
-                float mf[4];
-                if (f.mask_bf16) {
-                  const uint2 mw = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.mask) + off);
-                  mf[0] = bf16_bits_to_float(mw.x & 0xFFFFu); mf[1] = bf16_bits_to_float(mw.x >> 16);
-                  mf[2] = bf16_bits_to_float(mw.y & 0xFFFFu); mf[3] = bf16_bits_to_float(mw.y >> 16);
-                } else {
-                  const float4 mw = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.mask) + off);
-                  mf[0] = mw.x; mf[1] = mw.y; mf[2] = mw.z; mf[3] = mw.w;
-                }
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (!(mf[e] > 0.f)) v[e] = 0.f;
-              }
-#pragma unroll
-              for (int e = 0; e < 4; ++e) cs[e] += v[e];
-              if (f.resid) {
-                if (a.resid_bf16) {
-                  const uint2 rw = *reinterpret_cast<const uint2*>(reinterpret_cast<const __nv_bfloat16*>(a.resid) + off);
-                  v[0] += bf16_bits_to_float(rw.x & 0xFFFFu); v[1] += bf16_bits_to_float(rw.x >> 16);
-                  v[2] += bf16_bits_to_float(rw.y & 0xFFFFu); v[3] += bf16_bits_to_float(rw.y >> 16);
-                } else {
-                  const float4 rw = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.resid) + off);
-                  v[0] += rw.x; v[1] += rw.y; v[2] += rw.z; v[3] += rw.w;
-                }
-              }
-              if (f.c_bf16)
-                *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off) = make_uint2(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]));
-              else
-                *reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off) = make_float4(v[0], v[1], v[2], v[3]);
-            }
-          }
-          if (f.rsum) {                                      // lanes that share columns add up, the first of each set reports
-            for (int o = lanes_per_row; o < 32; o <<= 1) {
-#pragma unroll
-              for (int e = 0; e < 4; ++e) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], o);
-            }
-            if (lr == 0 && col_ok) {
-#pragma unroll
-              for (int e = 0; e < 4; ++e) atomicAdd(a.rsum + n + e, cs[e]);
-            }
-          }
-        }
+        __syncwarp();
       }
     }
   }
@@ -1072,6 +1032,29 @@ int sm_count() {
   return n;
 }
 
+// Clears 32-bit words (the fused reduce_sum output, the arrival counters of shared tiles).  A kernel
+// rather than a memset so that it can sit in a chain of programmatically dependent launches: it
+// waits for the kernel before it, and the contraction after it overlaps its set-up with this one.
+__global__ void zero_words_kernel(uint32_t* p, long long n) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) p[i] = 0u;
+}
+
+mtf_status zero_words(void* p, long long n, cudaStream_t st) {
+  if (n <= 0) return MTF_OK;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  const long long blocks = std::min<long long>((n + 255) / 256, 4 * sm_count());
+  cfg.gridDim = dim3((unsigned)blocks, 1, 1); cfg.blockDim = dim3(256, 1, 1); cfg.stream = st; cfg.attrs = at; cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, zero_words_kernel, reinterpret_cast<uint32_t*>(p), n);
+  if (e != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "zero_words_kernel: %s", cudaGetErrorString(e));
+  mtf::count_launch();
+  return MTF_OK;
+}
+
 // One kernel variant: shared-memory opt-in and the number of clusters that can be resident at once
 // are looked up on first use; the grid is that many clusters (persistent) or fewer.
 template <bool kPair, int CM, int CN, int EPI>
@@ -1147,10 +1130,10 @@ size_t tc_workspace_bytes(const TcParams& t) {
     // two fp32 fragments per tile plus counters, for tiles of up to 512 rows (upper bound over the tile shapes)
     int64_t area = ((t.M / t.sm + 511) / 512 * 512) * t.sm * (((t.N / t.sn + t.block_n - 1) / t.block_n) * t.block_n) * t.sn;
     for (int j = 0; j < t.n_outer; ++j) area *= t.outer_size[j];
-    return (size_t)area * 2 * sizeof(float) + (size_t)(area / (32 * 64)) * 2 * sizeof(unsigned) + 1024;
+    return (size_t)area * 2 * sizeof(float) + (size_t)(area / (32 * 64)) * 4 * sizeof(unsigned) + 1024;
   }
   const int64_t tiles = tc_total_tiles(t);
-  return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * 2 * sizeof(unsigned) + 256;
+  return (size_t)tiles * t.sk * tc_tile_rows(t) * t.block_n * sizeof(float) + (size_t)tiles * (tc_tile_rows(t) / 32) * 4 * sizeof(unsigned) + 256;
 }
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
@@ -1214,7 +1197,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.resid = resid; a.resid_bf16 = dtRes == MTF_BF16;
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
-  a.ws_partials = nullptr; a.ws_counters = nullptr;
+  a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
   a.kb_tile = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
   a.slots = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.sk : 2;
   a.balanced = 0;
@@ -1229,13 +1212,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     const long long rounds = (a.total_tiles + workers - 1) / workers;
     const bool worth = a.total_tiles >= workers && (double)a.total_tiles / (double)(rounds * workers) <= 0.92;
     const size_t part_bytes = (size_t)a.total_tiles * 2 * tile_rows * a.block_n * sizeof(float);
-    const size_t cnt_bytes = (size_t)a.total_tiles * (tile_rows / 32) * 2 * sizeof(unsigned);
+    a.ws_ncounters = a.total_tiles * (tile_rows / 32) * 2;
+    const size_t cnt_bytes = (size_t)a.ws_ncounters * 2 * sizeof(unsigned);     // arrivals, fragments written
     if (worth && workspace_bytes >= ((part_bytes + 255) / 256) * 256 + cnt_bytes) {
       a.balanced = 1;
       a.ws_partials = reinterpret_cast<float*>(workspace);
       a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
-      cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, cnt_bytes, st);
-      if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+      mtf_status zs = zero_words(a.ws_counters, (long long)(cnt_bytes / sizeof(unsigned)), st);
+      if (zs != MTF_OK) return zs;
     }
   }
   if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
@@ -1245,13 +1229,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     const size_t part_bytes = (size_t)a.total_tiles * a.sk * tile_rows * a.block_n * sizeof(float);
     a.ws_partials = reinterpret_cast<float*>(workspace);
     a.ws_counters = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(workspace) + ((part_bytes + 255) / 256) * 256);
-    cudaError_t e = cudaMemsetAsync(a.ws_counters, 0, (size_t)a.total_tiles * (tile_rows / 32) * 2 * sizeof(unsigned), st);
-    if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    a.ws_ncounters = a.total_tiles * (tile_rows / 32) * 2;
+    mtf_status zs = zero_words(a.ws_counters, a.ws_ncounters * 2, st);
+    if (zs != MTF_OK) return zs;
   }
 
   if (rsum) {
-    cudaError_t e = cudaMemsetAsync(rsum, 0, (size_t)t.N * sizeof(float), st);
-    if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    mtf_status zs = zero_words(rsum, t.N, st);
+    if (zs != MTF_OK) return zs;
   }
   CUtensorMap map_a, map_b, map_c, map_m;
   mtf_status s;
@@ -1280,8 +1265,9 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // epilogue kind: the common combinations have kernels of their own, everything else (and every
   // launch that assembles tiles from fragments) takes the generic one
   int epi = EPI_GENERIC;
-  if (!a.ws_partials && scale == 1.f && !resid) {
+  if (scale == 1.f && !resid) {
     if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
+    else if (a.ws_partials) epi = EPI_GENERIC;
     else if (bias && !a.bias_along_m && relu && !mask && !rsum && a.c_bf16) epi = EPI_BIAS_RELU_BF16;
     else if (a.mask_tma && rsum && !bias && !relu) epi = EPI_MASK_RSUM_BF16;
   }
