@@ -552,13 +552,18 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 // 16 KB / CN + 16 KB / CM per k-block through L2 instead of 32 KB.  A stage may be refilled when
 // every pair that reads what this CTA writes has retired its MMAs: CM + CN - 1 pair leaders signal
 // each CTA's "empty" barrier.
-template <bool kPair, int CM, int CN, int EPI>
+template <bool kPair, int CM, int CN, int EPI, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
                     const __grid_constant__ CUtensorMap map_w, const TcArgs a) {
-  constexpr int kStages = kPair ? 5 : 3;
-  constexpr int kStageBytes = kPair ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
+  // kWide (pairs only): the pair owns a 256 x 512 tile, which fills the tensor memory: one accumulator,
+  // so a tile's epilogue is not overlapped with the next tile's MMAs, but a CTA pulls 48 KB per
+  // k-block through L2 for twice the flops (24 KB per 256 x 256 x 64 instead of 32 KB).  For long K,
+  // where the contraction is bound by the L2-to-SM traffic and the exposed epilogue is small.
+  static_assert(!kWide || (kPair && CM == 1 && CN == 1), "wide tiles: plain CTA pairs only");
+  constexpr int kStages = (kPair && !kWide) ? 5 : 3;
+  constexpr int kStageBytes = (kPair && !kWide) ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
   constexpr int kTileRows = kPairRows * CM;            // rows of C owned by a work item
   constexpr bool kCluster = CM * CN > 1;
@@ -622,7 +627,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  const int n_local = kPair ? a.block_n / 2 : a.block_n;       // N columns of B this CTA stages
+  const int n_local = kPair ? a.block_n / 2 : a.block_n;       // N columns of B this CTA stages (wide: two runs of 128)
   const uint32_t b_bytes = (uint32_t)n_local * BK * 2;
 
   if (warp == 0) {
@@ -673,7 +678,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             else tma_load_5d_multicast(sb + (uint32_t)(pm * (n_local / CM)) * 128u, &map_b, fb, mask, k0, n0 + pm * (n_local / CM), tl.o[2], tl.o[1], tl.o[0]);
           } else
 #endif
-          if (a.b_mn_major) {
+          if (kWide) {
+            // columns [256 j + 128 rank, + 128) of the tile for MMA j = 0, 1: two runs of 128, 16 KB each
+            for (int h2 = 0; h2 < 2; ++h2) {
+              const int nh = tl.n0 + 256 * h2 + cta_rank * 128;
+              if (a.b_mn_major) {
+                tma_load_5d<kPair>(sb + 16384 * h2, &map_b, fb, nh, k0, tl.o[2], tl.o[1], tl.o[0]);
+                tma_load_5d<kPair>(sb + 16384 * h2 + 8192, &map_b, fb, nh + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
+              } else {
+                tma_load_5d<kPair>(sb + 16384 * h2, &map_b, fb, k0, nh, tl.o[2], tl.o[1], tl.o[0]);
+              }
+            }
+          } else if (a.b_mn_major) {
             for (int j = 0; j < n_local / 64; ++j)
               tma_load_5d<kPair>(sb + 8192 * j, &map_b, fb, n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
@@ -687,7 +703,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------- MMA issuer (even CTA of a pair only) -------
     if (lane == 0 && leader) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.a_mn_major << 15) |
-                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)(a.block_n >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+                             ((uint32_t)a.b_mn_major << 16) | ((uint32_t)((kWide ? 256 : a.block_n) >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
       // completion signals: this pair's two CTAs, and every CTA whose loads land in this pair's tiles
       // (the pairs of this pair's cluster row and column)
       const uint16_t pair_mask = (uint16_t)(3u << (2 * pair_idx));
@@ -705,8 +721,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       Seg sg;
       for (; ok && it.next(sg); ++iter) {
         const int kb_count = sg.kb_count;
-        const int acc = iter & 1;
-        const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
+        const int acc = kWide ? 0 : (iter & 1);
+        const uint32_t acc_phase = kWide ? ((uint32_t)iter & 1u) : ((uint32_t)(iter >> 1) & 1u);
         if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, 0x200 + acc, abort_flag))) break;
         tcgen05_fence_after();
         const uint32_t tmem_c = tmem_base + (uint32_t)acc * kMaxBN;
@@ -720,6 +736,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const uint64_t da = make_smem_desc(sa + k * a_kstep, a.a_mn_major);
             const uint64_t db = make_smem_desc(sb + k * b_kstep, a.b_mn_major);
             umma_bf16<kPair>(tmem_c, da, db, idesc, (kb | k) != 0);
+            if (kWide) umma_bf16<kPair>(tmem_c + 256u, da, make_smem_desc(sb + 16384u + k * b_kstep, a.b_mn_major), idesc, (kb | k) != 0);
           }
           umma_commit<kPair>(empty_bar(stage), empty_mask);   // frees the stage in every CTA that writes into this pair's tiles
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -747,8 +764,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       Tile tl = decode_tile(a, t, kTileRows, a.block_n * CN);
       tl.m0 += pm * kPairRows;            // this pair's 256 x block_n part of the cluster's super-tile
       tl.n0 += pn * a.block_n;
-      const int acc = iter & 1;
-      const uint32_t acc_phase = (uint32_t)(iter >> 1) & 1u;
+      const int acc = kWide ? 0 : (iter & 1);
+      const uint32_t acc_phase = kWide ? ((uint32_t)iter & 1u) : ((uint32_t)(iter >> 1) & 1u);
       const int pair_row = cta_rank * BM + q * 32 + lane;       // row inside the pair's part of the tile
       const int tile_row = pm * kPairRows + pair_row;            // row inside the work item's tile
       const int row = tl.m0 + pair_row;
@@ -1057,7 +1074,7 @@ mtf_status zero_words(void* p, long long n, cudaStream_t st) {
 
 // One kernel variant: shared-memory opt-in and the number of clusters that can be resident at once
 // are looked up on first use; the grid is that many clusters (persistent) or fewer.
-template <bool kPair, int CM, int CN, int EPI>
+template <bool kPair, int CM, int CN, int EPI, bool kWide = false>
 mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
                           const CUtensorMap& map_w, const TcArgs& a, cudaStream_t st) {
   constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
@@ -1065,9 +1082,9 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   static cudaError_t attr_err = cudaSuccess;
   static int max_clusters = 0;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (attr_err != cudaSuccess) return;
-    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (attr_err != cudaSuccess) return;
     if (kCtas == 1) { max_clusters = sm_count(); return; }
     cudaLaunchConfig_t q = {};
@@ -1077,7 +1094,7 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     q.gridDim = dim3(kCtas * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
     q.attrs = at; q.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI>, &q) == cudaSuccess && n > 0) max_clusters = n;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, &q) == cudaSuccess && n > 0) max_clusters = n;
     else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
   });
   if (attr_err != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
@@ -1091,7 +1108,7 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   at[1].val.clusterDim.x = kCtas; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   cfg.gridDim = dim3((unsigned)(kCtas * clusters), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = kCtas > 1 ? 2 : 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI>, map_a, map_b, map_c, map_m, map_w, a);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, map_a, map_b, map_c, map_m, map_w, a);
   if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d,%d>: %s", (int)kPair, CM, CN, EPI, cudaGetErrorString(le));
   return MTF_OK;
 }
@@ -1162,10 +1179,24 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.ldc = t.ldc;
   a.reduce_mode = t.reduce_mode;
   a.k_sliced = (t.sk > 1 && a.Ks % BK == 0) ? 1 : 0;
+  // Wide tiles (256 x 512 per pair) for long contractions with a plain epilogue: per tile about 1.5x
+  // the time of a 256 x 256 one (twice the MMAs at 3/4 of the L2 traffic each, epilogue exposed), so
+  // they win when they halve the number of waves.
+  bool wide = false;
+  const bool plain_epi = scale == 1.f && !resid && !bias && !relu && !mask && !rsum;
+  if (t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && a.Ns % 512 == 0 && t.K >= 64 * BK) {
+    long long tiles = (long long)((a.Ms + 2 * BM - 1) / (2 * BM)) * (a.Ns / 256) * a.sm * a.sn;
+    for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
+    const long long workers = sm_count() / 2;
+    const long long waves_narrow = (tiles + workers - 1) / workers, waves_wide = (tiles / 2 + workers - 1) / workers;
+    wide = 3 * waves_wide < 2 * waves_narrow;
+    if (const char* dbg = getenv("MTF_DBG_WIDE")) wide = dbg[0] == '1';
+  }
+  if (wide) a.block_n = 512;
   // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads
   int cm = 1, cn = 1;
 #if defined(MTF_TMA_MULTICAST)
-  if (t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
+  if (!wide && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
     // measured on the FFN shapes: sharing B between two pairs that are neighbours along M is worth
     // 5-10 % on the contractions whose epilogue is light; with a relu mask or a fused reduction in the
     // epilogue the coupling of the two pairs costs more than the saved traffic; 2 x 2 clusters lose
@@ -1204,7 +1235,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (t.balance && cn == 1 && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+  if (t.balance && cn == 1 && !wide && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
     // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
     // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
     // the workspace by whichever worker finishes last (arrive, never wait).
@@ -1272,7 +1303,10 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     else if (a.mask_tma && rsum && !bias && !relu) epi = EPI_MASK_RSUM_BF16;
   }
   mtf_status ls;
-  if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
+  if (wide) {
+    if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, a, st);
+    else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, a, st);
+  } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
 #if defined(MTF_TMA_MULTICAST)
   else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
   else if (cm == 2 && cn == 1) ls = launch_kind<true, 2, 1, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
