@@ -184,7 +184,9 @@ mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* eq
                                       void* stream);
 /* Testing hook: force the kernel family / reduce mode of plans created afterwards by this thread
  * (-1 = planner's choice; kernel_kind 2 = tensor cores with one CTA per tile, i.e. without the
- * two-CTA pairs the planner prefers on tall slices; reduce_mode 3 = keep the planner's reduce mode
+ * two-CTA pairs the planner prefers on tall slices; kernel_kind 3 / 4 = tensor cores with the
+ * 256 x 512 pair tiles wherever the shape allows them (pairs, plain epilogue, N slice a multiple of
+ * 512) / never, instead of the launcher's count of waves; reduce_mode 3 = keep the planner's reduce mode
  * but, where the output tiles leave a partly filled last wave, give every worker an equal range of
  * (tile, k-block) units and assemble cut tiles from fragments in the workspace).  A forced choice
  * the shape cannot run gives MTF_ERR_UNSUPPORTED. */

@@ -346,7 +346,7 @@ mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, 
 }
 
 mtf_status mtf_plan_force(int32_t kernel_kind, int32_t reduce_mode) {
-  if (kernel_kind < -1 || kernel_kind > 2 || reduce_mode < -1 || reduce_mode > 3)
+  if (kernel_kind < -1 || kernel_kind > 4 || reduce_mode < -1 || reduce_mode > 3)
     return fail(MTF_ERR_INVALID_ARG, "plan_force: value out of range");
   g_force_kernel = kernel_kind;
   g_force_reduce = reduce_mode;

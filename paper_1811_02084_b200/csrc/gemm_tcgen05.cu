@@ -1184,13 +1184,15 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // they win when they halve the number of waves.
   bool wide = false;
   const bool plain_epi = scale == 1.f && !resid && !bias && !relu && !mask && !rsum;
-  if (t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && a.Ns % 512 == 0 && t.K >= 64 * BK) {
+  const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && a.Ns % 512 == 0;
+  if (t.wide_pref == 1 && !wide_legal)
+    return fail(MTF_ERR_UNSUPPORTED, "wide tiles need CTA pairs, a plain epilogue, no workspace reduction and an N slice that is a multiple of 512");
+  if (wide_legal && t.wide_pref != 0) {
     long long tiles = (long long)((a.Ms + 2 * BM - 1) / (2 * BM)) * (a.Ns / 256) * a.sm * a.sn;
     for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
     const long long workers = sm_count() / 2;
     const long long waves_narrow = (tiles + workers - 1) / workers, waves_wide = (tiles / 2 + workers - 1) / workers;
-    wide = 3 * waves_wide < 2 * waves_narrow;
-    if (const char* dbg = getenv("MTF_DBG_WIDE")) wide = dbg[0] == '1';
+    wide = t.wide_pref == 1 || (t.K >= 64 * BK && 3 * waves_wide < 2 * waves_narrow);
   }
   if (wide) a.block_n = 512;
   // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads

@@ -90,6 +90,7 @@ struct TcParams {
   int64_t a_ld = 0, b_ld = 0;                // element stride of the non-contiguous one of (M|N, K)
   int64_t ldc = 0;                           // element stride of M in C (N is contiguous)
   int block_n = 256;
+  int wide_pref = -1;                        // 256 x 512 pair tiles: -1 = launcher's wave heuristic, 0 = never, 1 = wherever the shape allows
   int balance = 0;                           // tiles leave a partly filled last wave: balanced k-range schedule (needs workspace)
   int cta_pair = 0;                          // two CTAs (a cluster) own a 256-row tile, tcgen05 cta_group::2
   int swapped = 0;                           // in[0] and in[1] exchanged so that N is contiguous in C

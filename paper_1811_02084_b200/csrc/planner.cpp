@@ -461,8 +461,10 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
   // ---- kernel family and reduce mode ----
   std::string why;
   const int force_single_cta = force_kernel == 2 ? 1 : 0;     // testing hook: tensor cores without CTA pairs
-  if (force_kernel == 2) force_kernel = MTF_KERNEL_TCGEN05;
+  const int wide_pref = force_kernel == 3 ? 1 : (force_kernel == 4 ? 0 : -1);   // testing hook: wide pair tiles always / never
+  if (force_kernel >= 2) force_kernel = MTF_KERNEL_TCGEN05;
   bool tc_ok = plan_tc(P.get(), &why, force_single_cta);
+  if (tc_ok) P->tc.wide_pref = wide_pref;
   if (!P->has_B && force_kernel == MTF_KERNEL_TCGEN05) force_kernel = -1;   // forcing concerns contractions only
   if (!P->has_B && force_reduce == MTF_REDUCE_WORKSPACE) force_reduce = -1;
   if (force_kernel == MTF_KERNEL_TCGEN05 && !tc_ok) return fail(MTF_ERR_UNSUPPORTED, "tensor-core path cannot run this einsum: %s", why.c_str());

@@ -99,6 +99,52 @@ def test_tensor_core_operand_majors(mtf, name, out_dtype, kind):
     assert parity_error(got, ref) <= TOL["bf16"]
 
 
+# 256 x 512 pair tiles (kernel_kind 3 forces them; the launcher refuses shapes they cannot run):
+# ragged M, several k-blocks with a remainder, every operand major-ness, both output types
+WIDE = {
+    "K-major x MN-major": ([("i", 300), ("k", 200)], [("k", 200), ("j", 1024)]),
+    "K-major x K-major": ([("i", 300), ("k", 200)], [("j", 1024), ("k", 200)]),
+    "MN-major x MN-major": ([("k", 200), ("i", 304)], [("k", 200), ("j", 1024)]),
+    "MN-major x K-major": ([("k", 200), ("i", 304)], [("j", 1024), ("k", 200)]),
+}
+
+
+@pytest.mark.parametrize("name", list(WIDE))
+@pytest.mark.parametrize("out_dtype", ["bf16", "f32"])
+def test_wide_pair_tiles(mtf, name, out_dtype):
+    a, b = WIDE[name]
+    out_dims = [a[0] if a[0][0] == "i" else a[1], b[1] if b[1][0] == "j" else b[0]]
+    got, ref, info = run_einsum(mtf, layout(mtf, [("all", 1)], []), [a, b], out_dims, "bf16", out_dtype, force=(3, -1))
+    assert info["kernel_kind"] == mtf.MTF_KERNEL_TCGEN05
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("mesh_dims,rules", [([("all", 2)], [("j", "all")]), ([("all", 4)], [("k", "all")]),
+                                             ([("a", 2), ("b", 2)], [("o", "a"), ("k", "b")])],
+                         ids=["n-split", "k-split-chained", "m-and-k-split"])
+def test_wide_pair_tiles_under_layouts(mtf, mesh_dims, rules):
+    # several tiles per worker in sequence (single accumulator: each tile's epilogue must finish
+    # before the next tile's first MMA), batch dim, split N (slices of 512) and chained group sums
+    a, b = [("o", 4), ("i", 960), ("k", 512)], [("k", 512), ("j", 1024)]      # o and i merge into M = 3840
+    k_split = any(t == "k" for t, _ in rules)       # (the workspace reduce mode has no wide tiles: ask for the chained one)
+    got, ref, info = run_einsum(mtf, layout(mtf, mesh_dims, rules), [a, b], [("o", 4), ("i", 960), ("j", 1024)], "bf16",
+                                force=(3, 1 if k_split else -1))
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
+def test_wide_pair_tiles_refuse_what_they_cannot_run(mtf):
+    lay = layout(mtf, [("all", 1)], [])
+    with pytest.raises(mtf.MtfError) as e:      # N is not a multiple of 512
+        run_einsum(mtf, lay, [[("i", 512), ("k", 128)], [("k", 128), ("j", 768)]], [("i", 512), ("j", 768)], "bf16", force=(3, -1))
+    assert e.value.code == "MTF_ERR_UNSUPPORTED"
+    with pytest.raises(mtf.MtfError) as e:      # not a plain epilogue
+        run_einsum(mtf, lay, [[("i", 512), ("k", 128)], [("k", 128), ("j", 1024)]], [("i", 512), ("j", 1024)], "bf16", force=(3, -1),
+                   epilogue={"relu": True})
+    assert e.value.code == "MTF_ERR_UNSUPPORTED"
+    got, ref, _ = run_einsum(mtf, lay, [[("i", 512), ("k", 128)], [("k", 128), ("j", 1024)]], [("i", 512), ("j", 1024)], "bf16", force=(4, -1))
+    assert parity_error(got, ref) <= TOL["bf16"]
+
+
 def test_tensor_core_transposed_output_swaps_operands(mtf):
     # out[j, i]: the contiguous output dim comes from the first operand
     a, b = [("i", 256), ("k", 128)], [("k", 128), ("j", 192)]
