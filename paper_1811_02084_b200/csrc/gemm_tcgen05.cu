@@ -97,6 +97,7 @@ struct TcArgs {
   const void* mask;
   int mask_bf16;
   int mask_tma;            // bf16 mask boxes are loaded by TMA into the output staging buffers (bf16 output only)
+  int resid_tma;           // residual boxes (same type as the output) are loaded the same way when there is no mask
   const void* resid;
   int resid_bf16;
   float scale;
@@ -384,18 +385,18 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
 // far fewer registers and instructions per chunk.
 enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_KINDS = 5 };
 struct EpiFlags {
-  bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, rsum, c_bf16, shared_tiles;
+  bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
 };
 template <int EPI>
 __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
   EpiFlags f;
   if (EPI == EPI_GENERIC) {
     f.scale = a.scale != 1.f; f.bias = a.bias != nullptr; f.bias_m = a.bias_along_m != 0; f.relu = a.relu != 0;
-    f.mask = a.mask != nullptr; f.mask_bf16 = a.mask_bf16 != 0; f.mask_tma = a.mask_tma != 0; f.resid = a.resid != nullptr;
+    f.mask = a.mask != nullptr; f.mask_bf16 = a.mask_bf16 != 0; f.mask_tma = a.mask_tma != 0; f.resid = a.resid != nullptr; f.resid_tma = a.resid_tma != 0;
     f.rsum = a.rsum != nullptr; f.c_bf16 = a.c_bf16 != 0; f.shared_tiles = true;
   } else {
     f.scale = false; f.bias = EPI == EPI_BIAS_RELU_BF16; f.bias_m = false; f.relu = EPI == EPI_BIAS_RELU_BF16;
-    f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = false;
+    f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = f.resid_tma = false;
     f.c_bf16 = EPI != EPI_PLAIN_F32;
     f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
   }
@@ -783,16 +784,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         bias_row = a.bias_bf16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.bias)[row]) : reinterpret_cast<const float*>(a.bias)[row];
       const int row0 = tl.m0 + cta_rank * BM + q * 32;           // first row of this warp
       const bool rows_full = row0 + 32 <= tl.m_end;
+      // an epilogue operand that arrives box by box in the staging buffers and is consumed in place:
+      // the bf16 relu mask, or the residual
       const bool mask_tma = f.mask_tma && !ws_mode && rows_full;
-      if (mask_tma && lane == 0) {
-        // pull this warp's boxes of the mask tile towards L2 and request the first one into the
+      const bool resid_tma = f.resid_tma && !ws_mode && rows_full;
+      const bool in_tma = mask_tma || resid_tma;
+      const int box_cols = f.c_bf16 ? 64 : 32;
+      if (in_tma && lane == 0) {
+        // pull this warp's boxes of the operand's tile towards L2 and request the first one into the
         // staging box it will be processed in (free once all but the latest store have been read out)
-        for (int b = col_half * 64; b < a.block_n; b += 128)
-          if (tl.n0 + b + 64 <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
-        if (col_half * 64 < a.block_n && tl.n0 + col_half * 64 + 64 <= tl.n_end) {
+        for (int b = col_half * box_cols; b < a.block_n; b += 2 * box_cols)
+          if (tl.n0 + b + box_cols <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
+        if (col_half * box_cols < a.block_n && tl.n0 + col_half * box_cols + box_cols <= tl.n_end) {
           asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
           mbar_expect_tx(mfull_bar(buf), 4096u);
-          tma_load_5d<false>(stg + buf * 4096u, &map_m, mfull_bar(buf), tl.n0 + col_half * 64, row0, tl.o[2], tl.o[1], tl.o[0]);
+          tma_load_5d<false>(stg + buf * 4096u, &map_m, mfull_bar(buf), tl.n0 + col_half * box_cols, row0, tl.o[2], tl.o[1], tl.o[0]);
         }
       }
       ok = mbar_wait_warp(tfull_bar(acc), acc_phase, 0x400 + acc, abort_flag, lane);
@@ -833,7 +839,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
-        const int box_cols = f.c_bf16 ? 64 : 32;
         float bias_cur = bias_at(tl.n0 + col_half * box_cols + lane);      // lane l keeps column l of the current chunk
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
@@ -849,7 +854,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const int half = (c0 >> 5) & 1;
           const uint32_t box = stg + buf * 4096u;
           if (staged && (c0 & (box_cols - 1)) == 0) {           // first chunk of a box
-            if (mask_tma) {                                     // its relu mask was requested a box ago, in place
+            if (in_tma) {                                       // its mask / residual was requested a box ago, in place
               mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag);
               mask_phase ^= 1u << buf;
             } else {                                            // the box must be free: all but the latest store read out
@@ -895,7 +900,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
           epilogue_math(a, f, v, bias_cur, bias_row, mk, row_off + n_first, live, n_valid);
           bias_cur = bias_next;
-          epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
+          if (staged && resid_tma) {                 // this lane's part of the residual box, where the result will go
+            const uint32_t srow = box + (uint32_t)lane * 128u;
+            const uint32_t sw = (uint32_t)(lane & 7);
+            if (f.c_bf16) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                float r8[8];
+                unpack_bf16x8(ld_shared_v4(srow + ((((uint32_t)(half * 4 + i)) ^ sw) << 4)), r8);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[i * 8 + e] += r8[e];
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const uint4 r4 = ld_shared_v4(srow + (((uint32_t)i ^ sw) << 4));
+                v[4 * i] += __uint_as_float(r4.x); v[4 * i + 1] += __uint_as_float(r4.y);
+                v[4 * i + 2] += __uint_as_float(r4.z); v[4 * i + 3] += __uint_as_float(r4.w);
+              }
+            }
+          } else {
+            epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
+          }
           if (staged) store_staged(f, v, box, lane, half);
           else if (live) store_direct(a, f, v, row_off + n_first, n_valid);
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
@@ -905,7 +931,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
               // request the mask of this warp's next box of the tile into the other staging box
               const int next_n0 = box_n0 + 2 * box_cols;
-              if (mask_tma && next_n0 < tl.n0 + a.block_n && next_n0 + box_cols <= tl.n_end) {
+              if (in_tma && next_n0 < tl.n0 + a.block_n && next_n0 + box_cols <= tl.n_end) {
                 asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                 mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
                 tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
@@ -927,7 +953,6 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // fragment `ks` of the tile -> workspace, the way a finished tile leaves: 32-row x 128-byte
         // boxes through the staging buffers and TMA stores (the chunks this warp owns in the regular
         // epilogue, so that the finisher finds them under the same counter)
-        const int box_cols = f.c_bf16 ? 64 : 32;
         const long long part_row0 = (t * a.slots + ks) * (long long)kTileRows + warp_tile_row;
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
@@ -1228,6 +1253,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.mask = mask; a.mask_bf16 = dtMask == MTF_BF16;
   a.mask_tma = (mask && a.mask_bf16 && a.c_bf16) ? 1 : 0;
   a.resid = resid; a.resid_bf16 = dtRes == MTF_BF16;
+  a.resid_tma = (resid && !a.mask_tma && a.resid_bf16 == a.c_bf16) ? 1 : 0;
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
@@ -1285,6 +1311,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if ((s = make_map(&map_c, C, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
   map_m = map_c;
   if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
+  if (a.resid_tma && (s = make_map(&map_m, resid, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
   // fragments of shared tiles: the workspace as one fp32 matrix of block_n columns, a tile slot after the other
   CUtensorMap map_w = map_c;
   if (a.ws_partials) {
