@@ -34,7 +34,7 @@ bool dims_match(const std::vector<Dim>& want, const mtf_tensor& t) {
 }
 
 mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epi,
-                     void* workspace, size_t workspace_bytes, void* stream) {
+                     void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1, const void* const* extra_operands = nullptr) {
   if (!P || !in || !out) return fail(MTF_ERR_INVALID_ARG, "einsum exec: NULL argument");
   if (!dims_match(P->dimsA, in[0]) || (P->has_B && !dims_match(P->dimsB, in[1])) || !dims_match(P->dimsC, *out))
     return fail(MTF_ERR_SIZE_MISMATCH, "einsum exec: operand dims differ from the planned ones");
@@ -74,7 +74,8 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
   const int relu = P->epi.on ? (epi->relu != 0) : 0;
   if (P->kernel_kind == MTF_KERNEL_TCGEN05)
     return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
-                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream);
+                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands);
+  if (n_terms != 1) return fail(MTF_ERR_UNSUPPORTED, "multi-term contraction on the generic kernel");
   SimtParams s = P->simt;
   s.A = in[0].data;
   s.B = P->has_B ? in[1].data : nullptr;
@@ -439,6 +440,28 @@ mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, con
 }
 
 }  // extern "C"
+
+mtf_status mtf::einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tensor (*terms)[2], mtf_tensor* out,
+                             const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!layout || !terms || !out || n_terms < 1 || n_terms > 3) return fail(MTF_ERR_INVALID_ARG, "einsum_terms: bad argument");
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 2, terms[0], out, epilogue, &P);
+  if (st != MTF_OK) return st;
+  if (n_terms == 1) return exec_plan(P, terms[0], out, epilogue, workspace, workspace_bytes, stream);
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->reduce_mode == MTF_REDUCE_WORKSPACE)
+    return fail(MTF_ERR_UNSUPPORTED, "einsum_terms: this plan takes one product per launch");
+  const void* extra[4] = {nullptr, nullptr, nullptr, nullptr};
+  for (int i = 1; i < n_terms; ++i)
+    for (int q = 0; q < 2; ++q) {
+      const mtf_tensor& a = terms[0][q];
+      const mtf_tensor& b = terms[i][q];
+      bool same = a.ndim == b.ndim && a.dtype == b.dtype && b.data != nullptr;
+      for (int d = 0; same && d < a.ndim; ++d) same = a.dims[d].size == b.dims[d].size;
+      if (!same) return fail(MTF_ERR_SIZE_MISMATCH, "einsum_terms: term %d operand %d differs in shape or type from term 0", i, q);
+      extra[2 * (i - 1) + q] = b.data;
+    }
+  return exec_plan(P, terms[0], out, epilogue, workspace, workspace_bytes, stream, n_terms, extra);
+}
 
 // dx_residual (NULL or a tensor with dx's dims) is added to dx in the last einsum's epilogue.
 mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,

@@ -298,6 +298,13 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   // last einsum adds the running sum and writes dx once
   mtf_epilogue er = epi_none();
   er.residual = dx_residual;
+  {
+    // one launch where the plan allows it: the k loop runs through dq.wq, then dkk.wk, then dvv.wv
+    // into one accumulator (same shapes; the key / value side carries the memory_length name)
+    const mtf_tensor terms[3][2] = {{dq.t, *wq}, {dkk.t, *wk}, {dvv.t, *wv}};
+    st = mtf::einsum_terms(layout, 3, terms, dx, dx_residual ? &er : nullptr, rest, rest_bytes, stream);
+    if (st != MTF_ERR_UNSUPPORTED) return st;
+  }
   if ((st = ein(layout, dq.t, *wq, &dx32.t, dx_residual ? &er : nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   TD dx32m = renamed(dx32.t, s.l.name, kMemory);
   mtf_epilogue ea = epi_none();

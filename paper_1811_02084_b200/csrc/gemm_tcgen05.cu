@@ -88,7 +88,9 @@ struct TcArgs {
   int n_fastest;           // tile order inside a slice: 1 = walk the n tiles of one m tile first
   long long tiles_per_slice, total_tiles, total_work;
   int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
-  int kb_tile;             // k-blocks of one whole tile
+  int kb_tile;             // k-blocks of one whole tile (all terms)
+  int n_terms;             // sum of n_terms products A_i . B_i of identical shape in one accumulator (1..3)
+  int kb_term;             // k-blocks of one term
   int slots;               // partial-tile slots per tile in the workspace (sk, or 2 when balanced)
   void* C;
   int c_bf16;
@@ -107,6 +109,11 @@ struct TcArgs {
   unsigned* ws_counters;     // per (tile, 32-row group, column part): arrivals, then as many again: fragments written
   long long ws_ncounters;
   FastDiv fd_tiles_per_slice, fd_n_tiles, fd_m_tiles, fd_outer_local[3], fd_sn, fd_sm, fd_outer_split[3], fd_sk;
+};
+
+// Operand maps of the second and third product of a multi-term launch (A_1, B_1, A_2, B_2).
+struct ExtraMaps {
+  CUtensorMap m[4];
 };
 
 struct Tile {
@@ -557,7 +564,7 @@ template <bool kPair, int CM, int CN, int EPI, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
-                    const __grid_constant__ CUtensorMap map_w, const TcArgs a) {
+                    const __grid_constant__ CUtensorMap map_w, const __grid_constant__ ExtraMaps extra, const TcArgs a) {
   // kWide (pairs only): the pair owns a 256 x 512 tile, which fills the tensor memory: one accumulator,
   // so a tile's epilogue is not overlapped with the next tile's MMAs, but a CTA pulls 48 KB per
   // k-block through L2 for twice the flops (24 KB per 256 x 256 x 64 instead of 32 KB).  For long K,
@@ -644,10 +651,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const Tile tl = decode_tile(a, sg.tile, kTileRows, a.block_n * CN);
         const int m0 = tl.m0 + pm * kPairRows + cta_rank * BM;
         const int n0 = tl.n0 + pn * a.block_n + cta_rank * n_local;
+        int term = kb_first / a.kb_term, kt = kb_first - term * a.kb_term;
         for (int kb = 0; kb < kb_count; ++kb) {
           // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
-          // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor)
-          const int k0 = (kb_first + kb) * BK;
+          // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor); a
+          // multi-term launch then goes on with the next product's operands
+          const int k0 = kt * BK;
+          const CUtensorMap* const pa = term == 0 ? &map_a : &extra.m[2 * (term - 1)];
+          const CUtensorMap* const pb = term == 0 ? &map_b : &extra.m[2 * (term - 1) + 1];
+          if (++kt == a.kb_term) { kt = 0; ++term; }
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, 0x100 + stage, abort_flag))) break;
           // a pair's loads all count on the even CTA's barrier, which expects both CTAs' bytes
           if (!kPair) mbar_expect_tx(full_bar(stage), kAStageBytes + b_bytes);
@@ -660,23 +672,23 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // this CTA's 1/CN share of its 128 rows of A goes to the same-position CTA of every pair in its cluster row
             uint16_t mask = 0;
             for (int j = 0; j < CN; ++j) mask |= (uint16_t)(1u << (2 * (pm * CN + j) + cta_rank));
-            if (a.a_mn_major) tma_load_5d_multicast(sa + 8192u * pn, &map_a, fb, mask, m0 + 64 * pn, k0, tl.o[2], tl.o[1], tl.o[0]);
-            else tma_load_5d_multicast(sa + (uint32_t)(pn * (BM / CN)) * 128u, &map_a, fb, mask, k0, m0 + pn * (BM / CN), tl.o[2], tl.o[1], tl.o[0]);
+            if (a.a_mn_major) tma_load_5d_multicast(sa + 8192u * pn, pa, fb, mask, m0 + 64 * pn, k0, tl.o[2], tl.o[1], tl.o[0]);
+            else tma_load_5d_multicast(sa + (uint32_t)(pn * (BM / CN)) * 128u, pa, fb, mask, k0, m0 + pn * (BM / CN), tl.o[2], tl.o[1], tl.o[0]);
           } else
 #endif
           if (a.a_mn_major) {
-            tma_load_5d<kPair>(sa, &map_a, fb, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
-            tma_load_5d<kPair>(sa + 8192, &map_a, fb, m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa, pa, fb, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa + 8192, pa, fb, m0 + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
-            tma_load_5d<kPair>(sa, &map_a, fb, k0, m0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sa, pa, fb, k0, m0, tl.o[2], tl.o[1], tl.o[0]);
           }
 #if defined(MTF_TMA_MULTICAST)
           if (CM > 1) {
             // this CTA's 1/CM share of its half of B's columns goes to the same-position CTA of every pair in its cluster column
             uint16_t mask = 0;
             for (int j = 0; j < CM; ++j) mask |= (uint16_t)(1u << (2 * (j * CN + pn) + cta_rank));
-            if (a.b_mn_major) tma_load_5d_multicast(sb + 8192u * pm, &map_b, fb, mask, n0 + 64 * pm, k0, tl.o[2], tl.o[1], tl.o[0]);
-            else tma_load_5d_multicast(sb + (uint32_t)(pm * (n_local / CM)) * 128u, &map_b, fb, mask, k0, n0 + pm * (n_local / CM), tl.o[2], tl.o[1], tl.o[0]);
+            if (a.b_mn_major) tma_load_5d_multicast(sb + 8192u * pm, pb, fb, mask, n0 + 64 * pm, k0, tl.o[2], tl.o[1], tl.o[0]);
+            else tma_load_5d_multicast(sb + (uint32_t)(pm * (n_local / CM)) * 128u, pb, fb, mask, k0, n0 + pm * (n_local / CM), tl.o[2], tl.o[1], tl.o[0]);
           } else
 #endif
           if (kWide) {
@@ -684,17 +696,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             for (int h2 = 0; h2 < 2; ++h2) {
               const int nh = tl.n0 + 256 * h2 + cta_rank * 128;
               if (a.b_mn_major) {
-                tma_load_5d<kPair>(sb + 16384 * h2, &map_b, fb, nh, k0, tl.o[2], tl.o[1], tl.o[0]);
-                tma_load_5d<kPair>(sb + 16384 * h2 + 8192, &map_b, fb, nh + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
+                tma_load_5d<kPair>(sb + 16384 * h2, pb, fb, nh, k0, tl.o[2], tl.o[1], tl.o[0]);
+                tma_load_5d<kPair>(sb + 16384 * h2 + 8192, pb, fb, nh + 64, k0, tl.o[2], tl.o[1], tl.o[0]);
               } else {
-                tma_load_5d<kPair>(sb + 16384 * h2, &map_b, fb, k0, nh, tl.o[2], tl.o[1], tl.o[0]);
+                tma_load_5d<kPair>(sb + 16384 * h2, pb, fb, k0, nh, tl.o[2], tl.o[1], tl.o[0]);
               }
             }
           } else if (a.b_mn_major) {
             for (int j = 0; j < n_local / 64; ++j)
-              tma_load_5d<kPair>(sb + 8192 * j, &map_b, fb, n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
+              tma_load_5d<kPair>(sb + 8192 * j, pb, fb, n0 + 64 * j, k0, tl.o[2], tl.o[1], tl.o[0]);
           } else {
-            tma_load_5d<kPair>(sb, &map_b, fb, k0, n0, tl.o[2], tl.o[1], tl.o[0]);
+            tma_load_5d<kPair>(sb, pb, fb, k0, n0, tl.o[2], tl.o[1], tl.o[0]);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -1101,7 +1113,7 @@ mtf_status zero_words(void* p, long long n, cudaStream_t st) {
 // are looked up on first use; the grid is that many clusters (persistent) or fewer.
 template <bool kPair, int CM, int CN, int EPI, bool kWide = false>
 mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
-                          const CUtensorMap& map_w, const TcArgs& a, cudaStream_t st) {
+                          const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
   constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -1133,7 +1145,7 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   at[1].val.clusterDim.x = kCtas; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   cfg.gridDim = dim3((unsigned)(kCtas * clusters), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = kCtas > 1 ? 2 : 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, map_a, map_b, map_c, map_m, map_w, a);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, map_a, map_b, map_c, map_m, map_w, extra, a);
   if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d,%d>: %s", (int)kPair, CM, CN, EPI, cudaGetErrorString(le));
   return MTF_OK;
 }
@@ -1142,14 +1154,14 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
 // shapes that are never used with a mask).
 template <bool kPair, int CM, int CN, bool kAllKinds>
 mtf_status launch_kind(int epi, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
-                       const CUtensorMap& map_w, const TcArgs& a, cudaStream_t st) {
+                       const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
   switch (epi) {
-    case EPI_PLAIN_BF16: return launch_variant<kPair, CM, CN, EPI_PLAIN_BF16>(map_a, map_b, map_c, map_m, map_w, a, st);
-    case EPI_PLAIN_F32: return launch_variant<kPair, CM, CN, EPI_PLAIN_F32>(map_a, map_b, map_c, map_m, map_w, a, st);
-    case EPI_BIAS_RELU_BF16: return launch_variant<kPair, CM, CN, EPI_BIAS_RELU_BF16>(map_a, map_b, map_c, map_m, map_w, a, st);
+    case EPI_PLAIN_BF16: return launch_variant<kPair, CM, CN, EPI_PLAIN_BF16>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    case EPI_PLAIN_F32: return launch_variant<kPair, CM, CN, EPI_PLAIN_F32>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    case EPI_BIAS_RELU_BF16: return launch_variant<kPair, CM, CN, EPI_BIAS_RELU_BF16>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     case EPI_MASK_RSUM_BF16:
-      if (kAllKinds) return launch_variant<kPair, CM, CN, kAllKinds ? EPI_MASK_RSUM_BF16 : EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, a, st);
-    default: return launch_variant<kPair, CM, CN, EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, a, st);
+      if (kAllKinds) return launch_variant<kPair, CM, CN, kAllKinds ? EPI_MASK_RSUM_BF16 : EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    default: return launch_variant<kPair, CM, CN, EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
   }
 }
 
@@ -1180,9 +1192,11 @@ size_t tc_workspace_bytes(const TcParams& t) {
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
-                     void* workspace, size_t workspace_bytes, void* stream) {
+                     void* workspace, size_t workspace_bytes, void* stream, int n_terms, const void* const* extra_operands) {
   const TcParams& t = plan.tc;
   if (t.swapped) std::swap(A, B);
+  if (n_terms < 1 || n_terms > 3 || (n_terms > 1 && !extra_operands)) return fail(MTF_ERR_INVALID_ARG, "1 to 3 terms");
+  if (n_terms > 1 && t.reduce_mode == MTF_REDUCE_WORKSPACE) return fail(MTF_ERR_UNSUPPORTED, "a multi-term contraction cannot use the workspace reduce mode");
   if (t.M > 0x7fffffffLL || t.N > 0x7fffffffLL || t.K > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "extent beyond 2^31");
   if (reinterpret_cast<uintptr_t>(C) & 15) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned output");
   if (bias && !t.bias_along_m && (reinterpret_cast<uintptr_t>(bias) & 15)) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned bias");
@@ -1217,7 +1231,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
     const long long workers = sm_count() / 2;
     const long long waves_narrow = (tiles + workers - 1) / workers, waves_wide = (tiles / 2 + workers - 1) / workers;
-    wide = t.wide_pref == 1 || (t.K >= 64 * BK && 3 * waves_wide < 2 * waves_narrow);
+    wide = t.wide_pref == 1 || (t.K * n_terms >= 64 * BK && 3 * waves_wide < 2 * waves_narrow);
   }
   if (wide) a.block_n = 512;
   // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads
@@ -1257,13 +1271,15 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
-  a.kb_tile = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
+  a.kb_term = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
+  a.n_terms = n_terms;
+  a.kb_tile = a.kb_term * n_terms;
   a.slots = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.sk : 2;
   a.balanced = 0;
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (t.balance && cn == 1 && !wide && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+  if (t.balance && cn == 1 && !wide && n_terms == 1 && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
     // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
     // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
     // the workspace by whichever worker finishes last (arrive, never wait).
@@ -1306,6 +1322,18 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (s != MTF_OK) return s;
   s = t.b_mn_major ? make_map(&map_b, B, 2, t.N, t.K, t.b_ld, 64, BK, t, t.outer_sB) : make_map(&map_b, B, 2, t.K, t.N, t.b_ld, 64, b_rows, t, t.outer_sB);
   if (s != MTF_OK) return s;
+  ExtraMaps extra;
+  for (int i = 0; i < 4; ++i) extra.m[i] = i % 2 == 0 ? map_a : map_b;
+  for (int i = 1; i < n_terms; ++i) {
+    const void* Ai = extra_operands[2 * (i - 1)];
+    const void* Bi = extra_operands[2 * (i - 1) + 1];
+    if (t.swapped) std::swap(Ai, Bi);
+    if (!Ai || !Bi) return fail(MTF_ERR_INVALID_ARG, "multi-term contraction: NULL operand");
+    s = t.a_mn_major ? make_map(&extra.m[2 * (i - 1)], Ai, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&extra.m[2 * (i - 1)], Ai, 2, t.K, t.M, t.a_ld, 64, BM / cn, t, t.outer_sA);
+    if (s != MTF_OK) return s;
+    s = t.b_mn_major ? make_map(&extra.m[2 * (i - 1) + 1], Bi, 2, t.N, t.K, t.b_ld, 64, BK, t, t.outer_sB) : make_map(&extra.m[2 * (i - 1) + 1], Bi, 2, t.K, t.N, t.b_ld, 64, b_rows, t, t.outer_sB);
+    if (s != MTF_OK) return s;
+  }
   // output: (N contiguous, M rows), boxes of 32 rows x 128 bytes for the staged stores
   const int c_bytes = plan.dtC == MTF_BF16 ? 2 : 4;
   if ((s = make_map(&map_c, C, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
@@ -1333,14 +1361,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   }
   mtf_status ls;
   if (wide) {
-    if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, a, st);
-    else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, a, st);
-  } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
+    if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+  } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
 #if defined(MTF_TMA_MULTICAST)
-  else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
-  else if (cm == 2 && cn == 1) ls = launch_kind<true, 2, 1, false>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
+  else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
+  else if (cm == 2 && cn == 1) ls = launch_kind<true, 2, 1, false>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
 #endif
-  else ls = launch_kind<true, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, a, st);
+  else ls = launch_kind<true, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
   if (ls != MTF_OK) return ls;
   count_launch();
   cudaError_t e = cudaGetLastError();
@@ -1390,7 +1418,7 @@ mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, cons
   if (st != MTF_OK) return st;
   // the tile counters inside the scratch are cleared by the launcher on the stream; partial tiles are
   // overwritten before they are read, so the previous call's contents do not matter
-  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream);
+  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr);
 }
 
 mtf_status read_device_status(int* code) {

@@ -155,7 +155,13 @@ std::string plan_key(int n_in, const mtf_tensor* in, const mtf_tensor* out, cons
 mtf_status launch_simt(const SimtParams& p, int64_t rsum_elems, void* stream);
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
-                     void* workspace, size_t workspace_bytes, void* stream);
+                     void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1,
+                     const void* const* extra_operands = nullptr);   // extra_operands: A_1, B_1 (, A_2, B_2) of a multi-term launch
+// Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes
+// and types may not) in one launch, one accumulator.  MTF_ERR_UNSUPPORTED when this plan cannot
+// (generic kernel, workspace reduce mode): the caller then chains einsums through the residual stage.
+mtf_status einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tensor (*terms)[2], mtf_tensor* out,
+                        const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream);
 size_t tc_workspace_bytes(const TcParams& t);
 size_t builtin_scratch_capacity();
 mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
