@@ -34,7 +34,8 @@ bool dims_match(const std::vector<Dim>& want, const mtf_tensor& t) {
 }
 
 mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epi,
-                     void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1, const void* const* extra_operands = nullptr) {
+                     void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1, const void* const* extra_operands = nullptr,
+                     int row_softmax = 0) {
   if (!P || !in || !out) return fail(MTF_ERR_INVALID_ARG, "einsum exec: NULL argument");
   if (!dims_match(P->dimsA, in[0]) || (P->has_B && !dims_match(P->dimsB, in[1])) || !dims_match(P->dimsC, *out))
     return fail(MTF_ERR_SIZE_MISMATCH, "einsum exec: operand dims differ from the planned ones");
@@ -74,8 +75,8 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
   const int relu = P->epi.on ? (epi->relu != 0) : 0;
   if (P->kernel_kind == MTF_KERNEL_TCGEN05)
     return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
-                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands);
-  if (n_terms != 1) return fail(MTF_ERR_UNSUPPORTED, "multi-term contraction on the generic kernel");
+                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands, row_softmax);
+  if (n_terms != 1 || row_softmax) return fail(MTF_ERR_UNSUPPORTED, "multi-term contraction or fused softmax on the generic kernel");
   SimtParams s = P->simt;
   s.A = in[0].data;
   s.B = P->has_B ? in[1].data : nullptr;
@@ -461,6 +462,19 @@ mtf_status mtf::einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_
       extra[2 * (i - 1) + q] = b.data;
     }
   return exec_plan(P, terms[0], out, epilogue, workspace, workspace_bytes, stream, n_terms, extra);
+}
+
+mtf_status mtf::einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* weights, float scale,
+                                   int causal, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!layout || !a || !b || !weights) return fail(MTF_ERR_INVALID_ARG, "einsum_row_softmax: NULL argument");
+  mtf_epilogue e;
+  e.scale = scale; e.relu = 0; e.bias = nullptr; e.relu_mask = nullptr; e.residual = nullptr; e.reduce_sum_out = nullptr;
+  const mtf_tensor in[2] = {*a, *b};
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 2, in, weights, &e, &P);
+  if (st != MTF_OK) return st;
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->tc.swapped) return fail(MTF_ERR_UNSUPPORTED, "einsum_row_softmax: not on this plan");
+  return exec_plan(P, in, weights, &e, workspace, workspace_bytes, stream, 1, nullptr, causal ? 2 : 1);
 }
 
 // dx_residual (NULL or a tensor with dx's dims) is added to dx in the last einsum's epilogue.

@@ -248,8 +248,14 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
   if ((st = ein(layout, xm.t, *wv, vv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   mtf_epilogue es = epi_none();
   es.scale = (float)s.scale;
-  if ((st = ein(layout, *q, *kk, &lg.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = mtf_softmax_forward(layout, &lg.t, causal, weights, stream)) != MTF_OK) return st;
+  // logits and softmax in one launch where a row of logits fits a tile (the fp32 logits then never
+  // leave the tensor memory); otherwise the logits go through the workspace and the row kernel
+  st = mtf::einsum_row_softmax(layout, q, kk, weights, (float)s.scale, causal, rest, rest_bytes, stream);
+  if (st == MTF_ERR_UNSUPPORTED) {
+    if ((st = ein(layout, *q, *kk, &lg.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
+    st = mtf_softmax_forward(layout, &lg.t, causal, weights, stream);
+  }
+  if (st != MTF_OK) return st;
   if ((st = ein(layout, *weights, *vv, o, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   mtf_epilogue er = epi_none();
   er.residual = residual;

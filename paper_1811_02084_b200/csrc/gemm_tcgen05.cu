@@ -89,6 +89,7 @@ struct TcArgs {
   long long tiles_per_slice, total_tiles, total_work;
   int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
   int kb_tile;             // k-blocks of one whole tile (all terms)
+  int softmax_causal;      // row-softmax epilogue: columns beyond the row's own position are masked out
   int n_terms;             // sum of n_terms products A_i . B_i of identical shape in one accumulator (1..3)
   int kb_term;             // k-blocks of one term
   int slots;               // partial-tile slots per tile in the workspace (sk, or 2 when balanced)
@@ -390,7 +391,7 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
 // Which component-wise stages a launch runs.  EPI_GENERIC reads them from the arguments; the other
 // kinds fix them at compile time, so that the common epilogues carry no branches on them and need
 // far fewer registers and instructions per chunk.
-enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_KINDS = 5 };
+enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_KINDS = 6 };
 struct EpiFlags {
   bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
 };
@@ -405,6 +406,7 @@ __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
     f.scale = false; f.bias = EPI == EPI_BIAS_RELU_BF16; f.bias_m = false; f.relu = EPI == EPI_BIAS_RELU_BF16;
     f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = f.resid_tma = false;
     f.c_bf16 = EPI != EPI_PLAIN_F32;
+    if (EPI == EPI_ROW_SOFTMAX) f.scale = true;
     f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
   }
   return f;
@@ -570,7 +572,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // k-block through L2 for twice the flops (24 KB per 256 x 256 x 64 instead of 32 KB).  For long K,
   // where the contraction is bound by the L2-to-SM traffic and the exposed epilogue is small.
   static_assert(!kWide || (kPair && CM == 1 && CN == 1), "wide tiles: plain CTA pairs only");
-  constexpr int kStages = (kPair && !kWide) ? 5 : 3;
+  // (the row-softmax kind keeps one stage less: its two warps per lane quarter exchange row statistics
+  // through the 32 KB that frees at the end of the ring)
+  constexpr int kStages = (kPair && !kWide) ? (EPI == EPI_ROW_SOFTMAX ? 4 : 5) : 3;
   constexpr int kStageBytes = (kPair && !kWide) ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
   constexpr int kTileRows = kPairRows * CM;            // rows of C owned by a work item
@@ -615,6 +619,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
   }
+  const uint32_t xchg_base = tiles_base + (uint32_t)(kStages * kStageBytes);     // [2 slots][8 warps][32 lanes] x 8 bytes
+  if (EPI == EPI_ROW_SOFTMAX)
+    for (int i = threadIdx.x; i < 2 * kEpilogueWarps * 32; i += kThreads)
+      asm volatile("st.shared.v2.b32 [%0], {%1, %1};" ::"r"(xchg_base + 8u * i), "r"(0u) : "memory");
   if (warp == 1) {   // TMEM allocation is a warp-wide operation (the same warp of both CTAs of a pair)
     if (kPair) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
@@ -818,6 +826,93 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (!ok) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
+      if (EPI == EPI_ROW_SOFTMAX) {
+        // The tile holds whole rows of logits (one tile column per slice).  Softmax over each row in
+        // three passes over the accumulator, which stays in tensor memory: maximum, sum of
+        // exponentials, normalised weights (bf16).  A row lives in one lane; the two warps of a lane
+        // quarter own alternate 64-column boxes and exchange their partial maximum and sum through
+        // shared memory (value + sequence number, bounded wait).
+        const float sl2 = a.scale * 1.4426950408889634f;                   // logits in units of log 2
+        const int ncols = min(a.block_n, tl.n_end - tl.n0);
+        const int lim = a.softmax_causal ? min(ncols, row + 1) : ncols;    // columns [0, lim) take part (row = position in `length`)
+        const int lim_warp = __shfl_sync(0xffffffffu, lim, 31);            // rows ascend with the lane: the warp's widest row
+        const uint32_t my_slot = xchg_base + 8u * (uint32_t)((warp - 2) * 32 + lane);
+        const uint32_t peer_slot = xchg_base + 8u * (uint32_t)((((warp - 2) ^ 4)) * 32 + lane);
+        const uint32_t seq = (uint32_t)iter + 1u;
+        auto exchange = [&](int slot, float mine, bool take_max) -> float {
+          const uint32_t off = (uint32_t)slot * (8u * kEpilogueWarps * 32u);
+          asm volatile("st.volatile.shared.v2.b32 [%0], {%1, %2};" ::"r"(my_slot + off), "r"(__float_as_uint(mine)), "r"(seq) : "memory");
+          uint32_t vb = 0, sq = 0;
+          int tries = 0;
+          do {
+            asm volatile("ld.volatile.shared.v2.b32 {%0, %1}, [%2];" : "=r"(vb), "=r"(sq) : "r"(peer_slot + off) : "memory");
+          } while (sq != seq && ++tries < (1 << 24) && !*abort_flag);
+          if (sq != seq) { atomicCAS(&g_status, 0, 0x700 + slot); *abort_flag = 1; }
+          const float other = __uint_as_float(vb);
+          return take_max ? fmaxf(mine, other) : mine + other;
+        };
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c0 = col_half * 64; c0 < lim_warp; c0 += (c0 & 32) ? 96 : 32) {
+          uint32_t raw[32];
+          tmem_ld32(taddr + c0, raw);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < lim) mx = fmaxf(mx, __uint_as_float(raw[j]) * sl2);
+        }
+        mx = exchange(0, mx, true);
+        float sum = 0.f;
+#pragma unroll 1
+        for (int c0 = col_half * 64; c0 < lim_warp; c0 += (c0 & 32) ? 96 : 32) {
+          uint32_t raw[32];
+          tmem_ld32(taddr + c0, raw);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (c0 + j < lim) sum += exp2f(__uint_as_float(raw[j]) * sl2 - mx);
+        }
+        sum = exchange(1, sum, false);
+        const float inv = 1.f / sum;
+#pragma unroll 1
+        for (int c0 = col_half * 64; c0 < a.block_n; c0 += (c0 & 32) ? 96 : 32) {
+          const int n_first = tl.n0 + c0;
+          int n_valid = tl.n_end - n_first;
+          n_valid = n_valid > 32 ? 32 : n_valid;
+          const bool live = row_ok && n_valid > 0;
+          const int box_n0 = tl.n0 + (c0 & ~63);
+          const bool staged = rows_full && box_n0 + 64 <= tl.n_end;
+          const int half = (c0 >> 5) & 1;
+          const uint32_t box = stg + buf * 4096u;
+          float v[32];
+          if (c0 < lim_warp) {
+            uint32_t raw[32];
+            tmem_ld32(taddr + c0, raw);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (c0 + j < lim) ? exp2f(__uint_as_float(raw[j]) * sl2 - mx) * inv : 0.f;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+          }
+          if (staged && half == 0) {
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+          }
+          if (staged) store_staged(f, v, box, lane, half);
+          else if (live) store_direct(a, f, v, row_off + n_first, n_valid);
+          if (staged && half == 1) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+            buf ^= 1u;
+          }
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
+        continue;
+      }
       // A tile shared by several workers: every worker but the last to arrive (per 32-row group and
       // column part) leaves its fragment in the workspace; the last one keeps its own in registers,
       // adds the others in ascending order of the fragments (= of the processors of the group) and
@@ -1192,7 +1287,8 @@ size_t tc_workspace_bytes(const TcParams& t) {
 
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
-                     void* workspace, size_t workspace_bytes, void* stream, int n_terms, const void* const* extra_operands) {
+                     void* workspace, size_t workspace_bytes, void* stream, int n_terms, const void* const* extra_operands,
+                     int row_softmax) {
   const TcParams& t = plan.tc;
   if (t.swapped) std::swap(A, B);
   if (n_terms < 1 || n_terms > 3 || (n_terms > 1 && !extra_operands)) return fail(MTF_ERR_INVALID_ARG, "1 to 3 terms");
@@ -1222,7 +1318,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // the time of a 256 x 256 one (twice the MMAs at 3/4 of the L2 traffic each, epilogue exposed), so
   // they win when they halve the number of waves.
   bool wide = false;
-  const bool plain_epi = scale == 1.f && !resid && !bias && !relu && !mask && !rsum;
+  const bool plain_epi = scale == 1.f && !resid && !bias && !relu && !mask && !rsum && !row_softmax;
+  if (row_softmax) {
+    // whole rows in one tile: the N slice is the whole dimension and fits a tile (256 columns, or 512 with a wide pair tile)
+    const bool fits = a.sn == 1 && (a.Ns <= a.block_n || (a.Ns == 512 && t.cta_pair && t.block_n == 256));
+    if (!fits || plan.dtC != MTF_BF16 || resid || bias || relu || mask || rsum || t.reduce_mode == MTF_REDUCE_WORKSPACE || n_terms != 1)
+      return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a bf16 result whose rows fit one tile (N <= 256, or 512 with CTA pairs) and no other stage");
+    wide = a.Ns == 512;
+  }
   const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && a.Ns % 512 == 0;
   if (t.wide_pref == 1 && !wide_legal)
     return fail(MTF_ERR_UNSUPPORTED, "wide tiles need CTA pairs, a plain epilogue, no workspace reduction and an N slice that is a multiple of 512");
@@ -1237,7 +1340,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads
   int cm = 1, cn = 1;
 #if defined(MTF_TMA_MULTICAST)
-  if (!wide && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
+  if (!wide && !row_softmax && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
     // measured on the FFN shapes: sharing B between two pairs that are neighbours along M is worth
     // 5-10 % on the contractions whose epilogue is light; with a relu mask or a fused reduction in the
     // epilogue the coupling of the two pairs costs more than the saved traffic; 2 x 2 clusters lose
@@ -1273,13 +1376,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
   a.kb_term = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
   a.n_terms = n_terms;
+  a.softmax_causal = row_softmax == 2 ? 1 : 0;
   a.kb_tile = a.kb_term * n_terms;
   a.slots = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.sk : 2;
   a.balanced = 0;
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (t.balance && cn == 1 && !wide && n_terms == 1 && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+  if (t.balance && cn == 1 && !wide && n_terms == 1 && !row_softmax && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
     // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
     // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
     // the workspace by whichever worker finishes last (arrive, never wait).
@@ -1353,14 +1457,19 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // epilogue kind: the common combinations have kernels of their own, everything else (and every
   // launch that assembles tiles from fragments) takes the generic one
   int epi = EPI_GENERIC;
-  if (scale == 1.f && !resid) {
+  if (row_softmax) epi = EPI_ROW_SOFTMAX;
+  else if (scale == 1.f && !resid) {
     if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
     else if (a.ws_partials) epi = EPI_GENERIC;
     else if (bias && !a.bias_along_m && relu && !mask && !rsum && a.c_bf16) epi = EPI_BIAS_RELU_BF16;
     else if (a.mask_tma && rsum && !bias && !relu) epi = EPI_MASK_RSUM_BF16;
   }
   mtf_status ls;
-  if (wide) {
+  if (row_softmax) {
+    if (wide) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else if (t.cta_pair) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else ls = launch_variant<false, 1, 1, EPI_ROW_SOFTMAX, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+  } else if (wide) {
     if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
   } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
@@ -1418,7 +1527,7 @@ mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, cons
   if (st != MTF_OK) return st;
   // the tile counters inside the scratch are cleared by the launcher on the stream; partial tiles are
   // overwritten before they are read, so the previous call's contents do not matter
-  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr);
+  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr, 0);
 }
 
 mtf_status read_device_status(int* code) {

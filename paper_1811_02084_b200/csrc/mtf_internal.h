@@ -156,7 +156,12 @@ mtf_status launch_simt(const SimtParams& p, int64_t rsum_elems, void* stream);
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1,
-                     const void* const* extra_operands = nullptr);   // extra_operands: A_1, B_1 (, A_2, B_2) of a multi-term launch
+                     const void* const* extra_operands = nullptr,    // A_1, B_1 (, A_2, B_2) of a multi-term launch
+                     int row_softmax = 0);                           // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue
+// weights[.., l, m] = softmax_m(scale * sum_k a b (causal: only m <= l)) in one launch, bf16 result.
+// MTF_ERR_UNSUPPORTED when the plan cannot (rows longer than a tile, generic kernel, split rows).
+mtf_status einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* weights, float scale,
+                              int causal, void* workspace, size_t workspace_bytes, void* stream);
 // Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes
 // and types may not) in one launch, one accumulator.  MTF_ERR_UNSUPPORTED when this plan cannot
 // (generic kernel, workspace reduce mode): the caller then chains einsums through the residual stage.
