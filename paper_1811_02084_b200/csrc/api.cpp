@@ -477,6 +477,19 @@ mtf_status mtf::einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor*
   return exec_plan(P, in, weights, &e, workspace, workspace_bytes, stream, 1, nullptr, causal ? 2 : 1);
 }
 
+mtf_status mtf::einsum_row_softmax_bwd(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, const mtf_tensor* weights,
+                                       mtf_tensor* dlogits, int causal, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!layout || !a || !b || !weights || !dlogits) return fail(MTF_ERR_INVALID_ARG, "einsum_row_softmax_bwd: NULL argument");
+  mtf_epilogue e;
+  e.scale = 1.f; e.relu = 0; e.bias = nullptr; e.relu_mask = weights; e.residual = nullptr; e.reduce_sum_out = nullptr;
+  const mtf_tensor in[2] = {*a, *b};
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 2, in, dlogits, &e, &P);
+  if (st != MTF_OK) return st;
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->tc.swapped) return fail(MTF_ERR_UNSUPPORTED, "einsum_row_softmax_bwd: not on this plan");
+  return exec_plan(P, in, dlogits, &e, workspace, workspace_bytes, stream, 1, nullptr, causal ? 4 : 3);
+}
+
 // dx_residual (NULL or a tensor with dx's dims) is added to dx in the last einsum's epilogue.
 mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,
                                   const mtf_tensor* h_saved, const mtf_tensor* dy, mtf_tensor* dx, const mtf_tensor* dx_residual,

@@ -289,9 +289,14 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   TD xm = renamed(*x, s.l.name, kMemory);
   if ((st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, *dy, *wo, &dob.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, dob.t, *vv, &dP.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  // dP and the softmax backward in one launch where a row fits a tile (dP then stays in tensor
+  // memory); otherwise dP goes through the workspace in fp32 and the row kernel follows
+  st = mtf::einsum_row_softmax_bwd(layout, &dob.t, vv, weights, &dlg.t, 0 /* zeros of a causal P give zeros here without being told */, rest, rest_bytes, stream);
+  const bool fused_bwd = st == MTF_OK;
+  if (st != MTF_OK && st != MTF_ERR_UNSUPPORTED) return st;
+  if (!fused_bwd && (st = ein(layout, dob.t, *vv, &dP.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, *weights, dob.t, &dvv.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = mtf_softmax_backward(layout, weights, &dP.t, &dlg.t, stream)) != MTF_OK) return st;
+  if (!fused_bwd && (st = mtf_softmax_backward(layout, weights, &dP.t, &dlg.t, stream)) != MTF_OK) return st;
   mtf_epilogue es = epi_none();
   es.scale = (float)s.scale;
   if ((st = ein(layout, dlg.t, *kk, &dq.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;

@@ -391,7 +391,7 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
 // Which component-wise stages a launch runs.  EPI_GENERIC reads them from the arguments; the other
 // kinds fix them at compile time, so that the common epilogues carry no branches on them and need
 // far fewer registers and instructions per chunk.
-enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_KINDS = 6 };
+enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_ROW_SOFTMAX_BWD = 6, EPI_KINDS = 7 };
 struct EpiFlags {
   bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
 };
@@ -407,6 +407,7 @@ __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
     f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = f.resid_tma = false;
     f.c_bf16 = EPI != EPI_PLAIN_F32;
     if (EPI == EPI_ROW_SOFTMAX) f.scale = true;
+    if (EPI == EPI_ROW_SOFTMAX_BWD) f.mask = f.mask_bf16 = true;      // the weights P arrive like a mask, by TMA
     f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
   }
   return f;
@@ -574,7 +575,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   static_assert(!kWide || (kPair && CM == 1 && CN == 1), "wide tiles: plain CTA pairs only");
   // (the row-softmax kind keeps one stage less: its two warps per lane quarter exchange row statistics
   // through the 32 KB that frees at the end of the ring)
-  constexpr int kStages = (kPair && !kWide) ? (EPI == EPI_ROW_SOFTMAX ? 4 : 5) : 3;
+  constexpr int kStages = (kPair && !kWide) ? ((EPI == EPI_ROW_SOFTMAX || EPI == EPI_ROW_SOFTMAX_BWD) ? 4 : 5) : 3;
   constexpr int kStageBytes = (kPair && !kWide) ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
   constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
   constexpr int kTileRows = kPairRows * CM;            // rows of C owned by a work item
@@ -620,7 +621,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
   }
   const uint32_t xchg_base = tiles_base + (uint32_t)(kStages * kStageBytes);     // [2 slots][8 warps][32 lanes] x 8 bytes
-  if (EPI == EPI_ROW_SOFTMAX)
+  if (EPI == EPI_ROW_SOFTMAX || EPI == EPI_ROW_SOFTMAX_BWD)
     for (int i = threadIdx.x; i < 2 * kEpilogueWarps * 32; i += kThreads)
       asm volatile("st.shared.v2.b32 [%0], {%1, %1};" ::"r"(xchg_base + 8u * i), "r"(0u) : "memory");
   if (warp == 1) {   // TMEM allocation is a warp-wide operation (the same warp of both CTAs of a pair)
@@ -808,8 +809,23 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       // the bf16 relu mask, or the residual
       const bool mask_tma = f.mask_tma && !ws_mode && rows_full;
       const bool resid_tma = f.resid_tma && !ws_mode && rows_full;
-      const bool in_tma = mask_tma || resid_tma;
+      const bool in_tma = (mask_tma || resid_tma) && EPI != EPI_ROW_SOFTMAX_BWD;
       const int box_cols = f.c_bf16 ? 64 : 32;
+      // softmax backward: the boxes of P this warp visits (twice: row dot products, then the result);
+      // under the causal limit the boxes right of the warp's widest row hold zeros and are not read
+      int sb_lim = 0, sb_lim_warp = 0, sb_nbox = 0;
+      if (EPI == EPI_ROW_SOFTMAX_BWD) {
+        const int ncols = min(a.block_n, tl.n_end - tl.n0);
+        sb_lim = a.softmax_causal ? min(ncols, row + 1) : ncols;
+        sb_lim_warp = __shfl_sync(0xffffffffu, sb_lim, 31);
+        if (rows_full)                     // (a warp is inside its slice with all 32 rows or with none)
+          for (int b = col_half * 64; b < sb_lim_warp; b += 128) ++sb_nbox;
+        if (sb_nbox > 0 && lane == 0) {
+          asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          mbar_expect_tx(mfull_bar(buf), 4096u);
+          tma_load_5d<false>(stg + buf * 4096u, &map_m, mfull_bar(buf), tl.n0 + col_half * 64, row0, tl.o[2], tl.o[1], tl.o[0]);
+        }
+      }
       if (in_tma && lane == 0) {
         // pull this warp's boxes of the operand's tile towards L2 and request the first one into the
         // staging box it will be processed in (free once all but the latest store have been read out)
@@ -826,6 +842,92 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (!ok) break;
       tcgen05_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)acc * kMaxBN + ((uint32_t)(q * 32) << 16);
+      if (EPI == EPI_ROW_SOFTMAX_BWD) {
+        // The accumulator holds whole rows of dP = do . vv^T; with the weights P of the same rows
+        // (64-column boxes by TMA into the staging buffers, one box ahead) the result is
+        // dlogits = P (dP - sum_m dP P): a first visit of every box for the row sums, the two warps of
+        // a lane quarter exchange their parts, a second visit writes the result over the box and stores it.
+        // (exchange slots alternate with the tile, so a warp that runs ahead cannot overwrite what its partner has not read)
+        const uint32_t slot_off = (uint32_t)(iter & 1) * (8u * kEpilogueWarps * 32u);
+        const uint32_t my_slot = xchg_base + slot_off + 8u * (uint32_t)((warp - 2) * 32 + lane);
+        const uint32_t peer_slot = xchg_base + slot_off + 8u * (uint32_t)((((warp - 2) ^ 4)) * 32 + lane);
+        const uint32_t seq = (uint32_t)iter + 1u;
+        float dot = 0.f;
+        auto exchange_dot = [&]() {
+          asm volatile("st.volatile.shared.v2.b32 [%0], {%1, %2};" ::"r"(my_slot), "r"(__float_as_uint(dot)), "r"(seq) : "memory");
+          uint32_t vb = 0, sq = 0;
+          int tries = 0;
+          do {
+            asm volatile("ld.volatile.shared.v2.b32 {%0, %1}, [%2];" : "=r"(vb), "=r"(sq) : "r"(peer_slot) : "memory");
+          } while (sq != seq && ++tries < (1 << 24) && !*abort_flag);
+          if (sq != seq) { atomicCAS(&g_status, 0, 0x710); *abort_flag = 1; }
+          dot += __uint_as_float(vb);
+        };
+        if (sb_nbox == 0) exchange_dot();                // no box of its own: the partner still needs a zero from this warp
+        const int visits = 2 * sb_nbox;
+#pragma unroll 1
+        for (int vis = 0; vis < visits; ++vis) {
+          const bool second = vis >= sb_nbox;
+          const int bc = col_half * 64 + 128 * (second ? vis - sb_nbox : vis);     // first column of the box inside the tile
+          const uint32_t box = stg + buf * 4096u;
+          if (!mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag)) { ok = false; break; }
+          mask_phase ^= 1u << buf;
+          const uint32_t srow = box + (uint32_t)lane * 128u;
+          const uint32_t sw = (uint32_t)(lane & 7);
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t raw[32];
+            tmem_ld32(taddr + bc + 32 * half, raw);
+            float pw[32];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) unpack_bf16x8(ld_shared_v4(srow + ((((uint32_t)(half * 4 + i)) ^ sw) << 4)), pw + 8 * i);
+            tmem_ld_wait();
+            float* v = reinterpret_cast<float*>(raw);
+            if (!second) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) dot = fmaf(v[j], pw[j], dot);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = pw[j] * (v[j] - dot);
+              store_staged(f, v, box, lane, half);
+            }
+          }
+          if (second) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) tma_store_5d(&map_c, box, tl.n0 + bc, row0, tl.o[2], tl.o[1], tl.o[0]);
+          }
+          if (vis + 1 < visits && lane == 0) {           // next visit's box into the other staging box
+            const int nv = vis + 1;
+            const int nbc = col_half * 64 + 128 * (nv >= sb_nbox ? nv - sb_nbox : nv);
+            if (second) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
+            tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), tl.n0 + nbc, row0, tl.o[2], tl.o[1], tl.o[0]);
+          }
+          __syncwarp();
+          buf ^= 1u;
+          if (vis == sb_nbox - 1) exchange_dot();        // all first visits done: the row's dot product
+        }
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        // boxes right of every row's causal limit: zeros
+#pragma unroll 1
+        for (int bc = col_half * 64 + 128 * sb_nbox; rows_full && bc < a.block_n && tl.n0 + bc + 64 <= tl.n_end; bc += 128) {
+          const uint32_t box = stg + buf * 4096u;
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 8; ++i) st_shared_v4(box + (uint32_t)lane * 128u + 16u * i, 0u, 0u, 0u, 0u);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) tma_store_5d(&map_c, box, tl.n0 + bc, row0, tl.o[2], tl.o[1], tl.o[0]);
+          buf ^= 1u;
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
+        continue;
+      }
       if (EPI == EPI_ROW_SOFTMAX) {
         // The tile holds whole rows of logits (one tile column per slice).  Softmax over each row in
         // three passes over the accumulator, which stays in tensor memory: maximum, sum of
@@ -1322,7 +1424,9 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (row_softmax) {
     // whole rows in one tile: the N slice is the whole dimension and fits a tile (256 columns, or 512 with a wide pair tile)
     const bool fits = a.sn == 1 && (a.Ns <= a.block_n || (a.Ns == 512 && t.cta_pair && t.block_n == 256));
-    if (!fits || plan.dtC != MTF_BF16 || resid || bias || relu || mask || rsum || t.reduce_mode == MTF_REDUCE_WORKSPACE || n_terms != 1)
+    const bool bwd = row_softmax >= 3;      // backward: the weights come in as the mask operand, whole boxes only
+    if (!fits || plan.dtC != MTF_BF16 || resid || bias || relu || rsum || t.reduce_mode == MTF_REDUCE_WORKSPACE || n_terms != 1 ||
+        (bwd ? (!mask || dtMask != MTF_BF16 || scale != 1.f || a.Ms % 32 != 0 || a.Ns % 64 != 0) : mask != nullptr))
       return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a bf16 result whose rows fit one tile (N <= 256, or 512 with CTA pairs) and no other stage");
     wide = a.Ns == 512;
   }
@@ -1376,7 +1480,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
   a.kb_term = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
   a.n_terms = n_terms;
-  a.softmax_causal = row_softmax == 2 ? 1 : 0;
+  a.softmax_causal = (row_softmax == 2 || row_softmax == 4) ? 1 : 0;
   a.kb_tile = a.kb_term * n_terms;
   a.slots = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.sk : 2;
   a.balanced = 0;
@@ -1457,7 +1561,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // epilogue kind: the common combinations have kernels of their own, everything else (and every
   // launch that assembles tiles from fragments) takes the generic one
   int epi = EPI_GENERIC;
-  if (row_softmax) epi = EPI_ROW_SOFTMAX;
+  if (row_softmax) epi = row_softmax >= 3 ? EPI_ROW_SOFTMAX_BWD : EPI_ROW_SOFTMAX;
   else if (scale == 1.f && !resid) {
     if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
     else if (a.ws_partials) epi = EPI_GENERIC;
@@ -1465,7 +1569,11 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     else if (a.mask_tma && rsum && !bias && !relu) epi = EPI_MASK_RSUM_BF16;
   }
   mtf_status ls;
-  if (row_softmax) {
+  if (row_softmax >= 3) {
+    if (wide) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX_BWD, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else if (t.cta_pair) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX_BWD, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else ls = launch_variant<false, 1, 1, EPI_ROW_SOFTMAX_BWD, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+  } else if (row_softmax) {
     if (wide) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     else if (t.cta_pair) ls = launch_variant<true, 1, 1, EPI_ROW_SOFTMAX, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     else ls = launch_variant<false, 1, 1, EPI_ROW_SOFTMAX, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);

@@ -157,9 +157,13 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1,
                      const void* const* extra_operands = nullptr,    // A_1, B_1 (, A_2, B_2) of a multi-term launch
-                     int row_softmax = 0);                           // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue
+                     int row_softmax = 0);                           // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue;
+                                                                     // 3 / 4 (causal): its backward, P (A . B - rowsum(P A . B)), P = the mask operand
 // weights[.., l, m] = softmax_m(scale * sum_k a b (causal: only m <= l)) in one launch, bf16 result.
 // MTF_ERR_UNSUPPORTED when the plan cannot (rows longer than a tile, generic kernel, split rows).
+// dlogits[.., l, m] = P (dP - sum_m dP P) with dP = sum_v a b, in one launch (same conditions, whole 32 x 64 boxes only).
+mtf_status einsum_row_softmax_bwd(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, const mtf_tensor* weights,
+                                  mtf_tensor* dlogits, int causal, void* workspace, size_t workspace_bytes, void* stream);
 mtf_status einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* weights, float scale,
                               int causal, void* workspace, size_t workspace_bytes, void* stream);
 // Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes
