@@ -224,6 +224,24 @@ mtf_status mtf_softmax_forward(const mtf_layout_t* layout, const mtf_tensor* log
 /* dlogits = weights * (dweights - sum over the last dim of dweights * weights); dweights f32. */
 mtf_status mtf_softmax_backward(const mtf_layout_t* layout, const mtf_tensor* weights, const mtf_tensor* dweights,
                                 mtf_tensor* dlogits, void* stream);
+/* Einsum and softmax in one launch: weights = softmax over the LAST dimension of scale * einsum(a, b)
+ * (the attention logits of Section 9's Transformer; bf16 operands, bf16 weights, device pointers).
+ * The f32 logits stay in the tensor cores' accumulator memory and never reach HBM.  Only for
+ * contractions whose whole output row fits one tile: the last output dimension is not split by the
+ * layout and has at most 256 entries (512 when the second-to-last dimension has more than 128);
+ * anything else, and any plan the tensor-core kernel cannot run, returns MTF_ERR_UNSUPPORTED and
+ * leaves `weights` untouched (call mtf_einsum + mtf_softmax_forward instead).  causal as in
+ * mtf_softmax_forward (the two last output dimensions are the query and memory positions).
+ * workspace: unused today (pass what mtf_einsum would get); stream: CUDA stream or NULL. */
+mtf_status mtf_einsum_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, float scale,
+                              int32_t causal, mtf_tensor* weights, void* workspace, size_t workspace_bytes, void* stream);
+/* Its backward, also one launch: dlogits = weights * (dw - sum over the last dim of dw * weights)
+ * with dw = einsum(a, b) (a = gradient of the attention output, b = values).  `weights` has the dims
+ * of dlogits (bf16).  Same shape conditions, and in addition the two last output dimensions must be
+ * multiples of 32 and 64 inside every slice; otherwise MTF_ERR_UNSUPPORTED. */
+mtf_status mtf_einsum_softmax_backward(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b,
+                                       const mtf_tensor* weights, mtf_tensor* dlogits, void* workspace,
+                                       size_t workspace_bytes, void* stream);
 /* y = gamma * (x - mean) * (var + eps)^-1/2 + beta over the LAST dimension (biased variance).
  * stats: f32 tensor with two values per row (mean, reciprocal standard deviation), kept for backward. */
 mtf_status mtf_layernorm_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* gamma,

@@ -90,6 +90,8 @@ def _load():
         "mtf_reduce_sum": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
         "mtf_softmax_forward": [vp, POINTER(mtf_tensor), c_int32, POINTER(mtf_tensor), vp],
         "mtf_softmax_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_einsum_softmax": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), c_float, c_int32, POINTER(mtf_tensor), vp, c_size_t, vp],
+        "mtf_einsum_softmax_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp, c_size_t, vp],
         "mtf_layernorm_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), c_float, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
         "mtf_layernorm_backward": [vp] + [POINTER(mtf_tensor)] * 8 + [vp],
         "mtf_attention_forward": [vp] + [POINTER(mtf_tensor)] * 5 + [c_int32] + [POINTER(mtf_tensor)] * 7 + [vp, c_size_t, vp],
@@ -382,6 +384,16 @@ def mtf_softmax_forward(layout, logits: Named, causal: bool, weights: Named, str
 
 def mtf_softmax_backward(layout, weights: Named, dweights: Named, dlogits: Named, stream=None) -> None:
     _check(_lib.mtf_softmax_backward(layout.handle, _p(weights), _p(dweights), _p(dlogits), _stream(stream)))
+
+
+def mtf_einsum_softmax(layout, a: Named, b: Named, scale: float, causal: bool, weights: Named, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_einsum_softmax(layout.handle, _p(a), _p(b), float(scale), 1 if causal else 0, _p(weights), wp, wb, _stream(stream)))
+
+
+def mtf_einsum_softmax_backward(layout, a: Named, b: Named, weights: Named, dlogits: Named, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_einsum_softmax_backward(layout.handle, _p(a), _p(b), _p(weights), _p(dlogits), wp, wb, _stream(stream)))
 
 
 def mtf_layernorm_forward(layout, x, gamma, beta, eps, y, stats, stream=None) -> None:

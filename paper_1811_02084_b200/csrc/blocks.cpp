@@ -216,6 +216,16 @@ mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* 
 // q[b,l,h,k] = sum_d x wq; kk[b,m,h,k] = sum_d xm wk; vv[b,m,h,v] = sum_d xm wv (xm = x with `length`
 // renamed memory_length); logits[b,h,l,m] = d_k^-1/2 sum_k q kk; weights = softmax_m (causal: m <= l);
 // o[b,l,h,v] = sum_m weights vv; y[b,l,d] = sum_{h,v} o wo (+ residual).
+mtf_status mtf_einsum_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, float scale, int32_t causal,
+                              mtf_tensor* weights, void* workspace, size_t workspace_bytes, void* stream) {
+  return mtf::einsum_row_softmax(layout, a, b, weights, scale, causal ? 1 : 0, workspace, workspace_bytes, stream);
+}
+
+mtf_status mtf_einsum_softmax_backward(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, const mtf_tensor* weights,
+                                       mtf_tensor* dlogits, void* workspace, size_t workspace_bytes, void* stream) {
+  return mtf::einsum_row_softmax_bwd(layout, a, b, weights, dlogits, 0, workspace, workspace_bytes, stream);
+}
+
 mtf_status mtf_attention_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq, const mtf_tensor* wv, size_t* bytes) {
   if (!layout || !x || !wq || !wv || !bytes || x->ndim != 3 || wq->ndim != 3 || wv->ndim != 3) return fail(MTF_ERR_INVALID_ARG, "attention_workspace_bytes: bad argument");
   const int64_t B = x->dims[0].size, L = x->dims[1].size, H = wq->dims[1].size, K = wq->dims[2].size, V = wv->dims[2].size;

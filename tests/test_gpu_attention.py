@@ -76,6 +76,96 @@ def test_softmax_forward_backward(mtf, causal):
     assert parity_error(from_torch(dlg), want) <= TOL["bf16"]
 
 
+# ---- einsum + softmax in one launch -------------------------------------------------------------------------
+
+FUSED_SHAPES = [
+    # (batch, heads, length, memory_length, d_k): a 128-row tile with a ragged tail, the single-CTA kernel
+    (2, 2, 136, 136, 64),
+    # CTA pairs, rows of three 64-column boxes (the two warps of a lane quarter own 2 and 1), 64 rows of the 256-row tile unused
+    (2, 4, 192, 192, 64),
+    # rows of 512: the wide pair tile (one accumulator)
+    (1, 2, 512, 512, 32),
+]
+
+
+def _fused_case(seed, B, H, L, M, K):
+    q = si.normal(seed, "q", [B, L, H, K], "bf16")
+    kk = si.normal(seed, "kk", [B, M, H, K], "bf16")
+    x = np.einsum("blhk,bmhk->bhlm", q.f64, kk.f64) * K ** -0.5
+    return q, kk, x
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("mesh_dims,rules", [([("all", 1)], []), ([("a", 2), ("b", 2)], [("batch", "a"), ("heads", "b")])][:2], ids=["one", "2x2"])
+def test_einsum_softmax_one_launch(mtf, shape, causal, mesh_dims, rules):
+    B, H, L, M, K = shape
+    if B % 2 and len(mesh_dims) > 1:
+        pytest.skip("batch of 1 cannot be split")
+    q, kk, x = _fused_case(21, B, H, L, M, K)
+    if causal:
+        x = np.where(np.triu(np.ones((L, M)), 1) > 0, -np.inf, x)
+    e = np.exp(x - x.max(-1, keepdims=True))
+    P = e / e.sum(-1, keepdims=True)
+    lay = layout(mtf, mesh_dims, rules)
+    wdims = [("batch", B), ("heads", H), ("length", L), ("memory_length", M)]
+    w = alloc(wdims, "bf16")
+    n0 = mtf.mtf_launch_count()
+    mtf.mtf_einsum_softmax(lay, mtf.named(to_torch(q), ["batch", "length", "heads", "d_k"]), mtf.named(to_torch(kk), ["batch", "memory_length", "heads", "d_k"]),
+                           K ** -0.5, causal, mtf.named(w, [n for n, _ in wdims]))
+    assert mtf.mtf_launch_count() - n0 == 1
+    mtf.mtf_device_status()
+    got = from_torch(w)
+    assert parity_error(got, P) <= TOL["bf16"]
+    if causal:
+        iu = np.triu_indices(L, 1)
+        assert (got[..., iu[0], iu[1]] == 0.0).all()
+    assert np.abs(got.sum(-1) - 1.0).max() <= 2e-2          # rows of bf16 weights still sum to 1 within rounding
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES[1:], ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("causal", [False, True])
+def test_einsum_softmax_backward_one_launch(mtf, shape, causal):
+    B, H, L, M, V = shape
+    do = si.normal(22, "do", [B, L, H, V], "bf16")
+    vv = si.normal(22, "vv", [B, M, H, V], "bf16")
+    lg = si.normal(22, "lg", [B, H, L, M], "f32", 2.0).f64
+    if causal:
+        lg = np.where(np.triu(np.ones((L, M)), 1) > 0, -np.inf, lg)
+    e = np.exp(lg - lg.max(-1, keepdims=True))
+    P = si.store(e / e.sum(-1, keepdims=True), "bf16")       # the weights as the forward pass keeps them
+    dP = np.einsum("blhv,bmhv->bhlm", do.f64, vv.f64)
+    want = P.f64 * (dP - (dP * P.f64).sum(-1, keepdims=True))
+    lay = layout(mtf, [("a", 2)], [("heads", "a")])
+    wdims = [("batch", B), ("heads", H), ("length", L), ("memory_length", M)]
+    names = [n for n, _ in wdims]
+    dlg = alloc(wdims, "bf16")
+    n0 = mtf.mtf_launch_count()
+    mtf.mtf_einsum_softmax_backward(lay, mtf.named(to_torch(do), ["batch", "length", "heads", "d_v"]),
+                                    mtf.named(to_torch(vv), ["batch", "memory_length", "heads", "d_v"]), mtf.named(to_torch(P), names),
+                                    mtf.named(dlg, names))
+    assert mtf.mtf_launch_count() - n0 == 1
+    mtf.mtf_device_status()
+    assert parity_error(from_torch(dlg), want) <= TOL["bf16"]
+
+
+def test_einsum_softmax_refuses_rows_that_do_not_fit(mtf):
+    lay = layout(mtf, [("all", 1)], [])
+    q, kk, _ = _fused_case(23, 1, 1, 64, 640, 64)             # 640 columns: more than a tile
+    w = alloc([("batch", 1), ("heads", 1), ("length", 64), ("memory_length", 640)], "bf16")
+    with pytest.raises(mtf.MtfError) as e:
+        mtf.mtf_einsum_softmax(lay, mtf.named(to_torch(q), ["batch", "length", "heads", "d_k"]), mtf.named(to_torch(kk), ["batch", "memory_length", "heads", "d_k"]),
+                               0.125, False, mtf.named(w, ["batch", "heads", "length", "memory_length"]))
+    assert e.value.code == "MTF_ERR_UNSUPPORTED"
+    lay2 = layout(mtf, [("all", 2)], [("memory_length", "all")])      # rows split over processors
+    q, kk, _ = _fused_case(23, 1, 1, 64, 128, 64)
+    w = alloc([("batch", 1), ("heads", 1), ("length", 64), ("memory_length", 128)], "bf16")
+    with pytest.raises(mtf.MtfError) as e:
+        mtf.mtf_einsum_softmax(lay2, mtf.named(to_torch(q), ["batch", "length", "heads", "d_k"]), mtf.named(to_torch(kk), ["batch", "memory_length", "heads", "d_k"]),
+                               0.125, False, mtf.named(w, ["batch", "heads", "length", "memory_length"]))
+    assert e.value.code == "MTF_ERR_UNSUPPORTED"
+
+
 # ---- layer norm --------------------------------------------------------------------------------------------
 
 def test_layernorm_forward_backward(mtf):
