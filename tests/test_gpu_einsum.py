@@ -188,7 +188,12 @@ def test_workspace_and_chained_agree_with_unsplit(mtf):
         got, ref, info = run_einsum(mtf, layout(mtf, mesh_dims, rules), [a, b], out, "bf16", "f32", force=force)
         assert parity_error(got, ref) <= TOL["bf16"], tag
         res[tag] = (got, info)
-    assert res["auto"][1]["reduce_mode"] == mtf.MTF_REDUCE_WORKSPACE      # 2 output tiles only: slices spread over CTAs
+    # one output tile: the planner spreads the slices over CTAs only when that takes enough k-blocks
+    # off the critical path to pay for the fragments (K = 2048 does not, K = 16384 does)
+    assert res["auto"][1]["reduce_mode"] == mtf.MTF_REDUCE_CHAINED
+    big = mtf.mtf_einsum_plan(layout(mtf, [("all", 8)], [("k", "all")]), [mtf.desc([("k", 16384), ("i", 256)], "bf16"), mtf.desc([("k", 16384), ("j", 256)], "bf16")],
+                              mtf.desc(out, "f32"))
+    assert mtf.mtf_plan_info(big)["reduce_mode"] == mtf.MTF_REDUCE_WORKSPACE
     # fp32 sums in different orders: equal to rounding, and the deterministic modes repeat bit for bit
     assert np.abs(res["chained"][0] - res["unsplit"][0]).max() <= 1e-3 * np.abs(res["unsplit"][0]).max()
     again, _, _ = run_einsum(mtf, layout(mtf, [("all", 8)], [("k", "all")]), [a, b], out, "bf16", "f32", force=(1, 2))
