@@ -1086,7 +1086,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           tmem_ld_wait();
           float* v = reinterpret_cast<float*>(raw);
           if (ws_mode) {
-            const float* prow = a.ws_partials + ((size_t)(t * a.slots) * kTileRows + (size_t)tile_row) * a.block_n + c0;
+            // fragment layout: per 32-row x 32-column chunk 4 KB, piece j of lane l at j * 512 + l * 16 bytes,
+            // so that every 16-byte access of a warp covers 512 contiguous bytes
+            const float* prow = a.ws_partials + (((size_t)(t * a.slots) * (kTileRows / 32) + (size_t)(warp_tile_row / 32)) * (a.block_n / 32) + (size_t)(c0 / 32)) * 1024 + lane * 4;
             const size_t slot_stride = (size_t)kTileRows * a.block_n;
             float pre[32];
 #pragma unroll
@@ -1099,7 +1101,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const float4* sp = reinterpret_cast<const float4*>(prow + (size_t)s2 * slot_stride);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                  const float4 x4 = __ldcg(sp + j);
+                  const float4 x4 = __ldcg(sp + 32 * j);
                   pre[4 * j] += x4.x; pre[4 * j + 1] += x4.y; pre[4 * j + 2] += x4.z; pre[4 * j + 3] += x4.w;
                 }
               }
@@ -1159,38 +1161,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __syncwarp();
         if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
       } else {
-        // fragment `ks` of the tile -> workspace, the way a finished tile leaves: 32-row x 128-byte
-        // boxes through the staging buffers and TMA stores (the chunks this warp owns in the regular
-        // epilogue, so that the finisher finds them under the same counter)
-        const long long part_row0 = (t * a.slots + ks) * (long long)kTileRows + warp_tile_row;
+        // fragment `ks` of the tile -> workspace, straight from registers in the chunk layout described
+        // at the reading side (the chunks this warp owns in the regular epilogue, so that the finisher
+        // finds them under the same counter)
+        float* pbase = a.ws_partials + (((size_t)(t * a.slots + ks) * (kTileRows / 32) + (size_t)(warp_tile_row / 32)) * (a.block_n / 32)) * 1024 + lane * 4;
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
           if (((c0 / box_cols) & 1) != col_half) continue;
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
-          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-          __syncwarp();
-          const uint32_t box = stg + buf * 4096u;
-          const uint32_t srow = box + (uint32_t)lane * 128u;
-          const uint32_t sw = (uint32_t)(lane & 7);
+          float4* pp = reinterpret_cast<float4*>(pbase + (size_t)(c0 / 32) * 1024);
           tmem_ld_wait();
 #pragma unroll
           for (int j = 0; j < 8; ++j)
-            st_shared_v4(srow + (((uint32_t)j ^ sw) << 4), raw[4 * j], raw[4 * j + 1], raw[4 * j + 2], raw[4 * j + 3]);
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) tma_store_5d(&map_w, box, c0, (int)part_row0, 0, 0, 0);
-          buf ^= 1u;
+            __stcg(pp + 32 * j, make_float4(__uint_as_float(raw[4 * j]), __uint_as_float(raw[4 * j + 1]), __uint_as_float(raw[4 * j + 2]), __uint_as_float(raw[4 * j + 3])));
         }
         tcgen05_fence_before();
         __syncwarp();
         if (lane == 0) {
           mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
-          asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");       // the fragment has been written, not only read out
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __threadfence();
-          atomicAdd(&a.ws_counters[a.ws_ncounters + ws_ci], 1u);
         }
+        __threadfence();                                   // every lane's part of the fragment, then the flag
+        __syncwarp();
+        if (lane == 0) atomicAdd(&a.ws_counters[a.ws_ncounters + ws_ci], 1u);
         __syncwarp();
       }
     }
@@ -1548,15 +1541,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   map_m = map_c;
   if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
   if (a.resid_tma && (s = make_map(&map_m, resid, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
-  // fragments of shared tiles: the workspace as one fp32 matrix of block_n columns, a tile slot after the other
-  CUtensorMap map_w = map_c;
-  if (a.ws_partials) {
-    const long long ws_rows = a.total_tiles * a.slots * tile_rows;
-    if (ws_rows > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "workspace of more than 2^31 rows");
-    TcParams flat = t;
-    flat.n_outer = 0;
-    if ((s = make_map(&map_w, a.ws_partials, 4, a.block_n, ws_rows, a.block_n, 32, 32, flat, t.outer_sC)) != MTF_OK) return s;
-  }
+  CUtensorMap map_w = map_c;      // (spare tensor-map slot of the kernel)
 
   // epilogue kind: the common combinations have kernels of their own, everything else (and every
   // launch that assembles tiles from fragments) takes the generic one

@@ -483,10 +483,11 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
       const int64_t rows = t.cta_pair ? 256 : 128;
       int64_t tiles = ((t.M / t.sm + rows - 1) / rows) * t.sm * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sn;
       for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
-      // measured: a workspace launch costs ~40 us beyond its (shorter) main loop, the chained one ~7 us,
-      // and a k-block takes ~0.33 us, so the k-blocks taken off the critical path must be worth the difference
+      // measured: a workspace launch costs ~22 us beyond its (shorter) main loop (clearing the counters,
+      // writing and adding the fragments), the chained one ~7 us, and a k-block takes ~0.33 us, so the
+      // k-blocks taken off the critical path must be worth the difference
       const int64_t kb_total = t.K / 64, kb_saved = kb_total - kb_total / t.sk;
-      if (tiles * (t.cta_pair ? 4 : 2) <= 148 && t.K / t.sk >= 256 && kb_saved >= 160) mode = MTF_REDUCE_WORKSPACE;
+      if (tiles * (t.cta_pair ? 4 : 2) <= 148 && t.K / t.sk >= 256 && kb_saved >= 64) mode = MTF_REDUCE_WORKSPACE;
     }
     t.reduce_mode = mode;
     P->reduce_mode = mode;
