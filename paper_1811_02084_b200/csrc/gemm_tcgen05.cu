@@ -350,6 +350,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+      ::"r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]),
+        "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]),
+        "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]), "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 // Shared-memory matrix descriptor for a 128B-swizzled bf16 tile (descriptor version 1).
 //   K-major  (rows of 64 K-elements = 128 B; 8-row groups 1024 B apart): LBO unused (1), SBO = 1024 B
@@ -953,27 +970,48 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const float other = __uint_as_float(vb);
           return take_max ? fmaxf(mine, other) : mine + other;
         };
+        const int lim_all = __shfl_sync(0xffffffffu, lim, 0);             // columns below it take part in every row of the warp
         float mx = -INFINITY;
 #pragma unroll 1
         for (int c0 = col_half * 64; c0 < lim_warp; c0 += (c0 & 32) ? 96 : 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
           tmem_ld_wait();
+          if (c0 + 32 <= lim_all) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < lim) mx = fmaxf(mx, __uint_as_float(raw[j]) * sl2);
+            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(raw[j]));
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c0 + j < lim) mx = fmaxf(mx, __uint_as_float(raw[j]));
+          }
         }
-        mx = exchange(0, mx, true);
+        // (the maximum is taken over the raw accumulator: scale > 0 keeps the order; a negative scale would need the minimum)
+        mx = exchange(0, mx, true) * sl2;
         float sum = 0.f;
 #pragma unroll 1
         for (int c0 = col_half * 64; c0 < lim_warp; c0 += (c0 & 32) ? 96 : 32) {
           uint32_t raw[32];
           tmem_ld32(taddr + c0, raw);
           tmem_ld_wait();
+          if (c0 + 32 <= lim_all) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c0 + j < lim) sum += exp2f(__uint_as_float(raw[j]) * sl2 - mx);
+            for (int j = 0; j < 32; ++j) {
+              const float e = ex2_approx(fmaf(__uint_as_float(raw[j]), sl2, -mx));
+              sum += e;
+              raw[j] = __float_as_uint(e);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float e = (c0 + j < lim) ? ex2_approx(fmaf(__uint_as_float(raw[j]), sl2, -mx)) : 0.f;
+              sum += e;
+              raw[j] = __float_as_uint(e);
+            }
+          }
+          tmem_st32(taddr + c0, raw);                 // the exponentials replace the logits: the last pass only scales them
         }
+        tmem_st_wait();
         sum = exchange(1, sum, false);
         const float inv = 1.f / sum;
 #pragma unroll 1
@@ -992,7 +1030,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             tmem_ld32(taddr + c0, raw);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (c0 + j < lim) ? exp2f(__uint_as_float(raw[j]) * sl2 - mx) * inv : 0.f;
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(raw[j]) * inv;
           } else {
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = 0.f;
@@ -1418,6 +1456,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     // whole rows in one tile: the N slice is the whole dimension and fits a tile (256 columns, or 512 with a wide pair tile)
     const bool fits = a.sn == 1 && (a.Ns <= a.block_n || (a.Ns == 512 && t.cta_pair && t.block_n == 256));
     const bool bwd = row_softmax >= 3;      // backward: the weights come in as the mask operand, whole boxes only
+    if (!bwd && !(scale > 0.f)) return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a positive scale");
     if (!fits || plan.dtC != MTF_BF16 || resid || bias || relu || rsum || t.reduce_mode == MTF_REDUCE_WORKSPACE || n_terms != 1 ||
         (bwd ? (!mask || dtMask != MTF_BF16 || scale != 1.f || a.Ms % 32 != 0 || a.Ns % 64 != 0) : mask != nullptr))
       return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a bf16 result whose rows fit one tile (N <= 256, or 512 with CTA pairs) and no other stage");
