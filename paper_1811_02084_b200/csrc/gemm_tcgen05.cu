@@ -881,14 +881,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           dot += __uint_as_float(vb);
         };
         if (sb_nbox == 0) exchange_dot();                // no box of its own: the partner still needs a zero from this warp
+        const int first_visits = sb_nbox;
         const int visits = 2 * sb_nbox;
 #pragma unroll 1
         for (int vis = 0; vis < visits; ++vis) {
-          const bool second = vis >= sb_nbox;
-          const int bc = col_half * 64 + 128 * (second ? vis - sb_nbox : vis);     // first column of the box inside the tile
+          const bool second = vis >= first_visits;
+          const int bc = col_half * 64 + 128 * (second ? vis - first_visits : vis);     // first column of the box inside the tile
           const uint32_t box = stg + buf * 4096u;
           if (!mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag)) { ok = false; break; }
           mask_phase ^= 1u << buf;
+          if (vis + 1 < visits && lane == 0) {           // next visit's box into the other staging box, while this one is worked on
+            const int nv = vis + 1;
+            const int nbc = col_half * 64 + 128 * (nv >= first_visits ? nv - first_visits : nv);
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
+            tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), tl.n0 + nbc, row0, tl.o[2], tl.o[1], tl.o[0]);
+          }
           const uint32_t srow = box + (uint32_t)lane * 128u;
           const uint32_t sw = (uint32_t)(lane & 7);
 #pragma unroll
@@ -914,17 +922,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             __syncwarp();
             if (lane == 0) tma_store_5d(&map_c, box, tl.n0 + bc, row0, tl.o[2], tl.o[1], tl.o[0]);
           }
-          if (vis + 1 < visits && lane == 0) {           // next visit's box into the other staging box
-            const int nv = vis + 1;
-            const int nbc = col_half * 64 + 128 * (nv >= sb_nbox ? nv - sb_nbox : nv);
-            if (second) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-            else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
-            tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), tl.n0 + nbc, row0, tl.o[2], tl.o[1], tl.o[0]);
-          }
           __syncwarp();
           buf ^= 1u;
-          if (vis == sb_nbox - 1) exchange_dot();        // all first visits done: the row's dot product
+          if (vis == first_visits - 1) exchange_dot();   // all first visits done: the row's dot product
         }
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         // boxes right of every row's causal limit: zeros
@@ -1104,6 +1104,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (in_tma) {                                       // its mask / residual was requested a box ago, in place
               mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag);
               mask_phase ^= 1u << buf;
+              // the operand of this warp's next box of the tile into the other staging box (free once the
+              // store issued from it a box ago has been read out), so that it arrives while this box is worked on
+              const int next_n0 = box_n0 + 2 * box_cols;
+              if (lane == 0 && next_n0 < tl.n0 + a.block_n && next_n0 + box_cols <= tl.n_end) {
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
+                tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+              }
             } else {                                            // the box must be free: all but the latest store read out
               if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
               __syncwarp();
@@ -1176,16 +1184,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) {
-              tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
-              // request the mask of this warp's next box of the tile into the other staging box
-              const int next_n0 = box_n0 + 2 * box_cols;
-              if (in_tma && next_n0 < tl.n0 + a.block_n && next_n0 + box_cols <= tl.n_end) {
-                asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
-                tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), next_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
-              }
-            }
+            if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
             buf ^= 1u;
           }
           if (f.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now

@@ -159,6 +159,11 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
                      const void* const* extra_operands = nullptr,    // A_1, B_1 (, A_2, B_2) of a multi-term launch
                      int row_softmax = 0);                           // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue;
                                                                      // 3 / 4 (causal): its backward, P (A . B - rowsum(P A . B)), P = the mask operand
+// Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes
+// and types may not) in one launch, one accumulator.  MTF_ERR_UNSUPPORTED when this plan cannot
+// (generic kernel, workspace reduce mode): the caller then chains einsums through the residual stage.
+mtf_status einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tensor (*terms)[2], mtf_tensor* out,
+                        const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream);
 // weights[.., l, m] = softmax_m(scale * sum_k a b (causal: only m <= l)) in one launch, bf16 result.
 // MTF_ERR_UNSUPPORTED when the plan cannot (rows longer than a tile, generic kernel, split rows).
 // dlogits[.., l, m] = P (dP - sum_m dP P) with dP = sum_v a b, in one launch (same conditions, whole 32 x 64 boxes only).
