@@ -38,7 +38,8 @@ constexpr int kAStageBytes = BM * BK * 2;        // 16 KB
 constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stages half of it)
 constexpr int kRingBytes = 5 * (kAStageBytes + kBStageBytes / 2);   // pairs: 5 x (16 KB + 16 KB); single CTAs: 3 x 48 KB fit too
 constexpr int kStagingBytes = kEpilogueWarps * 2 * 4096;   // per epilogue warp: two 32-row x 128-byte boxes for TMA stores
-constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kMaxStages = 8;                      // ring slots with barriers; a launch uses as many as fit its stage size
+constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 320 /*barriers*/;
 constexpr int kThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
@@ -88,6 +89,7 @@ struct TcArgs {
   int n_fastest;           // tile order inside a slice: 1 = walk the n tiles of one m tile first
   long long tiles_per_slice, total_tiles, total_work;
   int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
+  int n_stages, stage_bytes;   // operand ring: 16 KB of A plus this CTA's part of B per stage, as many stages as fit
   int kb_tile;             // k-blocks of one whole tile (all terms)
   int softmax_causal;      // row-softmax epilogue: columns beyond the row's own position are masked out
   int n_terms;             // sum of n_terms products A_i . B_i of identical shape in one accumulator (1..3)
@@ -590,10 +592,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // k-block through L2 for twice the flops (24 KB per 256 x 256 x 64 instead of 32 KB).  For long K,
   // where the contraction is bound by the L2-to-SM traffic and the exposed epilogue is small.
   static_assert(!kWide || (kPair && CM == 1 && CN == 1), "wide tiles: plain CTA pairs only");
-  // (the row-softmax kind keeps one stage less: its two warps per lane quarter exchange row statistics
-  // through the 32 KB that frees at the end of the ring)
-  constexpr int kStages = (kPair && !kWide) ? ((EPI == EPI_ROW_SOFTMAX || EPI == EPI_ROW_SOFTMAX_BWD) ? 4 : 5) : 3;
-  constexpr int kStageBytes = (kPair && !kWide) ? (kAStageBytes + kBStageBytes / 2) : (kAStageBytes + kBStageBytes);
+  // The ring has a.n_stages stages of a.stage_bytes (32 KB for a pair with 256-column tiles: 5 stages;
+  // 48 KB for wide and single-CTA 256-column tiles: 3 stages; narrower tiles get deeper rings).  The
+  // row-softmax kinds leave 2 KB at the end of the ring for the exchange of row statistics.
+  const int kStages = a.n_stages;
+  const int kStageBytes = a.stage_bytes;
   constexpr int kPairRows = kPair ? 2 * BM : BM;       // rows of C owned by one CTA pair (or single CTA)
   constexpr int kTileRows = kPairRows * CM;            // rows of C owned by a work item
   constexpr bool kCluster = CM * CN > 1;
@@ -606,14 +609,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // after the ring: per epilogue warp two 4 KB staging boxes for the output stores, then the barriers
   const uint32_t staging_base = tiles_base + kRingBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(gen_base + kRingBytes + kStagingBytes);
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty
+  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem_full, [2S+2..2S+4) tmem_empty  (S = kMaxStages slots)
   const uint32_t bar_base = staging_base + kStagingBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kStages + i); };
-  auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kStages + 2 + i); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kMaxStages + s); };
+  auto tfull_bar = [&](int i) { return bar_base + 8u * (2 * kMaxStages + i); };
+  auto tempty_bar = [&](int i) { return bar_base + 8u * (2 * kMaxStages + 2 + i); };
   // then [2S+4..2S+20): per epilogue warp two barriers for relu-mask boxes loaded into its staging buffers
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4 + 2 * kEpilogueWarps);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4 + 2 * kEpilogueWarps);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -630,7 +633,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), CM + CN - 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), (kPair ? 2 : 1) * kEpilogueWarps); }
-    for (int i = 0; i < 2 * kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kStages + 4 + i), 1);
+    for (int i = 0; i < 2 * kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kMaxStages + 4 + i), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -791,7 +794,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t stg = staging_base + (uint32_t)(warp - 2) * 8192u;      // this warp's two staging boxes
     uint32_t buf = 0;                              // staging box the next output box goes through
     uint32_t mask_phase = 0;                       // bit b: phase of this warp's mask barrier b
-    auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
+    auto mfull_bar = [&](uint32_t b) { return bar_base + 8u * (2 * kMaxStages + 4 + (uint32_t)(warp - 2) * 2 + b); };
     int iter = 0;
     bool ok = true;
     SegIter it(a, work_first, work_step);
@@ -1509,6 +1512,12 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
+  {
+    const int b_cols = (t.cta_pair ? a.block_n / 2 : a.block_n);          // B columns staged by one CTA (wide: two runs of 128)
+    a.stage_bytes = kAStageBytes + b_cols * BK * 2;
+    const int ring = kRingBytes - (row_softmax ? 2048 : 0);
+    a.n_stages = std::min(kMaxStages, ring / a.stage_bytes);
+  }
   a.kb_term = a.k_sliced ? a.sk * (a.Ks / BK) : (a.K + BK - 1) / BK;
   a.n_terms = n_terms;
   a.softmax_causal = (row_softmax == 2 || row_softmax == 4) ? 1 : 0;
