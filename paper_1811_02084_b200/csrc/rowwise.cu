@@ -8,6 +8,7 @@
 // own shuffle reduction over the whole row.  The column sums (reduce out the token dims, i.e. the
 // gradient Allreduce of Algorithm 1 under a batch split) accumulate per block and finish with fp32
 // atomics.  All loads and stores are 16-byte vectors, coalesced along the row.
+#include <algorithm>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -197,6 +198,169 @@ layernorm_bwd_dx_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat1
   }
 }
 
+// Rows of exactly NCH * 256 columns: a lane keeps its NCH pieces of 8 columns in registers, so the row
+// is read from memory once and all its loads are in flight together.
+template <int NCH>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+layernorm_fwd_rows_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                          __nv_bfloat16* __restrict__ y, float* __restrict__ stats, int64_t rows, float eps) {
+  constexpr int n = NCH * 256;
+  const int64_t row = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const __nv_bfloat16* xr = x + row * n + lane * 8;
+  uint4 xv[NCH];
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) xv[i] = *reinterpret_cast<const uint4*>(xr + i * 256);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    float f[8];
+    bf16x8_to_float(xv[i], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s += f[e];
+  }
+  const float mu = warp_sum(s) / (float)n;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    float f[8];
+    bf16x8_to_float(xv[i], f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) q += (f[e] - mu) * (f[e] - mu);
+  }
+  const float rstd = rsqrtf(warp_sum(q) / (float)n + eps);
+  if (lane == 0) { stats[2 * row] = mu; stats[2 * row + 1] = rstd; }
+  __nv_bfloat16* yr = y + row * n + lane * 8;
+#pragma unroll
+  for (int i = 0; i < NCH; ++i) {
+    const int c = i * 256 + lane * 8;
+    float f[8], o[8];
+    bf16x8_to_float(xv[i], f);
+    const float4 g0 = *reinterpret_cast<const float4*>(gamma + c), g1 = *reinterpret_cast<const float4*>(gamma + c + 4);
+    const float4 b0 = *reinterpret_cast<const float4*>(beta + c), b1 = *reinterpret_cast<const float4*>(beta + c + 4);
+    const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+    const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e) o[e] = g[e] * (f[e] - mu) * rstd + b[e];
+    *reinterpret_cast<uint4*>(yr + i * 256) = float_to_bf16x8(o);
+  }
+}
+
+// Backward for rows of NCH * 256 columns, dx and the parameter gradients in one pass over dy and x:
+// a persistent grid of 8-warp blocks, every warp walks rows with both rows in registers and keeps
+// its lanes' partial dgamma / dbeta sums in registers; at the end the block adds them up in shared
+// memory and issues one fp32 atomic per column and block.
+// kSmemAcc (the 2048-column case, whose 128 partial sums per lane do not fit the registers next to
+// the two rows): every warp keeps its partial sums in a shared-memory strip of its own instead.
+template <int NCH, bool kSmemAcc>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 1)
+layernorm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ x, const float* __restrict__ stats,
+                          const float* __restrict__ gamma, const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ dx,
+                          float* __restrict__ dgamma, float* __restrict__ dbeta, int64_t rows) {
+  constexpr int n = NCH * 256;
+  constexpr int kAccRegs = kSmemAcc ? 1 : NCH;
+  extern __shared__ float4 sh_dyn[];
+  float* const sh = reinterpret_cast<float*>(sh_dyn);                 // [2][n] block sums, then (kSmemAcc) [warps][2][n] strips
+  const int n_sh = 2 * n * (kSmemAcc ? 1 + kWarpsPerBlock : 1);
+  for (int i = threadIdx.x; i < n_sh; i += kWarpsPerBlock * 32) sh[i] = 0.f;
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  float* const strip = sh + 2 * n * (1 + (threadIdx.x >> 5));           // this warp's strip: [2][n]
+  const int64_t wid = (int64_t)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5), nw = (int64_t)gridDim.x * kWarpsPerBlock;
+  float ag[kAccRegs][8], ab[kAccRegs][8];
+#pragma unroll
+  for (int i = 0; i < kAccRegs; ++i)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { ag[i][e] = 0.f; ab[i][e] = 0.f; }
+  for (int64_t row = wid; row < rows; row += nw) {
+    const __nv_bfloat16* xr = x + row * n + lane * 8;
+    const __nv_bfloat16* dr = dy + row * n + lane * 8;
+    uint4 xv[NCH], dv[NCH];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) { xv[i] = *reinterpret_cast<const uint4*>(xr + i * 256); dv[i] = *reinterpret_cast<const uint4*>(dr + i * 256); }
+    const float mu = stats[2 * row], rstd = stats[2 * row + 1];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+      const int c = i * 256 + lane * 8;
+      float xf[8], df[8];
+      bf16x8_to_float(xv[i], xf);
+      bf16x8_to_float(dv[i], df);
+      const float4 g0 = *reinterpret_cast<const float4*>(gamma + c), g1 = *reinterpret_cast<const float4*>(gamma + c + 4);
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      if (kSmemAcc) {
+        float4* pg = reinterpret_cast<float4*>(strip + c);
+        float4* pb = reinterpret_cast<float4*>(strip + n + c);
+        float4 a0 = pg[0], a1 = pg[1], b0 = pb[0], b1 = pb[1];
+        float ga[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w}, be[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float xh = (xf[e] - mu) * rstd;
+          const float gg = df[e] * g[e];
+          s1 += gg;
+          s2 += gg * xh;
+          ga[e] += df[e] * xh;
+          be[e] += df[e];
+        }
+        pg[0] = make_float4(ga[0], ga[1], ga[2], ga[3]); pg[1] = make_float4(ga[4], ga[5], ga[6], ga[7]);
+        pb[0] = make_float4(be[0], be[1], be[2], be[3]); pb[1] = make_float4(be[4], be[5], be[6], be[7]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float xh = (xf[e] - mu) * rstd;
+          const float gg = df[e] * g[e];
+          s1 += gg;
+          s2 += gg * xh;
+          ag[kSmemAcc ? 0 : i][e] += df[e] * xh;
+          ab[kSmemAcc ? 0 : i][e] += df[e];
+        }
+      }
+    }
+    const float m1 = warp_sum(s1) / (float)n, m2 = warp_sum(s2) / (float)n;
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+      const int c = i * 256 + lane * 8;
+      float xf[8], df[8], o[8], rf[8];
+      bf16x8_to_float(xv[i], xf);
+      bf16x8_to_float(dv[i], df);
+      if (residual) bf16x8_to_float(*reinterpret_cast<const uint4*>(residual + row * n + c), rf);
+      const float4 g0 = *reinterpret_cast<const float4*>(gamma + c), g1 = *reinterpret_cast<const float4*>(gamma + c + 4);
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float xh = (xf[e] - mu) * rstd;
+        o[e] = rstd * (df[e] * g[e] - m1 - xh * m2) + (residual ? rf[e] : 0.f);
+      }
+      *reinterpret_cast<uint4*>(dx + row * n + c) = float_to_bf16x8(o);
+    }
+  }
+  if (dgamma && dbeta) {
+    if (kSmemAcc) {
+      __syncthreads();
+      for (int c = threadIdx.x; c < 2 * n; c += kWarpsPerBlock * 32) {
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarpsPerBlock; ++w) t += sh[2 * n * (1 + w) + c];
+        atomicAdd((c < n ? dgamma : dbeta) + (c < n ? c : c - n), t);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < kAccRegs; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          atomicAdd(&sh[i * 256 + lane * 8 + e], ag[i][e]);
+          atomicAdd(&sh[n + i * 256 + lane * 8 + e], ab[i][e]);
+        }
+      __syncthreads();
+      for (int c = threadIdx.x; c < n; c += kWarpsPerBlock * 32) {
+        atomicAdd(dgamma + c, sh[c]);
+        atomicAdd(dbeta + c, sh[n + c]);
+      }
+    }
+  }
+}
+
 // dgamma[c] += sum_rows dy * xh,  dbeta[c] += sum_rows dy.  Block = 32 x 8 threads: 64 columns
 // (two per thread), the 8 thread rows interleave over a chunk of token rows; fp32 atomics finish.
 __global__ void __launch_bounds__(256)
@@ -273,7 +437,17 @@ mtf_status launch_layernorm_fwd(const void* x, const float* gamma, const float* 
   if (rows <= 0) return MTF_OK;
   const int64_t blocks = (rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if (blocks > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "layernorm: too many rows");
-  layernorm_fwd_kernel<<<(unsigned)blocks, kWarpsPerBlock * 32, 0, (cudaStream_t)stream>>>(reinterpret_cast<const __nv_bfloat16*>(x), gamma, beta, reinterpret_cast<__nv_bfloat16*>(y), stats, rows, n, eps);
+  const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(x);
+  __nv_bfloat16* yb = reinterpret_cast<__nv_bfloat16*>(y);
+  cudaStream_t st = (cudaStream_t)stream;
+  // rows of 256, 512, 1024 or 2048 columns stay in registers; other lengths re-read the row per pass
+  switch (n) {
+    case 256: layernorm_fwd_rows_kernel<1><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(xb, gamma, beta, yb, stats, rows, eps); break;
+    case 512: layernorm_fwd_rows_kernel<2><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(xb, gamma, beta, yb, stats, rows, eps); break;
+    case 1024: layernorm_fwd_rows_kernel<4><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(xb, gamma, beta, yb, stats, rows, eps); break;
+    case 2048: layernorm_fwd_rows_kernel<8><<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(xb, gamma, beta, yb, stats, rows, eps); break;
+    default: layernorm_fwd_kernel<<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(xb, gamma, beta, yb, stats, rows, n, eps);
+  }
   count_launch();
   return check("layernorm_fwd_kernel");
 }
@@ -284,6 +458,37 @@ mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stat
     return fail(MTF_ERR_UNSUPPORTED, "layernorm backward: row length must be a multiple of 8 and pointers 16-byte aligned");
   if (rows <= 0) return MTF_OK;
   cudaStream_t st = (cudaStream_t)stream;
+  if (n == 256 || n == 512 || n == 1024 || n == 2048) {
+    // one pass over dy and x for dx and the parameter gradients (persistent grid, one block per SM)
+    if (dgamma && dbeta) {
+      cudaError_t e = cudaMemsetAsync(dgamma, 0, (size_t)n * sizeof(float), st);
+      if (e == cudaSuccess) e = cudaMemsetAsync(dbeta, 0, (size_t)n * sizeof(float), st);
+      if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+    }
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const unsigned grid = (unsigned)std::min<int64_t>((rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 2 * (int64_t)sms);
+    const __nv_bfloat16* db = reinterpret_cast<const __nv_bfloat16*>(dy);
+    const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(x);
+    const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(residual);
+    __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(dx);
+    float* dg = (dgamma && dbeta) ? dgamma : nullptr;
+    float* dbp = (dgamma && dbeta) ? dbeta : nullptr;
+    const size_t sm_small = 2 * (size_t)n * sizeof(float), sm_big = sm_small * (1 + kWarpsPerBlock);       // 144 KB for 2048 columns
+    switch (n) {
+      case 256: layernorm_bwd_rows_kernel<1, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
+      case 512: layernorm_bwd_rows_kernel<2, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
+      case 1024: layernorm_bwd_rows_kernel<4, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
+      default: {
+        static cudaError_t attr = cudaFuncSetAttribute(layernorm_bwd_rows_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * 2048 * sizeof(float) * (1 + kWarpsPerBlock)));
+        if (attr != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr));
+        layernorm_bwd_rows_kernel<8, true><<<std::min(grid, (unsigned)sms), kWarpsPerBlock * 32, sm_big, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows);
+      }
+    }
+    count_launch();
+    return check("layernorm_bwd_rows_kernel");
+  }
   const int64_t blocks = (rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if (blocks > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "layernorm backward: too many rows");
   layernorm_bwd_dx_kernel<<<(unsigned)blocks, kWarpsPerBlock * 32, 0, st>>>(reinterpret_cast<const __nv_bfloat16*>(dy), reinterpret_cast<const __nv_bfloat16*>(x), stats, gamma,
