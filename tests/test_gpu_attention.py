@@ -168,17 +168,20 @@ def test_einsum_softmax_refuses_rows_that_do_not_fit(mtf):
 
 # ---- layer norm --------------------------------------------------------------------------------------------
 
-def test_layernorm_forward_backward(mtf):
+# 136: the kernels that re-read the row per pass; 256..2048: rows kept in registers (2048: partial
+# parameter sums in shared-memory strips); 50 rows per batch entry leave the last block ragged
+@pytest.mark.parametrize("D", [136, 256, 512, 1024, 2048])
+def test_layernorm_forward_backward(mtf, D):
     import torch
     from oracle import NT, DenseOps, blocks
     ops = DenseOps()
-    dims = [("batch", 3), ("length", 50), ("d_model", 136)]
+    dims = [("batch", 3), ("length", 50), ("d_model", D)]
     names = [n for n, _ in dims]
-    x = si.normal(12, "x", [3, 50, 136], "bf16", 2.0, 0.5)
-    dy = si.normal(12, "dy", [3, 50, 136], "bf16")
-    res = si.normal(12, "res", [3, 50, 136], "bf16")
-    gamma = si.normal(12, "g", [136], "f32", 0.1, 1.0)
-    beta = si.normal(12, "b", [136], "f32", 0.1)
+    x = si.normal(12, "x", [3, 50, D], "bf16", 2.0, 0.5)
+    dy = si.normal(12, "dy", [3, 50, D], "bf16")
+    res = si.normal(12, "res", [3, 50, D], "bf16")
+    gamma = si.normal(12, "g", [D], "f32", 0.1, 1.0)
+    beta = si.normal(12, "b", [D], "f32", 0.1)
     eps = 1e-6
     f = blocks.layernorm_forward(ops, NT(dims, x.f64), NT(dims[2:], gamma.f64), NT(dims[2:], beta.f64), eps)
     g = blocks.layernorm_backward(ops, NT(dims[2:], gamma.f64), f, NT(dims, dy.f64))
