@@ -179,7 +179,7 @@ def run_ours(args):
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
     torch.cuda.set_device(local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or os.environ.get("MTF_BENCH_DIST"):      # (the variable: exercise the N > 1 code path with one rank)
         import torch.distributed as dist_mod
         dist = dist_mod
         dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local_rank))
@@ -221,12 +221,44 @@ def run_ours(args):
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
 
+    dhp = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda") if dist is not None else None
+    sync = multi_gpu.GradientSync(dist)
+
+    def backward(lay, xin, dyin, dxout):
+        """The feed-forward backward pass.  On one GPU: mtf_ffn_backward.  On several: the same four
+        contractions issued one by one (what mtf_ffn_backward does inside), so that the all-reduce of a
+        parameter gradient (Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs)
+        starts right behind the contraction that produces it and runs while the later ones compute."""
+        if dist is None:
+            mtf.mtf_ffn_backward(lay, xin, N["w"], N["v"], N["h"], dyin, dxout, N["dw"], N["dbias"], N["dv"], ws)
+            return
+        ndhp = mtf.named(dhp, ["batch", "length", "d_ff"])
+        mtf.mtf_einsum(lay, None, [dyin, N["v"]], ndhp, mtf.Epilogue(relu_mask=N["h"], reduce_sum_out=N["dbias"]), workspace=ws)
+        mtf.mtf_einsum(lay, None, [N["h"], dyin], N["dv"], None, workspace=ws)
+        sync.start(dv)
+        sync.start(dbias)
+        mtf.mtf_einsum(lay, None, [xin, ndhp], N["dw"], None, workspace=ws)
+        sync.start(dw)
+        mtf.mtf_einsum(lay, None, [ndhp, N["w"]], dxout, None, workspace=ws)
+        sync.finish()
+
     def step(lay):
         mtf.mtf_ffn_forward(lay, N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
-        mtf.mtf_ffn_backward(lay, N["x"], N["w"], N["v"], N["h"], N["dy"], N["dx"], N["dw"], N["dbias"], N["dv"], ws)
-        # Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs sums the
-        # parameter gradients across ranks (no-op on one GPU)
-        multi_gpu.allreduce_gradients(dist, (dw, dv, dbias))
+        backward(lay, N["x"], N["dy"], N["dx"])
+
+    if dist is not None:
+        # the contractions issued one by one give what the block entry point gives
+        mtf.mtf_ffn_forward(layouts[args.layout], N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
+        mtf.mtf_ffn_backward(layouts[args.layout], N["x"], N["w"], N["v"], N["h"], N["dy"], N["dx"], N["dw"], N["dbias"], N["dv"], ws)
+        want = [t_.clone() for t_ in (dx, dw, dv, dbias)]
+        ndhp = mtf.named(dhp, ["batch", "length", "d_ff"])
+        mtf.mtf_einsum(layouts[args.layout], None, [N["dy"], N["v"]], ndhp, mtf.Epilogue(relu_mask=N["h"], reduce_sum_out=N["dbias"]), workspace=ws)
+        mtf.mtf_einsum(layouts[args.layout], None, [N["h"], N["dy"]], N["dv"], None, workspace=ws)
+        mtf.mtf_einsum(layouts[args.layout], None, [N["x"], ndhp], N["dw"], None, workspace=ws)
+        mtf.mtf_einsum(layouts[args.layout], None, [ndhp, N["w"]], N["dx"], None, workspace=ws)
+        torch.cuda.synchronize()
+        for got, ref, nm in zip((dx, dw, dv, dbias), want, ("dx", "dw", "dv", "dbias")):
+            assert torch.allclose(got.float(), ref.float(), rtol=1e-3, atol=1e-3 * float(ref.float().abs().max())), f"{nm}: the einsum sequence differs from mtf_ffn_backward"
 
     def timed(lay, steps, warmup, sampler=None):
         for _ in range(warmup):
@@ -303,8 +335,7 @@ def run_ours(args):
         stream.wait_event(in_ready[q])
         stream.wait_event(out_done[q])                  # the results of the step that last used this output set are on the host
         mtf.mtf_ffn_forward(lay, names["x"], N["w"], N["bias"], N["v"], N["h"], names["y"], ws)
-        mtf.mtf_ffn_backward(lay, names["x"], N["w"], N["v"], N["h"], names["dy"], names["dx"], N["dw"], N["dbias"], N["dv"], ws)
-        multi_gpu.allreduce_gradients(dist, (dw, dv, dbias))
+        backward(lay, names["x"], names["dy"], names["dx"])
         done[q].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(done[q])

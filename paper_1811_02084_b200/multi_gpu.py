@@ -26,6 +26,26 @@ def allreduce_gradients(dist, grads) -> None:
         dist.all_reduce(g)
 
 
+class GradientSync:
+    """Sums gradients over the ranks while later kernels of the backward pass still run: ``start`` is
+    called right after the launch that produces a gradient and enqueues its all-reduce without
+    blocking (the collective waits for that launch on its own stream), ``finish`` makes the calling
+    stream wait for every all-reduce started since.  With one rank (``dist`` None) both do nothing."""
+
+    def __init__(self, dist):
+        self.dist = dist
+        self.pending = []
+
+    def start(self, tensor) -> None:
+        if self.dist is not None:
+            self.pending.append(self.dist.all_reduce(tensor, async_op=True))
+
+    def finish(self) -> None:
+        for work in self.pending:
+            work.wait()
+        self.pending = []
+
+
 def max_over_ranks(dist, value: float, device="cpu") -> float:
     """The slowest rank's value (timings of a multi-rank step are reported as the maximum)."""
     if dist is None:

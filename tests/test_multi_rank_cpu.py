@@ -41,7 +41,13 @@ def _worker(rank, world, port, out_dir):
     f = blocks.ffn_forward(ops, xs, w, bias, v)
     g = blocks.ffn_backward(ops, xs, w, v, f["h"], dys)
     grads = [torch.from_numpy(g[k].a.copy()) for k in ("dw", "dv", "dbias")]
-    multi_gpu.allreduce_gradients(dist, grads)
+    # dw and dv through the non-blocking path the bench uses between its launches, dbias through the blocking one
+    sync = multi_gpu.GradientSync(dist)
+    sync.start(grads[1])
+    sync.start(grads[0])
+    sync.finish()
+    assert sync.pending == []
+    multi_gpu.allreduce_gradients(dist, grads[2:])
     slowest = multi_gpu.max_over_ranks(dist, float(rank + 1))
     np.savez(os.path.join(out_dir, f"rank{rank}.npz"), dw=grads[0].numpy(), dv=grads[1].numpy(), dbias=grads[2].numpy(),
              dx=g["dx"].a, y=f["y"].a, slowest=slowest, block=np.array([b0, b1]))
@@ -78,4 +84,7 @@ def test_rank_block_rules():
     with pytest.raises(ValueError):
         multi_gpu.rank_block(30, 8, 0)
     multi_gpu.allreduce_gradients(None, [torch.ones(2)])          # single process: no-op
+    one = multi_gpu.GradientSync(None)
+    one.start(torch.ones(2))
+    one.finish()
     assert multi_gpu.max_over_ranks(None, 3.5) == 3.5
