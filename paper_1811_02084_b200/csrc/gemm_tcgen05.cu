@@ -412,7 +412,7 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
 // far fewer registers and instructions per chunk.
 enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_ROW_SOFTMAX_BWD = 6, EPI_KINDS = 7 };
 struct EpiFlags {
-  bool scale, bias, bias_m, relu, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
+  bool scale, bias, bias_m, relu, relu_in_pack, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
 };
 template <int EPI>
 __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
@@ -420,11 +420,12 @@ __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
   if (EPI == EPI_GENERIC) {
     f.scale = a.scale != 1.f; f.bias = a.bias != nullptr; f.bias_m = a.bias_along_m != 0; f.relu = a.relu != 0;
     f.mask = a.mask != nullptr; f.mask_bf16 = a.mask_bf16 != 0; f.mask_tma = a.mask_tma != 0; f.resid = a.resid != nullptr; f.resid_tma = a.resid_tma != 0;
-    f.rsum = a.rsum != nullptr; f.c_bf16 = a.c_bf16 != 0; f.shared_tiles = true;
+    f.rsum = a.rsum != nullptr; f.c_bf16 = a.c_bf16 != 0; f.shared_tiles = true; f.relu_in_pack = false;
   } else {
     f.scale = false; f.bias = EPI == EPI_BIAS_RELU_BF16; f.bias_m = false; f.relu = EPI == EPI_BIAS_RELU_BF16;
     f.mask = f.mask_bf16 = f.mask_tma = f.rsum = EPI == EPI_MASK_RSUM_BF16; f.resid = f.resid_tma = false;
     f.c_bf16 = EPI != EPI_PLAIN_F32;
+    f.relu_in_pack = EPI == EPI_BIAS_RELU_BF16;      // relu is the last stage there: it rides in the conversion to bf16
     if (EPI == EPI_ROW_SOFTMAX) f.scale = true;
     if (EPI == EPI_ROW_SOFTMAX_BWD) f.mask = f.mask_bf16 = true;      // the weights P arrive like a mask, by TMA
     f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
@@ -445,6 +446,16 @@ __device__ __forceinline__ void mask_fetch(const TcArgs& a, long long off, bool 
 // scale, bias (broadcast), relu, relu mask; the value then feeds the fused reduce_sum; residual last.
 //   bias_lane : bias of column (n_first + lane), handed to every lane by shuffle (bias along n)
 //   bias_row  : bias of this thread's row (bias along m)
+// Keeps a (b) where the lower (upper) bf16 of m is greater than zero, else makes it zero: one packed
+// compare for two mask values (ordered: a NaN mask keeps nothing, like the scalar comparison).
+__device__ __forceinline__ void keep_where_positive(uint32_t m, float& a, float& b) {
+  asm("{\n\t.reg .pred p, q;\n\t"
+      "setp.gt.bf16x2 p|q, %2, %3;\n\t"
+      "selp.f32 %0, %0, 0f00000000, p;\n\t"
+      "selp.f32 %1, %1, 0f00000000, q;\n\t}"
+      : "+f"(a), "+f"(b) : "r"(m), "r"(0u));
+}
+
 __device__ __forceinline__ void epilogue_math(const TcArgs& a, const EpiFlags& f, float* v, float bias_lane, float bias_row,
                                               const uint4* mk, long long off, bool live, int n_valid) {
   if (f.scale) {
@@ -460,7 +471,7 @@ __device__ __forceinline__ void epilogue_math(const TcArgs& a, const EpiFlags& f
       for (int j = 0; j < 32; ++j) v[j] += __shfl_sync(0xffffffffu, bias_lane, j);
     }
   }
-  if (f.relu) {
+  if (f.relu && !f.relu_in_pack) {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = fmaxf(v[j], 0.f);
   }
@@ -468,11 +479,9 @@ __device__ __forceinline__ void epilogue_math(const TcArgs& a, const EpiFlags& f
     if (f.mask_bf16) {
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        float f[8];
-        unpack_bf16x8(mk[q], f);
+        const uint32_t w[4] = {mk[q].x, mk[q].y, mk[q].z, mk[q].w};
 #pragma unroll
-        for (int e = 0; e < 8; ++e)
-          if (!(f[e] > 0.f)) v[q * 8 + e] = 0.f;
+        for (int e = 0; e < 4; ++e) keep_where_positive(w[e], v[q * 8 + 2 * e], v[q * 8 + 2 * e + 1]);
       }
     } else if (live) {
       const float* mp = reinterpret_cast<const float*>(a.mask) + off;
@@ -503,20 +512,29 @@ __device__ __forceinline__ void epilogue_residual(const TcArgs& a, const EpiFlag
   }
 }
 
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 h2 = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&h2);
 }
 
 // 16-byte stores of one chunk straight from registers (ragged tiles and the workspace mode).
+__device__ __forceinline__ uint32_t pack_out(const EpiFlags& f, float lo, float hi) {
+  return f.relu_in_pack ? pack_bf16x2_relu(lo, hi) : pack_bf16x2(lo, hi);
+}
+
 __device__ __forceinline__ void store_direct(const TcArgs& a, const EpiFlags& f, const float* v, long long off, int n_valid) {
   if (f.c_bf16) {
     uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
       if (q * 8 < n_valid)
-        cp[q] = make_uint4(pack_bf16x2(v[q * 8], v[q * 8 + 1]), pack_bf16x2(v[q * 8 + 2], v[q * 8 + 3]),
-                           pack_bf16x2(v[q * 8 + 4], v[q * 8 + 5]), pack_bf16x2(v[q * 8 + 6], v[q * 8 + 7]));
+        cp[q] = make_uint4(pack_out(f, v[q * 8], v[q * 8 + 1]), pack_out(f, v[q * 8 + 2], v[q * 8 + 3]),
+                           pack_out(f, v[q * 8 + 4], v[q * 8 + 5]), pack_out(f, v[q * 8 + 6], v[q * 8 + 7]));
   } else {
     float4* cp = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off);
 #pragma unroll
@@ -548,9 +566,9 @@ __device__ __forceinline__ void store_staged(const EpiFlags& f, const float* v, 
   if (f.c_bf16) {
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-      st_shared_v4(row + ((((uint32_t)(half * 4 + q)) ^ sw) << 4), pack_bf16x2(v[q * 8], v[q * 8 + 1]),
-                   pack_bf16x2(v[q * 8 + 2], v[q * 8 + 3]), pack_bf16x2(v[q * 8 + 4], v[q * 8 + 5]),
-                   pack_bf16x2(v[q * 8 + 6], v[q * 8 + 7]));
+      st_shared_v4(row + ((((uint32_t)(half * 4 + q)) ^ sw) << 4), pack_out(f, v[q * 8], v[q * 8 + 1]),
+                   pack_out(f, v[q * 8 + 2], v[q * 8 + 3]), pack_out(f, v[q * 8 + 4], v[q * 8 + 5]),
+                   pack_out(f, v[q * 8 + 6], v[q * 8 + 7]));
   } else {
 #pragma unroll
     for (int q = 0; q < 8; ++q)
@@ -1191,8 +1209,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             buf ^= 1u;
           }
           if (f.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
+            if (!(rows_full && n_valid == 32)) {       // ragged chunk: rows and columns outside the slice add nothing
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (live && j < n_valid) ? v[j] : 0.f;
+              for (int j = 0; j < 32; ++j) v[j] = (live && j < n_valid) ? v[j] : 0.f;
+            }
             const float col = warp_column_sums(v, lane);
             if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
           }
