@@ -29,7 +29,7 @@ LAYOUTS = {
     "dp8": ([("all", 8)], [("batch", "all")]),
     "mp8": ([("all", 8)], [("d_ff", "all")]),
 }
-NCU_DRAM_BYTES_PER_LAUNCH = 170.3e6
+NCU_DRAM_BYTES_PER_LAUNCH = 169.7e6
 METRIC = "transformer_ffn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
