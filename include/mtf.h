@@ -58,7 +58,8 @@ typedef struct mtf_mesh_s mtf_mesh_t;
 typedef struct mtf_layout_s mtf_layout_t;
 typedef struct mtf_plan_s mtf_plan_t;
 
-/* A named dimension (Section 4): name + static size. */
+/* A named dimension (Section 4): name + static size.  Sizes are at least 1: a tensor with an empty
+ * dimension has no slices to lay out and every call that sees one returns MTF_ERR_INVALID_ARG. */
 typedef struct { const char* name; int64_t size; } mtf_dim;
 
 /* A named tensor: non-owning view.  `data` is a device pointer (ignored where stated). */

@@ -474,6 +474,9 @@ mtf_status mtf::einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor*
   mtf_status st = cached_plan(layout, 2, in, weights, &e, &P);
   if (st != MTF_OK) return st;
   if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->tc.swapped) return fail(MTF_ERR_UNSUPPORTED, "einsum_row_softmax: not on this plan");
+  // the causal limit compares a row's position with the column: the rows of the contraction must be one dimension
+  if (causal && (weights->ndim < 2 || weights->dims[weights->ndim - 2].size != P->tc.M || weights->dims[weights->ndim - 1].size != P->tc.N))
+    return fail(MTF_ERR_UNSUPPORTED, "einsum_row_softmax: a causal mask needs the two last output dimensions to be the rows and columns of the contraction");
   return exec_plan(P, in, weights, &e, workspace, workspace_bytes, stream, 1, nullptr, causal ? 2 : 1);
 }
 

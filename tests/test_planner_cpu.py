@@ -51,6 +51,17 @@ def test_mesh_coords_match_oracle():
         mtf.mtf_mesh_coords(mtf.mtf_mesh_create([("a", 2)]), 2)
 
 
+def test_empty_dimensions_are_refused():
+    L = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 2)]), [("batch", "all")])
+    a, b = mtf.desc([("batch", 4), ("k", 0)], "bf16"), mtf.desc([("k", 0), ("j", 8)], "bf16")
+    with pytest.raises(mtf.MtfError) as e:
+        mtf.mtf_einsum_plan(L, [a, b], mtf.desc([("batch", 4), ("j", 8)], "bf16"))
+    assert e.value.code == "MTF_ERR_INVALID_ARG"
+    with pytest.raises(mtf.MtfError) as e:
+        mtf.mtf_layout_check_tensor(L, [("batch", 0)])
+    assert e.value.code == "MTF_ERR_INVALID_ARG"
+
+
 def both(mesh_dims, rules):
     return mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules), Layout(Mesh(mesh_dims), rules)
 
