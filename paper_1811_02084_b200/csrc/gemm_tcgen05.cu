@@ -549,11 +549,6 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   return r;
 }
 
-__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
-  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global [%0, {%1, %2, %3, %4, %5}];"
-               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
-}
-
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
 }
@@ -865,10 +860,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
       }
       if (in_tma && lane == 0) {
-        // pull this warp's boxes of the operand's tile towards L2 and request the first one into the
-        // staging box it will be processed in (free once all but the latest store have been read out)
-        for (int b = col_half * box_cols; b < a.block_n; b += 2 * box_cols)
-          if (tl.n0 + b + box_cols <= tl.n_end) tma_prefetch_5d(&map_m, tl.n0 + b, row0, tl.o[2], tl.o[1], tl.o[0]);
+        // request the first box into the staging box it will be processed in (free once all but the latest
+        // store have been read out); asking for the later boxes to be brought to L2 here measured slower
         if (col_half * box_cols < a.block_n && tl.n0 + col_half * box_cols + box_cols <= tl.n_end) {
           asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
           mbar_expect_tx(mfull_bar(buf), 4096u);
