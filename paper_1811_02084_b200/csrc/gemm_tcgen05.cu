@@ -1098,7 +1098,55 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (!ok) break;
         }
       }
-      if (finisher) {
+      if (EPI == EPI_MASK_RSUM_BF16 && rows_full && tl.n0 + a.block_n <= tl.n_end) {
+        // A tile that lies wholly inside its slice, for the kind whose epilogue sets the pace of its
+        // contraction (dhp): a box (two 32-column chunks) at a time, both tensor-memory loads in flight
+        // together and the two chunks' arithmetic interleaved (3 us of 117; the same for bias + relu lost 1 us).
+#pragma unroll 1
+        for (int c0 = col_half * 64; c0 < a.block_n; c0 += 128) {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(taddr + c0, r0);
+          tmem_ld32(taddr + c0 + 32, r1);
+          const uint32_t box = stg + buf * 4096u;
+          const uint32_t srow = box + (uint32_t)lane * 128u;
+          const uint32_t sw = (uint32_t)(lane & 7);
+          uint4 mk[8];
+          mbar_wait(mfull_bar(buf), (mask_phase >> buf) & 1u, 0x500 + (int)buf, abort_flag);   // its relu mask, requested a box ago
+          mask_phase ^= 1u << buf;
+          if (lane == 0 && c0 + 128 < a.block_n) {                                             // the next box's mask into the other staging box
+            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            mbar_expect_tx(mfull_bar(buf ^ 1u), 4096u);
+            tma_load_5d<false>(stg + (buf ^ 1u) * 4096u, &map_m, mfull_bar(buf ^ 1u), tl.n0 + c0 + 128, row0, tl.o[2], tl.o[1], tl.o[0]);
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) mk[i] = ld_shared_v4(srow + (((uint32_t)i ^ sw) << 4));
+          tmem_ld_wait();
+          float* v0 = reinterpret_cast<float*>(r0);
+          float* v1 = reinterpret_cast<float*>(r1);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t w0[4] = {mk[i].x, mk[i].y, mk[i].z, mk[i].w}, w1[4] = {mk[4 + i].x, mk[4 + i].y, mk[4 + i].z, mk[4 + i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              keep_where_positive(w0[e], v0[i * 8 + 2 * e], v0[i * 8 + 2 * e + 1]);
+              keep_where_positive(w1[e], v1[i * 8 + 2 * e], v1[i * 8 + 2 * e + 1]);
+            }
+          }
+          store_staged(f, v0, box, lane, 0);
+          store_staged(f, v1, box, lane, 1);
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) tma_store_5d(&map_c, box, tl.n0 + c0, row0, tl.o[2], tl.o[1], tl.o[0]);
+          buf ^= 1u;
+          const float s0 = warp_column_sums(v0, lane);      // the column sums while the store drains (v0, v1 are destroyed)
+          const float s1 = warp_column_sums(v1, lane);
+          atomicAdd(a.rsum + tl.n0 + c0 + lane, s0);
+          atomicAdd(a.rsum + tl.n0 + c0 + 32 + lane, s1);
+        }
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_pair<kPair>(tempty_bar(acc), (uint32_t)(2 * pair_idx));
+      } else if (finisher) {
         // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
