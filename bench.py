@@ -28,6 +28,7 @@ LAYOUTS = {
     "none": ([("all", 1)], []),
     "dp8": ([("all", 8)], [("batch", "all")]),
     "mp8": ([("all", 8)], [("d_ff", "all")]),
+    "mp16": ([("all", 16)], [("d_ff", "all")]),
 }
 NCU_DRAM_BYTES_PER_LAUNCH = 169.7e6
 METRIC = "transformer_ffn_fwd_bwd_tflops"
@@ -383,6 +384,28 @@ def run_ours(args):
                 "frac_of_measured_burst": achieved / peaks["bf16_burst"], "flops_per_launch": flops_per_launch,
                 "avg_launch_ms": avg_launch_ms}
 
+    # which way the sums over a split reduced dimension were realised (Section 6: the Allreduce of the
+    # mesh group) in the contractions of this layout that have one, and the workspace they moved
+    mode_name = {0: "none", 1: "chained in the accumulator", 2: "fp32 fragments in the workspace"}
+    hname = ["batch", "length", "d_ff"]
+    dsc = lambda t_, names: mtf.desc(list(zip(names, t_.shape)), "bf16" if t_.dtype == torch.bfloat16 else "f32")
+    group_sums = {}
+    for tag, ins, out in (("y", [(h, hname), (t["v"], vn)], (y, act)), ("dx", [(h, hname), (t["w"], wn)], (dx, act)),
+                          ("dw", [(t["x"], act), (h, hname)], (dw, wn)), ("dv", [(h, hname), (t["dy"], act)], (dv, vn))):
+        plan = mtf.mtf_einsum_plan(lay, [dsc(a_, n_) for a_, n_ in ins], dsc(*out))
+        info = mtf.mtf_plan_info(plan)
+        if info["group_size"] > 1:
+            group_sums[tag] = {"group_size": info["group_size"], "mode": mode_name.get(info["reduce_mode"], str(info["reduce_mode"])),
+                               "workspace_bytes": mtf.mtf_plan_workspace_bytes(plan) if info["reduce_mode"] == 2 else 0}
+
+    # the same step back to back for two seconds: the rate the GPU settles at under its power limit
+    sustained = None
+    if world == 1 and not args.no_sustained:
+        n_sus = max(int(2000.0 / ms_step), 50)
+        ms_sus, _, clocks_sus = timed(lay, n_sus, 3, ClockSampler(physical_gpu_index(local_rank)))
+        sustained = {"ms_per_step": ms_sus, "value": flops_step / (ms_sus * 1e-3) / 1e12, "unit": UNIT, "steps": n_sus,
+                     "sm_mhz": clocks_sus.get("sm_mhz") if clocks_sus else None, "reasons": clocks_sus.get("reasons") if clocks_sus else None}
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cores = len(os.sched_getaffinity(0))
@@ -401,6 +424,7 @@ def run_ours(args):
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
                                       "d2h_bytes_per_step": 2 * act_bytes, "ms_per_step": e2e_ms},
             "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu, "per_layout_tflops": per_layout,
+            "group_sums": group_sums, "sustained_2s": sustained,
             "frac_of_datasheet_bf16_peak": value / world / 2250.0}
     print(json.dumps(line), flush=True)
     if dist is not None:
@@ -504,11 +528,14 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="mp8", choices=sorted(LAYOUTS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the extra two-second back-to-back run")
+    ap.add_argument("--d-ff", type=int, default=WORKLOAD["d_ff"], help="4096 = config 2, 65536 (with --layout mp16) = config 4")
     ap.add_argument("--batch", type=int, default=WORKLOAD["batch"], help="sequences of 256 tokens per GPU (smaller only for profiler captures)")
     ap.add_argument("--main-only", action="store_true", help="skip the per-layout table and the end-to-end leg (profiler captures)")
     ap.add_argument("--workload", default="ffn", choices=["ffn", "attention", "decoder"], help="ffn = the headline line; the others print a secondary line")
     args = ap.parse_args()
     WORKLOAD["batch"] = args.batch
+    WORKLOAD["d_ff"] = args.d_ff
     if args.impl == "reference":
         run_reference(args)
     elif args.workload != "ffn":
