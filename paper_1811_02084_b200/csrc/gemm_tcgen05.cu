@@ -429,6 +429,7 @@ __device__ __forceinline__ EpiFlags epi_flags(const TcArgs& a) {
     f.c_bf16 = EPI != EPI_PLAIN_F32;
     f.relu_in_pack = EPI == EPI_BIAS_RELU_BF16;      // relu is the last stage there: it rides in the conversion to bf16
     if (EPI == EPI_ROW_SOFTMAX) f.scale = true;
+    if (EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32) f.scale = a.scale != 1.f;      // one uniform branch: s . (a . b) stays on the fast kinds
     if (EPI == EPI_ROW_SOFTMAX_BWD) f.mask = f.mask_bf16 = true;      // the weights P arrive like a mask, by TMA
     f.shared_tiles = EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32;     // the other fixed kinds never split a tile
   }
@@ -1661,6 +1662,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // launch that assembles tiles from fragments) takes the generic one
   int epi = EPI_GENERIC;
   if (row_softmax) epi = row_softmax >= 3 ? EPI_ROW_SOFTMAX_BWD : EPI_ROW_SOFTMAX;
+  else if (!resid && !bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
   else if (scale == 1.f && !resid) {
     if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
     else if (a.ws_partials) epi = EPI_GENERIC;
