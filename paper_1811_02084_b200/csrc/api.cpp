@@ -35,7 +35,7 @@ bool dims_match(const std::vector<Dim>& want, const mtf_tensor& t) {
 
 mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epi,
                      void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1, const void* const* extra_operands = nullptr,
-                     int row_softmax = 0) {
+                     int row_softmax = 0, int n_groups = 1, const void* const* group_operands = nullptr) {
   if (!P || !in || !out) return fail(MTF_ERR_INVALID_ARG, "einsum exec: NULL argument");
   if (!dims_match(P->dimsA, in[0]) || (P->has_B && !dims_match(P->dimsB, in[1])) || !dims_match(P->dimsC, *out))
     return fail(MTF_ERR_SIZE_MISMATCH, "einsum exec: operand dims differ from the planned ones");
@@ -75,8 +75,8 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
   const int relu = P->epi.on ? (epi->relu != 0) : 0;
   if (P->kernel_kind == MTF_KERNEL_TCGEN05)
     return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
-                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands, row_softmax);
-  if (n_terms != 1 || row_softmax) return fail(MTF_ERR_UNSUPPORTED, "multi-term contraction or fused softmax on the generic kernel");
+                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands, row_softmax, n_groups, group_operands);
+  if (n_terms != 1 || row_softmax || n_groups != 1) return fail(MTF_ERR_UNSUPPORTED, "multi-term, grouped or fused-softmax contraction on the generic kernel");
   SimtParams s = P->simt;
   s.A = in[0].data;
   s.B = P->has_B ? in[1].data : nullptr;
@@ -462,6 +462,28 @@ mtf_status mtf::einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_
       extra[2 * (i - 1) + q] = b.data;
     }
   return exec_plan(P, terms[0], out, epilogue, workspace, workspace_bytes, stream, n_terms, extra);
+}
+
+mtf_status mtf::einsum_group(const mtf_layout_t* layout, int n_groups, const mtf_tensor (*ins)[2], mtf_tensor* const* outs,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+  if (!layout || !ins || !outs || n_groups < 1 || n_groups > 3) return fail(MTF_ERR_INVALID_ARG, "einsum_group: bad argument");
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 2, ins[0], outs[0], nullptr, &P);
+  if (st != MTF_OK) return st;
+  if (n_groups == 1) return exec_plan(P, ins[0], outs[0], nullptr, workspace, workspace_bytes, stream);
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05) return fail(MTF_ERR_UNSUPPORTED, "einsum_group: this plan runs one problem per launch");
+  const void* ops[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  for (int g = 1; g < n_groups; ++g) {
+    const mtf_tensor* cand[3] = {&ins[g][0], &ins[g][1], outs[g]};
+    const mtf_tensor* ref[3] = {&ins[0][0], &ins[0][1], outs[0]};
+    for (int q = 0; q < 3; ++q) {
+      bool same = cand[q] && cand[q]->ndim == ref[q]->ndim && cand[q]->dtype == ref[q]->dtype && cand[q]->data != nullptr;
+      for (int d = 0; same && d < ref[q]->ndim; ++d) same = cand[q]->dims[d].size == ref[q]->dims[d].size;
+      if (!same) return fail(MTF_ERR_SIZE_MISMATCH, "einsum_group: problem %d tensor %d differs in shape or type from problem 0", g, q);
+      ops[3 * (g - 1) + q] = cand[q]->data;
+    }
+  }
+  return exec_plan(P, ins[0], outs[0], nullptr, workspace, workspace_bytes, stream, 1, nullptr, 0, n_groups, ops);
 }
 
 mtf_status mtf::einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* weights, float scale,

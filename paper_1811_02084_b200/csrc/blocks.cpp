@@ -253,9 +253,18 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
   void* rest = ar.base + ar.used;
   const size_t rest_bytes = ar.size - ar.used;
   TD xm = renamed(*x, s.l.name, kMemory);
-  if ((st = ein(layout, *x, *wq, q, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, xm.t, *wk, kk, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, xm.t, *wv, vv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  {
+    // the three projections are problems of one shape: one grouped launch where the plan allows it
+    const mtf_tensor gin[3][2] = {{*x, *wq}, {xm.t, *wk}, {xm.t, *wv}};
+    mtf_tensor* const gout[3] = {q, kk, vv};
+    st = (s.k.size == s.v.size) ? mtf::einsum_group(layout, 3, gin, gout, rest, rest_bytes, stream) : MTF_ERR_UNSUPPORTED;
+    if (st == MTF_ERR_UNSUPPORTED) {
+      if ((st = ein(layout, *x, *wq, q, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+      if ((st = ein(layout, xm.t, *wk, kk, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+      st = ein(layout, xm.t, *wv, vv, nullptr, rest, rest_bytes, stream);
+    }
+    if (st != MTF_OK) return st;
+  }
   mtf_epilogue es = epi_none();
   es.scale = (float)s.scale;
   // logits and softmax in one launch where a row of logits fits a tile (the fp32 logits then never
@@ -311,9 +320,19 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   es.scale = (float)s.scale;
   if ((st = ein(layout, dlg.t, *kk, &dq.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, dlg.t, *q, &dkk.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, *x, dq.t, dwq, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, xm.t, dkk.t, dwk, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, xm.t, dvv.t, dwv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  {
+    // the three weight gradients are problems of one shape (few output tiles each): one grouped launch
+    const mtf_tensor gin[3][2] = {{*x, dq.t}, {xm.t, dkk.t}, {xm.t, dvv.t}};
+    mtf_tensor* const gout[3] = {dwq, dwk, dwv};
+    st = (s.k.size == s.v.size && dwq->dtype == dwk->dtype && dwq->dtype == dwv->dtype) ? mtf::einsum_group(layout, 3, gin, gout, rest, rest_bytes, stream)
+                                                                                      : MTF_ERR_UNSUPPORTED;
+    if (st == MTF_ERR_UNSUPPORTED) {
+      if ((st = ein(layout, *x, dq.t, dwq, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+      if ((st = ein(layout, xm.t, dkk.t, dwk, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+      st = ein(layout, xm.t, dvv.t, dwv, nullptr, rest, rest_bytes, stream);
+    }
+    if (st != MTF_OK) return st;
+  }
   // the three contributions to dx are accumulated through the residual stage, in an fp32 buffer
   // (viewed with the memory_length name for the two that come from the key / value side); the
   // last einsum adds the running sum and writes dx once

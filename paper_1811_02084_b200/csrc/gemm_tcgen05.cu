@@ -94,6 +94,8 @@ struct TcArgs {
   int n_stages, stage_bytes;   // operand ring: 16 KB of A plus this CTA's part of B per stage, as many stages as fit
   int kb_tile;             // k-blocks of one whole tile (all terms)
   int softmax_causal;      // row-softmax epilogue: columns beyond the row's own position are masked out
+  int n_groups;            // grouped launch: n_groups (1..3) independent problems of identical shape, tiles of problem g follow those of g - 1
+  void* C_group[2];        // outputs of problems 1 and 2
   int n_terms;             // sum of n_terms products A_i . B_i of identical shape in one accumulator (1..3)
   int kb_term;             // k-blocks of one term
   int slots;               // partial-tile slots per tile in the workspace (sk, or 2 when balanced)
@@ -116,9 +118,11 @@ struct TcArgs {
   FastDiv fd_tiles_per_slice, fd_n_tiles, fd_m_tiles, fd_outer_local[3], fd_sn, fd_sm, fd_outer_split[3], fd_sk;
 };
 
-// Operand maps of the second and third product of a multi-term launch (A_1, B_1, A_2, B_2).
+// Operand maps of the second and third product of a multi-term launch, or of the second and third
+// problem of a grouped launch (A_1, B_1, A_2, B_2).
 struct ExtraMaps {
   CUtensorMap m[4];
+  CUtensorMap c[2];       // grouped launch: the outputs of problems 1 and 2
 };
 
 struct Tile {
@@ -159,6 +163,7 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long tile, int
 struct Seg {
   long long tile;
   int kb_begin, kb_count, frag, nfrag;
+  int group;               // problem of a grouped launch
 };
 
 // The sequence of segments of worker `w` of `W`.  Three schedules:
@@ -179,6 +184,7 @@ struct SegIter {
   }
   __device__ long long owner(long long unit) const { return ((unit + 1) * W - 1) / total_units; }
   __device__ bool next(Seg& s) {
+    s.group = 0;
     if (a.balanced) {
       if (u >= u_end) return false;
       s.tile = u / a.kb_tile;
@@ -201,7 +207,9 @@ struct SegIter {
       s.kb_begin = s.frag * kb_per_slice;
       s.kb_count = kb_per_slice;
     } else {
-      s.tile = a.reverse ? a.total_tiles - 1 - work : work;
+      long long w2 = a.reverse ? a.total_work - 1 - work : work;
+      if (a.n_groups > 1) { s.group = (int)(w2 / a.total_tiles); w2 -= (long long)s.group * a.total_tiles; }
+      s.tile = w2;
       s.frag = 0;
       s.nfrag = 1;
       s.kb_begin = 0;
@@ -530,16 +538,17 @@ __device__ __forceinline__ uint32_t pack_out(const EpiFlags& f, float lo, float 
   return f.relu_in_pack ? pack_bf16x2_relu(lo, hi) : pack_bf16x2(lo, hi);
 }
 
-__device__ __forceinline__ void store_direct(const TcArgs& a, const EpiFlags& f, const float* v, long long off, int n_valid) {
+__device__ __forceinline__ void store_direct(const TcArgs& a, const EpiFlags& f, const float* v, long long off, int n_valid, void* c_base = nullptr) {
+  if (!c_base) c_base = a.C;
   if (f.c_bf16) {
-    uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(a.C) + off);
+    uint4* cp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(c_base) + off);
 #pragma unroll
     for (int q = 0; q < 4; ++q)
       if (q * 8 < n_valid)
         cp[q] = make_uint4(pack_out(f, v[q * 8], v[q * 8 + 1]), pack_out(f, v[q * 8 + 2], v[q * 8 + 3]),
                            pack_out(f, v[q * 8 + 4], v[q * 8 + 5]), pack_out(f, v[q * 8 + 6], v[q * 8 + 7]));
   } else {
-    float4* cp = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.C) + off);
+    float4* cp = reinterpret_cast<float4*>(reinterpret_cast<float*>(c_base) + off);
 #pragma unroll
     for (int q = 0; q < 8; ++q)
       if (q * 4 < n_valid) cp[q] = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
@@ -702,8 +711,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor); a
           // multi-term launch then goes on with the next product's operands
           const int k0 = kt * BK;
-          const CUtensorMap* const pa = term == 0 ? &map_a : &extra.m[2 * (term - 1)];
-          const CUtensorMap* const pb = term == 0 ? &map_b : &extra.m[2 * (term - 1) + 1];
+          const int sel = a.n_groups > 1 ? sg.group : term;          // operand pair: the problem of a grouped launch, else the term
+          const CUtensorMap* const pa = sel == 0 ? &map_a : &extra.m[2 * (sel - 1)];
+          const CUtensorMap* const pb = sel == 0 ? &map_b : &extra.m[2 * (sel - 1) + 1];
           if (++kt == a.kb_term) { kt = 0; ++term; }
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, 0x100 + stage, abort_flag))) break;
           // a pair's loads all count on the even CTA's barrier, which expects both CTAs' bytes
@@ -1151,6 +1161,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // whole boxes of 32 rows x 128 B that lie inside the slice leave through the staging
         // buffers and TMA stores (a bf16 relu mask of such a box arrives the same way, in place);
         // ragged edges are read and stored from registers
+        const CUtensorMap* const pc = sg.group == 0 ? &map_c : &extra.c[sg.group - 1];       // (grouped launch: this problem's output)
+        void* const c_base = sg.group == 0 ? a.C : a.C_group[sg.group - 1];
         float bias_cur = bias_at(tl.n0 + col_half * box_cols + lane);      // lane l keeps column l of the current chunk
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
@@ -1245,11 +1257,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
           }
           if (staged) store_staged(f, v, box, lane, half);
-          else if (live) store_direct(a, f, v, row_off + n_first, n_valid);
+          else if (live) store_direct(a, f, v, row_off + n_first, n_valid, c_base);
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) tma_store_5d(&map_c, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
+            if (lane == 0) tma_store_5d(pc, box, box_n0, row0, tl.o[2], tl.o[1], tl.o[0]);
             buf ^= 1u;
           }
           if (f.rsum && n_valid > 0) {       // fused reduce_sum (never combined with a residual): v may be destroyed now
@@ -1487,11 +1499,13 @@ size_t tc_workspace_bytes(const TcParams& t) {
 mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream, int n_terms, const void* const* extra_operands,
-                     int row_softmax) {
+                     int row_softmax, int n_groups, const void* const* group_operands) {
   const TcParams& t = plan.tc;
   if (t.swapped) std::swap(A, B);
   if (n_terms < 1 || n_terms > 3 || (n_terms > 1 && !extra_operands)) return fail(MTF_ERR_INVALID_ARG, "1 to 3 terms");
   if (n_terms > 1 && t.reduce_mode == MTF_REDUCE_WORKSPACE) return fail(MTF_ERR_UNSUPPORTED, "a multi-term contraction cannot use the workspace reduce mode");
+  if (n_groups < 1 || n_groups > 3 || (n_groups > 1 && (!group_operands || n_terms != 1 || row_softmax || bias || mask || resid || rsum || relu)))
+    return fail(MTF_ERR_INVALID_ARG, "a grouped launch takes 1 to 3 plain problems");
   if (t.M > 0x7fffffffLL || t.N > 0x7fffffffLL || t.K > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "extent beyond 2^31");
   if (reinterpret_cast<uintptr_t>(C) & 15) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned output");
   if (bias && !t.bias_along_m && (reinterpret_cast<uintptr_t>(bias) & 15)) return fail(MTF_ERR_INVALID_ARG, "tensor-core path needs a 16-byte aligned bias");
@@ -1511,7 +1525,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.a_mn_major = t.a_mn_major; a.b_mn_major = t.b_mn_major;
   a.block_n = t.block_n;
   a.ldc = t.ldc;
-  a.reduce_mode = t.reduce_mode;
+  a.reduce_mode = (n_groups > 1 && t.reduce_mode == MTF_REDUCE_WORKSPACE) ? MTF_REDUCE_CHAINED : t.reduce_mode;     // a group has tiles enough: no fragments
   a.k_sliced = (t.sk > 1 && a.Ks % BK == 0) ? 1 : 0;
   // Wide tiles (256 x 512 per pair) for long contractions with a plain epilogue: per tile about 1.5x
   // the time of a 256 x 256 one (twice the MMAs at 3/4 of the L2 traffic each, epilogue exposed), so
@@ -1561,7 +1575,9 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   long long out_slices = (long long)a.sm * a.sn;
   for (int j = 0; j < a.n_outer; ++j) out_slices *= a.outer_split[j];
   a.total_tiles = a.tiles_per_slice * out_slices;
-  a.total_work = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.total_tiles * a.sk : a.total_tiles;
+  a.total_work = a.reduce_mode == MTF_REDUCE_WORKSPACE ? a.total_tiles * a.sk : a.total_tiles * n_groups;
+  a.n_groups = n_groups;
+  a.C_group[0] = a.C_group[1] = nullptr;
   if (a.total_work >= 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "more than 2^31 tiles");
   a.fd_tiles_per_slice = make_fastdiv(a.tiles_per_slice);
   a.fd_n_tiles = make_fastdiv(a.n_tiles); a.fd_m_tiles = make_fastdiv(a.m_tiles);
@@ -1595,7 +1611,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (t.balance && cn == 1 && !wide && n_terms == 1 && !row_softmax && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+  if (t.balance && cn == 1 && !wide && n_terms == 1 && n_groups == 1 && !row_softmax && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
     // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
     // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
     // the workspace by whichever worker finishes last (arrive, never wait).
@@ -1653,6 +1669,20 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // output: (N contiguous, M rows), boxes of 32 rows x 128 bytes for the staged stores
   const int c_bytes = plan.dtC == MTF_BF16 ? 2 : 4;
   if ((s = make_map(&map_c, C, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
+  extra.c[0] = extra.c[1] = map_c;
+  for (int g = 1; g < n_groups; ++g) {          // grouped launch: problem g's operands (caller's order) and output
+    const void* Ag = group_operands[3 * (g - 1)];
+    const void* Bg = group_operands[3 * (g - 1) + 1];
+    void* Cg = const_cast<void*>(group_operands[3 * (g - 1) + 2]);
+    if (t.swapped) std::swap(Ag, Bg);
+    if (!Ag || !Bg || !Cg || (reinterpret_cast<uintptr_t>(Cg) & 15)) return fail(MTF_ERR_INVALID_ARG, "grouped launch: NULL or misaligned operand");
+    s = t.a_mn_major ? make_map(&extra.m[2 * (g - 1)], Ag, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&extra.m[2 * (g - 1)], Ag, 2, t.K, t.M, t.a_ld, 64, BM / cn, t, t.outer_sA);
+    if (s != MTF_OK) return s;
+    s = t.b_mn_major ? make_map(&extra.m[2 * (g - 1) + 1], Bg, 2, t.N, t.K, t.b_ld, 64, BK, t, t.outer_sB) : make_map(&extra.m[2 * (g - 1) + 1], Bg, 2, t.K, t.N, t.b_ld, 64, b_rows, t, t.outer_sB);
+    if (s != MTF_OK) return s;
+    if ((s = make_map(&extra.c[g - 1], Cg, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
+    a.C_group[g - 1] = Cg;
+  }
   map_m = map_c;
   if (a.mask_tma && (s = make_map(&map_m, mask, 2, t.N, t.M, t.ldc, 64, 32, t, t.outer_sC)) != MTF_OK) return s;
   if (a.resid_tma && (s = make_map(&map_m, resid, c_bytes, t.N, t.M, t.ldc, 128 / c_bytes, 32, t, t.outer_sC)) != MTF_OK) return s;
@@ -1736,7 +1766,7 @@ mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, cons
   if (st != MTF_OK) return st;
   // the tile counters inside the scratch are cleared by the launcher on the stream; partial tiles are
   // overwritten before they are read, so the previous call's contents do not matter
-  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr, 0);
+  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr, 0, 1, nullptr);
 }
 
 mtf_status read_device_status(int* code) {

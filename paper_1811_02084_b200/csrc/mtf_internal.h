@@ -157,8 +157,15 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
                      const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
                      void* workspace, size_t workspace_bytes, void* stream, int n_terms = 1,
                      const void* const* extra_operands = nullptr,    // A_1, B_1 (, A_2, B_2) of a multi-term launch
-                     int row_softmax = 0);                           // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue;
+                     int row_softmax = 0,                            // 1 / 2 (causal): softmax over each row of scale * (A . B) in the epilogue;
                                                                      // 3 / 4 (causal): its backward, P (A . B - rowsum(P A . B)), P = the mask operand
+                     int n_groups = 1,                               // grouped launch: up to 3 independent problems of this plan's shape
+                     const void* const* group_operands = nullptr);   // A_1, B_1, C_1 (, A_2, B_2, C_2)
+// n_groups (1..3) independent einsums with the dims of group 0 (names may differ, sizes and types may
+// not) in one launch, so that contractions with few output tiles fill the GPU together.
+// MTF_ERR_UNSUPPORTED when the plan cannot (generic kernel): the caller then runs them one by one.
+mtf_status einsum_group(const mtf_layout_t* layout, int n_groups, const mtf_tensor (*ins)[2], mtf_tensor* const* outs,
+                        void* workspace, size_t workspace_bytes, void* stream);
 // Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes
 // and types may not) in one launch, one accumulator.  MTF_ERR_UNSUPPORTED when this plan cannot
 // (generic kernel, workspace reduce mode): the caller then chains einsums through the residual stage.
