@@ -1,19 +1,26 @@
 // Grouped bf16 contraction on the 5th-generation tensor cores (sm_100a): the per-slice local einsum
 // of Section 6 for every virtual processor of a call in ONE persistent launch, with the sum over a
 // reduce group (the paper's Allreduce within a mesh group) fused in:
-//   CHAINED   - the CTA that owns an output tile runs the K loops of the group's slices back to back
+//   CHAINED   - the worker that owns an output tile runs the K loops of the group's slices back to back
 //               (ascending processor order) into one TMEM accumulator;
-//   WORKSPACE - every (tile, slice) pair is its own work item, writes an fp32 partial, and the warp
-//               that arrives last for its 32 rows adds the partials in ascending processor order.
-// Component-wise work (scale, bias, relu, relu mask, residual, cast) is applied on the way out.
+//   WORKSPACE - every (tile, slice) pair is its own work item; all but the last to arrive leave an fp32
+//               fragment in the workspace, the last one adds them in ascending processor order.
+// Component-wise work (scale, bias, relu, relu mask, residual, cast), a fused column sum, and for
+// attention a whole-row softmax (forward and backward) are applied on the way out.  One launch can
+// also sum up to three operand pairs into one accumulator, or run up to three independent problems
+// of one shape.
 //
-// Structure of a CTA (192 threads, one CTA per SM, persistent over work items):
-//   warp 0   : TMA producer   - cp.async.bulk.tensor loads (128B swizzle) into a 4-stage smem ring
+// Structure of a CTA (320 threads, one CTA per SM, persistent over work items; by default two CTAs
+// form a pair that owns a 256-row tile through tcgen05 cta_group::2):
+//   warp 0   : TMA producer   - cp.async.bulk.tensor loads (128B swizzle) into a shared-memory ring
+//                               (16 KB of A plus this CTA's part of B per stage, as many stages as fit)
 //   warp 1   : MMA issuer     - tcgen05.mma kind::f16 (bf16 x bf16 -> fp32), accumulators in TMEM,
 //                               two 128 x 256 accumulators so the epilogue of tile i overlaps tile i+1
-//   warps 2-5: epilogue       - tcgen05.ld of the warp's 32 TMEM lanes, fused epilogue, 16-byte stores
-// Every mbarrier wait is bounded: after ~2 s it records a code in the device status word, raises a
-// CTA-wide abort flag, and all roles fall through to the common teardown (TMEM is freed).
+//                               (one 128 x 512 accumulator for the wide tiles)
+//   warps 2-9: epilogue       - two warps per TMEM lane quarter, alternate 64-column boxes: tcgen05.ld,
+//                               the fused stages, 32-row x 128-byte swizzled staging boxes, TMA stores
+// Every wait is bounded: after ~2 s it records a code in the device status word, raises a CTA-wide
+// abort flag, and all roles fall through to the common teardown (TMEM is freed).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
