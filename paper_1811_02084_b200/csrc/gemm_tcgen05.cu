@@ -597,9 +597,9 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 
-// kPair = false: one CTA owns a 128 x block_n tile (tcgen05 cta_group::1), 4-stage ring of 48 KB.
+// kPair = false: one CTA owns a 128 x block_n tile (tcgen05 cta_group::1); 3 stages of 48 KB at block_n = 256.
 // kPair = true : a cluster of two CTAs owns a 256 x block_n tile (tcgen05 cta_group::2).  Each CTA
-//   stages its own 128 rows of A and its own half of the N columns of B (32 KB per stage, 6 stages),
+//   stages its own 128 rows of A and its own half of the N columns of B (32 KB per stage, 5 stages at block_n = 256),
 //   the even CTA of the pair issues every MMA for both, each CTA's TMEM receives its own 128 rows of
 //   the result, and each CTA runs the epilogue on its own rows.  Compared with kPair = false a CTA
 //   pulls 2/3 of the bytes through L2 per flop and holds 1.5x as many k-blocks in flight.
