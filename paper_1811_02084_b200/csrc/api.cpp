@@ -22,6 +22,7 @@ using mtf::fail;
 namespace {
 
 thread_local int g_force_kernel = -1;
+thread_local bool g_next_independent = false;
 thread_local int g_force_reduce = -1;
 
 int elem_bytes(int dt) { return dt == MTF_BF16 ? 2 : 4; }
@@ -300,11 +301,15 @@ mtf_status mtf_einsum_exec(const mtf_plan_t* plan, const mtf_tensor* in, mtf_ten
 
 mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in, mtf_tensor* out,
                       const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream) {
+  const bool independent = mtf::take_independent_hint();     // (cleared whatever happens below)
   const mtf_plan_t* P = nullptr;
   mtf_status st = cached_plan(layout, n_in, in, out, epilogue, &P);
   if (st != MTF_OK) return st;
   if (equation && (st = check_equation(equation, n_in, in, out)) != MTF_OK) return st;
-  return exec_plan(P, in, out, epilogue, workspace, workspace_bytes, stream);
+  if (independent && P->kernel_kind == MTF_KERNEL_TCGEN05) mtf::hint_next_launch_independent();
+  st = exec_plan(P, in, out, epilogue, workspace, workspace_bytes, stream);
+  (void)mtf::take_independent_hint();
+  return st;
 }
 
 mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in,
@@ -464,6 +469,13 @@ mtf_status mtf::einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_
   return exec_plan(P, terms[0], out, epilogue, workspace, workspace_bytes, stream, n_terms, extra);
 }
 
+void mtf::hint_next_launch_independent() { g_next_independent = true; }
+bool mtf::take_independent_hint() {
+  const bool v = g_next_independent;
+  g_next_independent = false;
+  return v;
+}
+
 mtf_status mtf::einsum_group(const mtf_layout_t* layout, int n_groups, const mtf_tensor (*ins)[2], mtf_tensor* const* outs,
                              void* workspace, size_t workspace_bytes, void* stream) {
   if (!layout || !ins || !outs || n_groups < 1 || n_groups > 3) return fail(MTF_ERR_INVALID_ARG, "einsum_group: bad argument");
@@ -544,6 +556,7 @@ mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* 
   if ((st = mtf_einsum(layout, nullptr, 2, in1, &dhp, &e1, rest, rest_bytes, stream)) != MTF_OK) return st;
   // dv = h^T . dy  and  dw = x^T . dhp  reduce out the token dims (Section 8.1)
   mtf_tensor in2[2] = {*h_saved, *dy};
+  mtf::hint_next_launch_independent();        // dv reads h and dy, which the dhp launch only reads, and writes dv
   if ((st = mtf_einsum(layout, nullptr, 2, in2, dv, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   mtf_tensor in3[2] = {*x, dhp};
   if ((st = mtf_einsum(layout, nullptr, 2, in3, dw, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
@@ -552,6 +565,7 @@ mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* 
   mtf_tensor in4[2] = {dhp, *w};
   mtf_epilogue e4;
   e4.scale = 1.f; e4.relu = 0; e4.bias = nullptr; e4.relu_mask = nullptr; e4.residual = dx_residual; e4.reduce_sum_out = nullptr;
+  if (!(dbias && !fuse_dbias)) mtf::hint_next_launch_independent();      // dx reads dhp and w and writes dx; the dw launch before it reads x and dhp and writes dw
   return mtf_einsum(layout, nullptr, 2, in4, dx, dx_residual ? &e4 : nullptr, rest, rest_bytes, stream);
 }
 

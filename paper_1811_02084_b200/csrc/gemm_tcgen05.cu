@@ -97,6 +97,7 @@ struct TcArgs {
   int n_fastest;           // tile order inside a slice: 1 = walk the n tiles of one m tile first
   long long tiles_per_slice, total_tiles, total_work;
   int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
+  int late_wait;           // programmatic dependent launch: wait for the previous launch at the end instead of the start
   int reverse;             // walk the tiles from the last to the first (see launch_tc)
   int n_stages, stage_bytes;   // operand ring: 16 KB of A plus this CTA's part of B per stage, as many stages as fit
   int kb_tile;             // k-blocks of one whole tile (all terms)
@@ -693,7 +694,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // Programmatic dependent launch: everything above (barriers, TMEM, tensor-map prefetch) may overlap
   // the tail of the previous kernel on the stream; nothing below touches global memory before that
   // kernel has completed.  The next kernel on the stream may start its own set-up right away.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // (late_wait: this launch reads and writes nothing that the launch before it on the stream touches, so it
+  // starts at once and fills the SMs that launch's last tiles leave idle; it waits for it before exiting
+  // instead, so that whatever follows on the stream still sees every earlier launch complete.)
+  if (!a.late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int n_local = kPair ? a.block_n / 2 : a.block_n;       // N columns of B this CTA stages (wide: two runs of 128)
@@ -1322,6 +1326,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   tcgen05_fence_before();
   __syncthreads();
   if (kPair) cluster_sync();      // the partner may still signal this CTA's barriers or read its tiles
+  if (a.late_wait) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (warp == 1) {
     __syncwarp();
     tcgen05_fence_after();
@@ -1609,6 +1614,9 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.n_terms = n_terms;
   a.softmax_causal = (row_softmax == 2 || row_softmax == 4) ? 1 : 0;
   a.kb_tile = a.kb_term * n_terms;
+  // the caller's word that this launch is independent of the one before it (consumed here); only honoured
+  // for launches that clear nothing beforehand and use no workspace
+  a.late_wait = (take_independent_hint() && !rsum && t.reduce_mode != MTF_REDUCE_WORKSPACE && !t.balance) ? 1 : 0;
   // Successive launches walk their tiles in opposite directions: a contraction that reads what the launch
   // before it wrote (h then y, the attention weights then P.v) starts with the part that is still in L2.
   static std::atomic<unsigned> launch_parity{0};

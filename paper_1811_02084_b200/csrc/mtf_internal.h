@@ -161,6 +161,10 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
                                                                      // 3 / 4 (causal): its backward, P (A . B - rowsum(P A . B)), P = the mask operand
                      int n_groups = 1,                               // grouped launch: up to 3 independent problems of this plan's shape
                      const void* const* group_operands = nullptr);   // A_1, B_1, C_1 (, A_2, B_2, C_2)
+// Hint for the next tensor-core launch of this thread: it neither reads nor writes anything the launch
+// before it on the same stream touches (set by the block compositions, consumed by the launch).
+void hint_next_launch_independent();
+bool take_independent_hint();
 // n_groups (1..3) independent einsums with the dims of group 0 (names may differ, sizes and types may
 // not) in one launch, so that contractions with few output tiles fill the GPU together.
 // MTF_ERR_UNSUPPORTED when the plan cannot (generic kernel): the caller then runs them one by one.
