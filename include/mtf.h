@@ -131,7 +131,12 @@ mtf_status mtf_slice_gather(const mtf_layout_t* layout, const mtf_tensor* global
  * n_in must be 2 (MTF_ERR_UNSUPPORTED otherwise).  `data` of the descriptors is ignored here.
  * Errors: duplicate names, size mismatch, output dim in no input (MTF_ERR_UNKNOWN_DIM), illegal
  * layout for any operand or for the whole iteration space, non-divisible split sizes, and
- * MTF_ERR_UNSUPPORTED for a dimension that only one input has and the output lacks. */
+ * MTF_ERR_UNSUPPORTED for a dimension that only one input has and the output lacks.
+ * A bf16 x bf16 einsum that the tensor-core kernel cannot take (strides that are not 16-byte aligned,
+ * an N slice that is not a multiple of 8, a reduced dimension that only one operand has, more than
+ * three batch dimensions) runs on the generic one-thread-per-element kernel only up to 2^30
+ * multiply-adds; above that the plan is refused with MTF_ERR_UNSUPPORTED and the reason in
+ * mtf_last_error(), unless mtf_plan_force(MTF_KERNEL_SIMT, ..) asked for the generic kernel. */
 mtf_status mtf_einsum_plan(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in_desc,
                            const mtf_tensor* out_desc, const mtf_epilogue* epilogue, mtf_plan_t** out);
 mtf_status mtf_plan_destroy(mtf_plan_t* plan);

@@ -12,9 +12,33 @@ from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32,
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _BASE_LIB = os.path.join(_HERE, "libmtf_b200.so")
-_MC_LIB = os.path.join(_HERE, "libmtf_b200_mc.so")     # optional single-GPU build with cluster-multicast operand loads
-_multi_rank = int(os.environ.get("WORLD_SIZE", "1")) > 1
-LIB_PATH = _MC_LIB if (os.path.exists(_MC_LIB) and not _multi_rank and not os.environ.get("MTF_NO_MULTICAST")) else _BASE_LIB
+_SHARE_LIB = os.path.join(_HERE, "libmtf_b200_mc.so")     # optional single-GPU build whose CTA clusters share operand tiles
+
+
+def _single_gpu_process() -> bool:
+    """True only when this process can drive exactly one GPU and no multi-rank launcher started it."""
+    for var in ("WORLD_SIZE", "LOCAL_WORLD_SIZE", "OMPI_COMM_WORLD_SIZE", "PMI_SIZE", "SLURM_NTASKS"):
+        try:
+            if int(os.environ.get(var, "1")) > 1:
+                return False
+        except ValueError:
+            return False
+    try:
+        import torch
+        return torch.cuda.device_count() == 1
+    except Exception:
+        return False
+
+
+def _choose_library() -> str:
+    """libmtf_b200.so always, unless MTF_CLUSTER_SHARE=1 asks for the single-GPU build AND that
+    library exists AND this is a single-GPU, single-rank process."""
+    if os.environ.get("MTF_CLUSTER_SHARE") == "1" and os.path.exists(_SHARE_LIB) and _single_gpu_process():
+        return _SHARE_LIB
+    return _BASE_LIB
+
+
+LIB_PATH = _choose_library()
 
 MTF_F32, MTF_BF16 = 0, 1
 MTF_KERNEL_SIMT, MTF_KERNEL_TCGEN05 = 0, 1

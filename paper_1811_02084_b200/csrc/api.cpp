@@ -323,23 +323,12 @@ mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* eq
   if (P->workspace_bytes > mtf::builtin_scratch_capacity())
     return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "this einsum needs %zu scratch bytes, the built-in scratch holds %zu; use mtf_einsum with a caller-provided workspace",
                 P->workspace_bytes, mtf::builtin_scratch_capacity());
-  // same argument checks as the regular path, then the launch on the library's own scratch
-  if (!in || !out || !in[0].data || !in[1].data || !out->data) return fail(MTF_ERR_INVALID_ARG, "einsum: NULL data pointer");
-  if (!dims_match(P->dimsA, in[0]) || !dims_match(P->dimsB, in[1]) || !dims_match(P->dimsC, *out))
-    return fail(MTF_ERR_SIZE_MISMATCH, "einsum: operand dims differ from the planned ones");
-  const void* bias = nullptr;
-  const void* mask = nullptr;
-  const void* resid = nullptr;
-  float* rsum = nullptr;
-  if (P->epi.on) {
-    if (!epilogue) return fail(MTF_ERR_INVALID_ARG, "einsum: the plan has an epilogue, none was passed");
-    if (P->epi.has_bias) { if (!epilogue->bias || !epilogue->bias->data) return fail(MTF_ERR_INVALID_ARG, "einsum: bias has no data"); bias = epilogue->bias->data; }
-    if (P->epi.has_mask) { if (!epilogue->relu_mask || !epilogue->relu_mask->data) return fail(MTF_ERR_INVALID_ARG, "einsum: relu_mask has no data"); mask = epilogue->relu_mask->data; }
-    if (P->epi.has_res) { if (!epilogue->residual || !epilogue->residual->data) return fail(MTF_ERR_INVALID_ARG, "einsum: residual has no data"); resid = epilogue->residual->data; }
-    if (P->epi.has_rsum) { if (!epilogue->reduce_sum_out || !epilogue->reduce_sum_out->data) return fail(MTF_ERR_INVALID_ARG, "einsum: reduce_sum_out has no data"); rsum = reinterpret_cast<float*>(epilogue->reduce_sum_out->data); }
-  }
-  return mtf::launch_tc_builtin_scratch(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid, P->epi.dtRes,
-                                        P->epi.on ? epilogue->scale : 1.f, P->epi.on ? (epilogue->relu != 0) : 0, rsum, stream);
+  // the regular execution path (one validator for both entry points), on the library's own scratch: the
+  // tile counters inside it are cleared on the stream before the launch and partial tiles are written
+  // before they are read, so what the previous call left there does not matter
+  void* ws = nullptr;
+  if ((st = mtf::builtin_scratch_ptr(&ws)) != MTF_OK) return st;
+  return exec_plan(P, in, out, epilogue, ws, mtf::builtin_scratch_capacity(), stream);
 }
 
 mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in, const mtf_tensor* out,

@@ -31,10 +31,9 @@
 
 #include "mtf_internal.h"
 
-// Cluster-multicast operand loads exist only in the optional single-GPU build (see tma_multicast.cuh).
-#if defined(MTF_TMA_MULTICAST)
-#include "tma_multicast.cuh"
-#endif
+// MTF_CLUSTER_SHARE: defined only by a header that the optional single-GPU build force-includes
+// (operand tiles shared between the CTA pairs of a cluster).  The regular library is compiled
+// without that header; nothing in this file issues or names such a load.
 
 namespace {
 
@@ -733,14 +732,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const uint32_t fb = kPair ? (full_bar(stage) & 0xFEFFFFFFu) : full_bar(stage);
           const uint32_t sa = tiles_base + stage * kStageBytes;
           const uint32_t sb = sa + kAStageBytes;
-#if defined(MTF_TMA_MULTICAST)
-          if (CN > 1) {
-            // this CTA's 1/CN share of its 128 rows of A goes to the same-position CTA of every pair in its cluster row
-            uint16_t mask = 0;
-            for (int j = 0; j < CN; ++j) mask |= (uint16_t)(1u << (2 * (pm * CN + j) + cta_rank));
-            if (a.a_mn_major) tma_load_5d_multicast(sa + 8192u * pn, pa, fb, mask, m0 + 64 * pn, k0, tl.o[2], tl.o[1], tl.o[0]);
-            else tma_load_5d_multicast(sa + (uint32_t)(pn * (BM / CN)) * 128u, pa, fb, mask, k0, m0 + pn * (BM / CN), tl.o[2], tl.o[1], tl.o[0]);
-          } else
+#if defined(MTF_CLUSTER_SHARE)
+          if (CN > 1) cluster_share_load_a(sa, pa, fb, pm, pn, CN, cta_rank, a.a_mn_major, BM / CN, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
+          else
 #endif
           if (a.a_mn_major) {
             tma_load_5d<kPair>(sa, pa, fb, m0, k0, tl.o[2], tl.o[1], tl.o[0]);
@@ -748,14 +742,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           } else {
             tma_load_5d<kPair>(sa, pa, fb, k0, m0, tl.o[2], tl.o[1], tl.o[0]);
           }
-#if defined(MTF_TMA_MULTICAST)
-          if (CM > 1) {
-            // this CTA's 1/CM share of its half of B's columns goes to the same-position CTA of every pair in its cluster column
-            uint16_t mask = 0;
-            for (int j = 0; j < CM; ++j) mask |= (uint16_t)(1u << (2 * (j * CN + pn) + cta_rank));
-            if (a.b_mn_major) tma_load_5d_multicast(sb + 8192u * pm, pb, fb, mask, n0 + 64 * pm, k0, tl.o[2], tl.o[1], tl.o[0]);
-            else tma_load_5d_multicast(sb + (uint32_t)(pm * (n_local / CM)) * 128u, pb, fb, mask, k0, n0 + pm * (n_local / CM), tl.o[2], tl.o[1], tl.o[0]);
-          } else
+#if defined(MTF_CLUSTER_SHARE)
+          if (CM > 1) cluster_share_load_b(sb, pb, fb, pm, pn, CM, CN, cta_rank, a.b_mn_major, n_local / CM, n0, k0, tl.o[2], tl.o[1], tl.o[0]);
+          else
 #endif
           if (kWide) {
             // columns [256 j + 128 rank, + 128) of the tile for MMA j = 0, 1: two runs of 128, 16 KB each
@@ -1393,13 +1382,23 @@ mtf_status make_map(CUtensorMap* map, const void* base, int elem_bytes, int64_t 
   return MTF_OK;
 }
 
+constexpr int kMaxDevices = 64;
+
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = 0;
+  return dev;
+}
+
+// SM count of the current device (looked up once per device).
 int sm_count() {
-  static int n = 0;
+  static std::atomic<int> cached[kMaxDevices];
+  const int dev = current_device();
+  int n = cached[dev].load(std::memory_order_relaxed);
   if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
     if (n <= 0) n = 148;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
   return n;
 }
@@ -1433,10 +1432,13 @@ template <bool kPair, int CM, int CN, int EPI, bool kWide = false>
 mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
                           const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
   constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  static int max_clusters = 0;
-  std::call_once(once, [] {
+  // the shared-memory opt-in and the number of resident clusters are properties of a device: one set-up per device
+  struct PerDevice { std::once_flag once; cudaError_t attr_err = cudaSuccess; int max_clusters = 0; };
+  static PerDevice per_device[kMaxDevices];
+  PerDevice& pd = per_device[current_device()];
+  std::call_once(pd.once, [&pd] {
+    cudaError_t& attr_err = pd.attr_err;
+    int& max_clusters = pd.max_clusters;
     attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (attr_err != cudaSuccess) return;
     if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
@@ -1452,6 +1454,8 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, &q) == cudaSuccess && n > 0) max_clusters = n;
     else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
   });
+  const cudaError_t attr_err = pd.attr_err;
+  const int max_clusters = pd.max_clusters;
   if (attr_err != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr_err));
   // balanced schedule: every resident cluster takes an equal share of the k-block units
   const long long clusters = a.balanced ? std::min<long long>(a.total_tiles, max_clusters) : std::min<long long>(a.total_work, max_clusters);
@@ -1565,10 +1569,11 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     wide = t.wide_pref == 1 || (t.K * n_terms >= 64 * BK && 3 * waves_wide < 2 * waves_narrow);
   }
   if (wide) a.block_n = 512;
-  // optional single-GPU build: clusters of CTA pairs that share operand tiles through multicast loads
+  // optional single-GPU build: clusters of CTA pairs that share operand tiles
   int cm = 1, cn = 1;
-#if defined(MTF_TMA_MULTICAST)
-  if (!wide && !row_softmax && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE) {
+#if defined(MTF_CLUSTER_SHARE)
+  if (!wide && !row_softmax && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && n_terms == 1 && n_groups == 1 &&
+      cluster_share_operands_local(A, B)) {      // both operands are allocations of the GPU this launch runs on
     // measured on the FFN shapes: sharing B between two pairs that are neighbours along M is worth
     // 5-10 % on the contractions whose epilogue is light; with a relu mask or a fused reduction in the
     // epilogue the coupling of the two pairs costs more than the saved traffic; 2 x 2 clusters lose
@@ -1663,7 +1668,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   CUtensorMap map_a, map_b, map_c, map_m;
   mtf_status s;
   // operands: K-major = (K contiguous, M|N rows), box 64 x rows;  MN-major = (M|N contiguous, K rows), box 64 x 64
-  // (a CTA of a multicast cluster loads 1/cn of its A rows and 1/cm of its B columns per box)
+  // (a CTA of a sharing cluster loads 1/cn of its A rows and 1/cm of its B columns per box)
   const int b_rows = (t.cta_pair ? t.block_n / 2 : t.block_n) / cm;
   s = t.a_mn_major ? make_map(&map_a, A, 2, t.M, t.K, t.a_ld, 64, BK, t, t.outer_sA) : make_map(&map_a, A, 2, t.K, t.M, t.a_ld, 64, BM / cn, t, t.outer_sA);
   if (s != MTF_OK) return s;
@@ -1727,7 +1732,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
   } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
-#if defined(MTF_TMA_MULTICAST)
+#if defined(MTF_CLUSTER_SHARE)
   else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
   else if (cm == 2 && cn == 1) ls = launch_kind<true, 2, 1, false>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
 #endif
@@ -1749,15 +1754,17 @@ static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratch
 
 size_t builtin_scratch_capacity() { return kBuiltinScratchBytes; }
 
+int device_sm_count() { return sm_count(); }
+
 // The array's name is only a host-side handle; the device address comes from the runtime, once per
 // device, with that device current.
-static mtf_status builtin_scratch_ptr(void** out) {
+mtf_status builtin_scratch_ptr(void** out) {
   static std::mutex mu;
-  static void* cached[64] = {nullptr};
+  static void* cached[kMaxDevices] = {nullptr};
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
-  if (dev < 0 || dev >= 64) return fail(MTF_ERR_UNSUPPORTED, "device ordinal %d outside [0, 64)", dev);
+  if (dev < 0 || dev >= kMaxDevices) return fail(MTF_ERR_UNSUPPORTED, "device ordinal %d outside [0, %d)", dev, kMaxDevices);
   std::lock_guard<std::mutex> lock(mu);
   if (!cached[dev]) {
     void* p = nullptr;
@@ -1767,21 +1774,6 @@ static mtf_status builtin_scratch_ptr(void** out) {
   }
   *out = cached[dev];
   return MTF_OK;
-}
-
-mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
-                                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
-                                     void* stream) {
-  const size_t need = tc_workspace_bytes(plan.tc);
-  if (need > kBuiltinScratchBytes)
-    return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "this einsum needs %zu scratch bytes, the built-in scratch holds %zu; use mtf_einsum with a caller-provided workspace",
-                need, kBuiltinScratchBytes);
-  void* ws = nullptr;
-  mtf_status st = builtin_scratch_ptr(&ws);
-  if (st != MTF_OK) return st;
-  // the tile counters inside the scratch are cleared by the launcher on the stream; partial tiles are
-  // overwritten before they are read, so the previous call's contents do not matter
-  return launch_tc(plan, A, B, C, bias, dtBias, mask, dtMask, resid, dtRes, scale, relu, rsum, ws, kBuiltinScratchBytes, stream, 1, nullptr, 0, 1, nullptr);
 }
 
 mtf_status read_device_status(int* code) {

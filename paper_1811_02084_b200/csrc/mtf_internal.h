@@ -189,9 +189,10 @@ mtf_status einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tenso
                         const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream);
 size_t tc_workspace_bytes(const TcParams& t);
 size_t builtin_scratch_capacity();
-mtf_status launch_tc_builtin_scratch(const mtf_plan_t& plan, const void* A, const void* B, void* C, const void* bias, int dtBias,
-                                     const void* mask, int dtMask, const void* resid, int dtRes, float scale, int relu, float* rsum,
-                                     void* stream);
+// SM count of the current device; 148 (a B200) when no device can be asked, so that planning works without one.
+int device_sm_count();
+// Device address of the library's own scratch array on the current device (resolved once per device).
+mtf_status builtin_scratch_ptr(void** out);
 mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes,
                                const int64_t* offs, const int64_t* gstrides, void* stream);
 void count_launch(int n = 1);

@@ -18,6 +18,9 @@ namespace mtf {
 
 static thread_local char g_err[512] = "";
 
+// bf16 contractions above this many multiply-adds are not sent to the generic kernel unasked (2^30: ~0.1 s there)
+constexpr double kGenericKernelMacLimit = 1073741824.0;
+
 void set_error(const char* fmt, ...) {
   va_list ap;
   va_start(ap, fmt);
@@ -469,6 +472,16 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
   if (!P->has_B && force_reduce == MTF_REDUCE_WORKSPACE) force_reduce = -1;
   if (force_kernel == MTF_KERNEL_TCGEN05 && !tc_ok) return fail(MTF_ERR_UNSUPPORTED, "tensor-core path cannot run this einsum: %s", why.c_str());
   P->kernel_kind = (tc_ok && force_kernel != MTF_KERNEL_SIMT) ? MTF_KERNEL_TCGEN05 : MTF_KERNEL_SIMT;
+  // A large bf16 contraction the tensor-core path declines would run ~100x slower on the generic
+  // kernel (one thread per output element): refuse it with the reason instead of a silent cliff.
+  // mtf_plan_force(MTF_KERNEL_SIMT, ..) is the opt-in for running it there all the same.
+  if (P->kernel_kind == MTF_KERNEL_SIMT && P->has_B && !tc_ok && force_kernel != MTF_KERNEL_SIMT && P->dtA == MTF_BF16 && P->dtB == MTF_BF16) {
+    double total_macs = 1.0;
+    for (auto& d : P->iter) total_macs *= (double)d.size;
+    if (total_macs > kGenericKernelMacLimit)
+      return fail(MTF_ERR_UNSUPPORTED, "this bf16 einsum (%.3g multiply-adds) cannot run on the tensor-core path (%s) and is too large for the generic kernel; "
+                  "change the shapes, or opt in with mtf_plan_force(MTF_KERNEL_SIMT, -1)", total_macs, why.c_str());
+  }
   P->reduce_mode = P->group_size > 1 ? MTF_REDUCE_CHAINED : MTF_REDUCE_NONE;
   P->workspace_bytes = 0;
   if (P->kernel_kind == MTF_KERNEL_TCGEN05) {
@@ -487,7 +500,7 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
       // writing and adding the fragments), the chained one ~7 us, and a k-block takes ~0.33 us, so the
       // k-blocks taken off the critical path must be worth the difference
       const int64_t kb_total = t.K / 64, kb_saved = kb_total - kb_total / t.sk;
-      if (tiles * (t.cta_pair ? 4 : 2) <= 148 && t.K / t.sk >= 256 && kb_saved >= 64) mode = MTF_REDUCE_WORKSPACE;
+      if (tiles * (t.cta_pair ? 4 : 2) <= device_sm_count() && t.K / t.sk >= 256 && kb_saved >= 64) mode = MTF_REDUCE_WORKSPACE;
     }
     t.reduce_mode = mode;
     P->reduce_mode = mode;
@@ -496,7 +509,7 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
     if (mode != MTF_REDUCE_WORKSPACE && t.cta_pair && t.K >= 32 * 64) {
       int64_t tiles = ((t.M / t.sm + 255) / 256) * t.sm * ((t.N / t.sn + t.block_n - 1) / t.block_n) * t.sn;
       for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
-      const int64_t workers = 74;     // CTA pairs of a B200; the launcher re-checks with the device's count
+      const int64_t workers = device_sm_count() / 2;     // CTA pairs of the device; the launcher re-checks
       const int64_t rounds = (tiles + workers - 1) / workers;
       // Measured on the FFN shapes the fragment traffic costs more than the idle tail it removes,
       // so the schedule is only taken when asked for (mtf_plan_force reduce_mode 3).
