@@ -10,6 +10,7 @@ Contents
   mesh.py         mesh, computation layout, legality, per-processor slice boxes
   lowering.py     per-processor simulation: local op on slices, then the group sum (Allreduce)
   blocks.py       feed-forward, attention, layer norm, decoder layer - forward and backward
+  stages.py       the same blocks one launch at a time (an einsum plus its fused component-wise stages, or a row reduction)
   cost.py         per-processor cost counts (Table 1, Appendix B)
   rounding.py     the one rounding step applied where the method stores an intermediate in bf16
 
@@ -21,7 +22,7 @@ from .named import (NT, DenseOps, DuplicateDim, IllegalLayout, NotDivisible, Ora
                     UnknownDim, einsum_arrays)
 from .mesh import Layout, Mesh
 from .lowering import LT, LoweredOps
-from . import blocks, cost, rounding
+from . import blocks, cost, rounding, stages
 
-__all__ = ["NT", "DenseOps", "LoweredOps", "LT", "Mesh", "Layout", "blocks", "cost", "einsum_arrays",
+__all__ = ["NT", "DenseOps", "LoweredOps", "LT", "Mesh", "Layout", "blocks", "stages", "cost", "einsum_arrays",
            "OracleError", "DuplicateDim", "UnknownDim", "SizeMismatch", "IllegalLayout", "NotDivisible"]
