@@ -308,6 +308,24 @@ mtf_status mtf_decoder_layer_workspace_bytes(const mtf_layout_t* layout, const m
  * slice, then the group sum across the mesh dims of reduced-out split dims, in one launch. */
 mtf_status mtf_reduce_sum(const mtf_layout_t* layout, const mtf_tensor* in, mtf_tensor* out, void* stream);
 
+/* ---- stage tap (verification aid) ----------------------------------------------------------------
+ * The block calls keep some results of their einsums only in scratch memory (the feed-forward
+ * block's dhp; the attention block's do, dlogits, dq, dkk, dvv; the decoder layer's gradient streams
+ * ds2, da, ds1), and reuse that scratch.  While a tap is open on the calling thread, every block call
+ * of that thread copies each such intermediate, right behind the launch that produced it and on the
+ * same stream, into `device_buffer` (device memory, 256-byte aligned, caller-owned), one after the
+ * other at 256-byte aligned offsets.  A checker can then hold every launch of a block to the
+ * single-einsum tolerance: the inputs the launch read and the output it wrote are all available.
+ *   mtf_stage_tap_begin : opens the tap (forgets the previous one's entries).
+ *   mtf_stage_tap_end   : closes it, returns the number of entries; MTF_ERR_WORKSPACE_TOO_SMALL when
+ *                         the buffer was too small (entries that did not fit were not copied).
+ *   mtf_stage_tap_entry : name (valid until the next begin on this thread), byte offset and size of
+ *                         entry `index`, in the order the intermediates were produced.
+ * With no tap open the block calls do no extra work.  (The paper has no counterpart.) */
+mtf_status mtf_stage_tap_begin(void* device_buffer, size_t bytes);
+mtf_status mtf_stage_tap_end(int32_t* n_entries);
+mtf_status mtf_stage_tap_entry(int32_t index, const char** name, size_t* offset, size_t* bytes);
+
 /* ---- status ------------------------------------------------------------------------------------- */
 const char* mtf_status_string(mtf_status s);
 const char* mtf_last_error(void);

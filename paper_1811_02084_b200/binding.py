@@ -125,6 +125,9 @@ def _load():
         "mtf_decoder_layer_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(mtf_decoder_saved), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_decoder_grads), vp, c_size_t, vp],
         "mtf_decoder_layer_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(c_size_t)],
         "mtf_device_status": [POINTER(c_int32)],
+        "mtf_stage_tap_begin": [vp, c_size_t],
+        "mtf_stage_tap_end": [POINTER(c_int32)],
+        "mtf_stage_tap_entry": [c_int32, POINTER(c_char_p), POINTER(c_size_t), POINTER(c_size_t)],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -490,6 +493,24 @@ def mtf_device_status() -> int:
     c = c_int32()
     _check(_lib.mtf_device_status(byref(c)))
     return c.value
+
+
+def mtf_stage_tap_begin(buffer) -> None:
+    """Open the stage tap on a device byte buffer (a contiguous torch tensor)."""
+    _check(_lib.mtf_stage_tap_begin(c_void_p(buffer.data_ptr()), buffer.numel() * buffer.element_size()))
+
+
+def mtf_stage_tap_end() -> int:
+    n = c_int32()
+    _check(_lib.mtf_stage_tap_end(byref(n)))
+    return n.value
+
+
+def mtf_stage_tap_entry(index: int):
+    """(name, byte offset, byte size) of one tapped intermediate."""
+    name, off, size = c_char_p(), c_size_t(), c_size_t()
+    _check(_lib.mtf_stage_tap_entry(index, byref(name), byref(off), byref(size)))
+    return name.value.decode(), off.value, size.value
 
 
 def mtf_launch_count() -> int:

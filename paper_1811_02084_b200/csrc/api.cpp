@@ -543,6 +543,7 @@ mtf_status mtf::ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* 
   e1.reduce_sum_out = fuse_dbias ? dbias : nullptr;
   mtf_tensor in1[2] = {*dy, *v};
   if ((st = mtf_einsum(layout, nullptr, 2, in1, &dhp, &e1, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("dhp", dhp, stream)) != MTF_OK) return st;
   // dv = h^T . dy  and  dw = x^T . dhp  reduce out the token dims (Section 8.1)
   mtf_tensor in2[2] = {*h_saved, *dy};
   mtf::hint_next_launch_independent();        // dv reads h and dy, which the dhp launch only reads, and writes dv
@@ -587,5 +588,9 @@ mtf_status mtf_device_status(int32_t* code) {
 }
 
 int64_t mtf_launch_count(void) { return mtf::launch_count(); }
+
+mtf_status mtf_stage_tap_begin(void* device_buffer, size_t bytes) { return mtf::tap_begin(device_buffer, bytes); }
+mtf_status mtf_stage_tap_end(int32_t* n_entries) { return mtf::tap_end(n_entries); }
+mtf_status mtf_stage_tap_entry(int32_t index, const char** name, size_t* offset, size_t* bytes) { return mtf::tap_entry(index, name, offset, bytes); }
 
 }  // extern "C"

@@ -308,6 +308,7 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   TD xm = renamed(*x, s.l.name, kMemory);
   if ((st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, *dy, *wo, &dob.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("do", dob.t, stream)) != MTF_OK) return st;
   // dP and the softmax backward in one launch where a row fits a tile (dP then stays in tensor
   // memory); otherwise dP goes through the workspace in fp32 and the row kernel follows
   st = mtf::einsum_row_softmax_bwd(layout, &dob.t, vv, weights, &dlg.t, 0 /* zeros of a causal P give zeros here without being told */, rest, rest_bytes, stream);
@@ -316,10 +317,12 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   if (!fused_bwd && (st = ein(layout, dob.t, *vv, &dP.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, *weights, dob.t, &dvv.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if (!fused_bwd && (st = mtf_softmax_backward(layout, weights, &dP.t, &dlg.t, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("dvv", dvv.t, stream)) != MTF_OK || (st = mtf::tap("dlogits", dlg.t, stream)) != MTF_OK) return st;
   mtf_epilogue es = epi_none();
   es.scale = (float)s.scale;
   if ((st = ein(layout, dlg.t, *kk, &dq.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, dlg.t, *q, &dkk.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("dq", dq.t, stream)) != MTF_OK || (st = mtf::tap("dkk", dkk.t, stream)) != MTF_OK) return st;
   {
     // the three weight gradients are problems of one shape (few output tiles each): one grouped launch
     const mtf_tensor gin[3][2] = {{*x, dq.t}, {xm.t, dkk.t}, {xm.t, dvv.t}};
@@ -401,10 +404,13 @@ mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tens
   const size_t rest_bytes = ar.size - ar.used;
   mtf_status st;
   if ((st = mtf_layernorm_backward(layout, dout, sv->s2, sv->stats2, p->ln2_gamma, nullptr, &ds2.t, g->dln2_gamma, g->dln2_beta, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("ds2", ds2.t, stream)) != MTF_OK) return st;
   // da = ds2 + dFFN/da
   if ((st = mtf::ffn_backward_impl(layout, sv->a, p->w, p->v, sv->h, &ds2.t, &da.t, &ds2.t, g->dw, g->dbias, g->dv, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("da", da.t, stream)) != MTF_OK) return st;
   // ds1 (reusing ds2's buffer) = LN1 backward; dx = ds1 + dAttention/dx
   if ((st = mtf_layernorm_backward(layout, &da.t, sv->s1, sv->stats1, p->ln1_gamma, nullptr, &ds2.t, g->dln1_gamma, g->dln1_beta, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("ds1", ds2.t, stream)) != MTF_OK) return st;
   return mtf_attention_backward(layout, x, p->wq, p->wk, p->wv, p->wo, sv->q, sv->kk, sv->vv, sv->weights, sv->o, &ds2.t, &ds2.t, dx, g->dwq, g->dwk,
                                 g->dwv, g->dwo, rest, rest_bytes, stream);
 }

@@ -12,6 +12,9 @@
 
 #include <atomic>
 
+#include <string>
+#include <vector>
+
 #include "mtf_internal.h"
 
 namespace {
@@ -143,6 +146,55 @@ mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int n
   slice_gather_kernel<<<(unsigned)blocks, 256, 0, (cudaStream_t)stream>>>(src, dst, g);
   count_launch();
   return check_launch("slice_gather_kernel");
+}
+
+// ---- stage tap: copies of scratch-resident intermediates for verification -----------------------------
+namespace {
+struct TapEntry { std::string name; size_t offset, bytes; };
+struct TapState {
+  uint8_t* base = nullptr;
+  size_t size = 0, used = 0;
+  bool active = false, overflow = false;
+  std::vector<TapEntry> entries;
+};
+thread_local TapState g_tap;
+}  // namespace
+
+mtf_status tap_begin(void* device_buffer, size_t bytes) {
+  if (!device_buffer || (reinterpret_cast<uintptr_t>(device_buffer) & 255)) return fail(MTF_ERR_INVALID_ARG, "stage tap: the buffer must be a 256-byte aligned device pointer");
+  g_tap.base = reinterpret_cast<uint8_t*>(device_buffer);
+  g_tap.size = bytes; g_tap.used = 0; g_tap.active = true; g_tap.overflow = false;
+  g_tap.entries.clear();
+  return MTF_OK;
+}
+
+mtf_status tap_end(int32_t* n_entries) {
+  g_tap.active = false;
+  if (n_entries) *n_entries = (int32_t)g_tap.entries.size();
+  if (g_tap.overflow) return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "stage tap: the buffer of %zu bytes was too small (needed %zu)", g_tap.size, g_tap.used);
+  return MTF_OK;
+}
+
+mtf_status tap_entry(int32_t i, const char** name, size_t* offset, size_t* bytes) {
+  if (i < 0 || i >= (int32_t)g_tap.entries.size()) return fail(MTF_ERR_INVALID_ARG, "stage tap: entry %d of %d", i, (int)g_tap.entries.size());
+  if (name) *name = g_tap.entries[i].name.c_str();
+  if (offset) *offset = g_tap.entries[i].offset;
+  if (bytes) *bytes = g_tap.entries[i].bytes;
+  return MTF_OK;
+}
+
+// Called by the block compositions right after the launch that produced `t`; does nothing unless a tap is open.
+mtf_status tap(const char* name, const mtf_tensor& t, void* stream) {
+  if (!g_tap.active || !t.data) return MTF_OK;
+  size_t n = t.dtype == MTF_BF16 ? 2 : 4;
+  for (int i = 0; i < t.ndim; ++i) n *= (size_t)t.dims[i].size;
+  const size_t off = g_tap.used;
+  g_tap.used += (n + 255) / 256 * 256;
+  if (g_tap.used > g_tap.size) { g_tap.overflow = true; return MTF_OK; }
+  cudaError_t e = cudaMemcpyAsync(g_tap.base + off, t.data, n, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "stage tap copy: %s", cudaGetErrorString(e));
+  g_tap.entries.push_back({name, off, n});
+  return MTF_OK;
 }
 
 }  // namespace mtf

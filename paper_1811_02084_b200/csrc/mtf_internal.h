@@ -196,5 +196,11 @@ mtf_status builtin_scratch_ptr(void** out);
 mtf_status launch_slice_gather(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes,
                                const int64_t* offs, const int64_t* gstrides, void* stream);
 void count_launch(int n = 1);
+// stage tap (mtf_stage_tap_*): while a tap is open on this thread, `tap` copies the named intermediate
+// into the caller's buffer on the stream, right behind the launch that produced it
+mtf_status tap_begin(void* device_buffer, size_t bytes);
+mtf_status tap_end(int32_t* n_entries);
+mtf_status tap_entry(int32_t i, const char** name, size_t* offset, size_t* bytes);
+mtf_status tap(const char* name, const mtf_tensor& t, void* stream);
 
 }  // namespace mtf

@@ -42,13 +42,41 @@ def rms_error(got, ref) -> float:
     return float(np.sqrt((d * d).sum()) / max(np.sqrt((ref * ref).sum()), 1e-300))
 
 
-TOL = {"bf16": 1e-2, "f32": 1e-4}
-# Blocks that chain four to six bf16-stored intermediates (attention, decoder layer): a GPU value and
-# the oracle's value of a stored intermediate may round to neighbouring bf16 numbers (one ulp = 0.78 %),
-# and outputs fed by few terms (the first rows under a causal mask) do not average that out.  Gates:
-# element-wise 2e-2 and rms 4e-3 against the oracle that stores the same intermediates in bf16;
-# 5e-2 / 1e-2 against exact mathematics (which that oracle itself misses by ~3.5e-2 element-wise).
-TOL_CHAIN = {"elem": 2e-2, "rms": 4e-3, "elem_exact": 5e-2, "rms_exact": 1e-2}
+TOL = {"bf16": 1e-2, "f32": 1e-4}      # the parity metric a single launch is held to, against exact fp64 mathematics
+
+
+class Guarded:
+    """Device allocations with guard bands: every tensor handed out sits inside a larger buffer whose
+    margins hold a sentinel byte pattern; ``check()`` asserts that no kernel wrote outside a tensor
+    (a stand-in for a memory checker: NaN pre-fill catches unwritten elements, the bands catch writes
+    that miss the tensor)."""
+    MARGIN = 4096
+    SENTINEL = 0xA5
+
+    def __init__(self):
+        self.items = []
+
+    def empty(self, shape, dtype, fill=float("nan")):
+        import torch
+        tdt = {"bf16": torch.bfloat16, "f32": torch.float32, "u8": torch.uint8}[dtype] if isinstance(dtype, str) else dtype
+        n = int(np.prod(shape)) if len(shape) else 1
+        nbytes = n * torch.empty(0, dtype=tdt).element_size()
+        padded = (nbytes + 255) // 256 * 256
+        raw = torch.full((padded + 2 * self.MARGIN,), self.SENTINEL, dtype=torch.uint8, device="cuda")
+        t = raw[self.MARGIN:self.MARGIN + nbytes].view(tdt).view(*shape)
+        if fill is not None and tdt != torch.uint8:
+            t.fill_(fill)
+        self.items.append((raw, nbytes))
+        return t
+
+    def check(self):
+        import torch
+        for raw, nbytes in self.items:
+            lo = raw[:self.MARGIN]
+            hi = raw[self.MARGIN + (nbytes + 255) // 256 * 256:]
+            tail = raw[self.MARGIN + nbytes:self.MARGIN + (nbytes + 255) // 256 * 256]
+            for band in (lo, hi, tail):
+                assert bool((band == self.SENTINEL).all()), "a kernel wrote outside a tensor (guard band overwritten)"
 
 
 def ffn_inputs(seed, tok_dims, d_model, d_ff, dtype, with_bias=True, io_name="d_model", hidden_name="d_ff"):
@@ -66,100 +94,30 @@ def ffn_inputs(seed, tok_dims, d_model, d_ff, dtype, with_bias=True, io_name="d_
     return out
 
 
-def run_ffn_gpu(mtf, layout, inp, act_dtype, grad_dtype="f32"):
-    """Forward + backward through the C ABI.  Returns dict of fp64 numpy outputs."""
-    import torch
-    tdt = {"bf16": torch.bfloat16, "f32": torch.float32}
-    dev = {k: to_torch(s) for k, (_, s) in inp.items()}
-    N = {k: mtf.named(dev[k], [n for n, _ in d]) for k, (d, _) in inp.items()}
-    xd, wd = inp["x"][0], inp["w"][0]
-    hd = xd[:-1] + [wd[1]]
-    h = torch.empty([s for _, s in hd], dtype=tdt[act_dtype], device="cuda")
-    y = torch.empty([s for _, s in xd], dtype=tdt[act_dtype], device="cuda")
-    dx = torch.empty_like(y)
-    dw = torch.empty([s for _, s in wd], dtype=tdt[grad_dtype], device="cuda")
-    dv = torch.empty([s for _, s in inp["v"][0]], dtype=tdt[grad_dtype], device="cuda")
-    dbias = torch.empty([wd[1][1]], dtype=tdt[grad_dtype], device="cuda")
-    nbytes = mtf.mtf_ffn_workspace_bytes(layout, N["x"], N["w"])
-    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    nm = lambda t, d: mtf.named(t, [n for n, _ in d])
-    mtf.mtf_ffn_forward(layout, N["x"], N["w"], N.get("bias"), N["v"], nm(h, hd), nm(y, xd), ws)
-    mtf.mtf_ffn_backward(layout, N["x"], N["w"], N["v"], nm(h, hd), N["dy"], nm(dx, xd), nm(dw, wd),
-                         nm(dbias, [wd[1]]) if "bias" in inp else None, nm(dv, inp["v"][0]), ws)
-    mtf.mtf_device_status()
-    out = {"h": h, "y": y, "dx": dx, "dw": dw, "dv": dv}
-    if "bias" in inp:
-        out["dbias"] = dbias
-    return {k: from_torch(t) for k, t in out.items()}
-
-
-def run_ffn_oracle(inp, store_dtype=None):
-    """Dense fp64 oracle on the same (rounded) inputs.  ``store_dtype`` = the type the method keeps
-    h and dhp in between einsums (None: exact mathematics, nothing rounded).  Also returns the
-    ambiguity sets of the relu decision: where |hp| is so small that fp32 accumulation may
-    legitimately decide [hp > 0] differently, the outputs that hinge on it are not unique."""
-    from oracle import NT, DenseOps, blocks, rounding
+def run_ffn_oracle(inp):
+    """The whole block in exact fp64 mathematics on the same (rounded) inputs, nothing rounded in
+    between: the end-to-end reference.  (The gate is stage-wise, see stagewise.py; end to end the
+    storage rounding of h and dhp and single relu decisions taken on values within rounding of zero
+    legitimately move outputs, so this comparison is reported and gated in the rms only.)"""
+    from oracle import NT, DenseOps, blocks
     ops = DenseOps()
-    store = rounding.make_store(ops, store_dtype)
     T = {k: NT(d, s.f64) for k, (d, s) in inp.items()}
-    f = blocks.ffn_forward(ops, T["x"], T["w"], T.get("bias"), T["v"], store)
-    g = blocks.ffn_backward(ops, T["x"], T["w"], T["v"], f["h"], T["dy"], store)
+    f = blocks.ffn_forward(ops, T["x"], T["w"], T.get("bias"), T["v"])
+    g = blocks.ffn_backward(ops, T["x"], T["w"], T["v"], f["h"], T["dy"])
     ref = {"h": f["h"].a, "y": f["y"].a, "dx": g["dx"].a, "dw": g["dw"].a, "dv": g["dv"].a}
     if "bias" in inp:
         ref["dbias"] = g["dbias"].a
-    hp = f["hp"].a
-    scale = float(np.sqrt(np.mean(hp * hp)))
-    amb = np.abs(hp) < 2e-5 * max(scale, 1e-30)
-    amb2 = amb.reshape(-1, amb.shape[-1])
-    return ref, {"tokens": np.unique(np.nonzero(amb2)[0]), "hidden": np.unique(np.nonzero(amb2)[1])}
+    return ref
 
 
-def max_norm_error(got, ref) -> float:
-    """max |g - r| / max |r|."""
-    ref = np.asarray(ref, dtype=np.float64)
-    return float(np.max(np.abs(np.asarray(got, dtype=np.float64) - ref)) / max(float(np.max(np.abs(ref))), 1e-300))
+def end_to_end_report(got, ref, what, rms_gate=1e-2):
+    """Parity metric and rms error of every output of a block against exact end-to-end mathematics.
+    Printed; only the rms is gated (at the single-launch tolerance)."""
+    rows = {k: (parity_error(got[k], ref[k]), rms_error(got[k], ref[k])) for k in ref}
+    print(f"[end to end] {what}: " + ", ".join(f"{k} elem {e:.2e} rms {r:.2e}" for k, (e, r) in rows.items()))
+    if rms_gate is not None:
+        bad = {k: r for k, (_, r) in rows.items() if not r <= rms_gate}
+        assert not bad, f"{what}: end-to-end rms error above {rms_gate}: {bad}"
+    return rows
 
 
-def check_ffn_block(got, inp, act_dtype):
-    """The parity gates of the feed-forward block.
-    1. Against the oracle that keeps h and dhp in the activation dtype (the method's storage
-       precision; arithmetic exact): parity metric within the tolerance of that dtype.
-    2. For bf16 also against exact mathematics with nothing rounded: the bf16 storage of h and dhp
-       alone moves an output element by up to ~6 sigma of 0.16 % of the output rms plus its own
-       final rounding (0.39 %), so this gate is 2e-2 in the parity metric and 1e-2 in max norm."""
-    ref_s, amb = run_ffn_oracle(inp, act_dtype if act_dtype == "bf16" else None)
-    errs = check_ffn(got, ref_s, amb, TOL[act_dtype])
-    if act_dtype == "bf16":
-        ref_e, amb_e = run_ffn_oracle(inp, None)
-        amb_u = {k: np.union1d(amb[k], amb_e[k]) for k in amb}
-        errs_exact = check_ffn(got, ref_e, amb_u, 2e-2)
-        for k in ref_e:
-            if k in ("dx", "dw", "dbias") and (len(amb_u["tokens"]) or len(amb_u["hidden"])):
-                continue
-            assert max_norm_error(got[k], ref_e[k]) <= 1e-2, k
-        errs = {**errs, **{k + "_vs_exact": e for k, e in errs_exact.items()}}
-    return errs
-
-
-def check_ffn(got, ref, amb, tol):
-    """Compare everything that is unique; rows / columns that hinge on an ambiguous relu decision are
-    checked for validity only (finite)."""
-    errs = {}
-    for k in ref:
-        g, r = got[k], ref[k]
-        assert np.isfinite(g).all(), k
-        if k == "dx":
-            g2, r2 = g.reshape(-1, g.shape[-1]), r.reshape(-1, r.shape[-1])
-            keep = np.setdiff1d(np.arange(g2.shape[0]), amb["tokens"])
-            errs[k] = parity_error(g2[keep], r2[keep])
-        elif k == "dw":
-            keep = np.setdiff1d(np.arange(g.shape[1]), amb["hidden"])
-            errs[k] = parity_error(g[:, keep], r[:, keep])
-        elif k == "dbias":
-            keep = np.setdiff1d(np.arange(g.shape[0]), amb["hidden"])
-            errs[k] = parity_error(g[keep], r[keep])
-        else:
-            errs[k] = parity_error(g, r)
-    bad = {k: e for k, e in errs.items() if not e <= tol}
-    assert not bad, f"parity above {tol}: {bad} (all: {errs})"
-    return errs

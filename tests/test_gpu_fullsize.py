@@ -1,20 +1,23 @@
 """GPU parity at the full sizes of the benchmark configurations, in the launch configuration the
-bench times (planner's choices, C ABI), on SAMPLED outputs the oracle can compute one by one:
+bench times (planner's choices, C ABI).
 
-  feed-forward (configs 2, 4 and the d_ff = 8192 target shape): for a seeded set of tokens - always
-  including the first and last token of every slice along a split dimension - the full rows of h, y
-  and dx; for a seeded set of hidden units (first / last of every slice included) the full columns
-  dw[:, j], rows dv[j, :] and dbias[j].  Every sampled output is summed over the FULL reduction
-  range, so the cross-slice sum is exercised end to end.
-  attention (config 3) and decoder layer (config 5): every output that belongs to one sampled batch
-  element (the blocks do not mix batch elements in the forward pass and in dx); parameter gradients
-  reduce over the whole batch and are compared across layouts instead (every layout against mesh [1]).
+Gate: stage-wise (stagewise.py) - every launch of the block against the exact fp64 oracle of that
+launch, evaluated on the inputs the GPU launch actually read, at 1e-2 in the parity metric, on SAMPLED
+outputs the oracle can compute one by one:
+  * rows of sampled tokens (always the first and last token of every slice along a split dimension)
+    for everything that has a token dimension;
+  * whole (batch, head) pairs for the attention core (corners of every slice included);
+  * columns of sampled hidden units / (head, d_k) pairs / d_model columns for the parameter
+    gradients, each summed over ALL tokens, so the cross-slice sums are exercised end to end.
+The elements that are not sampled are covered by comparing every layout's outputs with those of the
+un-split mesh [1] (GPU against GPU, all elements).
 """
 import numpy as np
 import pytest
 
 import seeded_inputs as si
-from helpers import TOL, TOL_CHAIN, from_torch, parity_error, rms_error, to_torch
+from helpers import TOL, ffn_inputs
+from stagewise import run_attention_stagewise, run_decoder_stagewise, run_ffn_stagewise
 
 pytestmark = pytest.mark.gpu
 
@@ -36,136 +39,113 @@ def slice_edges(extent, nsplit):
     return sorted({c * t for c in range(nsplit)} | {(c + 1) * t - 1 for c in range(nsplit)})
 
 
+def device_errors(g, r):
+    """(parity metric, rms error) of two device tensors, computed on the device in fp64 (the tensors
+    of the largest configuration would not fit a host array of doubles comfortably)."""
+    import torch
+    g, r = g.double().flatten(), r.double().flatten()
+    rms_r = r.pow(2).mean().sqrt().clamp_min(1e-300)
+    d = (g - r).abs()
+    par = (d / torch.maximum(r.abs(), rms_r)).max()
+    rms = d.pow(2).sum().sqrt() / r.pow(2).sum().sqrt().clamp_min(1e-300)
+    return float(par), float(rms)
+
+
+def cross_layout(res, base, keys, what, elem_gate=True):
+    """Every element of every output against the un-split run (same arithmetic, other tile boundaries
+    and summation order): a one-ulp flip of a stored bf16 value is the largest legitimate difference."""
+    for k in keys:
+        par, rms = device_errors(res[k], base[k])
+        assert rms <= 2e-3, (what, k, rms)
+        if elem_gate:
+            assert par <= TOL["bf16"], (what, k, par)
+
+
 FFN_CASES = {
-    "config2": dict(batch=32, length=256, d_model=1024, d_ff=4096,
+    "config2": dict(batch=32, length=256, d_model=1024, d_ff=4096, nsplit=8,
                     layouts=[([("all", 1)], []), ([("all", 8)], [("batch", "all")]), ([("all", 8)], [("d_ff", "all")])]),
-    "target": dict(batch=32, length=256, d_model=1024, d_ff=8192,
-                   layouts=[([("all", 8)], [("d_ff", "all")]), ([("all", 8)], [("batch", "all")])]),
-    "config4": dict(batch=32, length=256, d_model=1024, d_ff=65536, layouts=[([("all", 16)], [("d_ff", "all")])]),
+    "target": dict(batch=32, length=256, d_model=1024, d_ff=8192, nsplit=8,
+                   layouts=[([("all", 1)], []), ([("all", 8)], [("d_ff", "all")]), ([("all", 8)], [("batch", "all")])]),
+    "config4": dict(batch=32, length=256, d_model=1024, d_ff=65536, nsplit=16,
+                    layouts=[([("all", 1)], []), ([("all", 16)], [("d_ff", "all")])]),
 }
 
 
 @pytest.mark.parametrize("name", list(FFN_CASES))
-def test_ffn_full_size_sampled(mtf, name):
-    import torch
-    from oracle import NT, DenseOps, blocks, rounding
+def test_ffn_full_size_stagewise(mtf, name):
     c = FFN_CASES[name]
     B, L, D, F = c["batch"], c["length"], c["d_model"], c["d_ff"]
     T = B * L
-    seed = 0
-    x = si.normal(seed, "x", [B, L, D], "bf16")
-    dy = si.normal(seed, "dy", [B, L, D], "bf16")
-    w = si.normal(seed, "w", [D, F], "bf16", D ** -0.5)
-    v = si.normal(seed, "v", [F, D], "bf16", F ** -0.5)
-    bias = si.normal(seed, "bias", [F], "f32", 0.1)
-    dev = {k: to_torch(s) for k, s in dict(x=x, dy=dy, w=w, v=v, bias=bias).items()}
-    act, hn, wn, vn = ["batch", "length", "d_model"], ["batch", "length", "d_ff"], ["d_model", "d_ff"], ["d_ff", "d_model"]
-    N = mtf.named
-    h = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda")
-    y = torch.empty(B, L, D, dtype=torch.bfloat16, device="cuda")
-    dx = torch.empty_like(y)
-    dw = torch.empty(D, F, dtype=torch.float32, device="cuda")
-    dv = torch.empty(F, D, dtype=torch.float32, device="cuda")
-    dbias = torch.empty(F, dtype=torch.float32, device="cuda")
-
-    # sampled indices: slice edges of every split this case uses, plus seeded picks
-    tok = si.sample_indices(seed, "tokens", T, 6, must_include=slice_edges(B, 8)[:4] + [0, T - 1] + [b * L for b in slice_edges(B, 8)][-3:])
-    hid = si.sample_indices(seed, "hidden", F, 6, must_include=slice_edges(F, 16) if F > 8192 else slice_edges(F, 8))
-    hid = hid[:: max(1, len(hid) // 14)]
-    ops = DenseOps()
-    store = rounding.make_store(ops, "bf16")
-    xs, dys = x.f64.reshape(T, D), dy.f64.reshape(T, D)
-    # (1) sampled tokens: full rows of h, y, dx
-    Xt = NT([("tok", len(tok)), ("d_model", D)], xs[tok])
-    DYt = NT([("tok", len(tok)), ("d_model", D)], dys[tok])
-    Wn, Vn, Bn = NT([("d_model", D), ("d_ff", F)], w.f64), NT([("d_ff", F), ("d_model", D)], v.f64), NT([("d_ff", F)], bias.f64)
-    ft = blocks.ffn_forward(ops, Xt, Wn, Bn, Vn, store)
-    gt = blocks.ffn_backward(ops, Xt, Wn, Vn, ft["h"], DYt, store)
-    amb_tok = tok[np.unique(np.nonzero(np.abs(ft["hp"].a) < 2e-5 * np.sqrt(np.mean(ft["hp"].a ** 2)))[0])]
-    # (2) sampled hidden units: full columns / rows of dw, dv, dbias
-    Xa = NT([("tok", T), ("d_model", D)], xs)
-    DYa = NT([("tok", T), ("d_model", D)], dys)
-    Ws = NT([("d_model", D), ("d_ff", len(hid))], w.f64[:, hid])
-    Vs = NT([("d_ff", len(hid)), ("d_model", D)], v.f64[hid, :])
-    Bs = NT([("d_ff", len(hid))], bias.f64[hid])
-    fh = blocks.ffn_forward(ops, Xa, Ws, Bs, Vs, store)
-    gh = blocks.ffn_backward(ops, Xa, Ws, Vs, fh["h"], DYa, store)
-    amb_hid = np.unique(np.nonzero(np.abs(fh["hp"].a) < 2e-5 * np.sqrt(np.mean(fh["hp"].a ** 2)))[1])
-    keep_hid = np.setdiff1d(np.arange(len(hid)), amb_hid)
-    keep_tok = np.array([i for i, t in enumerate(tok) if t not in set(amb_tok.tolist())], dtype=np.int64)
-
+    inp = ffn_inputs(0, [("batch", B), ("length", L)], D, F, "bf16", True)
+    # sampled tokens: first / last token of every batch slice (8 ways) + seeded picks; sampled hidden
+    # units: first / last of every d_ff slice + seeded picks
+    tok_edges = [b * L for b in slice_edges(B, 8)[:3]] + [b * L + L - 1 for b in slice_edges(B, 8)[-3:]] + [0, T - 1]
+    tok = si.sample_indices(0, "tokens", T, 6, must_include=tok_edges)
+    hid_edges = slice_edges(F, c["nsplit"])
+    hid = si.sample_indices(0, "hidden", F, 6, must_include=hid_edges[:4] + hid_edges[-4:] + hid_edges[len(hid_edges) // 2:len(hid_edges) // 2 + 2])
+    base = None
     for mesh_dims, rules in c["layouts"]:
-        lay = layout(mtf, mesh_dims, rules)
-        ws = torch.empty(mtf.mtf_ffn_workspace_bytes(lay, N(dev["x"], act), N(dev["w"], wn)), dtype=torch.uint8, device="cuda")
-        for t in (h, y, dx, dw, dv, dbias):
-            t.fill_(float("nan"))
-        mtf.mtf_ffn_forward(lay, N(dev["x"], act), N(dev["w"], wn), N(dev["bias"], ["d_ff"]), N(dev["v"], vn), N(h, hn), N(y, act), ws)
-        mtf.mtf_ffn_backward(lay, N(dev["x"], act), N(dev["w"], wn), N(dev["v"], vn), N(h, hn), N(dev["dy"], act), N(dx, act), N(dw, wn),
-                             N(dbias, ["d_ff"]), N(dv, vn), ws)
-        mtf.mtf_device_status()
-        tok_t, hid_t = torch.from_numpy(tok).cuda(), torch.from_numpy(hid).cuda()
-        got = {"h": from_torch(h.view(T, F)[tok_t]), "y": from_torch(y.view(T, D)[tok_t]), "dx": from_torch(dx.view(T, D)[tok_t]),
-               "dw": from_torch(dw[:, hid_t]), "dv": from_torch(dv[hid_t, :]), "dbias": from_torch(dbias[hid_t])}
-        ref = {"h": ft["h"].a, "y": ft["y"].a, "dx": gt["dx"].a[keep_tok], "dw": gh["dw"].a[:, keep_hid], "dv": gh["dv"].a,
-               "dbias": gh["dbias"].a[keep_hid]}
-        got["dx"], got["dw"], got["dbias"] = got["dx"][keep_tok], got["dw"][:, keep_hid], got["dbias"][keep_hid]
-        errs = {k: parity_error(got[k], ref[k]) for k in ref}
-        assert all(e <= TOL["bf16"] for e in errs.values()), (name, rules, errs)
-        # nothing outside the sampled outputs was left unwritten
-        for t in (h, y, dx, dw, dv, dbias):
-            assert bool(torch.isfinite(t).all()), (name, rules)
+        errs, out = run_ffn_stagewise(mtf, layout(mtf, mesh_dims, rules), inp, "bf16", tok=tok, hid=hid, what=f"{name} {rules}")
+        print(name, rules, {k: f"{e:.2e}" for k, e in errs.items()})
+        if base is None:
+            base = out
+        else:
+            cross_layout(out, base, list(base), f"{name} {rules}")
 
 
-def test_attention_config3_full_size(mtf):
-    import torch
-    from test_gpu_attention import attention_case, run_attention_gpu, run_attention_oracle
+def attention_samples(B, L, H, K, b_split, h_split, seed=0):
+    bs, hs = slice_edges(B, b_split), slice_edges(H, h_split)
+    pairs = sorted({(bs[0], hs[0]), (bs[-1], hs[-1]), (bs[1], hs[-2]), (bs[-2], hs[1]), (bs[len(bs) // 2], hs[len(hs) // 2])})
+    tok = si.sample_indices(seed, "att_tokens", B * L, 6, must_include=[0, B * L - 1] + [b * L for b in bs[1:4]] + [b * L + L - 1 for b in bs[-4:-1]])
+    wcols = sorted({(hs[0], 0), (hs[-1], K - 1), (hs[1], K // 2), (hs[-2], 1), (hs[len(hs) // 2], K - 2)})
+    return tok, pairs, wcols
+
+
+def test_attention_config3_full_size_stagewise(mtf):
+    from test_gpu_attention import attention_case
     B, L, D, H, K = 16, 512, 1024, 16, 64
     inp = attention_case(0, B, L, D, H, K)
-    res = {}
+    tok, pairs, wcols = attention_samples(B, L, H, K, 4, 4)
+    base = None
     for tag, mesh_dims, rules in (("unsplit", [("all", 1)], []), ("4x4", [("rows", 4), ("cols", 4)], [("batch", "rows"), ("heads", "cols")])):
-        res[tag] = run_attention_gpu(mtf, layout(mtf, mesh_dims, rules), inp, False)
-    # sampled batch elements against the oracle (the forward pass and dx do not mix batch elements)
-    for b in (0, B - 1):
-        sub = {k: (d, s) if k not in ("x", "dy") else ([("batch", 1)] + d[1:], si.store(s.f64[b:b + 1], "bf16")) for k, (d, s) in inp.items()}
-        ref_s, ref_e = run_attention_oracle(sub, False, "bf16"), run_attention_oracle(sub, False, None)
-        for tag in res:
-            for k in ("y", "P", "o", "q", "dx"):
-                g = res[tag][k][b:b + 1]
-                assert parity_error(g, ref_s[k]) <= TOL_CHAIN["elem"] and rms_error(g, ref_s[k]) <= TOL_CHAIN["rms"], (tag, b, k)
-                assert rms_error(g, ref_e[k]) <= TOL_CHAIN["rms_exact"], (tag, b, k)
-    # parameter gradients reduce over the whole batch: every layout against mesh [1]
-    for k in ("dwq", "dwk", "dwv", "dwo"):
-        assert rms_error(res["4x4"][k], res["unsplit"][k]) <= 1e-3, k
-        assert parity_error(res["4x4"][k], res["unsplit"][k]) <= TOL["bf16"], k
+        errs, out = run_attention_stagewise(mtf, layout(mtf, mesh_dims, rules), inp, False, tok=tok, pairs=pairs, wcols=wcols, what=f"config3 {tag}")
+        print("config3", tag, {k: f"{e:.2e}" for k, e in errs.items()})
+        if base is None:
+            base = out
+        else:
+            cross_layout(out, base, list(base), f"config3 {tag}")
 
 
-def test_decoder_layer_config5_full_size(mtf):
-    from test_gpu_attention import PARAMS, decoder_case, run_decoder_gpu, run_decoder_oracle
+# the six mesh / layout combinations of the decoder-layer sweep that name dimensions the mesh has
+DECODER_SWEEP = {
+    "unsplit": ([("all", 1)], []),
+    "batch8": ([("all", 8)], [("batch", "all")]),
+    "model8": ([("all", 8)], [("d_ff", "all"), ("heads", "all")]),
+    "4x8-batch": ([("rows", 4), ("cols", 8)], [("batch", "rows")]),
+    "4x8-model": ([("rows", 4), ("cols", 8)], [("d_ff", "cols"), ("heads", "cols")]),
+    "4x8": ([("rows", 4), ("cols", 8)], [("batch", "rows"), ("d_ff", "cols"), ("heads", "cols")]),
+}
+
+
+def test_decoder_layer_config5_full_size_stagewise(mtf):
+    import torch
+    from test_gpu_attention import decoder_case
     B, L, D, H, K, F = 64, 256, 2048, 32, 64, 8192
     inp = decoder_case(0, B, L, D, H, K, F)
-    sweeps = {"unsplit": ([("all", 1)], []), "batch8": ([("all", 8)], [("batch", "all")]),
-              "model8": ([("all", 8)], [("d_ff", "all"), ("heads", "all")]),
-              "4x8": ([("rows", 4), ("cols", 8)], [("batch", "rows"), ("d_ff", "cols"), ("heads", "cols")])}
-    res = {tag: run_decoder_gpu(mtf, layout(mtf, md, rules), inp) for tag, (md, rules) in sweeps.items()}
-    # one sampled batch element against the oracle that stores the same intermediates in bf16
-    b = B - 1
-    sub = {k: (d, s) if k not in ("x", "dout") else ([("batch", 1)] + d[1:], si.store(s.f64[b:b + 1], "bf16")) for k, (d, s) in inp.items()}
-    ref_s, _ = run_decoder_oracle(sub, "bf16")
-    # `out` is unique up to storage rounding.  dx is not: with 256 x 8192 hidden activations per batch
-    # element, a few thousand relu decisions [h > 0] fall on inputs that the GPU and the oracle hold
-    # one bf16 ulp apart (each side decides in its own precision), and every such decision moves a
-    # whole row of the gradient stream; the sampled dx therefore agrees to ~1e-2 rms, gated at 3e-2.
-    for tag in res:
-        g = res[tag]["out"][b:b + 1]
-        assert rms_error(g, ref_s["out"]) <= TOL_CHAIN["rms"], (tag, rms_error(g, ref_s["out"]))
-        # element-wise: a one-ulp difference (0.78 %) of the stored residual sum s2 is scaled by
-        # |s2| / rms, which reaches 3-4 in the tails of half a million samples
-        assert parity_error(g, ref_s["out"]) <= 4e-2, (tag, parity_error(g, ref_s["out"]))
-        g = res[tag]["dx"][b:b + 1]
-        assert rms_error(g, ref_s["dx"]) <= 3e-2, (tag, rms_error(g, ref_s["dx"]))
-        # dx of every layout against mesh [1]: same decisions on both sides, so tight again
-        assert rms_error(res[tag]["dx"], res["unsplit"]["dx"]) <= 2e-3, tag
-    # parameter gradients reduce over the whole batch: every layout against mesh [1]
-    for tag in ("batch8", "model8", "4x8"):
-        for k in PARAMS:
-            assert rms_error(res[tag]["d_" + k], res["unsplit"]["d_" + k]) <= 2e-3, (tag, k)
+    tok, pairs, wcols = attention_samples(B, L, H, K, 8, 8)
+    hid_edges = slice_edges(F, 8)
+    hid = si.sample_indices(0, "dec_hidden", F, 4, must_include=hid_edges[:3] + hid_edges[-3:])
+    dcols = si.sample_indices(0, "dec_dcols", D, 6, must_include=[0, D - 1])
+    base = None
+    for tag, (mesh_dims, rules) in DECODER_SWEEP.items():
+        errs, res = run_decoder_stagewise(mtf, layout(mtf, mesh_dims, rules), inp, tok=tok, pairs=pairs, wcols=wcols, hid=hid, dcols=dcols,
+                                          what=f"config5 {tag}")
+        print("config5", tag, {k: f"{e:.2e}" for k, e in errs.items()})
+        if base is None:
+            base = {k: t.clone() for k, t in res.items()}
+        else:
+            # dx and the parameter gradients follow relu decisions and bf16 stores that both runs take
+            # in the same precision on the same values: tight again
+            cross_layout(res, base, list(base), f"config5 {tag}", elem_gate=False)
+        del res
+        torch.cuda.empty_cache()

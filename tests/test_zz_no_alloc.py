@@ -49,6 +49,23 @@ def test_builtin_scratch_matches_regular_entry_point_twice():
             # both entry points add the same partial tiles in the same (ascending processor) order
             assert parity_error(g, w) <= TOL["bf16"], call
             assert np.array_equal(g, w), call
+            # and what they compute is the einsum: against the fp64 oracle on the same inputs
+            from oracle import einsum_arrays
+            ref = einsum_arrays([a_dims, b_dims], [a.f64, b.f64], out_dims)
+            assert parity_error(g, ref) <= TOL["bf16"], call
+        # arguments are validated on every call, as through the regular entry point: a relu mask of the
+        # wrong shape handed in after a good call with the same stages is refused before any launch
+        mask_ok = torch.ones(256, 384, dtype=torch.float32, device="cuda")
+        mask_bad = torch.ones(128, 384, dtype=torch.float32, device="cuda")
+        out = torch.empty(256, 384, dtype=torch.float32, device="cuda")
+        mtf.mtf_einsum_builtin_scratch(lay, None, ins, mtf.named(out, ["i", "j"]), mtf.Epilogue(relu_mask=mtf.named(mask_ok, ["i", "j"])))
+        mtf.mtf_device_status()
+        assert np.array_equal(from_torch(out), from_torch(got))          # a mask of ones keeps everything
+        n0 = mtf.mtf_launch_count()
+        with pytest.raises(mtf.MtfError) as e:
+            mtf.mtf_einsum_builtin_scratch(lay, None, ins, mtf.named(out, ["i", "j"]), mtf.Epilogue(relu_mask=mtf.named(mask_bad, ["i", "j"])))
+        assert e.value.code in ("MTF_ERR_INVALID_ARG", "MTF_ERR_SIZE_MISMATCH")
+        assert mtf.mtf_launch_count() == n0
         # a contraction whose partial tiles do not fit the built-in array is refused before any launch
         big_a, big_b = mtf.desc([("k", 8192), ("i", 4096)], "bf16"), mtf.desc([("k", 8192), ("j", 4096)], "bf16")
         n0 = mtf.mtf_launch_count()
