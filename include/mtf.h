@@ -125,6 +125,43 @@ mtf_status mtf_slice_map(const mtf_layout_t* layout, int32_t ndim, const mtf_dim
 mtf_status mtf_slice_gather(const mtf_layout_t* layout, const mtf_tensor* global, int64_t processor,
                             void* out_slice, void* stream);
 
+/* ---- one mesh dimension across several GPUs (Section 2: a mesh is a naming abstraction over the
+ * physical processors; Section 3, Algorithm 1 line 2: the gradient Allreduce; Section 8.1 / 8.2 /
+ * Table 1 "Comm." column: which einsums need an Allreduce under which layout) ----------------------
+ * One process per GPU.  mtf_layout_bind_ranks maps mesh dimension `mesh_dim` (size m, divisible by
+ * `world`) onto `world` ranks: rank r owns the virtual processors whose coordinate on that mesh
+ * dimension lies in [r m / world, (r + 1) m / world).  The returned handle is a layout over THIS
+ * RANK'S part of the mesh (that mesh dimension has m / world processors in it), and every tensor
+ * handed to a call under it is the rank's box of the global tensor: a dimension that the layout
+ * splits over `mesh_dim` has its global size / world here (mtf_rank_box gives the box), everything
+ * else is whole (replicated across ranks).  All calls work as on one GPU; in addition
+ *   - an einsum (or reduction) that sums out a dimension split over `mesh_dim` leaves, on every
+ *     rank, a partial result that the ranks must add up: mtf_plan_needs_rank_sum says so, and when
+ *     collective hooks were given the library calls `start(user, data, count, dtype, stream)` right
+ *     behind the launch that produced the partial result (the hook enqueues a sum over all ranks, in
+ *     place, that begins when `stream` reaches this point, and returns without blocking);
+ *   - `wait(user, stream)` makes `stream` wait for every sum started so far.  The block calls
+ *     (mtf_ffn_*, mtf_attention_*, mtf_decoder_layer_*, mtf_layernorm_backward) call it before a
+ *     launch that reads a summed tensor and before they return; after a bare mtf_einsum call
+ *     mtf_rank_wait when the result is needed;
+ *   - component-wise stages that are not linear (bias, relu, relu_mask, a fused reduce_sum of such
+ *     values, a row softmax) cannot ride in a launch whose result is only a partial sum:
+ *     MTF_ERR_UNSUPPORTED.  A residual can: rank 0 adds it, the others do not.
+ * The hooks are the only place where ranks meet; the library itself links no communication library
+ * (the Python binding provides hooks over torch.distributed: NCCL on GPUs, gloo in CPU tests).
+ * Hooks may be NULL (both or neither): the caller then sums the flagged outputs itself.
+ * world = 1 is legal and changes nothing. */
+typedef mtf_status (*mtf_rank_allreduce_fn)(void* user, void* data, int64_t count, mtf_dtype dtype, void* stream);
+typedef mtf_status (*mtf_rank_wait_fn)(void* user, void* stream);
+mtf_status mtf_layout_bind_ranks(const mtf_layout_t* layout, const char* mesh_dim, int32_t world, int32_t rank,
+                                 mtf_rank_allreduce_fn start, mtf_rank_wait_fn wait, void* user, mtf_layout_t** out);
+/* This rank's box of a GLOBAL tensor under a rank-bound layout: host outputs offsets[ndim], sizes[ndim]. */
+mtf_status mtf_rank_box(const mtf_layout_t* bound_layout, int32_t ndim, const mtf_dim* global_dims, int64_t* offsets, int64_t* sizes);
+/* 1 when the plan's result is a partial sum the ranks still have to add up (bit 0: the output, bit 1:
+ * the fused reduce_sum output), else 0.  Always 0 under a layout that is not rank-bound. */
+mtf_status mtf_plan_needs_rank_sum(const mtf_plan_t* plan, int32_t* flags);
+mtf_status mtf_rank_wait(const mtf_layout_t* bound_layout, void* stream);
+
 /* ---- einsum (Section 6 "Einstein Summation"; Section 8 code fragment) ------------------------- */
 /* Plan  out[out dims] = sum over dims not in out of  in[0] * in[1]  under `layout`.
  * The equation is carried by the dimension names, as in mtf.einsum(x, w, output_shape=[...]).

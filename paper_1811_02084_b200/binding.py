@@ -74,6 +74,10 @@ class mtf_decoder_grads(Structure):
     _fields_ = [(n, POINTER(mtf_tensor)) for n in ("dwq", "dwk", "dwv", "dwo", "dln1_gamma", "dln1_beta", "dw", "dbias", "dv", "dln2_gamma", "dln2_beta")]
 
 
+RANK_ALLREDUCE_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p, c_int64, c_int, c_void_p)     # (user, data, count, dtype, stream) -> status
+RANK_WAIT_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p)                                    # (user, stream) -> status
+
+
 class MtfError(RuntimeError):
     def __init__(self, status: int, message: str):
         self.status = status
@@ -125,6 +129,10 @@ def _load():
         "mtf_decoder_layer_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(mtf_decoder_saved), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_decoder_grads), vp, c_size_t, vp],
         "mtf_decoder_layer_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(c_size_t)],
         "mtf_device_status": [POINTER(c_int32)],
+        "mtf_layout_bind_ranks": [vp, c_char_p, c_int32, c_int32, RANK_ALLREDUCE_FN, RANK_WAIT_FN, vp, POINTER(vp)],
+        "mtf_rank_box": [vp, c_int32, POINTER(mtf_dim), POINTER(c_int64), POINTER(c_int64)],
+        "mtf_plan_needs_rank_sum": [vp, POINTER(c_int32)],
+        "mtf_rank_wait": [vp, vp],
         "mtf_stage_tap_begin": [vp, c_size_t],
         "mtf_stage_tap_end": [POINTER(c_int32)],
         "mtf_stage_tap_entry": [c_int32, POINTER(c_char_p), POINTER(c_size_t), POINTER(c_size_t)],
@@ -298,6 +306,38 @@ def mtf_layout(mesh: Mesh, rules) -> Layout:
     h = c_void_p()
     _check(_lib.mtf_layout(mesh.handle, n, t, m, byref(h)))
     return Layout(h, list(mesh.dims), list(rules))
+
+
+def mtf_layout_bind_ranks(layout: Layout, mesh_dim: str, world: int, rank: int, collective=None) -> Layout:
+    """This rank's part of ``layout`` when mesh dimension ``mesh_dim`` is spread over ``world`` ranks.
+    ``collective``: an object with ctypes callbacks ``start_cb`` (RANK_ALLREDUCE_FN) and ``wait_cb``
+    (RANK_WAIT_FN), e.g. multi_gpu.RankCollective; None = the caller sums the flagged outputs itself."""
+    h = c_void_p()
+    start = collective.start_cb if collective is not None else RANK_ALLREDUCE_FN()
+    wait = collective.wait_cb if collective is not None else RANK_WAIT_FN()
+    _check(_lib.mtf_layout_bind_ranks(layout.handle, mesh_dim.encode(), int(world), int(rank), start, wait, None, byref(h)))
+    mesh_dims = [(n, s // world if n == mesh_dim else s) for n, s in layout.mesh_dims]
+    out = Layout(h, mesh_dims, list(layout.rules))
+    out.collective = collective          # keeps the callbacks alive as long as the handle
+    return out
+
+
+def mtf_rank_box(bound_layout: Layout, global_dims):
+    arr, _keep = _dims_array(global_dims)
+    offs = (c_int64 * max(len(global_dims), 1))()
+    sizes = (c_int64 * max(len(global_dims), 1))()
+    _check(_lib.mtf_rank_box(bound_layout.handle, len(global_dims), arr, offs, sizes))
+    return list(offs)[:len(global_dims)], list(sizes)[:len(global_dims)]
+
+
+def mtf_plan_needs_rank_sum(plan: Plan) -> int:
+    f = c_int32()
+    _check(_lib.mtf_plan_needs_rank_sum(plan.handle, byref(f)))
+    return f.value
+
+
+def mtf_rank_wait(bound_layout: Layout, stream=None) -> None:
+    _check(_lib.mtf_rank_wait(bound_layout.handle, _stream(stream)))
 
 
 def mtf_layout_check_tensor(layout: Layout, dims) -> None:

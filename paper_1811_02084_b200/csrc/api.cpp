@@ -27,6 +27,12 @@ thread_local int g_force_reduce = -1;
 
 int elem_bytes(int dt) { return dt == MTF_BF16 ? 2 : 4; }
 
+int64_t numel(const mtf_tensor& t) {
+  int64_t n = 1;
+  for (int i = 0; i < t.ndim; ++i) n *= t.dims[i].size;
+  return n;
+}
+
 bool dims_match(const std::vector<Dim>& want, const mtf_tensor& t) {
   if ((int)want.size() != t.ndim) return false;
   for (int i = 0; i < t.ndim; ++i)
@@ -62,6 +68,7 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
       if (!epi->residual || !epi->residual->data || !dims_match(P->dimsC, *epi->residual) || epi->residual->dtype != P->epi.dtRes)
         return fail(MTF_ERR_INVALID_ARG, "einsum exec: residual differs from the planned one");
       resid = epi->residual->data;
+      if (P->rank_sum && P->rank != 0) resid = nullptr;      // a partial sum across ranks: rank 0 alone adds the residual
     }
   }
   float* rsum = nullptr;
@@ -74,18 +81,39 @@ mtf_status exec_plan(const mtf_plan_t* P, const mtf_tensor* in, mtf_tensor* out,
   }
   const float scale = P->epi.on ? epi->scale : 1.f;
   const int relu = P->epi.on ? (epi->relu != 0) : 0;
-  if (P->kernel_kind == MTF_KERNEL_TCGEN05)
-    return mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
-                          P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands, row_softmax, n_groups, group_operands);
-  if (n_terms != 1 || row_softmax || n_groups != 1) return fail(MTF_ERR_UNSUPPORTED, "multi-term, grouped or fused-softmax contraction on the generic kernel");
-  SimtParams s = P->simt;
-  s.A = in[0].data;
-  s.B = P->has_B ? in[1].data : nullptr;
-  s.C = out->data;
-  s.bias = bias; s.mask = mask; s.resid = resid;
-  s.scale = scale; s.relu = relu;
-  s.rsum = rsum;
-  return mtf::launch_simt(s, rsum_elems, stream);
+  if (row_softmax && P->rank_sum) return fail(MTF_ERR_UNSUPPORTED, "a row softmax cannot follow a sum that is split across ranks");
+  mtf_status st;
+  if (P->kernel_kind == MTF_KERNEL_TCGEN05) {
+    st = mtf::launch_tc(*P, in[0].data, in[1].data, out->data, bias, P->epi.dtBias, mask, P->epi.dtMask, resid,
+                        P->epi.dtRes, scale, relu, rsum, workspace, workspace_bytes, stream, n_terms, extra_operands, row_softmax, n_groups, group_operands);
+  } else {
+    if (n_terms != 1 || row_softmax || n_groups != 1) return fail(MTF_ERR_UNSUPPORTED, "multi-term, grouped or fused-softmax contraction on the generic kernel");
+    SimtParams s = P->simt;
+    s.A = in[0].data;
+    s.B = P->has_B ? in[1].data : nullptr;
+    s.C = out->data;
+    s.bias = bias; s.mask = mask; s.resid = resid;
+    s.scale = scale; s.relu = relu;
+    s.rsum = rsum;
+    st = mtf::launch_simt(s, rsum_elems, stream);
+  }
+  if (st != MTF_OK) return st;
+  // one mesh dimension across ranks: the result is a partial sum; the caller's hook adds the ranks' parts up behind this launch
+  if (P->ar_start && (P->rank_sum || (P->rsum_rank_sum && rsum))) {
+    if (P->rank_sum) {
+      mtf_status hs = P->ar_start(P->ar_user, out->data, numel(*out), out->dtype, stream);
+      if (hs != MTF_OK) return fail(hs, "the rank collective hook (start) returned status %d", (int)hs);
+      for (int g = 1; g < n_groups; ++g) {       // grouped launch: the other problems' outputs (same shape and type)
+        hs = P->ar_start(P->ar_user, const_cast<void*>(group_operands[3 * (g - 1) + 2]), numel(*out), out->dtype, stream);
+        if (hs != MTF_OK) return fail(hs, "the rank collective hook (start) returned status %d", (int)hs);
+      }
+    }
+    if (P->rsum_rank_sum && rsum) {
+      mtf_status hs = P->ar_start(P->ar_user, rsum, rsum_elems, MTF_F32, stream);
+      if (hs != MTF_OK) return fail(hs, "the rank collective hook (start) returned status %d", (int)hs);
+    }
+  }
+  return MTF_OK;
 }
 
 // Plan through the layout's cache.  The returned pointer stays valid for the layout's lifetime.
@@ -134,12 +162,6 @@ mtf_status check_equation(const char* eq, int n_in, const mtf_tensor* in, const 
 }
 
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
-
-int64_t numel(const mtf_tensor& t) {
-  int64_t n = 1;
-  for (int i = 0; i < t.ndim; ++i) n *= t.dims[i].size;
-  return n;
-}
 
 struct FfnShapes {
   std::vector<mtf_dim> tok_hidden, hidden_only;
@@ -361,7 +383,8 @@ mtf_status mtf_reduce_sum(const mtf_layout_t* layout, const mtf_tensor* in, mtf_
 mtf_status mtf_ffn_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias,
                            const mtf_tensor* v, mtf_tensor* h_saved, mtf_tensor* y, void* workspace, size_t workspace_bytes,
                            void* stream) {
-  return mtf::ffn_forward_impl(layout, x, w, bias, v, h_saved, y, nullptr, workspace, workspace_bytes, stream);
+  mtf_status st = mtf::ffn_forward_impl(layout, x, w, bias, v, h_saved, y, nullptr, workspace, workspace_bytes, stream);
+  return st != MTF_OK ? st : mtf::rank_wait(layout, stream);
 }
 
 }  // extern "C"
@@ -431,7 +454,8 @@ mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor*
 mtf_status mtf_ffn_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v,
                             const mtf_tensor* h_saved, const mtf_tensor* dy, mtf_tensor* dx, mtf_tensor* dw, mtf_tensor* dbias,
                             mtf_tensor* dv, void* workspace, size_t workspace_bytes, void* stream) {
-  return mtf::ffn_backward_impl(layout, x, w, v, h_saved, dy, dx, nullptr, dw, dbias, dv, workspace, workspace_bytes, stream);
+  mtf_status st = mtf::ffn_backward_impl(layout, x, w, v, h_saved, dy, dx, nullptr, dw, dbias, dv, workspace, workspace_bytes, stream);
+  return st != MTF_OK ? st : mtf::rank_wait(layout, stream);
 }
 
 }  // extern "C"

@@ -207,9 +207,18 @@ mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* 
   if (residual && !residual->data) return fail(MTF_ERR_INVALID_ARG, "layernorm backward: residual has no data");
   mtf_status st = mtf_layout_check_tensor(layout, x->ndim, x->dims);
   if (st != MTF_OK) return st;
-  return mtf::launch_layernorm_bwd(dy->data, x->data, reinterpret_cast<const float*>(stats->data), reinterpret_cast<const float*>(gamma->data),
-                                   residual ? residual->data : nullptr, dx->data, dgamma ? reinterpret_cast<float*>(dgamma->data) : nullptr,
-                                   dbeta ? reinterpret_cast<float*>(dbeta->data) : nullptr, rows, n, stream);
+  st = mtf::launch_layernorm_bwd(dy->data, x->data, reinterpret_cast<const float*>(stats->data), reinterpret_cast<const float*>(gamma->data),
+                                 residual ? residual->data : nullptr, dx->data, dgamma ? reinterpret_cast<float*>(dgamma->data) : nullptr,
+                                 dbeta ? reinterpret_cast<float*>(dbeta->data) : nullptr, rows, n, stream);
+  if (st != MTF_OK || !dgamma) return st;
+  // the parameter gradients sum over the token dimensions: with one of them split across ranks they are partial sums
+  std::vector<std::string> reduced;
+  for (int i = 0; i + 1 < x->ndim; ++i) reduced.push_back(x->dims[i].name);
+  if (mtf::rank_sum_needed(layout, reduced)) {
+    if ((st = mtf::rank_allreduce_start(layout, dgamma->data, n, MTF_F32, stream)) != MTF_OK) return st;
+    if ((st = mtf::rank_allreduce_start(layout, dbeta->data, n, MTF_F32, stream)) != MTF_OK) return st;
+  }
+  return MTF_OK;
 }
 
 // ---- multi-head attention -----------------------------------------------------------------------------
@@ -278,7 +287,8 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
   if ((st = ein(layout, *weights, *vv, o, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   mtf_epilogue er = epi_none();
   er.residual = residual;
-  return ein(layout, *o, *wo, y, residual ? &er : nullptr, rest, rest_bytes, stream);
+  if ((st = ein(layout, *o, *wo, y, residual ? &er : nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  return mtf::rank_wait(layout, stream);        // heads split across ranks: y is summed over them before anyone reads it
 }
 
 // dwo = sum_{b,l} o dy; do = sum_d dy wo; dP = sum_v do vv; dvv = sum_l P do; dlogits = P (dP - sum_m dP P);
@@ -346,15 +356,19 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
     // into one accumulator (same shapes; the key / value side carries the memory_length name)
     const mtf_tensor terms[3][2] = {{dq.t, *wq}, {dkk.t, *wk}, {dvv.t, *wv}};
     st = mtf::einsum_terms(layout, 3, terms, dx, dx_residual ? &er : nullptr, rest, rest_bytes, stream);
+    if (st == MTF_OK) return mtf::rank_wait(layout, stream);
     if (st != MTF_ERR_UNSUPPORTED) return st;
   }
+  if (layout->bound_dim >= 0 && layout->world > 1 && mtf::rank_sum_needed(layout, {s.h.name, s.k.name, s.v.name}))
+    return fail(MTF_ERR_UNSUPPORTED, "attention_backward: with heads split across ranks dx needs the single three-term launch, which this plan cannot run");
   if ((st = ein(layout, dq.t, *wq, &dx32.t, dx_residual ? &er : nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   TD dx32m = renamed(dx32.t, s.l.name, kMemory);
   mtf_epilogue ea = epi_none();
   ea.residual = &dx32m.t;
   if ((st = ein(layout, dkk.t, *wk, &dx32m.t, &ea, rest, rest_bytes, stream)) != MTF_OK) return st;
   TD dxm = renamed(*dx, s.l.name, kMemory);
-  return ein(layout, dvv.t, *wv, &dxm.t, &ea, rest, rest_bytes, stream);
+  if ((st = ein(layout, dvv.t, *wv, &dxm.t, &ea, rest, rest_bytes, stream)) != MTF_OK) return st;
+  return mtf::rank_wait(layout, stream);
 }
 
 // ---- decoder layer: a = LN1(x + Attention(x)); out = LN2(a + FFN(a)) ------------------------------------
@@ -382,6 +396,7 @@ mtf_status mtf_decoder_layer_forward(const mtf_layout_t* layout, const mtf_tenso
   if ((st = mtf_layernorm_forward(layout, sv->s1, p->ln1_gamma, p->ln1_beta, eps, sv->a, sv->stats1, stream)) != MTF_OK) return st;
   // s2 = a + FFN(a); out = LN2(s2)
   if ((st = mtf::ffn_forward_impl(layout, sv->a, p->w, p->bias, p->v, sv->h, sv->s2, sv->a, workspace, workspace_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::rank_wait(layout, stream)) != MTF_OK) return st;        // d_ff split across ranks: s2 is summed before the layer norm reads it
   return mtf_layernorm_forward(layout, sv->s2, p->ln2_gamma, p->ln2_beta, eps, out, sv->stats2, stream);
 }
 
@@ -407,6 +422,7 @@ mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tens
   if ((st = mtf::tap("ds2", ds2.t, stream)) != MTF_OK) return st;
   // da = ds2 + dFFN/da
   if ((st = mtf::ffn_backward_impl(layout, sv->a, p->w, p->v, sv->h, &ds2.t, &da.t, &ds2.t, g->dw, g->dbias, g->dv, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::rank_wait(layout, stream)) != MTF_OK) return st;        // da (and the parameter gradients) summed across ranks
   if ((st = mtf::tap("da", da.t, stream)) != MTF_OK) return st;
   // ds1 (reusing ds2's buffer) = LN1 backward; dx = ds1 + dAttention/dx
   if ((st = mtf_layernorm_backward(layout, &da.t, sv->s1, sv->stats1, p->ln1_gamma, nullptr, &ds2.t, g->dln1_gamma, g->dln1_beta, stream)) != MTF_OK) return st;

@@ -121,6 +121,13 @@ struct mtf_plan_s {
   int64_t n_slices = 1, group_size = 1;
   uint32_t reduce_mask = 0;
   size_t workspace_bytes = 0;
+  // one mesh dimension mapped onto ranks (mtf_layout_bind_ranks): the on-device result is a partial sum
+  // that the ranks still have to add up when a reduced-out dimension is split over that mesh dimension
+  bool rank_sum = false;          // ... of the einsum's output
+  bool rsum_rank_sum = false;     // ... of the fused reduce_sum output
+  int rank = 0;
+  mtf_rank_allreduce_fn ar_start = nullptr;
+  void* ar_user = nullptr;
   // cost counts
   int64_t macs_per_proc = 0, allreduce_values = 0, slice_elems = 0;
   int n_reduce_mesh_dims = 0;
@@ -133,6 +140,14 @@ struct mtf_plan_s {
 struct mtf_layout_s {
   std::vector<mtf::Dim> mesh;
   std::vector<std::pair<std::string, int>> rules;   // tensor-dim name -> mesh-dim index
+  // rank binding: mesh dimension `bound_dim` (of global size bound_global) is spread over `world` ranks;
+  // this handle describes rank `rank`'s part, its mesh carries bound_global / world processors there
+  int bound_dim = -1;
+  int world = 1, rank = 0;
+  int64_t bound_global = 0;
+  mtf_rank_allreduce_fn ar_start = nullptr;
+  mtf_rank_wait_fn ar_wait = nullptr;
+  void* ar_user = nullptr;
   std::mutex mu;
   std::map<std::string, std::unique_ptr<mtf_plan_t>> cache;
   int mesh_dim_of(const std::string& tdim) const {
@@ -150,6 +165,13 @@ mtf_status slice_box(const mtf_layout_t* L, const std::vector<Dim>& dims, int64_
 mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, const mtf_tensor* out,
                      const mtf_epilogue* epi, int force_kernel, int force_reduce, std::unique_ptr<mtf_plan_t>* plan);
 std::string plan_key(int n_in, const mtf_tensor* in, const mtf_tensor* out, const mtf_epilogue* epi, int fk, int fr);
+
+// rank binding (ranks.cpp): does summing out `reduced` (dimension names) leave a sum across ranks to do?
+bool rank_sum_needed(const mtf_layout_t* L, const std::vector<std::string>& reduced);
+// start the sum across ranks of `count` values at `data` behind what is queued on `stream`; no-op without hooks
+mtf_status rank_allreduce_start(const mtf_layout_t* L, void* data, int64_t count, mtf_dtype dtype, void* stream);
+// make `stream` wait for every sum across ranks started so far; no-op without hooks
+mtf_status rank_wait(const mtf_layout_t* L, void* stream);
 
 // launchers (defined in the .cu files)
 mtf_status launch_simt(const SimtParams& p, int64_t rsum_elems, void* stream);

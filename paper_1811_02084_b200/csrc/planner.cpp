@@ -412,6 +412,25 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
   P->allreduce_values = P->reduce_mask ? out_slice : 0;
   P->slice_elems = out_slice + local_elems(P->dimsA) + (P->has_B ? local_elems(P->dimsB) : 0);
 
+  // ---- rank binding: which results are partial sums that the ranks still have to add up ----
+  if (L->bound_dim >= 0 && L->world > 1) {
+    P->rank = L->rank;
+    P->ar_start = L->ar_start;
+    P->ar_user = L->ar_user;
+    for (auto& d : P->iter)
+      if (!d.inC && L->mesh_dim_of(d.name) == L->bound_dim) P->rank_sum = true;
+    if (P->epi.has_rsum)
+      for (auto& d : P->iter) {
+        if (!d.inC || L->mesh_dim_of(d.name) != L->bound_dim) continue;
+        bool kept = false;
+        for (auto& r : P->epi.rsum_dims) kept = kept || r.name == d.name;
+        if (!kept) P->rsum_rank_sum = true;
+      }
+    if (P->rank_sum && (P->epi.has_bias || P->epi.relu || P->epi.has_mask || P->epi.has_rsum))
+      return fail(MTF_ERR_UNSUPPORTED, "this einsum sums out a dimension that is split across ranks: its result on one rank is a partial sum, "
+                  "which bias, relu, relu_mask and a fused reduce_sum cannot be applied to");
+  }
+
   // ---- generic strided kernel parameters (always built: it is the fallback family) ----
   SimtParams& s = P->simt;
   s.n_out = (int)P->dimsC.size();
