@@ -2,7 +2,7 @@
 """Benchmark of the hot path: Transformer feed-forward block, forward + backward, as layout-lowered
 named-dimension einsums on one B200 (or N replicas of the batch-split mesh dimension on N GPUs).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--layout mp8|dp8|none] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--layout mp8|dp8|none|mp16] [--split dp|mp] [--impl reference]
 
 One step = mtf_ffn_forward + mtf_ffn_backward through the C ABI on the workload
 tokens 8192 (batch 32 x length 256), d_model 1024, d_ff 8192, bf16 storage / fp32 accumulation
@@ -30,7 +30,10 @@ LAYOUTS = {
     "mp8": ([("all", 8)], [("d_ff", "all")]),
     "mp16": ([("all", 16)], [("d_ff", "all")]),
 }
+# dram__bytes_read.sum + dram__bytes_write.sum per contraction launch, averaged over the six launches of a
+# step of this workload (one ncu capture; the summary under profiles/ names the command and the commit)
 NCU_DRAM_BYTES_PER_LAUNCH = 169.7e6
+NCU_TRAFFIC_COMMIT = "12d0670"
 METRIC = "transformer_ffn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
@@ -169,8 +172,31 @@ def run_reference(args):
 # our arm
 # ------------------------------------------------------------------------------------------------------
 
-def run_ours(args):
+def to_device(s):
+    """seeded_inputs.Stored -> device tensor with exactly those bytes."""
     import numpy as np
+    import torch
+    if s.dtype == "bf16":
+        return torch.from_numpy(s.bits.view(np.int16)).view(torch.bfloat16).cuda()
+    return torch.from_numpy(s.bits).cuda()
+
+
+def event_time(fn, reps, stream, warmup=3):
+    """Average device time of fn() in ms: one CUDA-event pair around `reps` back-to-back calls."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(reps):
+        fn()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def run_ours(args):
     import torch
     import seeded_inputs as si
 
@@ -189,77 +215,51 @@ def run_ours(args):
 
     B, L, D, F = WORKLOAD["batch"], WORKLOAD["length"], WORKLOAD["d_model"], WORKLOAD["d_ff"]
     T = B * L
-    seed = 1000 * rank          # every rank owns its own shard of the (replica x batch) global batch
+    # Per-GPU work is fixed (weak scaling).  With N ranks one mesh dimension ("gpus") spans them:
+    #   --split dp: batch -> gpus   (global batch N x 32; every rank its own tokens; dw, dv, dbias are summed: Algorithm 1 line 2)
+    #   --split mp: d_ff  -> gpus   (global d_ff N x 8192; every rank its own hidden units; y and dx are summed: Section 8.2)
+    # The other dimension keeps the virtual mesh of --layout inside each rank.
+    seed_x = 1000 * rank if args.split == "dp" else 0
+    seed_w = 0 if args.split == "dp" else 1000 * rank
     host = {
-        "x": si.normal(seed, "x", [B, L, D], "bf16"),
-        "dy": si.normal(seed, "dy", [B, L, D], "bf16"),
-        "w": si.normal(0, "w", [D, F], "bf16", D ** -0.5),
-        "v": si.normal(0, "v", [F, D], "bf16", F ** -0.5),
-        "bias": si.normal(0, "bias", [F], "f32", 0.1),
+        "x": si.normal(seed_x, "x", [B, L, D], "bf16"),
+        "dy": si.normal(seed_x, "dy", [B, L, D], "bf16"),
+        "w": si.normal(seed_w, "w", [D, F], "bf16", D ** -0.5),
+        "v": si.normal(seed_w, "v", [F, D], "bf16", F ** -0.5),
+        "bias": si.normal(seed_w, "bias", [F], "f32", 0.1),
     }
-
-    def dev(s):
-        if s.dtype == "bf16":
-            return torch.from_numpy(s.bits.view(np.int16)).view(torch.bfloat16).cuda()
-        return torch.from_numpy(s.bits).cuda()
-
-    t = {k: dev(s) for k, s in host.items()}
+    t = {k: to_device(s) for k, s in host.items()}
     h = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda")
     y = torch.empty(B, L, D, dtype=torch.bfloat16, device="cuda")
     dx = torch.empty_like(y)
     dw = torch.empty(D, F, dtype=torch.float32, device="cuda")
     dv = torch.empty(F, D, dtype=torch.float32, device="cuda")
     dbias = torch.empty(F, dtype=torch.float32, device="cuda")
-    act, wn, vn = ["batch", "length", "d_model"], ["d_model", "d_ff"], ["d_ff", "d_model"]
+    act, wn, vn, hn = ["batch", "length", "d_model"], ["d_model", "d_ff"], ["d_ff", "d_model"], ["batch", "length", "d_ff"]
     N = {"x": mtf.named(t["x"], act), "dy": mtf.named(t["dy"], act), "w": mtf.named(t["w"], wn), "v": mtf.named(t["v"], vn),
-         "bias": mtf.named(t["bias"], ["d_ff"]), "h": mtf.named(h, ["batch", "length", "d_ff"]), "y": mtf.named(y, act),
+         "bias": mtf.named(t["bias"], ["d_ff"]), "h": mtf.named(h, hn), "y": mtf.named(y, act),
          "dx": mtf.named(dx, act), "dw": mtf.named(dw, wn), "dv": mtf.named(dv, vn), "dbias": mtf.named(dbias, ["d_ff"])}
 
+    collective = multi_gpu.RankCollective(dist) if dist is not None else None
     layouts = {}
     for name, (mesh_dims, rules) in LAYOUTS.items():
-        layouts[name] = mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules)
+        if dist is None:
+            layouts[name] = mtf.mtf_layout(mtf.mtf_mesh_create(mesh_dims), rules)
+            continue
+        # the rank-spanning mesh dimension in front of the virtual mesh; the dimension it takes leaves the inner rules
+        taken = "batch" if args.split == "dp" else "d_ff"
+        inner = [(td, md) for td, md in rules if td != taken]
+        glob = mtf.mtf_layout(mtf.mtf_mesh_create([("gpus", world)] + list(mesh_dims)), [(taken, "gpus")] + inner)
+        layouts[name] = mtf.mtf_layout_bind_ranks(glob, "gpus", world, rank, collective)
     ws_bytes = max(mtf.mtf_ffn_workspace_bytes(l, N["x"], N["w"]) for l in layouts.values())
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
 
-    dhp = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda") if dist is not None else None
-    sync = multi_gpu.GradientSync(dist)
-
-    def backward(lay, xin, dyin, dxout):
-        """The feed-forward backward pass.  On one GPU: mtf_ffn_backward.  On several: the same four
-        contractions issued one by one (what mtf_ffn_backward does inside), so that the all-reduce of a
-        parameter gradient (Algorithm 1, line 2: the batch-split mesh dimension that spans the GPUs)
-        starts right behind the contraction that produces it and runs while the later ones compute."""
-        if dist is None:
-            mtf.mtf_ffn_backward(lay, xin, N["w"], N["v"], N["h"], dyin, dxout, N["dw"], N["dbias"], N["dv"], ws)
-            return
-        ndhp = mtf.named(dhp, ["batch", "length", "d_ff"])
-        mtf.mtf_einsum(lay, None, [dyin, N["v"]], ndhp, mtf.Epilogue(relu_mask=N["h"], reduce_sum_out=N["dbias"]), workspace=ws)
-        mtf.mtf_einsum(lay, None, [N["h"], dyin], N["dv"], None, workspace=ws)
-        sync.start(dv)
-        sync.start(dbias)
-        mtf.mtf_einsum(lay, None, [xin, ndhp], N["dw"], None, workspace=ws)
-        sync.start(dw)
-        mtf.mtf_einsum(lay, None, [ndhp, N["w"]], dxout, None, workspace=ws)
-        sync.finish()
-
-    def step(lay):
-        mtf.mtf_ffn_forward(lay, N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
-        backward(lay, N["x"], N["dy"], N["dx"])
-
-    if dist is not None:
-        # the contractions issued one by one give what the block entry point gives
-        mtf.mtf_ffn_forward(layouts[args.layout], N["x"], N["w"], N["bias"], N["v"], N["h"], N["y"], ws)
-        mtf.mtf_ffn_backward(layouts[args.layout], N["x"], N["w"], N["v"], N["h"], N["dy"], N["dx"], N["dw"], N["dbias"], N["dv"], ws)
-        want = [t_.clone() for t_ in (dx, dw, dv, dbias)]
-        ndhp = mtf.named(dhp, ["batch", "length", "d_ff"])
-        mtf.mtf_einsum(layouts[args.layout], None, [N["dy"], N["v"]], ndhp, mtf.Epilogue(relu_mask=N["h"], reduce_sum_out=N["dbias"]), workspace=ws)
-        mtf.mtf_einsum(layouts[args.layout], None, [N["h"], N["dy"]], N["dv"], None, workspace=ws)
-        mtf.mtf_einsum(layouts[args.layout], None, [N["x"], ndhp], N["dw"], None, workspace=ws)
-        mtf.mtf_einsum(layouts[args.layout], None, [ndhp, N["w"]], N["dx"], None, workspace=ws)
-        torch.cuda.synchronize()
-        for got, ref, nm in zip((dx, dw, dv, dbias), want, ("dx", "dw", "dv", "dbias")):
-            assert torch.allclose(got.float(), ref.float(), rtol=1e-3, atol=1e-3 * float(ref.float().abs().max())), f"{nm}: the einsum sequence differs from mtf_ffn_backward"
+    def step(lay, xin=None, dyin=None, yout=None, dxout=None):
+        # the sums across ranks are started by the library behind the launch that produces each partial
+        # result (hooks of the rank-bound layout) and awaited before the block call returns
+        mtf.mtf_ffn_forward(lay, xin or N["x"], N["w"], N["bias"], N["v"], N["h"], yout or N["y"], ws)
+        mtf.mtf_ffn_backward(lay, xin or N["x"], N["w"], N["v"], N["h"], dyin or N["dy"], dxout or N["dx"], N["dw"], N["dbias"], N["dv"], ws)
 
     def timed(lay, steps, warmup, sampler=None):
         for _ in range(warmup):
@@ -290,6 +290,8 @@ def run_ours(args):
     sampler = ClockSampler(physical_gpu_index(local_rank))
     ms_step, launches, clocks = timed(layouts[args.layout], args.steps, max(args.warmup, 3), sampler)
     mtf.mtf_device_status()
+    if collective is not None and collective.error is not None:
+        raise collective.error
     value = world * flops_step / (ms_step * 1e-3) / 1e12
 
     per_layout = {}
@@ -335,8 +337,7 @@ def run_ours(args):
             in_ready[q].record(s_in)
         stream.wait_event(in_ready[q])
         stream.wait_event(out_done[q])                  # the results of the step that last used this output set are on the host
-        mtf.mtf_ffn_forward(lay, names["x"], N["w"], N["bias"], N["v"], N["h"], names["y"], ws)
-        backward(lay, names["x"], names["dy"], names["dx"])
+        step(lay, names["x"], names["dy"], names["y"], names["dx"])
         done[q].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(done[q])
@@ -370,41 +371,77 @@ def run_ours(args):
         return
 
     peaks = measured_peaks()
-    # dominant kernel: gemm_tcgen05_kernel, six launches per step of equal algorithmic work
-    gemm_launches_per_step = 6
-    flops_per_launch = flops_step / gemm_launches_per_step
-    avg_launch_ms = ms_step / gemm_launches_per_step        # includes launch gaps: a lower bound on the rate
+    # ---- the dominant kernel, launch by launch: the six contractions of a step timed one at a time (CUDA events
+    # on the launching stream, 50 back-to-back repeats each), next to torch.matmul on the same shapes
+    per_contraction, avg_launch_ms = None, ms_step / 6
+    if world == 1:
+        dhp = torch.empty(B, L, F, dtype=torch.bfloat16, device="cuda")
+        ndhp = mtf.named(dhp, hn)
+        calls = {
+            "h = relu(x.w + bias)": (lambda: mtf.mtf_einsum(lay, None, [N["x"], N["w"]], N["h"], mtf.Epilogue(relu=True, bias=N["bias"]), workspace=ws), (T, F, D)),
+            "y = h.v": (lambda: mtf.mtf_einsum(lay, None, [N["h"], N["v"]], N["y"], None, workspace=ws), (T, D, F)),
+            "dhp = (dy.v^T)*[h>0], dbias": (lambda: mtf.mtf_einsum(lay, None, [N["dy"], N["v"]], ndhp, mtf.Epilogue(relu_mask=N["h"], reduce_sum_out=N["dbias"]), workspace=ws), (T, F, D)),
+            "dv = h^T.dy": (lambda: mtf.mtf_einsum(lay, None, [N["h"], N["dy"]], N["dv"], None, workspace=ws), (F, D, T)),
+            "dw = x^T.dhp": (lambda: mtf.mtf_einsum(lay, None, [N["x"], ndhp], N["dw"], None, workspace=ws), (D, F, T)),
+            "dx = dhp.w^T": (lambda: mtf.mtf_einsum(lay, None, [ndhp, N["w"]], N["dx"], None, workspace=ws), (T, D, F)),
+        }
+        x2, dy2, h2, dhp2 = t["x"].view(T, D), t["dy"].view(T, D), h.view(T, F), dhp.view(T, F)
+        o_tf, o_td = torch.empty(T, F, dtype=torch.bfloat16, device="cuda"), torch.empty(T, D, dtype=torch.bfloat16, device="cuda")
+        o_fd, o_df = torch.empty(F, D, dtype=torch.bfloat16, device="cuda"), torch.empty(D, F, dtype=torch.bfloat16, device="cuda")
+        lib = {
+            "h = relu(x.w + bias)": lambda: torch.matmul(x2, t["w"], out=o_tf), "y = h.v": lambda: torch.matmul(h2, t["v"], out=o_td),
+            "dhp = (dy.v^T)*[h>0], dbias": lambda: torch.matmul(dy2, t["v"].t(), out=o_tf), "dv = h^T.dy": lambda: torch.matmul(h2.t(), dy2, out=o_fd),
+            "dw = x^T.dhp": lambda: torch.matmul(x2.t(), dhp2, out=o_df), "dx = dhp.w^T": lambda: torch.matmul(dhp2, t["w"].t(), out=o_td),
+        }
+        per_contraction = {}
+        for name, (fn, (m_, n_, k_)) in calls.items():
+            ms_c = event_time(fn, 50, stream)
+            ms_l = event_time(lib[name], 50, stream)
+            per_contraction[name] = {"ms": ms_c, "tflops": 2.0 * m_ * n_ * k_ / (ms_c * 1e-3) / 1e12, "torch_matmul_ms": ms_l,
+                                     "ratio_to_torch_matmul": ms_c / ms_l, "m_n_k": [m_, n_, k_]}
+        avg_launch_ms = sum(c["ms"] for c in per_contraction.values()) / len(per_contraction)
+        mtf.mtf_device_status()
+    flops_per_launch = flops_step / 6
     achieved = flops_per_launch / (avg_launch_ms * 1e-3) / 1e12
-    # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the six launches of a step,
-    # from the full-size ncu capture summarised in profiles/gemm_tcgen05_ffn_target_fullsize.md
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH if (T, D, F) == (8192, 1024, 8192) else None
-    roofline = {"bound": "tensor", "kernel": "gemm_tcgen05_kernel", "achieved": achieved, "peak": peaks["bf16_sustained"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16_sustained"], "traffic": traffic,
-                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "frac_of_datasheet_2250": achieved / 2250.0,
-                "frac_of_measured_burst": achieved / peaks["bf16_burst"], "flops_per_launch": flops_per_launch,
-                "avg_launch_ms": avg_launch_ms}
 
     # which way the sums over a split reduced dimension were realised (Section 6: the Allreduce of the
     # mesh group) in the contractions of this layout that have one, and the workspace they moved
     mode_name = {0: "none", 1: "chained in the accumulator", 2: "fp32 fragments in the workspace"}
-    hname = ["batch", "length", "d_ff"]
     dsc = lambda t_, names: mtf.desc(list(zip(names, t_.shape)), "bf16" if t_.dtype == torch.bfloat16 else "f32")
     group_sums = {}
-    for tag, ins, out in (("y", [(h, hname), (t["v"], vn)], (y, act)), ("dx", [(h, hname), (t["w"], wn)], (dx, act)),
-                          ("dw", [(t["x"], act), (h, hname)], (dw, wn)), ("dv", [(h, hname), (t["dy"], act)], (dv, vn))):
+    for tag, ins, out in (("y", [(h, hn), (t["v"], vn)], (y, act)), ("dx", [(h, hn), (t["w"], wn)], (dx, act)),
+                          ("dw", [(t["x"], act), (h, hn)], (dw, wn)), ("dv", [(h, hn), (t["dy"], act)], (dv, vn))):
         plan = mtf.mtf_einsum_plan(lay, [dsc(a_, n_) for a_, n_ in ins], dsc(*out))
         info = mtf.mtf_plan_info(plan)
-        if info["group_size"] > 1:
+        if info["group_size"] > 1 or mtf.mtf_plan_needs_rank_sum(plan):
             group_sums[tag] = {"group_size": info["group_size"], "mode": mode_name.get(info["reduce_mode"], str(info["reduce_mode"])),
-                               "workspace_bytes": mtf.mtf_plan_workspace_bytes(plan) if info["reduce_mode"] == 2 else 0}
+                               "workspace_bytes": mtf.mtf_plan_workspace_bytes(plan) if info["reduce_mode"] == 2 else 0,
+                               "summed_across_ranks": bool(mtf.mtf_plan_needs_rank_sum(plan) & 1)}
 
     # the same step back to back for two seconds: the rate the GPU settles at under its power limit
     sustained = None
     if world == 1 and not args.no_sustained:
         n_sus = max(int(2000.0 / ms_step), 50)
         ms_sus, _, clocks_sus = timed(lay, n_sus, 3, ClockSampler(physical_gpu_index(local_rank)))
-        sustained = {"ms_per_step": ms_sus, "value": flops_step / (ms_sus * 1e-3) / 1e12, "unit": UNIT, "steps": n_sus,
-                     "sm_mhz": clocks_sus.get("sm_mhz") if clocks_sus else None, "reasons": clocks_sus.get("reasons") if clocks_sus else None}
+        v_sus = flops_step / (ms_sus * 1e-3) / 1e12
+        sustained = {"ms_per_step": ms_sus, "value": v_sus, "unit": UNIT, "steps": n_sus,
+                     "sm_mhz": clocks_sus.get("sm_mhz") if clocks_sus else None, "reasons": clocks_sus.get("reasons") if clocks_sus else None,
+                     "peak": peaks["bf16_sustained"], "frac": v_sus / peaks["bf16_sustained"], "frac_of_datasheet_2250": v_sus / 2250.0,
+                     "note": "whole steps (launch gaps included) against the sustained torch.matmul rate: both seconds long, both under the power cap"}
+
+    # roofline of the dominant kernel: like for like.  A timed region under a second runs at the boost clock and
+    # is held against the burst peak (best-of-10 torch.matmul); seconds-long regions against the sustained peak.
+    region_s = ms_step * args.steps * 1e-3
+    regime = "sustained" if region_s >= 1.0 else "burst"
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH if (T, D, F) == (8192, 1024, 8192) else None
+    peak = peaks["bf16_sustained"] if regime == "sustained" else peaks["bf16_burst"]
+    roofline = {"bound": "tensor", "kernel": "gemm_tcgen05_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "traffic": traffic, "traffic_captured_at_commit": NCU_TRAFFIC_COMMIT, "regime": regime,
+                "peak_source": f"bf16_tflops{'_sustained' if regime == 'sustained' else ''} of MEASURED_PEAKS.json ({peaks['source']})",
+                "frac_of_datasheet_2250": achieved / 2250.0, "flops_per_launch": flops_per_launch, "avg_launch_ms": avg_launch_ms,
+                "avg_launch_ms_note": "mean of the six contractions timed one at a time (50 repeats each)" if per_contraction else "step time / 6",
+                "step_ms_over_6_launches": ms_step / 6, "per_contraction": per_contraction,
+                "sustained_regime": {"achieved": sustained["value"], "peak": peaks["bf16_sustained"], "frac": sustained["frac"]} if sustained else None}
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -414,57 +451,71 @@ def run_ours(args):
         cpu = {"value": tf, "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"ffn fwd+bwd on {tokens} of {T} tokens (full d_model, d_ff), fp64 loop nest, {dt:.1f} s"}
 
+    secondary = None
+    if world == 1 and not args.no_secondary:
+        del sets, hx, hdy, hy, hdx
+        torch.cuda.empty_cache()
+        secondary = run_secondary(mtf, peaks)
+
+    multi = "single GPU"
+    if world > 1:
+        multi = ("batch -> ranks (mesh dimension 'gpus'); dw, dv, dbias summed over ranks with NCCL, each started behind its contraction" if args.split == "dp"
+                 else "d_ff -> ranks (mesh dimension 'gpus'); y and dx summed over ranks with NCCL behind their contractions")
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
             "config": {"workload": f"transformer_ffn_fwd_bwd tokens={T} (batch {B} x length {L}) d_model={D} d_ff={F} per GPU",
                        "layout": args.layout, "mesh": LAYOUTS[args.layout][0], "rules": LAYOUTS[args.layout][1],
                        "grad_dtype": "f32", "l2": "inputs larger than L2 (working set ~0.6 GB per step), no flush",
-                       "multi_gpu": "batch split over ranks; NCCL all-reduce of dw, dv, dbias each step" if world > 1 else "single GPU"},
+                       "library": os.path.basename(mtf.binding.LIB_PATH), "multi_gpu": multi},
             "clocks": clocks, "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * act_bytes,
                                       "d2h_bytes_per_step": 2 * act_bytes, "ms_per_step": e2e_ms},
             "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu, "per_layout_tflops": per_layout,
             "group_sums": group_sums, "sustained_2s": sustained,
-            "frac_of_datasheet_bf16_peak": value / world / 2250.0}
+            "frac_of_datasheet_bf16_peak": value / world / 2250.0, "secondary": secondary}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
 
 # ------------------------------------------------------------------------------------------------------
-# secondary workloads (not the headline line): attention block (config 3) and decoder layer (config 5)
+# secondary workloads (records inside the headline line): attention block (config 3), decoder layer (config 5)
+# and the memory-bound kernels, on seeded inputs
 # ------------------------------------------------------------------------------------------------------
 
-def run_block(args):
-    """Times mtf_attention_* (config 3: batch 16, length 512, d_model 1024, 16 heads of 64, mesh [4,4]) or
-    mtf_decoder_layer_* (config 5: batch 64, length 256, d_model 2048, 32 heads, d_ff 8192, mesh [4,8],
-    causal) forward + backward on one GPU and prints one JSON line (random bf16 inputs made on the
-    device: this leg measures time only, parity is the tests' job)."""
+def block_case(seed, dec, B=None):
+    """Seeded inputs of config 3 (attention: batch 16, length 512, d_model 1024, 16 heads of 64) or config 5
+    (decoder layer: batch 64, length 256, d_model 2048, 32 heads of 64, d_ff 8192): name -> (Stored, dim names)."""
+    import seeded_inputs as si
+    B0, L, D, H, K, F = (64, 256, 2048, 32, 64, 8192) if dec else (16, 512, 1024, 16, 64, 0)
+    B = B or B0
+    act = ["batch", "length", "d_model"]
+    T = {"x": (si.normal(seed, "x", [B, L, D], "bf16"), act), "dout": (si.normal(seed, "dy", [B, L, D], "bf16"), act),
+         "wq": (si.normal(seed, "wq", [D, H, K], "bf16", D ** -0.5), ["d_model", "heads", "d_k"]),
+         "wk": (si.normal(seed, "wk", [D, H, K], "bf16", D ** -0.5), ["d_model", "heads", "d_k"]),
+         "wv": (si.normal(seed, "wv", [D, H, K], "bf16", D ** -0.5), ["d_model", "heads", "d_v"]),
+         "wo": (si.normal(seed, "wo", [H, K, D], "bf16", (H * K) ** -0.5), ["heads", "d_v", "d_model"])}
+    if dec:
+        T.update({"w": (si.normal(seed, "w", [D, F], "bf16", D ** -0.5), ["d_model", "d_ff"]),
+                  "v": (si.normal(seed, "v", [F, D], "bf16", F ** -0.5), ["d_ff", "d_model"]),
+                  "bias": (si.normal(seed, "bias", [F], "f32", 0.1), ["d_ff"])})
+        for n, shift in (("ln1_gamma", 1.0), ("ln1_beta", 0.0), ("ln2_gamma", 1.0), ("ln2_beta", 0.0)):
+            T[n] = (si.normal(seed, n, [D], "f32", 0.1, shift), ["d_model"])
+    return T, (B, L, D, H, K, F)
+
+
+def block_step(mtf, dec, B=None):
+    """Builds the step function of the attention block (config 3) or the decoder layer (config 5) on seeded inputs.
+    Returns (step, flops per step, description, tensors kept alive)."""
     import torch
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
-    import paper_1811_02084_b200 as mtf
-    torch.manual_seed(0)
     bf, f32 = torch.bfloat16, torch.float32
-    dec = args.workload == "decoder"
-    B, L, D, H, K, F = (64, 256, 2048, 32, 64, 8192) if dec else (16, 512, 1024, 16, 64, 0)
-    if args.batch != WORKLOAD["batch"]:
-        B = args.batch
+    host, (B, L, D, H, K, F) = block_case(0, dec, B)
     mesh, rules = ([("rows", 4), ("cols", 8)], [("batch", "rows"), ("heads", "cols"), ("d_ff", "cols")]) if dec else \
                   ([("rows", 4), ("cols", 4)], [("batch", "rows"), ("heads", "cols")])
     lay = mtf.mtf_layout(mtf.mtf_mesh_create(mesh), rules)
-    rn = lambda shape, scale, dt=bf: (torch.randn(*shape, device="cuda") * scale).to(dt)
     act = ["batch", "length", "d_model"]
-    T = {"x": (rn((B, L, D), 1.0), act), "dout": (rn((B, L, D), 1.0), act),
-         "wq": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_k"]), "wk": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_k"]),
-         "wv": (rn((D, H, K), D ** -0.5), ["d_model", "heads", "d_v"]), "wo": (rn((H, K, D), (H * K) ** -0.5), ["heads", "d_v", "d_model"])}
-    if dec:
-        T.update({"w": (rn((D, F), D ** -0.5), ["d_model", "d_ff"]), "v": (rn((F, D), F ** -0.5), ["d_ff", "d_model"]),
-                  "bias": (rn((F,), 0.1, f32), ["d_ff"])})
-        for n in ("ln1_gamma", "ln2_gamma"):
-            T[n] = (1.0 + rn((D,), 0.1, f32), ["d_model"])
-        for n in ("ln1_beta", "ln2_beta"):
-            T[n] = (rn((D,), 0.1, f32), ["d_model"])
-    N = {k: mtf.named(t, names) for k, (t, names) in T.items()}
+    T = {k: (to_device(s), names) for k, (s, names) in host.items()}
+    N = {k: mtf.named(t_, names) for k, (t_, names) in T.items()}
     m = "memory_length"
     sd = {"q": ((B, L, H, K), ["batch", "length", "heads", "d_k"]), "kk": ((B, L, H, K), ["batch", m, "heads", "d_k"]),
           "vv": ((B, L, H, K), ["batch", m, "heads", "d_v"]), "weights": ((B, H, L, L), ["batch", "heads", "length", m]),
@@ -499,25 +550,88 @@ def run_block(args):
                                       mtf.named(out, act), ws)
             mtf.mtf_attention_backward(lay, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], S["q"], S["kk"], S["vv"], S["weights"], S["o"], N["dout"], None,
                                        mtf.named(dx, act), G["dwq"], G["dwk"], G["dwv"], G["dwo"], ws)
+    desc = {"workload": ("decoder layer, config 5" if dec else "attention block, config 3") + f": batch={B} length={L} d_model={D} heads={H} d_k={K}" + (f" d_ff={F} causal" if dec else ""),
+            "mesh": mesh, "rules": rules, "flops_per_step": flops,
+            "flops_note": "dense-equivalent contraction flops (projections, attention core, FFN), 2 per multiply-add, forward + backward = 3x forward"}
+    return step, flops, desc, (T, keep, gt, out, dx, ws, lay)
+
+
+def run_secondary(mtf, peaks):
+    """Records for the other workloads and for the memory-bound kernels, each timed with CUDA events on seeded inputs."""
+    import torch
+    import seeded_inputs as si
+    stream = torch.cuda.current_stream()
+    out = []
+    for dec in (False, True):
+        step, flops, desc, keep = block_step(mtf, dec)
+        ms = event_time(step, 20, stream, warmup=3)
+        mtf.mtf_device_status()
+        tf = flops / (ms * 1e-3) / 1e12
+        out.append({"metric": "transformer_" + ("decoder_layer" if dec else "attention") + "_fwd_bwd_tflops", "value": tf, "unit": UNIT, "ms_per_step": ms,
+                    "dtype": "bf16", "data": "synthetic (seeded)", "config": desc,
+                    "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_burst"], "frac": tf / peaks["bf16_burst"], "unit": "TFLOP/s",
+                                 "note": "whole block (contractions + row kernels) against the burst torch.matmul rate; timed region well under a second"}})
+        del step, keep
+        torch.cuda.empty_cache()
+    # memory-bound kernels at the shapes of config 5 (layer norm rows of 2048) and config 3 (softmax rows of 512)
+    lay = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 8)]), [("batch", "all")])
+    B, L, D = 64, 256, 2048
+    x, dy = to_device(si.normal(5, "x", [B, L, D], "bf16")), to_device(si.normal(5, "dy", [B, L, D], "bf16"))
+    g, b = to_device(si.normal(5, "g", [D], "f32", 0.1, 1.0)), to_device(si.normal(5, "b", [D], "f32", 0.1))
+    yb, dxb = torch.empty_like(x), torch.empty_like(x)
+    stats = torch.empty(B, L, 2, dtype=torch.float32, device="cuda")
+    dg, db = torch.empty_like(g), torch.empty_like(b)
+    act = ["batch", "length", "d_model"]
+    Nn = mtf.named
+    rows = []
+    ms = event_time(lambda: mtf.mtf_layernorm_forward(lay, Nn(x, act), Nn(g, ["d_model"]), Nn(b, ["d_model"]), 1e-6, Nn(yb, act), Nn(stats, ["batch", "length", "stat"])), 50, stream)
+    rows.append(("layernorm_fwd_rows_kernel", f"{B * L} rows of {D}", 2 * x.numel() * 2, ms))
+    ms = event_time(lambda: mtf.mtf_layernorm_backward(lay, Nn(dy, act), Nn(x, act), Nn(stats, ["batch", "length", "stat"]), Nn(g, ["d_model"]), None, Nn(dxb, act),
+                                                       Nn(dg, ["d_model"]), Nn(db, ["d_model"])), 50, stream)
+    rows.append(("layernorm_bwd_rows_kernel", f"{B * L} rows of {D}", 3 * x.numel() * 2, ms))
+    Bs, H, Ls = 16, 16, 512
+    names = ["batch", "heads", "length", "memory_length"]
+    lg = to_device(si.normal(6, "lg", [Bs, H, Ls, Ls], "f32", 2.0))
+    dP = to_device(si.normal(6, "dP", [Bs, H, Ls, Ls], "f32"))
+    Pw, dlg = torch.empty(Bs, H, Ls, Ls, dtype=torch.bfloat16, device="cuda"), torch.empty(Bs, H, Ls, Ls, dtype=torch.bfloat16, device="cuda")
+    ms = event_time(lambda: mtf.mtf_softmax_forward(lay, Nn(lg, names), False, Nn(Pw, names)), 50, stream)
+    rows.append(("softmax_fwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (4 + 2), ms))
+    ms = event_time(lambda: mtf.mtf_softmax_backward(lay, Nn(Pw, names), Nn(dP, names), Nn(dlg, names)), 50, stream)
+    rows.append(("softmax_bwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (2 + 4 + 2), ms))
+    mtf.mtf_device_status()
+    for kernel, shape, nbytes, ms in rows:
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out.append({"metric": "row_kernel_gbs", "kernel": kernel, "value": gbs, "unit": "GB/s", "ms": ms, "config": {"workload": shape},
+                    "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "frac": gbs / peaks["hbm_gbs"], "unit": "GB/s",
+                                 "algorithmic_bytes": nbytes, "note": "read every input once, write every output once; inputs larger than L2"}})
+    return out
+
+
+def run_block(args):
+    """Times mtf_attention_* (config 3) or mtf_decoder_layer_* (config 5) forward + backward on one GPU, on seeded
+    inputs, and prints one JSON line (this leg measures time only, parity is the tests' job)."""
+    import torch
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    import paper_1811_02084_b200 as mtf
+    dec = args.workload == "decoder"
+    step, flops, desc, keep = block_step(mtf, dec, args.batch if args.batch != 32 else None)
+    stream = torch.cuda.current_stream()
+    n0 = None
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     n0 = mtf.mtf_launch_count()
-    e0.record()
+    e0.record(stream)
     for _ in range(args.steps):
         step()
-    e1.record()
+    e1.record(stream)
     torch.cuda.synchronize()
     mtf.mtf_device_status()
     ms = e0.elapsed_time(e1) / args.steps
     print(json.dumps({"metric": f"transformer_{args.workload}_fwd_bwd_tflops", "value": flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": 1,
                       "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16",
-                      "data": "synthetic", "gpu_launches": mtf.mtf_launch_count() - n0,
-                      "config": {"workload": f"{args.workload} batch={B} length={L} d_model={D} heads={H} d_k={K}" + (f" d_ff={F} causal" if dec else ""),
-                                 "mesh": mesh, "rules": rules, "flops_per_step": flops,
-                                 "flops_note": "dense-equivalent contraction flops (projections, attention core, FFN), 2 per multiply-add, forward + backward = 3x forward"}}),
-          flush=True)
+                      "data": "synthetic (seeded)", "gpu_launches": mtf.mtf_launch_count() - n0, "config": desc}), flush=True)
 
 
 def main():
@@ -527,8 +641,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layout", default="mp8", choices=sorted(LAYOUTS))
+    ap.add_argument("--split", default="dp", choices=["dp", "mp"], help="with N > 1 GPUs: which dimension the rank-spanning mesh dimension takes (dp: batch, mp: d_ff)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the extra two-second back-to-back run")
+    ap.add_argument("--no-secondary", action="store_true", help="skip the records of the other workloads and of the memory-bound kernels")
     ap.add_argument("--d-ff", type=int, default=WORKLOAD["d_ff"], help="4096 = config 2, 65536 (with --layout mp16) = config 4")
     ap.add_argument("--batch", type=int, default=WORKLOAD["batch"], help="sequences of 256 tokens per GPU (smaller only for profiler captures)")
     ap.add_argument("--main-only", action="store_true", help="skip the per-layout table and the end-to-end leg (profiler captures)")
