@@ -12,6 +12,9 @@ Contents
   blocks.py       feed-forward, attention, layer norm, decoder layer - forward and backward
   stages.py       the same blocks one launch at a time (an einsum plus its fused component-wise stages, or a row reduction)
   cost.py         per-processor cost counts (Table 1, Appendix B)
+  chooser.py      exhaustive search for the cheapest legal layout under those counts (Section 11's future work)
+  update.py       Algorithm 1 line 3: the parameter update (reading: SGD with momentum and weight decay)
+  vocab.py        embedding, logits einsum and softmax cross-entropy over a (split) vocab dimension
   rounding.py     the one rounding step applied where the method stores an intermediate in bf16
 
 Pins (tests that tie each part to something other than itself) are listed in the test files named
@@ -22,7 +25,7 @@ from .named import (NT, DenseOps, DuplicateDim, IllegalLayout, NotDivisible, Ora
                     UnknownDim, einsum_arrays)
 from .mesh import Layout, Mesh
 from .lowering import LT, LoweredOps
-from . import blocks, cost, rounding, stages
+from . import blocks, chooser, cost, rounding, stages, update, vocab
 
 __all__ = ["NT", "DenseOps", "LoweredOps", "LT", "Mesh", "Layout", "blocks", "stages", "cost", "einsum_arrays",
            "OracleError", "DuplicateDim", "UnknownDim", "SizeMismatch", "IllegalLayout", "NotDivisible"]

@@ -163,8 +163,60 @@ class LoweredOps:
         return self._reduce(x, out_names, "reduce_max", np.maximum)
 
     def rename(self, x, old, new):
-        """Rename one dimension.  Only the communication-free case is simulated: the old and the
-        new name must be split the same way (otherwise it is the re-layout of Section 6.1)."""
-        if self.layout.mesh_dim_of(old) != self.layout.mesh_dim_of(new):
-            raise OracleError("rename would change the layout (reshape with communication): not simulated")
-        return LT([(new if n == old else n, s) for n, s in x.dims], x.slices)
+        """Rename one dimension: the reshape of Section 6.1 with one name changed."""
+        return self.reshape(x, [new if n == old else n for n in x.names])
+
+    def reshape(self, x, out_names):
+        """Reshape that keeps the sizes and changes dimension names (Section 6.1), hence possibly the
+        layout.  Per mesh dimension the paper names three patterns:
+          * a tensor dimension split over it in the input but none in the output: Allgather over that
+            mesh dimension (every member of the group ends with the concatenation, in coordinate order);
+          * none in the input, one in the output: no communication, each processor keeps its stripe;
+          * different tensor dimensions in input and output: Alltoall over that mesh dimension (here
+            carried out as its definition: gather the group's blocks, keep the own stripe of the other
+            dimension; the elements a processor receives are counted as an Alltoall's).
+        All gathers run before all slicing, so that every step acts on whole stripes.
+        ``reshape_log`` receives (mesh-dim index, pattern, elements received per processor)."""
+        in_dims = x.dims
+        if len(out_names) != len(in_dims):
+            raise SizeMismatch("reshape keeps the number and the sizes of the dimensions")
+        out_dims = tuple((n, s) for n, (_, s) in zip(out_names, in_dims))
+        tl_in = {j: i for i, j in self.layout.tensor_layout(in_dims).items()}        # mesh dim -> position
+        tl_out = {j: i for i, j in self.layout.tensor_layout(out_dims).items()}
+        slices = [s.copy() for s in x.slices]
+        self.reshape_log = getattr(self, "reshape_log", [])
+        changed = [j for j in range(len(self.mesh.shape)) if tl_in.get(j) != tl_out.get(j)]
+        for j in changed:                                   # gathers
+            if j not in tl_in:
+                continue
+            pos, m = tl_in[j], self.mesh.shape[j]
+            local = int(slices[0].size)
+            gathered = []
+            for p in range(self.mesh.P):
+                grp = self.mesh.group(p, {j})               # ascending processor order = ascending coordinate j
+                gathered.append(np.concatenate([slices[q] for q in grp], axis=pos))
+            slices = gathered
+            if j in tl_out:                                 # an Alltoall keeps 1/m of what the gather brought
+                self.reshape_log.append((j, "alltoall", local * (m - 1) // m))
+            else:
+                self.reshape_log.append((j, "allgather", local * (m - 1)))
+        for j in changed:                                   # local slicing
+            if j not in tl_out:
+                continue
+            pos, m = tl_out[j], self.mesh.shape[j]
+            kept = []
+            for p in range(self.mesh.P):
+                c = self.mesh.coords(p)[j]
+                t = slices[p].shape[pos] // m
+                idx = [slice(None)] * slices[p].ndim
+                idx[pos] = slice(c * t, (c + 1) * t)
+                kept.append(np.require(slices[p][tuple(idx)], requirements="C").copy())
+            slices = kept
+            if j not in tl_in:
+                self.reshape_log.append((j, "slice", 0))
+        return LT(out_dims, slices)
+
+    def transpose(self, x, out_names):
+        """Same dimensions in another storage order: purely local (the layout goes by names)."""
+        perm = [x.names.index(n) for n in out_names]
+        return LT([x.dims[i] for i in perm], [np.require(np.transpose(s, perm), requirements="C").copy() for s in x.slices])

@@ -200,6 +200,15 @@ class DenseOps:
         """Same data, one dimension renamed (a reshape that changes only a name)."""
         return NT([(new if n == old else n, s) for n, s in x.dims], x.a)
 
+    def reshape(self, x, out_names):
+        """Same data, dimensions renamed position by position (sizes kept)."""
+        return NT([(n, s) for n, (_, s) in zip(out_names, x.dims)], x.a)
+
+    def transpose(self, x, out_names):
+        """Same dimensions in another storage order."""
+        perm = [x.names.index(n) for n in out_names]
+        return NT([x.dims[i] for i in perm], np.transpose(x.a, perm))
+
     def to_global(self, x):
         return x
 
