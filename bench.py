@@ -29,6 +29,10 @@ LAYOUTS = {
     "dp8": ([("all", 8)], [("batch", "all")]),
     "mp8": ([("all", 8)], [("d_ff", "all")]),
     "mp16": ([("all", 16)], [("d_ff", "all")]),
+    # Section 8.3: the two-dimensional layout (batch over rows, hidden over columns) and the three-dimensional one
+    # (additionally the input / output dimension over planes: every matrix tiled over two mesh dimensions)
+    "2d": ([("rows", 2), ("cols", 4)], [("batch", "rows"), ("d_ff", "cols")]),
+    "3d": ([("rows", 2), ("cols", 2), ("planes", 2)], [("batch", "rows"), ("d_ff", "cols"), ("d_model", "planes")]),
 }
 # dram__bytes_read.sum + dram__bytes_write.sum per contraction launch, averaged over the six launches of a
 # step of this workload (one ncu capture; the summary under profiles/ names the command and the commit)
@@ -598,6 +602,69 @@ def run_secondary(mtf, peaks):
     rows.append(("softmax_fwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (4 + 2), ms))
     ms = event_time(lambda: mtf.mtf_softmax_backward(lay, Nn(Pw, names), Nn(dP, names), Nn(dlg, names)), 50, stream)
     rows.append(("softmax_bwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (2 + 4 + 2), ms))
+    mtf.mtf_device_status()
+    # ---- the vocab dimension: embedding + logits + cross-entropy, forward and backward, vocab 32768, d_model 1024, tokens 8192
+    import numpy as np
+    Bv, Lv, Dv, V = 32, 256, 1024, 32768
+    Tv = Bv * Lv
+    layv = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 8)]), [("vocab", "all")])
+    rng = np.random.RandomState(7)
+    ids = torch.from_numpy(rng.randint(0, V, size=(Bv, Lv)).astype(np.int32)).cuda()
+    tgt = torch.from_numpy(rng.randint(0, V, size=(Bv, Lv)).astype(np.int32)).cuda()
+    E, Wo = to_device(si.normal(7, "E", [V, Dv], "bf16")), to_device(si.normal(7, "wout", [Dv, V], "bf16", Dv ** -0.5))
+    xv, lgt = torch.empty(Bv, Lv, Dv, dtype=torch.bfloat16, device="cuda"), torch.empty(Bv, Lv, V, dtype=torch.bfloat16, device="cuda")
+    lse, loss = torch.empty(Bv, Lv, dtype=torch.float32, device="cuda"), torch.empty(Bv, Lv, dtype=torch.float32, device="cuda")
+    dls = torch.full((Bv, Lv), 1.0 / Tv, dtype=torch.float32, device="cuda")
+    dhv, dWo, dE = torch.empty_like(xv), torch.empty(Dv, V, dtype=torch.float32, device="cuda"), torch.empty(V, Dv, dtype=torch.float32, device="cuda")
+    wsv = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    av, lv, tl = ["batch", "length", "d_model"], ["batch", "length", "vocab"], ["batch", "length"]
+
+    def vocab_step():
+        mtf.mtf_embedding_forward(layv, ids, Nn(E, ["vocab", "d_model"]), Nn(xv, av))
+        mtf.mtf_xent_forward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), wsv)
+        mtf.mtf_xent_backward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(dls, tl), Nn(dhv, av), Nn(dWo, ["d_model", "vocab"]), wsv)
+        mtf.mtf_embedding_backward(layv, ids, Nn(dhv, av), Nn(dE, ["vocab", "d_model"]))
+
+    ms = event_time(vocab_step, 10, stream)
+    mtf.mtf_device_status()
+    vflops = 6.0 * Tv * Dv * V
+    tf = vflops / (ms * 1e-3) / 1e12
+    out.append({"metric": "vocab_embedding_logits_xent_fwd_bwd_tflops", "value": tf, "unit": UNIT, "ms_per_step": ms, "dtype": "bf16", "data": "synthetic (seeded)",
+                "config": {"workload": f"embedding + logits + softmax cross-entropy, fwd+bwd: tokens={Tv} d_model={Dv} vocab={V}", "mesh": [["all", 8]],
+                           "rules": [["vocab", "all"]], "flops_per_step": vflops, "flops_note": "three contractions of 2 tokens d_model vocab"},
+                "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_burst"], "frac": tf / peaks["bf16_burst"], "unit": "TFLOP/s",
+                             "note": "whole step (3 contractions + 4 memory-bound kernels) against the burst torch.matmul rate"}})
+    # the memory-bound kernels of that step, each alone
+    ms = event_time(lambda: mtf.mtf_embedding_forward(layv, ids, Nn(E, ["vocab", "d_model"]), Nn(xv, av)), 50, stream)
+    rows.append(("embedding_gather_kernel", f"{Tv} rows of {Dv} (bf16) from a table of {V} rows", 2 * Tv * Dv * 2, ms))
+    mtf.mtf_xent_forward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), wsv)
+    ms = event_time(lambda: mtf.mtf_softmax_xent_forward(layv, Nn(lgt, lv), tgt, Nn(lse, tl), Nn(loss, tl)), 20, stream)
+    rows.append(("xent_rows_kernel", f"{Tv} rows of {V} (bf16 logits)", Tv * V * 2, ms))
+    ms = event_time(lambda: mtf.mtf_softmax_xent_backward(layv, Nn(lgt, lv), tgt, Nn(lse, tl), Nn(dls, tl)), 20, stream)
+    rows.append(("xent_backward_kernel", f"{Tv} rows of {V} (bf16, in place)", Tv * V * 4, ms))
+    del lgt, dWo, dE, E, Wo
+    torch.cuda.empty_cache()
+    # Algorithm 1 line 3 on the largest parameter of config 4 (d_model 1024 x d_ff 65536): momentum + weight decay + bf16 working copy
+    Dw, Fw = 1024, 65536
+    wm = to_device(si.normal(8, "w", [Dw, Fw], "f32", Dw ** -0.5))
+    gw = to_device(si.normal(8, "g", [Dw, Fw], "f32", 1e-3))
+    mo, wb16 = torch.zeros_like(wm), torch.empty(Dw, Fw, dtype=torch.bfloat16, device="cuda")
+    wn2 = ["d_model", "d_ff"]
+    layu = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 16)]), [("d_ff", "all")])
+    ms = event_time(lambda: mtf.mtf_update(layu, Nn(gw, wn2), Nn(wm, wn2), Nn(mo, wn2), Nn(wb16, wn2), 1e-3, 0.9, 0.01), 20, stream)
+    rows.append(("sgd_update_kernel", f"{Dw} x {Fw} f32 parameter with momentum and bf16 copy", Dw * Fw * 22, ms))
+    del wm, gw, mo, wb16
+    torch.cuda.empty_cache()
+    # Section 6.1: the block transpose between a batch split and a heads split, [batch, length, heads, d_k] -> [batch, heads, length, d_k]
+    Bt, Lt, Ht, Kt = 256, 256, 32, 64
+    qt = to_device(si.normal(9, "q", [Bt, Lt, Ht, Kt], "bf16"))
+    qo = torch.empty(Bt, Ht, Lt, Kt, dtype=torch.bfloat16, device="cuda")
+    ms = event_time(lambda: mtf.mtf_transpose(lay, Nn(qt, ["batch", "length", "heads", "d_k"]), Nn(qo, ["batch", "heads", "length", "d_k"])), 20, stream)
+    rows.append(("permute_copy_kernel", f"[{Bt}, {Lt}, {Ht}, {Kt}] bf16 -> [batch, heads, length, d_k]", 2 * qt.numel() * 2, ms))
+    xt2 = qt.view(Bt * Lt, Ht * Kt)
+    xo2 = qo.view(Ht * Kt, Bt * Lt)
+    ms = event_time(lambda: mtf.mtf_transpose(lay, Nn(xt2, ["tokens", "d_model"]), Nn(xo2, ["d_model", "tokens"])), 20, stream)
+    rows.append(("permute_transpose_kernel", f"[{Bt * Lt}, {Ht * Kt}] bf16 -> [d_model, tokens]", 2 * qt.numel() * 2, ms))
     mtf.mtf_device_status()
     for kernel, shape, nbytes, ms in rows:
         gbs = nbytes / (ms * 1e-3) / 1e9

@@ -340,6 +340,82 @@ mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tens
 mtf_status mtf_decoder_layer_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x,
                                              const mtf_decoder_params* params, size_t* bytes);
 
+/* ---- parameter update (Section 3, Algorithm 1 line 3: W(t+1) = Update(W(t), gradient)) -----------
+ * The paper leaves Update open.  This library's reading: stochastic gradient descent with optional
+ * momentum and decoupled weight decay on an f32 master copy, refreshing the bf16 working copy the
+ * contractions read, all in one memory-bound pass:
+ *     m <- momentum * m + g  (momentum tensor NULL: m = g);  W <- W - lr * (m + weight_decay * W);  Wb <- bf16(W)
+ * grad f32 or bf16; master f32 (updated in place); momentum f32 or NULL (updated in place; must be
+ * given when hp->momentum != 0); param bf16 or NULL.  All tensors have master's dims, are 16-byte
+ * aligned, device memory.  The update is component-wise (Section 6), hence local under every layout:
+ * each processor updates its own slice, which on one GPU is one pass over the stored tensor.  Under
+ * a rank-bound layout every rank updates its box after the gradients were summed across ranks. */
+typedef struct { float lr, momentum, weight_decay; } mtf_update_params;
+mtf_status mtf_update(const mtf_layout_t* layout, const mtf_tensor* grad, mtf_tensor* master, mtf_tensor* momentum, mtf_tensor* param,
+                      const mtf_update_params* hp, void* stream);
+
+/* ---- reshape and storage order (Section 6.1 "Reshape") ------------------------------------------------
+ * A reshape that keeps the sizes and changes dimension names changes the layout.  Per mesh dimension
+ * the paper names the communication it needs: a tensor dimension split over it before but none after
+ * = Allgather; none before, one after = local slicing; different tensor dimensions before and after
+ * = Alltoall.  On one GPU a tensor is stored once and slices are views, so such a reshape is a change
+ * of descriptor and moves no data; mtf_reshape_plan reports, for mesh dimension j, pattern[j] and the
+ * number of elements one processor would receive (host arrays of the mesh's ndim; all gathers are
+ * counted before any slicing, ascending mesh dimension).  Errors as mtf_layout_check_tensor, for the
+ * input and for the output dims. */
+typedef enum { MTF_RESHAPE_NONE = 0, MTF_RESHAPE_ALLGATHER = 1, MTF_RESHAPE_SLICE = 2, MTF_RESHAPE_ALLTOALL = 3 } mtf_reshape_pattern;
+mtf_status mtf_reshape_plan(const mtf_layout_t* layout, int32_t ndim, const mtf_dim* in_dims, const char* const* out_names, int32_t* pattern,
+                            int64_t* received_per_proc);
+/* What does move data on one GPU: a change of storage order.  out's dims are a permutation (by name)
+ * of in's; same dtype; device pointers; one launch, bound by HBM (each element read once, written
+ * once).  E.g. [batch, length, heads, d_k] -> [batch, heads, length, d_k], the block transpose an
+ * Alltoall between a batch split and a heads split performs. */
+mtf_status mtf_transpose(const mtf_layout_t* layout, const mtf_tensor* in, mtf_tensor* out, void* stream);
+/* Inverse of mtf_slice_gather: the dense row-major slice of `processor` (device, global's dtype) is
+ * written into its box of `global`.  (What an Allgather does with every processor's slice.) */
+mtf_status mtf_slice_scatter(const mtf_layout_t* layout, const void* slice, int64_t processor, mtf_tensor* global, void* stream);
+/* Layout search (Section 11 names it as future work; the cost model is Table 1's): over every
+ * assignment of the n_names candidate tensor dimensions to a mesh dimension or to none, legal for all
+ * n_einsums einsums in0[e] . in1[e] -> out[e] (descriptors; data ignored), minimise
+ *     sum_e  multiply-adds per processor + comm_weight * values entering an Allreduce per processor,
+ * ties going to the smaller sum of slice elements, then to the first assignment in enumeration order
+ * (first name slowest; unsplit, then mesh dimension 0, 1, ...).  chosen_mesh_dim[i] = index of the
+ * mesh dimension names[i] is split over, or -1.  MTF_ERR_ILLEGAL_LAYOUT when nothing is legal. Host only. */
+mtf_status mtf_layout_search(const mtf_mesh_t* mesh, int32_t n_einsums, const mtf_tensor* in0, const mtf_tensor* in1, const mtf_tensor* out,
+                             int32_t n_names, const char* const* names, double comm_weight, int32_t* chosen_mesh_dim, double* cost,
+                             int64_t* footprint);
+
+/* ---- the vocab dimension (Section 9: vocab, d_ff and heads are the split dimensions) ------------------
+ * Token ids and targets are device arrays of int32, one per token, values in [0, vocab); a value
+ * outside is skipped (zero row / zero loss) and reported by mtf_device_status as MTF_ERR_INVALID_ARG.
+ *   mtf_embedding_forward : x[t, :] = table[ids[t], :]   - the einsum onehot(ids) . table, which reduces
+ *       `vocab`; under a vocab split exactly one slice holds the row, and the table being stored once,
+ *       the group sum is a row lookup.  table [vocab, d], x [*tokens, d], same dtype (bf16 or f32).
+ *   mtf_embedding_backward: dtable[v, :] = sum over tokens with ids[t] = v of dx[t, :]  (f32, zeroed by
+ *       the call, fp32 atomics: order not fixed); summed across ranks when a token dim is split over them.
+ *   mtf_xent_forward      : logits[t, v] = sum_d h[t, d] wout[d, v] (bf16, through mtf_einsum under the
+ *       layout); per token lse = log sum_v exp(logits) - taken over the logits as stored, maximum
+ *       subtracted, the local reduction of every vocab slice and the combine over the group in one pass
+ *       (Section 6 "Reduction") - and loss = lse - logits[t, target[t]].  lse, loss: f32, one per token.
+ *   mtf_xent_backward     : dlogits = (exp(logits - lse) - onehot(target)) * dloss[t], written over
+ *       `logits`; dh = dlogits . wout^T (reduces vocab: the group sum of a vocab split);
+ *       dwout = h^T . dlogits (reduces the token dims).  dloss f32, one per token.
+ * A vocab dimension split across RANKS is refused (MTF_ERR_UNSUPPORTED): the row statistics would need
+ * a max / sum combine across ranks.  workspace: as for mtf_einsum. */
+mtf_status mtf_embedding_forward(const mtf_layout_t* layout, const int32_t* ids, const mtf_tensor* table, mtf_tensor* x, void* stream);
+mtf_status mtf_embedding_backward(const mtf_layout_t* layout, const int32_t* ids, const mtf_tensor* dx, mtf_tensor* dtable, void* stream);
+mtf_status mtf_xent_forward(const mtf_layout_t* layout, const mtf_tensor* h, const mtf_tensor* wout, const int32_t* targets, mtf_tensor* logits,
+                            mtf_tensor* lse, mtf_tensor* loss, void* workspace, size_t workspace_bytes, void* stream);
+/* The row parts of the two calls around this comment on their own, on logits that are already stored
+ * (bf16 [*tokens, vocab], vocab a multiple of 8): lse and loss per token; dlogits written over the logits. */
+mtf_status mtf_softmax_xent_forward(const mtf_layout_t* layout, const mtf_tensor* logits, const int32_t* targets, mtf_tensor* lse, mtf_tensor* loss,
+                                    void* stream);
+mtf_status mtf_softmax_xent_backward(const mtf_layout_t* layout, mtf_tensor* logits, const int32_t* targets, const mtf_tensor* lse,
+                                     const mtf_tensor* dloss, void* stream);
+mtf_status mtf_xent_backward(const mtf_layout_t* layout, const mtf_tensor* h, const mtf_tensor* wout, const int32_t* targets, mtf_tensor* logits,
+                             const mtf_tensor* lse, const mtf_tensor* dloss, mtf_tensor* dh, mtf_tensor* dwout, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
 /* ---- reductions (Section 6 "Reduction") --------------------------------------------------------- */
 /* out[out dims] = sum over the other dims of in (out dims a subset of in's).  Local reduction per
  * slice, then the group sum across the mesh dims of reduced-out split dims, in one launch. */
@@ -368,7 +444,8 @@ const char* mtf_status_string(mtf_status s);
 const char* mtf_last_error(void);
 /* Synchronises the current device and reads the sticky device status word: 0 = no kernel of this
  * library gave up on a bounded wait since the last call; non-zero = a code naming the wait.
- * Resets the word.  Returns MTF_ERR_TIMEOUT when it was non-zero. */
+ * Resets the word.  Returns MTF_ERR_TIMEOUT when it was non-zero, else MTF_ERR_INVALID_ARG when a
+ * token id or target outside [0, vocab) was seen by the vocab kernels since the last call. */
 mtf_status mtf_device_status(int32_t* code);
 /* Number of kernels this library has launched from this process (all threads). */
 int64_t mtf_launch_count(void);

@@ -78,6 +78,13 @@ RANK_ALLREDUCE_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p, c_int64, c_int, 
 RANK_WAIT_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p)                                    # (user, stream) -> status
 
 
+class mtf_update_params(Structure):
+    _fields_ = [("lr", c_float), ("momentum", c_float), ("weight_decay", c_float)]
+
+
+MTF_RESHAPE_NONE, MTF_RESHAPE_ALLGATHER, MTF_RESHAPE_SLICE, MTF_RESHAPE_ALLTOALL = 0, 1, 2, 3
+
+
 class MtfError(RuntimeError):
     def __init__(self, status: int, message: str):
         self.status = status
@@ -133,6 +140,19 @@ def _load():
         "mtf_rank_box": [vp, c_int32, POINTER(mtf_dim), POINTER(c_int64), POINTER(c_int64)],
         "mtf_plan_needs_rank_sum": [vp, POINTER(c_int32)],
         "mtf_rank_wait": [vp, vp],
+        "mtf_update": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_update_params), vp],
+        "mtf_reshape_plan": [vp, c_int32, POINTER(mtf_dim), POINTER(c_char_p), POINTER(c_int32), POINTER(c_int64)],
+        "mtf_transpose": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_slice_scatter": [vp, vp, c_int64, POINTER(mtf_tensor), vp],
+        "mtf_layout_search": [vp, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), c_int32, POINTER(c_char_p), ctypes.c_double,
+                              POINTER(c_int32), POINTER(ctypes.c_double), POINTER(c_int64)],
+        "mtf_embedding_forward": [vp, vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_embedding_backward": [vp, vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_softmax_xent_forward": [vp, POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_softmax_xent_backward": [vp, POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
+        "mtf_xent_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp, c_size_t, vp],
+        "mtf_xent_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor),
+                              POINTER(mtf_tensor), vp, c_size_t, vp],
         "mtf_stage_tap_begin": [vp, c_size_t],
         "mtf_stage_tap_end": [POINTER(c_int32)],
         "mtf_stage_tap_entry": [c_int32, POINTER(c_char_p), POINTER(c_size_t), POINTER(c_size_t)],
@@ -518,6 +538,70 @@ def mtf_decoder_layer_workspace_bytes(layout, x, params: dict) -> int:
     ps = _struct_of(mtf_decoder_params, params)
     _check(_lib.mtf_decoder_layer_workspace_bytes(layout.handle, _p(x), byref(ps), byref(b)))
     return b.value
+
+
+def mtf_update(layout, grad: Named, master: Named, momentum: Named | None, param: Named | None, lr: float, momentum_coef: float = 0.0,
+               weight_decay: float = 0.0, stream=None) -> None:
+    hp = mtf_update_params(float(lr), float(momentum_coef), float(weight_decay))
+    _check(_lib.mtf_update(layout.handle, _p(grad), _p(master), _p(momentum), _p(param), byref(hp), _stream(stream)))
+
+
+def mtf_reshape_plan(layout: Layout, in_dims, out_names):
+    """Per mesh dimension: (pattern code, elements one processor would receive)."""
+    arr, _keep = _dims_array(in_dims)
+    names = (c_char_p * max(len(out_names), 1))(*[n.encode() for n in out_names])
+    r = len(layout.mesh_dims)
+    pat, rec = (c_int32 * r)(), (c_int64 * r)()
+    _check(_lib.mtf_reshape_plan(layout.handle, len(in_dims), arr, names, pat, rec))
+    return list(pat), list(rec)
+
+
+def mtf_transpose(layout, inp: Named, out: Named, stream=None) -> None:
+    _check(_lib.mtf_transpose(layout.handle, _p(inp), _p(out), _stream(stream)))
+
+
+def mtf_slice_scatter(layout: Layout, slice_tensor, processor: int, glob: Named, stream=None) -> None:
+    _check(_lib.mtf_slice_scatter(layout.handle, c_void_p(slice_tensor.data_ptr()), processor, byref(glob.c), _stream(stream)))
+
+
+def mtf_layout_search(mesh: Mesh, einsums, names, comm_weight: float):
+    """einsums: [(in0, in1, out)] of descriptors.  Returns (rules, cost, footprint) of the cheapest legal layout."""
+    a0, a1, ao = _tensor_array([e[0] for e in einsums]), _tensor_array([e[1] for e in einsums]), _tensor_array([e[2] for e in einsums])
+    nm = (c_char_p * max(len(names), 1))(*[n.encode() for n in names])
+    chosen = (c_int32 * max(len(names), 1))()
+    cost, foot = ctypes.c_double(), c_int64()
+    _check(_lib.mtf_layout_search(mesh.handle, len(einsums), a0, a1, ao, len(names), nm, float(comm_weight), chosen, byref(cost), byref(foot)))
+    rules = [(n, mesh.dims[chosen[i]][0]) for i, n in enumerate(names) if chosen[i] >= 0]
+    return rules, cost.value, foot.value
+
+
+def mtf_embedding_forward(layout, ids, table: Named, x: Named, stream=None) -> None:
+    """ids: contiguous int32 device tensor, one id per token."""
+    _check(_lib.mtf_embedding_forward(layout.handle, c_void_p(ids.data_ptr()), _p(table), _p(x), _stream(stream)))
+
+
+def mtf_embedding_backward(layout, ids, dx: Named, dtable: Named, stream=None) -> None:
+    _check(_lib.mtf_embedding_backward(layout.handle, c_void_p(ids.data_ptr()), _p(dx), _p(dtable), _stream(stream)))
+
+
+def mtf_softmax_xent_forward(layout, logits: Named, targets, lse: Named, loss: Named, stream=None) -> None:
+    _check(_lib.mtf_softmax_xent_forward(layout.handle, _p(logits), c_void_p(targets.data_ptr()), _p(lse), _p(loss), _stream(stream)))
+
+
+def mtf_softmax_xent_backward(layout, logits: Named, targets, lse: Named, dloss: Named, stream=None) -> None:
+    _check(_lib.mtf_softmax_xent_backward(layout.handle, _p(logits), c_void_p(targets.data_ptr()), _p(lse), _p(dloss), _stream(stream)))
+
+
+def mtf_xent_forward(layout, h: Named, wout: Named, targets, logits: Named, lse: Named, loss: Named, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_xent_forward(layout.handle, _p(h), _p(wout), c_void_p(targets.data_ptr()), _p(logits), _p(lse), _p(loss), wp, wb, _stream(stream)))
+
+
+def mtf_xent_backward(layout, h: Named, wout: Named, targets, logits: Named, lse: Named, dloss: Named, dh: Named, dwout: Named, workspace=None,
+                      stream=None) -> None:
+    wp, wb = _ws(workspace)
+    _check(_lib.mtf_xent_backward(layout.handle, _p(h), _p(wout), c_void_p(targets.data_ptr()), _p(logits), _p(lse), _p(dloss), _p(dh), _p(dwout), wp, wb,
+                                  _stream(stream)))
 
 
 def mtf_status_string(status: int) -> str:

@@ -14,6 +14,7 @@ mtf_status ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, co
 const char* last_error();
 int64_t launch_count();
 mtf_status read_device_status(int* code);
+mtf_status read_bad_index(int* seen);
 }  // namespace mtf
 
 using mtf::Dim;
@@ -608,7 +609,11 @@ mtf_status mtf_device_status(int32_t* code) {
   int c = 0;
   mtf_status st = mtf::read_device_status(&c);
   if (code) *code = c;
-  return st;
+  if (st != MTF_OK) return st;
+  int bad = 0;
+  if ((st = mtf::read_bad_index(&bad)) != MTF_OK) return st;
+  if (bad) return fail(MTF_ERR_INVALID_ARG, "a token id or target outside [0, vocab) was seen by the vocab kernels");
+  return MTF_OK;
 }
 
 int64_t mtf_launch_count(void) { return mtf::launch_count(); }

@@ -240,6 +240,12 @@ static bool plan_tc(mtf_plan_t* P, std::string* why, int force_single_cta) {
   }
   for (int j = 0; j < t.n_outer; ++j)
     if (t.outer_sA[j] % 8 || t.outer_sB[j] % 8) { *why = "batch stride not 16-byte aligned"; return false; }
+  // A tensor-map copy must start on a 16-byte boundary along the contiguous dimension.  For an operand
+  // whose M / N dimension is the contiguous one the first column of a slice is a multiple of the slice
+  // extent, so that extent must be a multiple of 8 bf16 elements (k offsets are always multiples of a 64-element k-block:
+  // the slices of a split K are contiguous and walked as one range).
+  if (t.a_mn_major && t.sm > 1 && (t.M / t.sm) % 8) { *why = "M slices of an M-contiguous operand do not start on 16-byte boundaries"; return false; }
+  if (t.b_mn_major && t.sn > 1 && (t.N / t.sn) % 8) { *why = "N slices of an N-contiguous operand do not start on 16-byte boundaries"; return false; }
   // vectorised epilogue stores: rows of C must start 16-byte aligned
   int64_t cvec = P->dtC == MTF_BF16 ? 8 : 4;
   if (t.ldc % cvec) { *why = "output rows not 16-byte aligned"; return false; }

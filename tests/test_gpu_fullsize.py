@@ -65,7 +65,9 @@ FFN_CASES = {
     "config2": dict(batch=32, length=256, d_model=1024, d_ff=4096, nsplit=8,
                     layouts=[([("all", 1)], []), ([("all", 8)], [("batch", "all")]), ([("all", 8)], [("d_ff", "all")])]),
     "target": dict(batch=32, length=256, d_model=1024, d_ff=8192, nsplit=8,
-                   layouts=[([("all", 1)], []), ([("all", 8)], [("d_ff", "all")]), ([("all", 8)], [("batch", "all")])]),
+                   layouts=[([("all", 1)], []), ([("all", 8)], [("d_ff", "all")]), ([("all", 8)], [("batch", "all")]),
+                            ([("rows", 2), ("cols", 4)], [("batch", "rows"), ("d_ff", "cols")]),                                       # Section 8.3, two-dimensional
+                            ([("rows", 2), ("cols", 2), ("planes", 2)], [("batch", "rows"), ("d_ff", "cols"), ("d_model", "planes")])]),  # Section 8.3, three-dimensional
     "config4": dict(batch=32, length=256, d_model=1024, d_ff=65536, nsplit=16,
                     layouts=[([("all", 1)], []), ([("all", 16)], [("d_ff", "all")])]),
 }
