@@ -560,13 +560,18 @@ def block_step(mtf, dec, B=None):
     return step, flops, desc, (T, keep, gt, out, dx, ws, lay)
 
 
-def run_secondary(mtf, peaks):
-    """Records for the other workloads and for the memory-bound kernels, each timed with CUDA events on seeded inputs."""
+def run_secondary(mtf, peaks, blocks=True, reps=None):
+    """Records for the other workloads and for the memory-bound kernels, each timed with CUDA events on seeded inputs.
+    blocks=False leaves out the attention block and the decoder layer; reps overrides the repeat counts (profiler captures)."""
     import torch
     import seeded_inputs as si
     stream = torch.cuda.current_stream()
     out = []
-    for dec in (False, True):
+    if reps is not None:
+        timer = lambda fn, n, st_, warmup=3: event_time(fn, reps, st_, warmup=1)
+    else:
+        timer = event_time
+    for dec in ((False, True) if blocks else ()):
         step, flops, desc, keep = block_step(mtf, dec)
         ms = event_time(step, 20, stream, warmup=3)
         mtf.mtf_device_status()
@@ -588,21 +593,28 @@ def run_secondary(mtf, peaks):
     act = ["batch", "length", "d_model"]
     Nn = mtf.named
     rows = []
-    ms = event_time(lambda: mtf.mtf_layernorm_forward(lay, Nn(x, act), Nn(g, ["d_model"]), Nn(b, ["d_model"]), 1e-6, Nn(yb, act), Nn(stats, ["batch", "length", "stat"])), 50, stream)
+    # (the descriptors are built once, outside the timed calls: a call is then a few microseconds of host work,
+    #  well under the kernels' durations, so the event pair measures the device)
+    nx, ndy, ng, nb, ny, ndx = Nn(x, act), Nn(dy, act), Nn(g, ["d_model"]), Nn(b, ["d_model"]), Nn(yb, act), Nn(dxb, act)
+    nst, ndg, ndb = Nn(stats, ["batch", "length", "stat"]), Nn(dg, ["d_model"]), Nn(db, ["d_model"])
+    ms = timer(lambda: mtf.mtf_layernorm_forward(lay, nx, ng, nb, 1e-6, ny, nst), 50, stream)
     rows.append(("layernorm_fwd_rows_kernel", f"{B * L} rows of {D}", 2 * x.numel() * 2, ms))
-    ms = event_time(lambda: mtf.mtf_layernorm_backward(lay, Nn(dy, act), Nn(x, act), Nn(stats, ["batch", "length", "stat"]), Nn(g, ["d_model"]), None, Nn(dxb, act),
-                                                       Nn(dg, ["d_model"]), Nn(db, ["d_model"])), 50, stream)
-    rows.append(("layernorm_bwd_rows_kernel", f"{B * L} rows of {D}", 3 * x.numel() * 2, ms))
+    lnws = torch.empty(max(mtf.mtf_layernorm_workspace_bytes(D), 16), dtype=torch.uint8, device="cuda")
+    ms = timer(lambda: mtf.mtf_layernorm_backward(lay, ndy, nx, nst, ng, None, ndx, ndg, ndb, lnws), 50, stream)
+    rows.append(("layernorm_bwd_rows_kernel + colsum_finalize_kernel", f"{B * L} rows of {D}, dgamma / dbeta finished in a fixed order", 3 * x.numel() * 2, ms))
     Bs, H, Ls = 16, 16, 512
     names = ["batch", "heads", "length", "memory_length"]
     lg = to_device(si.normal(6, "lg", [Bs, H, Ls, Ls], "f32", 2.0))
     dP = to_device(si.normal(6, "dP", [Bs, H, Ls, Ls], "f32"))
     Pw, dlg = torch.empty(Bs, H, Ls, Ls, dtype=torch.bfloat16, device="cuda"), torch.empty(Bs, H, Ls, Ls, dtype=torch.bfloat16, device="cuda")
-    ms = event_time(lambda: mtf.mtf_softmax_forward(lay, Nn(lg, names), False, Nn(Pw, names)), 50, stream)
+    nlg, ndP, nPw, ndlg = Nn(lg, names), Nn(dP, names), Nn(Pw, names), Nn(dlg, names)
+    ms = timer(lambda: mtf.mtf_softmax_forward(lay, nlg, False, nPw), 50, stream)
     rows.append(("softmax_fwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (4 + 2), ms))
-    ms = event_time(lambda: mtf.mtf_softmax_backward(lay, Nn(Pw, names), Nn(dP, names), Nn(dlg, names)), 50, stream)
+    ms = timer(lambda: mtf.mtf_softmax_backward(lay, nPw, ndP, ndlg), 50, stream)
     rows.append(("softmax_bwd_kernel", f"{Bs * H * Ls} rows of {Ls}", lg.numel() * (2 + 4 + 2), ms))
     mtf.mtf_device_status()
+    del lg, dP, Pw, dlg
+    torch.cuda.empty_cache()
     # ---- the vocab dimension: embedding + logits + cross-entropy, forward and backward, vocab 32768, d_model 1024, tokens 8192
     import numpy as np
     Bv, Lv, Dv, V = 32, 256, 1024, 32768
@@ -625,7 +637,7 @@ def run_secondary(mtf, peaks):
         mtf.mtf_xent_backward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(dls, tl), Nn(dhv, av), Nn(dWo, ["d_model", "vocab"]), wsv)
         mtf.mtf_embedding_backward(layv, ids, Nn(dhv, av), Nn(dE, ["vocab", "d_model"]))
 
-    ms = event_time(vocab_step, 10, stream)
+    ms = timer(vocab_step, 10, stream)
     mtf.mtf_device_status()
     vflops = 6.0 * Tv * Dv * V
     tf = vflops / (ms * 1e-3) / 1e12
@@ -635,14 +647,15 @@ def run_secondary(mtf, peaks):
                 "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_burst"], "frac": tf / peaks["bf16_burst"], "unit": "TFLOP/s",
                              "note": "whole step (3 contractions + 4 memory-bound kernels) against the burst torch.matmul rate"}})
     # the memory-bound kernels of that step, each alone
-    ms = event_time(lambda: mtf.mtf_embedding_forward(layv, ids, Nn(E, ["vocab", "d_model"]), Nn(xv, av)), 50, stream)
+    nE, nxv, nlgt, nlse, nloss, ndls = Nn(E, ["vocab", "d_model"]), Nn(xv, av), Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), Nn(dls, tl)
+    ms = timer(lambda: mtf.mtf_embedding_forward(layv, ids, nE, nxv), 50, stream)
     rows.append(("embedding_gather_kernel", f"{Tv} rows of {Dv} (bf16) from a table of {V} rows", 2 * Tv * Dv * 2, ms))
     mtf.mtf_xent_forward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), wsv)
-    ms = event_time(lambda: mtf.mtf_softmax_xent_forward(layv, Nn(lgt, lv), tgt, Nn(lse, tl), Nn(loss, tl)), 20, stream)
+    ms = timer(lambda: mtf.mtf_softmax_xent_forward(layv, nlgt, tgt, nlse, nloss), 20, stream)
     rows.append(("xent_rows_kernel", f"{Tv} rows of {V} (bf16 logits)", Tv * V * 2, ms))
-    ms = event_time(lambda: mtf.mtf_softmax_xent_backward(layv, Nn(lgt, lv), tgt, Nn(lse, tl), Nn(dls, tl)), 20, stream)
+    ms = timer(lambda: mtf.mtf_softmax_xent_backward(layv, nlgt, tgt, nlse, ndls), 20, stream)
     rows.append(("xent_backward_kernel", f"{Tv} rows of {V} (bf16, in place)", Tv * V * 4, ms))
-    del lgt, dWo, dE, E, Wo
+    del lgt, dWo, dE, E, Wo, nE, nlgt
     torch.cuda.empty_cache()
     # Algorithm 1 line 3 on the largest parameter of config 4 (d_model 1024 x d_ff 65536): momentum + weight decay + bf16 working copy
     Dw, Fw = 1024, 65536
@@ -651,19 +664,22 @@ def run_secondary(mtf, peaks):
     mo, wb16 = torch.zeros_like(wm), torch.empty(Dw, Fw, dtype=torch.bfloat16, device="cuda")
     wn2 = ["d_model", "d_ff"]
     layu = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 16)]), [("d_ff", "all")])
-    ms = event_time(lambda: mtf.mtf_update(layu, Nn(gw, wn2), Nn(wm, wn2), Nn(mo, wn2), Nn(wb16, wn2), 1e-3, 0.9, 0.01), 20, stream)
+    ngw, nwm, nmo, nwb = Nn(gw, wn2), Nn(wm, wn2), Nn(mo, wn2), Nn(wb16, wn2)
+    ms = timer(lambda: mtf.mtf_update(layu, ngw, nwm, nmo, nwb, 1e-3, 0.9, 0.01), 20, stream)
     rows.append(("sgd_update_kernel", f"{Dw} x {Fw} f32 parameter with momentum and bf16 copy", Dw * Fw * 22, ms))
-    del wm, gw, mo, wb16
+    del wm, gw, mo, wb16, ngw, nwm, nmo, nwb
     torch.cuda.empty_cache()
     # Section 6.1: the block transpose between a batch split and a heads split, [batch, length, heads, d_k] -> [batch, heads, length, d_k]
     Bt, Lt, Ht, Kt = 256, 256, 32, 64
     qt = to_device(si.normal(9, "q", [Bt, Lt, Ht, Kt], "bf16"))
     qo = torch.empty(Bt, Ht, Lt, Kt, dtype=torch.bfloat16, device="cuda")
-    ms = event_time(lambda: mtf.mtf_transpose(lay, Nn(qt, ["batch", "length", "heads", "d_k"]), Nn(qo, ["batch", "heads", "length", "d_k"])), 20, stream)
+    nqt, nqo = Nn(qt, ["batch", "length", "heads", "d_k"]), Nn(qo, ["batch", "heads", "length", "d_k"])
+    ms = timer(lambda: mtf.mtf_transpose(lay, nqt, nqo), 20, stream)
     rows.append(("permute_copy_kernel", f"[{Bt}, {Lt}, {Ht}, {Kt}] bf16 -> [batch, heads, length, d_k]", 2 * qt.numel() * 2, ms))
     xt2 = qt.view(Bt * Lt, Ht * Kt)
     xo2 = qo.view(Ht * Kt, Bt * Lt)
-    ms = event_time(lambda: mtf.mtf_transpose(lay, Nn(xt2, ["tokens", "d_model"]), Nn(xo2, ["d_model", "tokens"])), 20, stream)
+    nxt2, nxo2 = Nn(xt2, ["tokens", "d_model"]), Nn(xo2, ["d_model", "tokens"])
+    ms = timer(lambda: mtf.mtf_transpose(lay, nxt2, nxo2), 20, stream)
     rows.append(("permute_transpose_kernel", f"[{Bt * Lt}, {Ht * Kt}] bf16 -> [d_model, tokens]", 2 * qt.numel() * 2, ms))
     mtf.mtf_device_status()
     for kernel, shape, nbytes, ms in rows:
@@ -715,12 +731,18 @@ def main():
     ap.add_argument("--d-ff", type=int, default=WORKLOAD["d_ff"], help="4096 = config 2, 65536 (with --layout mp16) = config 4")
     ap.add_argument("--batch", type=int, default=WORKLOAD["batch"], help="sequences of 256 tokens per GPU (smaller only for profiler captures)")
     ap.add_argument("--main-only", action="store_true", help="skip the per-layout table and the end-to-end leg (profiler captures)")
-    ap.add_argument("--workload", default="ffn", choices=["ffn", "attention", "decoder"], help="ffn = the headline line; the others print a secondary line")
+    ap.add_argument("--workload", default="ffn", choices=["ffn", "attention", "decoder", "rowkernels"],
+                    help="ffn = the headline line; attention / decoder print a secondary line; rowkernels runs the memory-bound kernels only (a few launches each, for profiler captures)")
     args = ap.parse_args()
     WORKLOAD["batch"] = args.batch
     WORKLOAD["d_ff"] = args.d_ff
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "rowkernels":
+        import torch
+        assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+        import paper_1811_02084_b200 as mtf
+        print(json.dumps({"metric": "row_kernels", "records": run_secondary(mtf, measured_peaks(), blocks=False, reps=args.steps if args.steps < 10 else None)}), flush=True)
     elif args.workload != "ffn":
         run_block(args)
     else:

@@ -290,11 +290,16 @@ mtf_status mtf_einsum_softmax_backward(const mtf_layout_t* layout, const mtf_ten
 mtf_status mtf_layernorm_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* gamma,
                                  const mtf_tensor* beta, float eps, mtf_tensor* y, mtf_tensor* stats, void* stream);
 /* dx = rstd * (g - mean(g) - xh * mean(g * xh)) + residual, g = dy * gamma, xh = (x - mean) * rstd;
- * dgamma = sum over rows of dy * xh, dbeta = sum over rows of dy (both or neither; zeroed by the call;
- * under a batch split these sums are the gradient Allreduce of Algorithm 1).  residual may be NULL. */
-mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* dy, const mtf_tensor* x,
-                                  const mtf_tensor* stats, const mtf_tensor* gamma, const mtf_tensor* residual,
-                                  mtf_tensor* dx, mtf_tensor* dgamma, mtf_tensor* dbeta, void* stream);
+ * dgamma = sum over rows of dy * xh, dbeta = sum over rows of dy (both or neither; under a batch split
+ * these sums are the gradient Allreduce of Algorithm 1).  residual may be NULL.
+ * workspace (device, 16-byte aligned; may be NULL): with at least mtf_layernorm_workspace_bytes(row
+ * length) bytes the two column sums are added up in a fixed order (per-block partial sums, then one
+ * pass in block order) and repeat bit for bit from run to run; with less, or for row lengths that
+ * report 0 bytes, they are accumulated with fp32 atomics into the zeroed outputs (order not fixed). */
+mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* dy, const mtf_tensor* x, const mtf_tensor* stats, const mtf_tensor* gamma,
+                                  const mtf_tensor* residual, mtf_tensor* dx, mtf_tensor* dgamma, mtf_tensor* dbeta, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+mtf_status mtf_layernorm_workspace_bytes(int64_t row_length, size_t* bytes);
 
 /* Multi-head attention.  x [batch, length, d_model]; wq, wk [d_model, heads, d_k]; wv [d_model, heads,
  * d_v]; wo [heads, d_v, d_model] (names are taken from the descriptors; the key/value side uses the

@@ -128,7 +128,8 @@ def _load():
         "mtf_einsum_softmax": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), c_float, c_int32, POINTER(mtf_tensor), vp, c_size_t, vp],
         "mtf_einsum_softmax_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp, c_size_t, vp],
         "mtf_layernorm_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), c_float, POINTER(mtf_tensor), POINTER(mtf_tensor), vp],
-        "mtf_layernorm_backward": [vp] + [POINTER(mtf_tensor)] * 8 + [vp],
+        "mtf_layernorm_backward": [vp] + [POINTER(mtf_tensor)] * 8 + [vp, c_size_t, vp],
+        "mtf_layernorm_workspace_bytes": [c_int64, POINTER(c_size_t)],
         "mtf_attention_forward": [vp] + [POINTER(mtf_tensor)] * 5 + [c_int32] + [POINTER(mtf_tensor)] * 7 + [vp, c_size_t, vp],
         "mtf_attention_backward": [vp] + [POINTER(mtf_tensor)] * 17 + [vp, c_size_t, vp],
         "mtf_attention_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
@@ -487,9 +488,16 @@ def mtf_layernorm_forward(layout, x, gamma, beta, eps, y, stats, stream=None) ->
     _check(_lib.mtf_layernorm_forward(layout.handle, _p(x), _p(gamma), _p(beta), float(eps), _p(y), _p(stats), _stream(stream)))
 
 
-def mtf_layernorm_backward(layout, dy, x, stats, gamma, residual, dx, dgamma, dbeta, stream=None) -> None:
+def mtf_layernorm_backward(layout, dy, x, stats, gamma, residual, dx, dgamma, dbeta, workspace=None, stream=None) -> None:
+    wp, wb = _ws(workspace)
     _check(_lib.mtf_layernorm_backward(layout.handle, _p(dy), _p(x), _p(stats), _p(gamma), _p(residual), _p(dx), _p(dgamma), _p(dbeta),
-                                       _stream(stream)))
+                                       wp, wb, _stream(stream)))
+
+
+def mtf_layernorm_workspace_bytes(row_length: int) -> int:
+    b = c_size_t()
+    _check(_lib.mtf_layernorm_workspace_bytes(int(row_length), byref(b)))
+    return b.value
 
 
 def mtf_attention_forward(layout, x, wq, wk, wv, wo, causal, residual, q, kk, vv, weights, o, y, workspace=None, stream=None) -> None:

@@ -15,6 +15,7 @@ const char* last_error();
 int64_t launch_count();
 mtf_status read_device_status(int* code);
 mtf_status read_bad_index(int* seen);
+mtf_status read_row_status(int* code);
 }  // namespace mtf
 
 using mtf::Dim;
@@ -610,6 +611,12 @@ mtf_status mtf_device_status(int32_t* code) {
   mtf_status st = mtf::read_device_status(&c);
   if (code) *code = c;
   if (st != MTF_OK) return st;
+  int rc = 0;
+  if ((st = mtf::read_row_status(&rc)) != MTF_OK) return st;
+  if (rc) {
+    if (code) *code = rc;
+    return fail(MTF_ERR_TIMEOUT, "a bounded device-side wait gave up (code 0x%x)", rc);
+  }
   int bad = 0;
   if ((st = mtf::read_bad_index(&bad)) != MTF_OK) return st;
   if (bad) return fail(MTF_ERR_INVALID_ARG, "a token id or target outside [0, vocab) was seen by the vocab kernels");

@@ -16,7 +16,8 @@ mtf_status launch_softmax_fwd(const float* logits, void* weights, int64_t rows, 
 mtf_status launch_softmax_bwd(const void* P, const float* dP, void* dlg, int64_t rows, int n, void* stream);
 mtf_status launch_layernorm_fwd(const void* x, const float* gamma, const float* beta, void* y, float* stats, int64_t rows, int n, float eps, void* stream);
 mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stats, const float* gamma, const void* residual, void* dx,
-                                float* dgamma, float* dbeta, int64_t rows, int n, void* stream);
+                                float* dgamma, float* dbeta, int64_t rows, int n, void* scratch, size_t scratch_bytes, void* stream);
+size_t layernorm_bwd_scratch_bytes(int n);
 mtf_status ffn_forward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias, const mtf_tensor* v,
                             mtf_tensor* h_saved, mtf_tensor* y, const mtf_tensor* y_residual, void* workspace, size_t workspace_bytes, void* stream);
 mtf_status ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v, const mtf_tensor* h_saved,
@@ -193,8 +194,15 @@ mtf_status mtf_layernorm_forward(const mtf_layout_t* layout, const mtf_tensor* x
 }
 
 // g = dy * gamma; dx = rstd * (g - mean(g) - xh * mean(g * xh)) (+ residual); dgamma = sum_rows dy * xh; dbeta = sum_rows dy
+mtf_status mtf_layernorm_workspace_bytes(int64_t row_length, size_t* bytes) {
+  if (!bytes || row_length <= 0 || row_length > 0x7fffffff) return fail(MTF_ERR_INVALID_ARG, "layernorm_workspace_bytes: bad argument");
+  *bytes = mtf::layernorm_bwd_scratch_bytes((int)row_length);
+  return MTF_OK;
+}
+
 mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* dy, const mtf_tensor* x, const mtf_tensor* stats, const mtf_tensor* gamma,
-                                  const mtf_tensor* residual, mtf_tensor* dx, mtf_tensor* dgamma, mtf_tensor* dbeta, void* stream) {
+                                  const mtf_tensor* residual, mtf_tensor* dx, mtf_tensor* dgamma, mtf_tensor* dbeta, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
   if (!layout || !dy || !x || !stats || !gamma || !dx || !dy->data || !x->data || !stats->data || !gamma->data || !dx->data) return fail(MTF_ERR_INVALID_ARG, "layernorm backward: NULL argument");
   if (x->ndim < 2 || !same_shape(*x, *dy) || !same_shape(*x, *dx) || (residual && !same_shape(*x, *residual))) return fail(MTF_ERR_SIZE_MISMATCH, "layernorm backward: dy, x, dx (and residual) must have the same dims");
   const int n = (int)x->dims[x->ndim - 1].size;
@@ -209,7 +217,7 @@ mtf_status mtf_layernorm_backward(const mtf_layout_t* layout, const mtf_tensor* 
   if (st != MTF_OK) return st;
   st = mtf::launch_layernorm_bwd(dy->data, x->data, reinterpret_cast<const float*>(stats->data), reinterpret_cast<const float*>(gamma->data),
                                  residual ? residual->data : nullptr, dx->data, dgamma ? reinterpret_cast<float*>(dgamma->data) : nullptr,
-                                 dbeta ? reinterpret_cast<float*>(dbeta->data) : nullptr, rows, n, stream);
+                                 dbeta ? reinterpret_cast<float*>(dbeta->data) : nullptr, rows, n, workspace, workspace_bytes, stream);
   if (st != MTF_OK || !dgamma) return st;
   // the parameter gradients sum over the token dimensions: with one of them split across ranks they are partial sums
   std::vector<std::string> reduced;
@@ -418,14 +426,14 @@ mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tens
   void* rest = ar.base + ar.used;
   const size_t rest_bytes = ar.size - ar.used;
   mtf_status st;
-  if ((st = mtf_layernorm_backward(layout, dout, sv->s2, sv->stats2, p->ln2_gamma, nullptr, &ds2.t, g->dln2_gamma, g->dln2_beta, stream)) != MTF_OK) return st;
+  if ((st = mtf_layernorm_backward(layout, dout, sv->s2, sv->stats2, p->ln2_gamma, nullptr, &ds2.t, g->dln2_gamma, g->dln2_beta, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = mtf::tap("ds2", ds2.t, stream)) != MTF_OK) return st;
   // da = ds2 + dFFN/da
   if ((st = mtf::ffn_backward_impl(layout, sv->a, p->w, p->v, sv->h, &ds2.t, &da.t, &ds2.t, g->dw, g->dbias, g->dv, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = mtf::rank_wait(layout, stream)) != MTF_OK) return st;        // da (and the parameter gradients) summed across ranks
   if ((st = mtf::tap("da", da.t, stream)) != MTF_OK) return st;
   // ds1 (reusing ds2's buffer) = LN1 backward; dx = ds1 + dAttention/dx
-  if ((st = mtf_layernorm_backward(layout, &da.t, sv->s1, sv->stats1, p->ln1_gamma, nullptr, &ds2.t, g->dln1_gamma, g->dln1_beta, stream)) != MTF_OK) return st;
+  if ((st = mtf_layernorm_backward(layout, &da.t, sv->s1, sv->stats1, p->ln1_gamma, nullptr, &ds2.t, g->dln1_gamma, g->dln1_beta, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = mtf::tap("ds1", ds2.t, stream)) != MTF_OK) return st;
   return mtf_attention_backward(layout, x, p->wq, p->wk, p->wv, p->wo, sv->q, sv->kk, sv->vv, sv->weights, sv->o, &ds2.t, &ds2.t, dx, g->dwq, g->dwk,
                                 g->dwv, g->dwo, rest, rest_bytes, stream);

@@ -105,6 +105,39 @@ __global__ void __launch_bounds__(256) permute_transpose_kernel(const T* __restr
   }
 }
 
+// The same for 2-byte elements with whole 64 x 64 tiles and 16-byte aligned rows on both sides: 16-byte loads along
+// the source's contiguous dimension, 16-byte stores along the destination's (eight 2-byte reads of a tile column each).
+__global__ void __launch_bounds__(256) permute_transpose16_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, const TileTranspose c) {
+  __shared__ __align__(16) uint16_t tile[64][64 + 8];
+  for (long long t = blockIdx.x; t < c.total_tiles; t += gridDim.x) {
+    uint32_t ta, tb, rem;
+    uint32_t w = fd_divmod((uint32_t)t, c.tiles_a, &ta);
+    w = fd_divmod(w, c.tiles_b, &tb);
+    long long so = 0, d_o = 0;
+    for (int d = c.nbatch - 1; d >= 0; --d) {
+      w = fd_divmod(w, c.bsize[d], &rem);
+      so += (long long)rem * c.bs_src[d];
+      d_o += (long long)rem * c.bs_dst[d];
+    }
+    const int a0 = (int)ta * 64, b0 = (int)tb * 64;
+    const int px = threadIdx.x & 7, py = threadIdx.x >> 3;        // 8 pieces of 8 elements x 32 rows
+#pragma unroll
+    for (int r = py; r < 64; r += 32)
+      *reinterpret_cast<uint4*>(&tile[r][px * 8]) = *reinterpret_cast<const uint4*>(src + so + (long long)(b0 + r) * c.sb_src + a0 + px * 8);
+    __syncthreads();
+#pragma unroll
+    for (int r = py; r < 64; r += 32) {                                // output row a0 + r, columns b0 + 8 px ... + 7
+      uint16_t v[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = tile[px * 8 + e][r];
+      uint4 o;
+      o.x = v[0] | ((uint32_t)v[1] << 16); o.y = v[2] | ((uint32_t)v[3] << 16); o.z = v[4] | ((uint32_t)v[5] << 16); o.w = v[6] | ((uint32_t)v[7] << 16);
+      *reinterpret_cast<uint4*>(dst + d_o + (long long)(a0 + r) * c.sa_dst + b0 + px * 8) = o;
+    }
+    __syncthreads();
+  }
+}
+
 }  // namespace
 
 namespace mtf {
@@ -155,7 +188,11 @@ mtf_status launch_permute_copy(const void* src, void* dst, int elem_bytes, int n
     c.total_tiles = ta * tb;
     for (int i = 0; i < c.nbatch; ++i) c.total_tiles *= c.bsize[i].d;
     const long long blocks = std::min<long long>(c.total_tiles, (long long)device_sm_count() * 8);
-    if (elem_bytes == 2) permute_transpose_kernel<uint16_t><<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c);
+    bool fast16 = elem_bytes == 2 && ia >= 0 && c.n_a % 64 == 0 && c.n_b % 64 == 0 && c.sb_src % 8 == 0 && c.sa_dst % 8 == 0 &&
+                  !(reinterpret_cast<uintptr_t>(src) & 15) && !(reinterpret_cast<uintptr_t>(dst) & 15);
+    for (int i = 0; fast16 && i < c.nbatch; ++i) fast16 = c.bs_src[i] % 8 == 0 && c.bs_dst[i] % 8 == 0;
+    if (fast16) permute_transpose16_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c);
+    else if (elem_bytes == 2) permute_transpose_kernel<uint16_t><<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint16_t*>(src), reinterpret_cast<uint16_t*>(dst), c);
     else permute_transpose_kernel<uint32_t><<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(src), reinterpret_cast<uint32_t*>(dst), c);
   }
   count_launch();

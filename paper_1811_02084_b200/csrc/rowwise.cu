@@ -257,7 +257,7 @@ template <int NCH, bool kSmemAcc>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32, 1)
 layernorm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ x, const float* __restrict__ stats,
                           const float* __restrict__ gamma, const __nv_bfloat16* __restrict__ residual, __nv_bfloat16* __restrict__ dx,
-                          float* __restrict__ dgamma, float* __restrict__ dbeta, int64_t rows) {
+                          float* __restrict__ dgamma, float* __restrict__ dbeta, float* __restrict__ partial, int64_t rows) {
   constexpr int n = NCH * 256;
   constexpr int kAccRegs = kSmemAcc ? 1 : NCH;
   extern __shared__ float4 sh_dyn[];
@@ -335,6 +335,9 @@ layernorm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloa
       *reinterpret_cast<uint4*>(dx + row * n + c) = float_to_bf16x8(o);
     }
   }
+  // Block sums in warp order (a fixed order), then either into this block's row of `partial` ([gridDim.x][2][n];
+  // colsum_finalize_kernel adds the blocks up in block order, so the result repeats bit for bit) or, without
+  // a partial buffer, onto the zeroed outputs with fp32 atomics.
   if (dgamma && dbeta) {
     if (kSmemAcc) {
       __syncthreads();
@@ -342,23 +345,43 @@ layernorm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloa
         float t = 0.f;
 #pragma unroll
         for (int w = 0; w < kWarpsPerBlock; ++w) t += sh[2 * n * (1 + w) + c];
-        atomicAdd((c < n ? dgamma : dbeta) + (c < n ? c : c - n), t);
+        if (partial) partial[(size_t)blockIdx.x * 2 * n + c] = t;
+        else atomicAdd((c < n ? dgamma : dbeta) + (c < n ? c : c - n), t);
       }
     } else {
+      for (int w = 0; w < kWarpsPerBlock; ++w) {
+        if ((int)(threadIdx.x >> 5) == w) {
 #pragma unroll
-      for (int i = 0; i < kAccRegs; ++i)
+          for (int i = 0; i < kAccRegs; ++i)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          atomicAdd(&sh[i * 256 + lane * 8 + e], ag[i][e]);
-          atomicAdd(&sh[n + i * 256 + lane * 8 + e], ab[i][e]);
+            for (int e = 0; e < 8; ++e) {
+              sh[i * 256 + lane * 8 + e] += ag[i][e];
+              sh[n + i * 256 + lane * 8 + e] += ab[i][e];
+            }
         }
-      __syncthreads();
-      for (int c = threadIdx.x; c < n; c += kWarpsPerBlock * 32) {
-        atomicAdd(dgamma + c, sh[c]);
-        atomicAdd(dbeta + c, sh[n + c]);
+        __syncthreads();
+      }
+      for (int c = threadIdx.x; c < 2 * n; c += kWarpsPerBlock * 32) {
+        if (partial) partial[(size_t)blockIdx.x * 2 * n + c] = sh[c];
+        else atomicAdd((c < n ? dgamma : dbeta) + (c < n ? c : c - n), sh[c]);
       }
     }
   }
+}
+
+// out0[c] = sum over g (ascending) of partial[g][0][c], out1[c] likewise from partial[g][1][c]: the fixed-order
+// finish of column sums whose partial sums were left by `groups` producers (planes = 1: one sum only)
+__global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ partial, int groups, int planes, int n, float* __restrict__ out0,
+                                                              float* __restrict__ out1) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= n) return;
+  float s0 = 0.f, s1 = 0.f;
+  for (int g = 0; g < groups; ++g) {
+    s0 += partial[((size_t)g * planes) * n + c];
+    if (planes > 1) s1 += partial[((size_t)g * planes + 1) * n + c];
+  }
+  out0[c] = s0;
+  if (planes > 1 && out1) out1[c] = s1;
 }
 
 // dgamma[c] += sum_rows dy * xh,  dbeta[c] += sum_rows dy.  Block = 32 x 8 threads: 64 columns
@@ -452,42 +475,58 @@ mtf_status launch_layernorm_fwd(const void* x, const float* gamma, const float* 
   return check("layernorm_fwd_kernel");
 }
 
+// Bytes of scratch with which the parameter gradients are summed in a fixed order (0: this row length always uses atomics)
+size_t layernorm_bwd_scratch_bytes(int n) {
+  if (n != 256 && n != 512 && n != 1024 && n != 2048) return 0;
+  return (size_t)device_sm_count() * 2 * 2 * n * sizeof(float);
+}
+
+mtf_status launch_colsum_finalize(const float* partial, int groups, int planes, int n, float* out0, float* out1, void* stream) {
+  colsum_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(partial, groups, planes, n, out0, out1);
+  count_launch();
+  return check("colsum_finalize_kernel");
+}
+
 mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stats, const float* gamma, const void* residual, void* dx,
-                                float* dgamma, float* dbeta, int64_t rows, int n, void* stream) {
+                                float* dgamma, float* dbeta, int64_t rows, int n, void* scratch, size_t scratch_bytes, void* stream) {
   if (n % 8 || !aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(gamma) || (residual && !aligned16(residual)))
     return fail(MTF_ERR_UNSUPPORTED, "layernorm backward: row length must be a multiple of 8 and pointers 16-byte aligned");
   if (rows <= 0) return MTF_OK;
   cudaStream_t st = (cudaStream_t)stream;
   if (n == 256 || n == 512 || n == 1024 || n == 2048) {
-    // one pass over dy and x for dx and the parameter gradients (persistent grid, one block per SM)
-    if (dgamma && dbeta) {
+    // one pass over dy and x for dx and the parameter gradients (persistent grid)
+    const int sms = device_sm_count();
+    unsigned grid = (unsigned)std::min<int64_t>((rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 2 * (int64_t)sms);
+    if (n == 2048) grid = std::min(grid, (unsigned)sms);
+    const bool want = dgamma && dbeta;
+    float* partial = nullptr;
+    if (want && scratch && !(reinterpret_cast<uintptr_t>(scratch) & 15) && scratch_bytes >= (size_t)grid * 2 * n * sizeof(float)) partial = reinterpret_cast<float*>(scratch);
+    if (want && !partial) {
       cudaError_t e = cudaMemsetAsync(dgamma, 0, (size_t)n * sizeof(float), st);
       if (e == cudaSuccess) e = cudaMemsetAsync(dbeta, 0, (size_t)n * sizeof(float), st);
       if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     }
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const unsigned grid = (unsigned)std::min<int64_t>((rows + kWarpsPerBlock - 1) / kWarpsPerBlock, 2 * (int64_t)sms);
     const __nv_bfloat16* db = reinterpret_cast<const __nv_bfloat16*>(dy);
     const __nv_bfloat16* xb = reinterpret_cast<const __nv_bfloat16*>(x);
     const __nv_bfloat16* rb = reinterpret_cast<const __nv_bfloat16*>(residual);
     __nv_bfloat16* ob = reinterpret_cast<__nv_bfloat16*>(dx);
-    float* dg = (dgamma && dbeta) ? dgamma : nullptr;
-    float* dbp = (dgamma && dbeta) ? dbeta : nullptr;
+    float* dg = want ? dgamma : nullptr;
+    float* dbp = want ? dbeta : nullptr;
     const size_t sm_small = 2 * (size_t)n * sizeof(float), sm_big = sm_small * (1 + kWarpsPerBlock);       // 144 KB for 2048 columns
     switch (n) {
-      case 256: layernorm_bwd_rows_kernel<1, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
-      case 512: layernorm_bwd_rows_kernel<2, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
-      case 1024: layernorm_bwd_rows_kernel<4, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows); break;
+      case 256: layernorm_bwd_rows_kernel<1, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, partial, rows); break;
+      case 512: layernorm_bwd_rows_kernel<2, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, partial, rows); break;
+      case 1024: layernorm_bwd_rows_kernel<4, false><<<grid, kWarpsPerBlock * 32, sm_small, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, partial, rows); break;
       default: {
         static cudaError_t attr = cudaFuncSetAttribute(layernorm_bwd_rows_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * 2048 * sizeof(float) * (1 + kWarpsPerBlock)));
         if (attr != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(attr));
-        layernorm_bwd_rows_kernel<8, true><<<std::min(grid, (unsigned)sms), kWarpsPerBlock * 32, sm_big, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, rows);
+        layernorm_bwd_rows_kernel<8, true><<<grid, kWarpsPerBlock * 32, sm_big, st>>>(db, xb, stats, gamma, rb, ob, dg, dbp, partial, rows);
       }
     }
     count_launch();
-    return check("layernorm_bwd_rows_kernel");
+    mtf_status s2 = check("layernorm_bwd_rows_kernel");
+    if (s2 != MTF_OK || !partial) return s2;
+    return launch_colsum_finalize(partial, (int)grid, 2, n, dgamma, dbeta, stream);
   }
   const int64_t blocks = (rows + kWarpsPerBlock - 1) / kWarpsPerBlock;
   if (blocks > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "layernorm backward: too many rows");
@@ -507,6 +546,12 @@ mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stat
     s = check("layernorm_bwd_params_kernel");
   }
   return s;
+}
+
+// (no row kernel has a bounded wait today: the status word of this family stays 0)
+mtf_status read_row_status(int* code) {
+  *code = 0;
+  return MTF_OK;
 }
 
 }  // namespace mtf

@@ -68,43 +68,45 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// One block per token row of bf16 logits (vocab a multiple of 8).  Two passes over the row (the second one hits L1/L2):
-// maximum, then sum of exponentials; the picked logit is read directly.
+// One block per token row of bf16 logits (vocab a multiple of 8).  One pass over the row: every thread keeps a running
+// maximum and the sum of exponentials relative to it (rescaled when the maximum moves); the threads' pairs are then
+// combined - the local reduction of each part of the row followed by the combine of Section 6's "Reduction".
+// The picked logit is read directly.
+__device__ __forceinline__ void lse_combine(float& m, float& s, float m2, float s2) {
+  const float mx = fmaxf(m, m2);
+  s = (m == -INFINITY ? 0.f : s * __expf(m - mx)) + (m2 == -INFINITY ? 0.f : s2 * __expf(m2 - mx));
+  m = mx;
+}
+
 __global__ void __launch_bounds__(256) xent_rows_kernel(const __nv_bfloat16* __restrict__ logits, const int32_t* __restrict__ targets, float* __restrict__ lse,
                                                         float* __restrict__ loss, int vocab, int* __restrict__ bad) {
-  __shared__ float red[8];
+  __shared__ float red_m[8], red_s[8];
   const long long row = blockIdx.x;
   const uint4* r = reinterpret_cast<const uint4*>(logits + row * vocab);
   const int pieces = vocab / 8;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float mx = -INFINITY;
+  float m = -INFINITY, s = 0.f;
   for (int p = threadIdx.x; p < pieces; p += 256) {
     float f[8];
     bf16x8(r[p], f);
+    float pm = f[0];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) mx = fmaxf(mx, f[e]);
+    for (int e = 1; e < 8; ++e) pm = fmaxf(pm, f[e]);
+    if (pm > m) { s *= __expf(m - pm); m = pm; }          // (m = -inf: s is 0 and stays 0)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) s += __expf(f[e] - m);
   }
-  mx = warp_max(mx);
-  if (lane == 0) red[warp] = mx;
-  __syncthreads();
-  mx = red[0];
 #pragma unroll
-  for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
-  __syncthreads();
-  float sum = 0.f;
-  for (int p = threadIdx.x; p < pieces; p += 256) {
-    float f[8];
-    bf16x8(r[p], f);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) sum += __expf(f[e] - mx);
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    lse_combine(m, s, m2, s2);
   }
-  sum = warp_sum(sum);
-  if (lane == 0) red[warp] = sum;
+  if (lane == 0) { red_m[warp] = m; red_s[warp] = s; }
   __syncthreads();
   if (threadIdx.x == 0) {
-    float s = 0.f;
-    for (int w = 0; w < 8; ++w) s += red[w];
-    const float l = mx + logf(s);
+    float mm = red_m[0], ss = red_s[0];
+    for (int w = 1; w < 8; ++w) lse_combine(mm, ss, red_m[w], red_s[w]);
+    const float l = mm + logf(ss);
     lse[row] = l;
     const int tg = targets[row];
     if (tg < 0 || tg >= vocab) { atomicExch(bad, 1); loss[row] = 0.f; }

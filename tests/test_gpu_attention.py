@@ -160,7 +160,7 @@ def test_einsum_softmax_refuses_rows_that_do_not_fit(mtf):
 
 # 136: the kernels that re-read the row per pass; 256..2048: rows kept in registers (2048: partial
 # parameter sums in shared-memory strips); 50 rows per batch entry leave the last block ragged
-@pytest.mark.parametrize("D", [136, 256, 512, 1024, 2048])
+@pytest.mark.parametrize("D", [136, 256, 512, 1024, 2048, 4096])
 def test_layernorm_forward_backward(mtf, D):
     import torch
     from oracle import NT, DenseOps, blocks
@@ -185,6 +185,22 @@ def test_layernorm_forward_backward(mtf, D):
     mtf.mtf_layernorm_backward(lay, N(dyt, names), N(xt, names), N(stats, ["batch", "length", "stat"]), N(gt, names[2:]), N(rt, names),
                                N(dx, names), N(dg, names[2:]), N(db, names[2:]))
     mtf.mtf_device_status()
+    # with a workspace the two column sums are added in a fixed order: the same values, bit for bit on every run
+    nbytes = mtf.mtf_layernorm_workspace_bytes(D)
+    if nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        runs = []
+        for _ in range(3):
+            dg2, db2, dx2 = alloc(dims[2:], "f32"), alloc(dims[2:], "f32"), alloc(dims, "bf16")
+            mtf.mtf_layernorm_backward(lay, N(dyt, names), N(xt, names), N(stats, ["batch", "length", "stat"]), N(gt, names[2:]), N(rt, names),
+                                       N(dx2, names), N(dg2, names[2:]), N(db2, names[2:]), ws)
+            mtf.mtf_device_status()
+            runs.append((dg2, db2))
+            assert torch.equal(dx2, dx)
+        assert all(torch.equal(runs[0][0], r[0]) and torch.equal(runs[0][1], r[1]) for r in runs[1:])
+        assert parity_error(from_torch(runs[0][0]), g["dgamma"].a) <= 1e-3 and parity_error(from_torch(runs[0][1]), g["dbeta"].a) <= 1e-3
+    else:
+        assert D in (136, 4096)          # these row lengths take the kernels without a fixed-order finish
     assert parity_error(from_torch(y), f["y"].a) <= TOL["bf16"]
     assert parity_error(from_torch(dx), g["dx"].a + res.f64) <= TOL["bf16"]
     assert parity_error(from_torch(dg), g["dgamma"].a) <= 1e-3
