@@ -441,12 +441,19 @@ mtf_status mtf_ffn_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor*
     mtf_tensor dy = {nullptr, x->dtype, x->ndim, yd};
     struct Case { mtf_tensor a, b, c; } cases[6] = {
         {xin, *w, hs}, {hs, v, dy}, {dy, v, dhp}, {hs, dy, {nullptr, MTF_F32, 2, vd}}, {xin, dhp, {nullptr, MTF_F32, 2, w->dims}}, {dhp, *w, xin}};
+    int idx = 0;
     for (auto& c : cases) {
       mtf_tensor in[2] = {c.a, c.b};
       size_t b = 0;
-      mtf_status st = mtf_einsum_workspace_bytes(layout, 2, in, &c.c, nullptr, &b);
+      // (the dhp launch carries the fused column sum for dbias: its fixed-order finish wants scratch too)
+      mtf_dim bd[1] = {w->dims[1]};
+      mtf_tensor dbias = {nullptr, MTF_F32, 1, bd};
+      mtf_epilogue e;
+      e.scale = 1.f; e.relu = 0; e.bias = nullptr; e.relu_mask = &hs; e.residual = nullptr; e.reduce_sum_out = &dbias;
+      mtf_status st = mtf_einsum_workspace_bytes(layout, 2, in, &c.c, idx == 2 ? &e : nullptr, &b);
       if (st != MTF_OK) return st;
       scratch = std::max(scratch, b);
+      ++idx;
     }
   }
   *bytes = align256((size_t)numel(dhp) * elem_bytes(dhp.dtype)) + align256(scratch) + 256;

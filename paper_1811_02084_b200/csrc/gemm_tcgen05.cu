@@ -119,6 +119,8 @@ struct TcArgs {
   float scale;
   int relu;
   float* rsum;             // fused reduce_sum over M of the epilogue value (fp32, pre-zeroed), indexed by n
+  float* rsum_partial;     // not NULL: every 32-row group leaves its column sums here ([row group][N]) instead of adding them to rsum with
+                           // atomics; a finishing launch adds the groups up in index order, so the sums repeat bit for bit
   float* ws_partials;
   unsigned* ws_counters;     // per (tile, 32-row group, column part): arrivals, then as many again: fragments written
   long long ws_ncounters;
@@ -136,6 +138,7 @@ struct Tile {
   int m0, m_end, n0, n_end;
   int o[3];
   long long c_off;         // element offset of the outer coordinates in C
+  long long row_id;        // index of the tile's block of rows among all blocks of rows of the launch (every index but the n tile's)
 };
 
 __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long tile, int tile_rows, int tile_cols) {
@@ -152,11 +155,16 @@ __device__ __forceinline__ Tile decode_tile(const TcArgs& a, long long tile, int
   slice = fd_divmod(slice, a.fd_sm, &im);
   r.c_off = 0;
   r.o[0] = r.o[1] = r.o[2] = 0;
+  long long so_lin = slice, ol_lin = 0;      // (what is left of `slice` is the linear index of the outer split coordinates)
+  for (int j = 0; j < a.n_outer; ++j) ol_lin = ol_lin * a.outer_local[j] + ol[j];
   for (int j = a.n_outer - 1; j >= 0; --j) {
     slice = fd_divmod(slice, a.fd_outer_split[j], &rem);
     r.o[j] = (int)rem * a.outer_local[j] + ol[j];
     r.c_off += (long long)r.o[j] * a.outer_sC[j];
   }
+  long long OL = 1;
+  for (int j = 0; j < a.n_outer; ++j) OL *= a.outer_local[j];
+  r.row_id = ((so_lin * a.sm + im) * OL + ol_lin) * a.m_tiles + mt;
   r.m0 = (int)im * a.Ms + (int)mt * tile_rows;
   r.m_end = ((int)im + 1) * a.Ms;
   r.n0 = (int)in * a.Ns + (int)nt * tile_cols;
@@ -1151,8 +1159,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           buf ^= 1u;
           const float s0 = warp_column_sums(v0, lane);      // the column sums while the store drains (v0, v1 are destroyed)
           const float s1 = warp_column_sums(v1, lane);
-          atomicAdd(a.rsum + tl.n0 + c0 + lane, s0);
-          atomicAdd(a.rsum + tl.n0 + c0 + 32 + lane, s1);
+          if (a.rsum_partial) {
+            float* const pr = a.rsum_partial + (size_t)(tl.row_id * (kTileRows / 32) + warp_tile_row / 32) * a.N + tl.n0 + c0 + lane;
+            pr[0] = s0;
+            pr[32] = s1;
+          } else {
+            atomicAdd(a.rsum + tl.n0 + c0 + lane, s0);
+            atomicAdd(a.rsum + tl.n0 + c0 + 32 + lane, s1);
+          }
         }
         tcgen05_fence_before();
         __syncwarp();
@@ -1270,7 +1284,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               for (int j = 0; j < 32; ++j) v[j] = (live && j < n_valid) ? v[j] : 0.f;
             }
             const float col = warp_column_sums(v, lane);
-            if (lane < n_valid) atomicAdd(a.rsum + n_first + lane, col);
+            if (lane < n_valid) {
+              if (a.rsum_partial) a.rsum_partial[(size_t)(tl.row_id * (kTileRows / 32) + warp_tile_row / 32) * a.N + n_first + lane] = col;
+              else atomicAdd(a.rsum + n_first + lane, col);
+            }
           }
         }
         tcgen05_fence_before();
@@ -1500,6 +1517,14 @@ static int64_t tc_total_tiles(const TcParams& t) {
   return tiles;
 }
 
+// Scratch for a fused reduce_sum whose column sums are finished in a fixed order: one fp32 row of N per 32-row group
+size_t tc_rsum_partial_bytes(const TcParams& t) {
+  const int rows = tc_tile_rows(t);
+  int64_t groups = ((t.M / t.sm + rows - 1) / rows) * (rows / 32) * t.sm;
+  for (int j = 0; j < t.n_outer; ++j) groups *= t.outer_size[j];
+  return (size_t)groups * t.N * sizeof(float);
+}
+
 size_t tc_workspace_bytes(const TcParams& t) {
   if (t.reduce_mode != MTF_REDUCE_WORKSPACE) {
     if (!t.balance) return 0;
@@ -1608,6 +1633,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.resid_tma = (resid && !a.mask_tma && a.resid_bf16 == a.c_bf16) ? 1 : 0;
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
+  a.rsum_partial = nullptr;
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
   {
     const int b_cols = (t.cta_pair ? a.block_n / 2 : a.block_n);          // B columns staged by one CTA (wide: two runs of 128)
@@ -1661,9 +1687,18 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     if (zs != MTF_OK) return zs;
   }
 
+  long long rsum_groups = 0;
   if (rsum) {
-    mtf_status zs = zero_words(rsum, t.N, st);
-    if (zs != MTF_OK) return zs;
+    // with room in the workspace the column sums are left per 32-row group and finished in group order by a small
+    // launch behind this one (repeatable bit for bit); otherwise they are added to the zeroed output with atomics
+    rsum_groups = (a.total_tiles / ((long long)a.n_tiles * a.sn)) * (tile_rows / 32);
+    const size_t need = (size_t)rsum_groups * t.N * sizeof(float);
+    if (!a.ws_partials && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 15) && workspace_bytes >= need) {
+      a.rsum_partial = reinterpret_cast<float*>(workspace);
+    } else {
+      mtf_status zs = zero_words(rsum, t.N, st);
+      if (zs != MTF_OK) return zs;
+    }
   }
   CUtensorMap map_a, map_b, map_c, map_m;
   mtf_status s;
@@ -1741,6 +1776,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel: %s", cudaGetErrorString(e));
+  if (a.rsum_partial) return launch_colsum_finalize(a.rsum_partial, (int)rsum_groups, 1, (int)t.N, rsum, nullptr, stream);
   return MTF_OK;
 }
 

@@ -210,6 +210,9 @@ mtf_status einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, c
 mtf_status einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tensor (*terms)[2], mtf_tensor* out,
                         const mtf_epilogue* epilogue, void* workspace, size_t workspace_bytes, void* stream);
 size_t tc_workspace_bytes(const TcParams& t);
+size_t tc_rsum_partial_bytes(const TcParams& t);
+// out0[c] (and out1[c] when planes = 2) = sum over g = 0 .. groups-1, in that order, of partial[g][plane][c]
+mtf_status launch_colsum_finalize(const float* partial, int groups, int planes, int n, float* out0, float* out1, void* stream);
 size_t builtin_scratch_capacity();
 // SM count of the current device; 148 (a B200) when no device can be asked, so that planning works without one.
 int device_sm_count();

@@ -541,6 +541,7 @@ mtf_status make_plan(const mtf_layout_t* L, int n_in, const mtf_tensor* in, cons
       if (force_reduce == 3 && tiles >= workers && (double)tiles / (double)(rounds * workers) <= 0.92) t.balance = 1;
     }
     P->workspace_bytes = tc_workspace_bytes(t);
+    if (P->epi.has_rsum && mode != MTF_REDUCE_WORKSPACE && !t.balance) P->workspace_bytes = std::max(P->workspace_bytes, tc_rsum_partial_bytes(t));
   } else if (force_reduce == MTF_REDUCE_WORKSPACE) {
     return fail(MTF_ERR_UNSUPPORTED, "workspace reduction exists only on the tensor-core path");
   }

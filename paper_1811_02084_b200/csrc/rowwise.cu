@@ -369,19 +369,43 @@ layernorm_bwd_rows_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloa
   }
 }
 
-// out0[c] = sum over g (ascending) of partial[g][0][c], out1[c] likewise from partial[g][1][c]: the fixed-order
-// finish of column sums whose partial sums were left by `groups` producers (planes = 1: one sum only)
+// Fixed-order finish of column sums whose partial sums were left by `groups` producers: partial is [groups][planes][n].
+// A block owns 32 columns; its eight warps each add up one contiguous eighth of the groups in ascending order (loads
+// issued four ahead), and the eight sums are then added in warp order.  The order depends on `groups` only, never on
+// timing, so the result repeats bit for bit.  planes = 2: out0 from plane 0, out1 from plane 1.
 __global__ void __launch_bounds__(256) colsum_finalize_kernel(const float* __restrict__ partial, int groups, int planes, int n, float* __restrict__ out0,
                                                               float* __restrict__ out1) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= n) return;
+  __shared__ float sh[2][8][32];
+  const int tx = threadIdx.x & 31, seg = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + tx;
+  const int g0 = (int)((long long)groups * seg / 8), g1 = (int)((long long)groups * (seg + 1) / 8);
   float s0 = 0.f, s1 = 0.f;
-  for (int g = 0; g < groups; ++g) {
-    s0 += partial[((size_t)g * planes) * n + c];
-    if (planes > 1) s1 += partial[((size_t)g * planes + 1) * n + c];
+  if (c < n) {
+    const size_t stride = (size_t)planes * n;
+    const float* p = partial + (size_t)g0 * stride + c;
+    int g = g0;
+    for (; g + 4 <= g1; g += 4, p += 4 * stride) {
+      const float a0 = p[0], a1 = p[stride], a2 = p[2 * stride], a3 = p[3 * stride];
+      float b0 = 0.f, b1 = 0.f, b2 = 0.f, b3 = 0.f;
+      if (planes > 1) { b0 = p[n]; b1 = p[stride + n]; b2 = p[2 * stride + n]; b3 = p[3 * stride + n]; }
+      s0 = ((s0 + a0) + a1) + a2 + a3;
+      s1 = ((s1 + b0) + b1) + b2 + b3;
+    }
+    for (; g < g1; ++g, p += stride) {
+      s0 += p[0];
+      if (planes > 1) s1 += p[n];
+    }
   }
-  out0[c] = s0;
-  if (planes > 1 && out1) out1[c] = s1;
+  sh[0][seg][tx] = s0;
+  sh[1][seg][tx] = s1;
+  __syncthreads();
+  if (seg == 0 && c < n) {
+    float t0 = sh[0][0][tx], t1 = sh[1][0][tx];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) { t0 += sh[0][w][tx]; t1 += sh[1][w][tx]; }
+    out0[c] = t0;
+    if (planes > 1 && out1) out1[c] = t1;
+  }
 }
 
 // dgamma[c] += sum_rows dy * xh,  dbeta[c] += sum_rows dy.  Block = 32 x 8 threads: 64 columns
@@ -482,7 +506,7 @@ size_t layernorm_bwd_scratch_bytes(int n) {
 }
 
 mtf_status launch_colsum_finalize(const float* partial, int groups, int planes, int n, float* out0, float* out1, void* stream) {
-  colsum_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, (cudaStream_t)stream>>>(partial, groups, planes, n, out0, out1);
+  colsum_finalize_kernel<<<(unsigned)((n + 31) / 32), 256, 0, (cudaStream_t)stream>>>(partial, groups, planes, n, out0, out1);
   count_launch();
   return check("colsum_finalize_kernel");
 }

@@ -81,3 +81,17 @@ def test_bf16_ffn_layouts(mtf, mesh_dims, rules, force):
 def test_bf16_outputs_bf16_grads(mtf):
     inp = ffn_inputs(4, [("batch", 4), ("length", 64)], 256, 512, "bf16", True)
     check_block(mtf, make_layout(mtf, [("all", 4)], [("batch", "all")]), inp, "bf16", grad_dtype="bf16")
+
+
+def test_column_sums_repeat_bit_for_bit(mtf):
+    """dbias = sum over tokens of dhp rides in the dhp launch; with the block's workspace its per-row-group partial
+    sums are finished in a fixed order, so - like every other output of the block - it is identical from run to run."""
+    import torch
+    inp = ffn_inputs(5, [("batch", 8), ("length", 72)], 320, 1088, "bf16", True)
+    runs = []
+    for _ in range(3):
+        _, out = run_ffn_stagewise(mtf, make_layout(mtf, [("rows", 2), ("cols", 4)], [("batch", "rows"), ("d_ff", "cols")]), inp, "bf16")
+        runs.append({k: t.clone() for k, t in out.items()})
+    for r in runs[1:]:
+        for k in runs[0]:
+            assert torch.equal(runs[0][k], r[k]), k
