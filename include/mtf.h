@@ -452,6 +452,15 @@ const char* mtf_last_error(void);
  * Resets the word.  Returns MTF_ERR_TIMEOUT when it was non-zero, else MTF_ERR_INVALID_ARG when a
  * token id or target outside [0, vocab) was seen by the vocab kernels since the last call. */
 mtf_status mtf_device_status(int32_t* code);
+/* Testing hook for the failure path of the bounded device-side waits.  limit_cycles > 0 sets how many SM
+ * cycles a wait may take before it gives up (<= 0 restores the default of about two seconds);
+ * withhold_one_signal != 0 makes every tensor-core launch leave out the "accumulator complete" signal
+ * of its first tile, so that the wait for it runs out: the kernel records a code, all its roles
+ * leave through the common teardown (copies and MMAs in flight are given time to land, tensor memory
+ * is freed), the launch ends normally, its output is unspecified, and the next mtf_device_status
+ * returns MTF_ERR_TIMEOUT.  Nothing traps or faults and the context stays usable.  Affects the current
+ * device until changed back; not for production use. */
+mtf_status mtf_debug_wait_test(int64_t limit_cycles, int32_t withhold_one_signal);
 /* Number of kernels this library has launched from this process (all threads). */
 int64_t mtf_launch_count(void);
 

@@ -154,6 +154,7 @@ def _load():
         "mtf_xent_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), vp, c_size_t, vp],
         "mtf_xent_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor),
                               POINTER(mtf_tensor), vp, c_size_t, vp],
+        "mtf_debug_wait_test": [c_int64, c_int32],
         "mtf_stage_tap_begin": [vp, c_size_t],
         "mtf_stage_tap_end": [POINTER(c_int32)],
         "mtf_stage_tap_entry": [c_int32, POINTER(c_char_p), POINTER(c_size_t), POINTER(c_size_t)],
@@ -643,6 +644,11 @@ def mtf_stage_tap_entry(index: int):
     name, off, size = c_char_p(), c_size_t(), c_size_t()
     _check(_lib.mtf_stage_tap_entry(index, byref(name), byref(off), byref(size)))
     return name.value.decode(), off.value, size.value
+
+
+def mtf_debug_wait_test(limit_cycles: int = 0, withhold_one_signal: bool = False) -> None:
+    """Testing hook: see mtf_debug_wait_test in include/mtf.h."""
+    _check(_lib.mtf_debug_wait_test(int(limit_cycles), 1 if withhold_one_signal else 0))
 
 
 def mtf_launch_count() -> int:

@@ -16,6 +16,7 @@ int64_t launch_count();
 mtf_status read_device_status(int* code);
 mtf_status read_bad_index(int* seen);
 mtf_status read_row_status(int* code);
+mtf_status debug_wait_test(long long limit_cycles, int skip_first_commit);
 }  // namespace mtf
 
 using mtf::Dim;
@@ -631,6 +632,8 @@ mtf_status mtf_device_status(int32_t* code) {
 }
 
 int64_t mtf_launch_count(void) { return mtf::launch_count(); }
+
+mtf_status mtf_debug_wait_test(int64_t limit_cycles, int32_t withhold_one_signal) { return mtf::debug_wait_test(limit_cycles, withhold_one_signal); }
 
 mtf_status mtf_stage_tap_begin(void* device_buffer, size_t bytes) { return mtf::tap_begin(device_buffer, bytes); }
 mtf_status mtf_stage_tap_end(int32_t* n_entries) { return mtf::tap_end(n_entries); }

@@ -52,6 +52,10 @@ constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
 
 __device__ int g_status = 0;
+// Testing hooks (mtf_debug_wait_test): the limit of the bounded waits in cycles, and a switch that makes the MMA
+// issuer leave out the "accumulator complete" signal of its first tile, so that the epilogue's wait for it runs out.
+__device__ long long g_wait_limit = kTimeoutCycles;
+__device__ int g_skip_first_commit = 0;
 
 // Division by a run-time constant as a multiply-high and a shift (exact for dividends below 2^31):
 // the tile decoder runs once per tile in every warp role and 64-bit divisions made it cost more
@@ -260,7 +264,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, int c
     for (int i = 0; i < 128; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kTimeoutCycles) {
+    if (clock64() - t0 > g_wait_limit) {
       atomicCAS(&g_status, 0, code);
       *abort_flag = 1;
       return false;
@@ -285,7 +289,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, in
         __nanosleep(100);
         if (mbar_try_wait(bar, parity)) break;
         if (*abort_flag) { ok = 0; break; }
-        if (clock64() - t0 > kTimeoutCycles) {
+        if (clock64() - t0 > g_wait_limit) {
           atomicCAS(&g_status, 0, code);
           *abort_flag = 1;
           ok = 0;
@@ -817,7 +821,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           umma_commit<kPair>(empty_bar(stage), empty_mask);   // frees the stage in every CTA that writes into this pair's tiles
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit<kPair>(tfull_bar(acc), pair_mask);   // accumulator complete (in both CTAs of the pair)
+        if (ok && !(iter == 0 && g_skip_first_commit)) umma_commit<kPair>(tfull_bar(acc), pair_mask);   // accumulator complete (in both CTAs of the pair)
       }
     }
   } else {
@@ -1109,7 +1113,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             while (*written < (unsigned)sg.nfrag - 1) {
               __nanosleep(64);
               if (*abort_flag) { good = 0; break; }
-              if (clock64() - t0 > kTimeoutCycles) { atomicCAS(&g_status, 0, 0x600); *abort_flag = 1; good = 0; break; }
+              if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, 0x600); *abort_flag = 1; good = 0; break; }
             }
             __threadfence();
           }
@@ -1809,6 +1813,16 @@ mtf_status builtin_scratch_ptr(void** out) {
     cached[dev] = p;
   }
   *out = cached[dev];
+  return MTF_OK;
+}
+
+// Testing hook: limit of the bounded device-side waits in SM cycles (<= 0: the default of about two seconds) and,
+// with skip_first_commit != 0, a signal that is deliberately never sent (see g_skip_first_commit).
+mtf_status debug_wait_test(long long limit_cycles, int skip_first_commit) {
+  const long long lim = limit_cycles > 0 ? limit_cycles : kTimeoutCycles;
+  cudaError_t e = cudaMemcpyToSymbol(g_wait_limit, &lim, sizeof(lim));
+  if (e == cudaSuccess) e = cudaMemcpyToSymbol(g_skip_first_commit, &skip_first_commit, sizeof(int));
+  if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemcpyToSymbol: %s", cudaGetErrorString(e));
   return MTF_OK;
 }
 
