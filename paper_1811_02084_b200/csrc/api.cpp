@@ -17,6 +17,7 @@ mtf_status read_device_status(int* code);
 mtf_status read_bad_index(int* seen);
 mtf_status read_row_status(int* code);
 mtf_status debug_wait_test(long long limit_cycles, int skip_first_commit);
+mtf_status read_attention_status(int* code);
 }  // namespace mtf
 
 using mtf::Dim;
@@ -620,7 +621,8 @@ mtf_status mtf_device_status(int32_t* code) {
   if (code) *code = c;
   if (st != MTF_OK) return st;
   int rc = 0;
-  if ((st = mtf::read_row_status(&rc)) != MTF_OK) return st;
+  if ((st = mtf::read_attention_status(&rc)) != MTF_OK) return st;
+  if (!rc && (st = mtf::read_row_status(&rc)) != MTF_OK) return st;
   if (rc) {
     if (code) *code = rc;
     return fail(MTF_ERR_TIMEOUT, "a bounded device-side wait gave up (code 0x%x)", rc);

@@ -18,6 +18,9 @@ mtf_status launch_layernorm_fwd(const void* x, const float* gamma, const float* 
 mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stats, const float* gamma, const void* residual, void* dx,
                                 float* dgamma, float* dbeta, int64_t rows, int n, void* scratch, size_t scratch_bytes, void* stream);
 size_t layernorm_bwd_scratch_bytes(int n);
+bool attention_fused_supported(int64_t L, int64_t d_k, int64_t d_v);
+mtf_status launch_attention_fwd_fused(const void* q, const void* kk, const void* vv, void* weights, void* o, int64_t B, int64_t H, int64_t L, float scale,
+                                      int causal, void* stream);
 mtf_status ffn_forward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias, const mtf_tensor* v,
                             mtf_tensor* h_saved, mtf_tensor* y, const mtf_tensor* y_residual, void* workspace, size_t workspace_bytes, void* stream);
 mtf_status ffn_backward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* v, const mtf_tensor* h_saved,
@@ -281,6 +284,30 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
       st = ein(layout, xm.t, *wv, vv, nullptr, rest, rest_bytes, stream);
     }
     if (st != MTF_OK) return st;
+  }
+  // The whole core - logits, softmax, weights . v - in one launch when the shapes allow it (d_k = d_v = 64, rows of at most
+  // 512 logits, only batch and heads split, tensors in the canonical dimension orders): every (batch, head) pair is an
+  // independent problem on the processor that owns it, so the layout only decides who computes which pair.
+  {
+    auto unsplit = [&](const mtf_dim& d) { const int j = layout->mesh_dim_of(d.name); return j < 0 || layout->mesh[j].size == 1; };
+    auto order = [](const mtf_tensor* t, std::initializer_list<mtf_dim> want) {
+      if (t->ndim != (int)want.size() || t->dtype != MTF_BF16 || !t->data) return false;
+      int i = 0;
+      for (auto& w : want) { if (strcmp(t->dims[i].name, w.name) != 0 || t->dims[i].size != w.size) return false; ++i; }
+      return true;
+    };
+    const bool canonical = order(q, {s.b, s.l, s.h, s.k}) && order(kk, {s.b, s.m, s.h, s.k}) && order(vv, {s.b, s.m, s.h, s.v}) &&
+                           order(weights, {s.b, s.h, s.l, s.m}) && order(o, {s.b, s.l, s.h, s.v});
+    // (legality and divisibility of the batch and heads splits were checked by the projections' plans above)
+    if (canonical && mtf::attention_fused_supported(s.l.size, s.k.size, s.v.size) && unsplit(s.l) && unsplit(s.m) && unsplit(s.k) && unsplit(s.v)) {
+      if ((st = mtf::launch_attention_fwd_fused(q->data, kk->data, vv->data, weights->data, o->data, s.b.size, s.h.size, s.l.size, (float)s.scale, causal ? 1 : 0,
+                                                stream)) != MTF_OK)
+        return st;
+      mtf_epilogue er2 = epi_none();
+      er2.residual = residual;
+      if ((st = ein(layout, *o, *wo, y, residual ? &er2 : nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+      return mtf::rank_wait(layout, stream);
+    }
   }
   mtf_epilogue es = epi_none();
   es.scale = (float)s.scale;
