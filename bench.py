@@ -682,6 +682,24 @@ def run_secondary(mtf, peaks, blocks=True, reps=None):
     ms = timer(lambda: mtf.mtf_transpose(lay, nxt2, nxo2), 20, stream)
     rows.append(("permute_transpose_kernel", f"[{Bt * Lt}, {Ht * Kt}] bf16 -> [d_model, tokens]", 2 * qt.numel() * 2, ms))
     mtf.mtf_device_status()
+    # the generic kernel (config 1: the fp32 example of Section 8 on mesh [2,2]; parity path, never tuned) and the slice gather
+    lay1 = mtf.mtf_layout(mtf.mtf_mesh_create([("rows", 2), ("cols", 2)]), [("batch", "rows"), ("hidden", "cols")])
+    x1, w1 = to_device(si.normal(0, "x", [8, 64], "f32")), to_device(si.normal(0, "w", [64, 256], "f32", 0.125))
+    h1 = torch.empty(8, 256, dtype=torch.float32, device="cuda")
+    nx1, nw1, nh1 = Nn(x1, ["batch", "io"]), Nn(w1, ["io", "hidden"]), Nn(h1, ["batch", "hidden"])
+    ms = timer(lambda: mtf.mtf_einsum(lay1, None, [nx1, nw1], nh1, None), 50, stream)
+    out.append({"metric": "einsum_simt_kernel_ms", "kernel": "einsum_simt_kernel", "value": ms, "unit": "ms", "ms": ms,
+                "config": {"workload": "config 1: x[8, 64] . w[64, 256] in fp32 on mesh [2,2] (131072 multiply-adds: launch-bound)"},
+                "roofline": {"bound": "alu", "achieved": 2.0 * 8 * 64 * 256 / (ms * 1e-3) / 1e12, "peak": 148 * 128 * 2 * 1.965e9 / 1e12, "unit": "TFLOP/s",
+                             "frac": 2.0 * 8 * 64 * 256 / (ms * 1e-3) / (148 * 128 * 2 * 1.965e9),
+                             "note": "fp32 FMA peak = 148 SMs x 128 lanes x 2 flop x 1.965 GHz; a 0.26 MFLOP problem measures launch latency only"}})
+    gl = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 8)]), [("d_ff", "all")])
+    gsrc = torch.empty(8192, 8192, dtype=torch.bfloat16, device="cuda")
+    gdst = torch.empty(8192, 1024, dtype=torch.bfloat16, device="cuda")
+    ngs = Nn(gsrc, ["tokens", "d_ff"])
+    ms = timer(lambda: mtf.mtf_slice_gather(gl, ngs, 3, gdst), 20, stream)
+    rows.append(("slice_gather_kernel", "processor 3's slice [8192, 1024] of a bf16 [8192, 8192] tensor (d_ff split 8 ways)", 2 * gdst.numel() * 2, ms))
+    mtf.mtf_device_status()
     for kernel, shape, nbytes, ms in rows:
         gbs = nbytes / (ms * 1e-3) / 1e9
         out.append({"metric": "row_kernel_gbs", "kernel": kernel, "value": gbs, "unit": "GB/s", "ms": ms, "config": {"workload": shape},
