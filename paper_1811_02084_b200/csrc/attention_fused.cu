@@ -9,17 +9,20 @@
 // 512} (a whole row of logits fits the 512 columns of tensor memory); other shapes take the launch-per-
 // einsum path.
 //
-// A persistent CTA (one per SM) walks (batch, head) pairs; K and V of the pair stay in shared memory for
-// all its query tiles of 128 rows.  Warp roles (320 threads):
-//   warp 0     TMA producer: K, V once per pair; Q per tile (two buffers)
+// A persistent CTA (one per SM) walks a contiguous, balanced range of (pair, query tile of 128 rows) items; K and V
+// of a (batch, head) pair stay in shared memory for all of the pair's tiles in the range, K of the next pair is
+// fetched as soon as the last logits of this one are complete, V as soon as its last weights . v is.
+// Warp roles (576 threads):
+//   warp 0     TMA producer: K, V once per pair; Q per tile
 //   warp 1     MMA issuer:   S = Q K^T (tcgen05.mma kind::f16, N up to 256 per instruction), then
 //                            O += P_c V_c for every 64-key chunk c of P as it arrives in shared memory
-//   warps 2-9  softmax:      two warps per tensor-memory lane quarter, each owns half of the row's columns;
-//                            row maximum and row sum are exchanged through shared memory; the normalised
-//                            weights are written as swizzled 32-row boxes (TMA store + MMA operand)
+//   warps 2-17 softmax:      four warps per tensor-memory lane quarter; warp part p owns the 64-key chunks c with
+//                            c mod 4 = p and the chunk buffer p; row maximum and row sum are exchanged through
+//                            shared memory at a named barrier of the quarter's 128 threads; the normalised weights
+//                            are written as swizzled 32-row boxes (TMA store + MMA operand)
 // O is accumulated in the tensor-memory columns of the first chunk of S, which are dead by then.
-// Every wait is bounded; on expiry a code is recorded in the status word, a CTA-wide abort flag is raised
-// and all roles leave through the teardown.
+// Every mbarrier wait is bounded; on expiry a code is recorded in the status word, a CTA-wide abort flag is raised,
+// the remaining waits return at once, work is skipped, and all roles leave through the teardown.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -31,10 +34,11 @@
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kSoftmaxWarps = 16;                 // four per tensor-memory lane quarter
+constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kQBytes = 128 * 64 * 2;            // one query tile
 constexpr int kPBufBytes = 128 * 64 * 2;         // one 64-key chunk of the weights for 128 rows
-constexpr int kPBufs = 3;
+constexpr int kPBufs = 4;                         // one chunk buffer per softmax part: a buffer is written by the same four warps every time
 constexpr int kMaxL = 512;
 constexpr long long kWaitCycles = 4000000000LL;
 
@@ -140,9 +144,6 @@ __device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t x, uint32_t y, ui
 
 // live 64-key chunks of query tile qt: all of them, or under the causal limit those that hold a key <= the tile's last row
 __device__ __forceinline__ int live_chunks(const AttArgs& a, int qt) { return a.causal ? min(a.L / 64, 2 * (qt + 1)) : a.L / 64; }
-// the order in which the chunks of a tile are produced and consumed: alternately from the first and the second half of the row
-// (position p = 0, 1, 2, ... -> chunk index); nc = chunks per row
-__device__ __forceinline__ int chunk_at(int p, int nc) { return (p & 1) ? nc / 2 + (p >> 1) : (p >> 1); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -152,22 +153,27 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const int L = a.L, nc = L / 64, q_tiles = L / 128;
-  // layout: Q[2] | K (L rows) | V (L rows) | P ring | zero box | exchange slots | barriers
-  const uint32_t sQ = base, sK = sQ + 2 * kQBytes, sV = sK + (uint32_t)L * 128u, sP = sV + (uint32_t)L * 128u;
+  // layout: Q | K (L rows) | V (L rows) | P chunk buffers | zero box | exchange slots | barriers
+  const uint32_t sQ = base, sK = sQ + kQBytes, sV = sK + (uint32_t)L * 128u, sP = sV + (uint32_t)L * 128u;
   const uint32_t sZero = sP + kPBufs * kPBufBytes;
-  const uint32_t sX = sZero + 4096u;                          // [2 slots][8 warps][32 lanes] x 8 bytes
-  const uint32_t bar0 = sX + 2u * 8u * 32u * 8u;
+  const uint32_t sX = sZero + 4096u;                          // [2 slots][16 warps][32 lanes] floats
+  const uint32_t bar0 = sX + 2u * kSoftmaxWarps * 32u * 4u;
   uint64_t* bars_gen = reinterpret_cast<uint64_t*>(gen + (bar0 - base));
-  // barriers: 0,1 q_full; 2,3 q_empty; 4 kv_full; 5 kv_empty; 6 s_full; 7 o_full; 8 o_empty; 9..11 p_full; 12..14 p_free
+  // barriers: 0 q_full; 1 q_empty; 2 v_full; 3 v_empty; 4 k_full; 5 k_empty; 6 s_full; 7 o_full; 8 o_empty; 9..12 p_full (the four quarter boxes of
+  // a chunk buffer are written); 13..16 p_free (the MMAs that read a chunk buffer have retired).  Every barrier has one set of
+  // waiters that see each of its phases in order, so a parity wait can never be a phase behind.
   auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 16);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars_gen + 24);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // this CTA's query tiles: a contiguous, balanced range of all (pair, tile) items
+  const long long total_tiles = a.units * q_tiles;
+  const long long g0 = total_tiles * blockIdx.x / gridDim.x, g1 = total_tiles * (blockIdx.x + 1) / gridDim.x;
 
   if (threadIdx.x == 0) {
     mb_init(bar(0), 1); mb_init(bar(1), 1); mb_init(bar(2), 1); mb_init(bar(3), 1);
     mb_init(bar(4), 1); mb_init(bar(5), 1); mb_init(bar(6), 1); mb_init(bar(7), 1); mb_init(bar(8), 4);
-    for (int i = 0; i < kPBufs; ++i) { mb_init(bar(9 + i), 4); mb_init(bar(12 + i), 1); }
+    for (int i = 0; i < kPBufs; ++i) { mb_init(bar(9 + i), 4); mb_init(bar(13 + i), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
@@ -176,7 +182,6 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_p) : "memory");
   }
   for (int i = threadIdx.x; i < 4096 / 16; i += kThreads) sts_v4(sZero + 16u * i, 0u, 0u, 0u, 0u);
-  for (int i = threadIdx.x; i < 2 * 8 * 32; i += kThreads) asm volatile("st.shared.v2.b32 [%0], {%1, %1};" ::"r"(sX + 8u * i), "r"(0u) : "memory");
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s_u32(tmem_slot)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -192,34 +197,50 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (warp == 0) {
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
-      long long tile_seq = 0, unit_seq = 0;
+      long long tile_seq = 0, unit_seq = -1;
       bool ok = true;
-      for (long long u = blockIdx.x; ok && u < a.units; u += gridDim.x, ++unit_seq) {
+      for (long long g = g0; ok && g < g1; ++g, ++tile_seq) {
+        const long long u = g / q_tiles;
+        const int qt = (int)(g % q_tiles);
         const int b = (int)(u / a.H), h = (int)(u % a.H);
-        if (!(ok = mb_wait(bar(5), ((uint32_t)unit_seq & 1u) ^ 1u, 0x901, abort_flag))) break;      // K, V of the previous pair are no longer read
-        mb_expect(bar(4), (uint32_t)L * 256u);
-        for (int r = 0; r < L; r += 128) tma_load_4d(sK + (uint32_t)r * 128u, &map_k, bar(4), 0, r, h, b);
-        for (int r = 0; r < L; r += 64) tma_load_4d(sV + (uint32_t)r * 128u, &map_v, bar(4), 0, r, h, b);
-        for (int qt = 0; qt < q_tiles; ++qt, ++tile_seq) {
-          const int qb = (int)(tile_seq & 1);
-          if (!(ok = mb_wait(bar(2 + qb), (((uint32_t)(tile_seq >> 1)) & 1u) ^ 1u, 0x902, abort_flag))) break;
-          mb_expect(bar(qb), kQBytes);
-          tma_load_4d(sQ + qb * kQBytes, &map_q, bar(qb), 0, qt * 128, h, b);
+        const bool new_unit = g == g0 || qt == 0;
+        if (new_unit) {
+          ++unit_seq;
+          if (!(ok = mb_wait(bar(5), ((uint32_t)unit_seq & 1u) ^ 1u, 0x901, abort_flag))) break;      // K of the previous pair is no longer read
+          mb_expect(bar(4), (uint32_t)L * 128u);
+          for (int r = 0; r < L; r += 128) tma_load_4d(sK + (uint32_t)r * 128u, &map_k, bar(4), 0, r, h, b);
+        }
+        if (!(ok = mb_wait(bar(1), ((uint32_t)tile_seq & 1u) ^ 1u, 0x902, abort_flag))) break;        // the logits of the previous tile are complete
+        mb_expect(bar(0), kQBytes);
+        tma_load_4d(sQ, &map_q, bar(0), 0, qt * 128, h, b);
+        if (new_unit) {
+          // V is wanted only after the softmax of the pair's first tile: its load waits for the previous pair's last MMA
+          // without holding up K and Q
+          if (!(ok = mb_wait(bar(3), ((uint32_t)unit_seq & 1u) ^ 1u, 0x903, abort_flag))) break;
+          mb_expect(bar(2), (uint32_t)L * 128u);
+          for (int r = 0; r < L; r += 64) tma_load_4d(sV + (uint32_t)r * 128u, &map_v, bar(2), 0, r, h, b);
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer ---------------------------------
     if (lane == 0) {
-      long long tile_seq = 0, unit_seq = 0, pseq = 0;
+      long long tile_seq = 0, unit_seq = -1;
+      uint32_t pu[kPBufs] = {0u, 0u, 0u, 0u};          // uses of every chunk buffer so far
+      const uint64_t dP0 = smem_desc(sP, 0), dV0 = smem_desc(sV, 1), dQ0 = smem_desc(sQ, 0), dK0 = smem_desc(sK, 0);
       bool ok = true;
-      for (long long u = blockIdx.x; ok && u < a.units; u += gridDim.x, ++unit_seq) {
-        if (!(ok = mb_wait(bar(4), (uint32_t)unit_seq & 1u, 0x911, abort_flag))) break;
-        for (int qt = 0; qt < q_tiles; ++qt, ++tile_seq) {
-          const int qb = (int)(tile_seq & 1);
+      {
+        for (long long g = g0; ok && g < g1; ++g, ++tile_seq) {
+          const int qt = (int)(g % q_tiles);
+          const bool new_unit = g == g0 || qt == 0;
+          const bool last_of_unit = qt == q_tiles - 1 || g == g1 - 1;
+          if (new_unit) {
+            ++unit_seq;
+            if (!(ok = mb_wait(bar(4), (uint32_t)unit_seq & 1u, 0x911, abort_flag))) break;
+          }
           const int live = live_chunks(a, qt);
           const int keys = live * 64 > L ? L : ((live * 64 + 127) / 128) * 128;      // logits columns to compute (whole 128-key blocks)
-          if (!(ok = mb_wait(bar(qb), ((uint32_t)(tile_seq >> 1)) & 1u, 0x912, abort_flag))) break;
+          if (!(ok = mb_wait(bar(0), (uint32_t)tile_seq & 1u, 0x912, abort_flag))) break;
           if (!(ok = mb_wait(bar(8), ((uint32_t)tile_seq & 1u) ^ 1u, 0x913, abort_flag))) break;       // O of the previous tile has been read out
           fence_after();
           // S = Q K^T: up to two instructions shapes of N <= 256 columns
@@ -228,208 +249,226 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(nn >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 #pragma unroll
             for (int k = 0; k < 4; ++k)
-              umma(tmem + (uint32_t)n0, smem_desc(sQ + qb * kQBytes + k * 32u, 0), smem_desc(sK + (uint32_t)n0 * 128u + k * 32u, 0), idesc, k != 0);
+              umma(tmem + (uint32_t)n0, dQ0 + 2u * k, dK0 + (uint64_t)(((uint32_t)n0 * 128u) >> 4) + 2u * k, idesc, k != 0);
           }
           umma_commit(bar(6));               // logits complete
-          umma_commit(bar(2 + qb));          // ... and this Q buffer may be refilled
+          umma_commit(bar(1));               // ... and the Q buffer may be refilled
+          if (last_of_unit) umma_commit(bar(5));           // ... and so may K
+          if (new_unit && !(ok = mb_wait(bar(2), (uint32_t)unit_seq & 1u, 0x915, abort_flag))) break;
           // O += P_c V_c, chunk by chunk in the order the softmax warps deliver them
           const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-          int done = 0;
-          for (int p = 0; p < nc && ok; ++p) {
-            const int c = chunk_at(p, nc);
-            if (c >= live) continue;
-            const int buf = (int)(pseq % kPBufs);
-            if (!(ok = mb_wait(bar(9 + buf), (uint32_t)(pseq / kPBufs) & 1u, 0x914, abort_flag))) break;
+          for (int c = 0; c < live && ok; ++c) {
+            const int buf = c & 3;
+            if (!(ok = mb_wait(bar(9 + buf), pu[buf] & 1u, 0x914, abort_flag))) break;
             fence_after();
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma(tmem, smem_desc(sP + buf * kPBufBytes + k * 32u, 0), smem_desc(sV + (uint32_t)c * 8192u + k * 2048u, 1), idesc_pv, (done | k) != 0);
-            umma_commit(bar(12 + buf));      // the chunk's buffer may be rewritten
-            ++done;
-            ++pseq;
+            const uint64_t da = dP0 + (uint64_t)((uint32_t)buf * (kPBufBytes >> 4));
+            const uint64_t db = dV0 + (uint64_t)((uint32_t)c * (8192u >> 4));
+            umma(tmem, da, db, idesc_pv, (uint32_t)c);
+            umma(tmem, da + 2u, db + (2048u >> 4), idesc_pv, 1u);
+            umma(tmem, da + 4u, db + 2u * (2048u >> 4), idesc_pv, 1u);
+            umma(tmem, da + 6u, db + 3u * (2048u >> 4), idesc_pv, 1u);
+            umma_commit(bar(13 + buf));      // the chunk's buffer may be rewritten
+            ++pu[buf];
           }
           if (!ok) break;
           umma_commit(bar(7));               // O complete
-          if (qt == q_tiles - 1) umma_commit(bar(5));      // K, V of this pair are no longer read
+          if (last_of_unit) umma_commit(bar(3));           // V of this pair is no longer read
         }
       }
     }
   } else {
     // ------------------------------- softmax warps ------------------------------
     const int q = warp & 3;                        // tensor-memory lane quarter this warp may access
-    // two warps share a lane quarter: warps with the same (warp & 3); the one with the smaller warp index takes the first half of the columns
-    const int my_half = (warp - 2) >= 4 ? 1 : 0;
-    const int peer_warp = my_half ? warp - 4 : warp + 4;
-    const uint32_t my_slot = sX + 8u * (uint32_t)((warp - 2) * 32 + lane);
-    const uint32_t peer_slot = sX + 8u * (uint32_t)((peer_warp - 2) * 32 + lane);
+    const int part = (warp - 2) >> 2;              // which of the four warps of the quarter: owns chunks c with c % 4 == part
+    const int slot_id = part * 4 + q;              // 0..15
     const float sl2 = a.scale * 1.4426950408889634f;
     const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16);
-    long long tile_seq = 0, pseq = 0;
+    long long tile_seq = 0;
+    uint32_t pu = 0;                               // uses of this part's chunk buffer so far
     bool ok = true;
-    auto exchange = [&](int slot, float mine, bool take_max, uint32_t seq) -> float {
-      const uint32_t off = (uint32_t)slot * (8u * 8u * 32u);
-      asm volatile("st.volatile.shared.v2.b32 [%0], {%1, %2};" ::"r"(my_slot + off), "r"(__float_as_uint(mine)), "r"(seq) : "memory");
-      uint32_t vb = 0, sq = 0;
-      int tries = 0;
-      do {
-        asm volatile("ld.volatile.shared.v2.b32 {%0, %1}, [%2];" : "=r"(vb), "=r"(sq) : "r"(peer_slot + off) : "memory");
-      } while (sq != seq && ++tries < (1 << 24) && !*abort_flag);
-      if (sq != seq) { atomicCAS(&g_att_status, 0, 0x920 + slot); *abort_flag = 1; }
-      const float other = __uint_as_float(vb);
-      return take_max ? fmaxf(mine, other) : mine + other;
+    // row statistics of the four warps that share a row: every warp publishes its value, the 128 threads of the lane quarter
+    // meet at a named barrier (the waiting warps take no issue slots), and each reads its three peers'.  The two exchanges
+    // of a tile use different slots, so a slot is rewritten only after the other slot's barrier.  Every softmax warp
+    // reaches every barrier, also after a failed wait (it skips the work, not the meeting).
+    auto exchange = [&](int slot, float mine, bool take_max) -> float {
+      const uint32_t off = sX + (uint32_t)slot * (4u * kSoftmaxWarps * 32u);
+      asm volatile("st.shared.b32 [%0], %1;" ::"r"(off + 4u * (uint32_t)(slot_id * 32 + lane)), "r"(__float_as_uint(mine)) : "memory");
+      asm volatile("bar.sync %0, 128;" ::"r"(1 + q) : "memory");
+      float r = mine;
+#pragma unroll
+      for (int pp = 1; pp < 4; ++pp) {
+        uint32_t vb;
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(vb) : "r"(off + 4u * (uint32_t)((((part + pp) & 3) * 4 + q) * 32 + lane)) : "memory");
+        const float other = __uint_as_float(vb);
+        r = take_max ? fmaxf(r, other) : r + other;
+      }
+      return r;
     };
-    for (long long u = blockIdx.x; ok && u < a.units; u += gridDim.x) {
-      const int b = (int)(u / a.H), h = (int)(u % a.H);
-      for (int qt = 0; qt < q_tiles && ok; ++qt, ++tile_seq) {
+    auto wait_all = [&](int b, uint32_t parity, int code) -> bool {      // all lanes wait (lane 0 polls first)
+      int w_ok = 1;
+      if (lane == 0) w_ok = mb_wait(bar(b), parity, code, abort_flag) ? 1 : 0;
+      w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
+      if (!w_ok) return false;
+      bool mine_ok = lane == 0 ? true : mb_wait(bar(b), parity, code, abort_flag);
+      return __all_sync(0xffffffffu, mine_ok);
+    };
+    // The trip counts below depend on the arguments alone: after a failed wait a warp keeps going through the tiles (waits
+    // then return at once, work is skipped) so that its peers never wait for it at a named barrier.
+    {
+      for (long long g = g0; g < g1; ++g, ++tile_seq) {
+        const long long u = g / q_tiles;
+        const int qt = (int)(g % q_tiles);
+        const int b = (int)(u / a.H), h = (int)(u % a.H);
         const int live = live_chunks(a, qt);
         const int row = qt * 128 + q * 32 + lane;                 // query position of this thread's row
         const int lim = a.causal ? min(L, row + 1) : L;            // columns [0, lim) take part
-        const int c_lo = my_half * (L / 2), c_hi = c_lo + L / 2;   // this warp's columns
         const int lim_warp = __shfl_sync(0xffffffffu, lim, 31);    // the warp's widest row
         const int lim_all = __shfl_sync(0xffffffffu, lim, 0);      // columns below it take part in every row of the warp
-        const uint32_t seq = (uint32_t)tile_seq + 1u;
-        {
-          int w_ok = 1;
-          if (lane == 0) w_ok = mb_wait(bar(6), (uint32_t)tile_seq & 1u, 0x921, abort_flag) ? 1 : 0;
-          w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
-          if (!w_ok) { ok = false; break; }
-          if (lane != 0 && !mb_wait(bar(6), (uint32_t)tile_seq & 1u, 0x921, abort_flag)) { ok = false; }
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-        }
+        if (ok) ok = wait_all(6, (uint32_t)tile_seq & 1u, 0x921);
         fence_after();
-        // pass 1: row maximum over this warp's live columns
+        // pass 1: row maximum over this warp's live columns (chunks part, part + 4, ...)
         float mx = -INFINITY;
+        if (ok) {
 #pragma unroll 1
-        for (int c0 = c_lo; c0 < min(c_hi, lim_warp); c0 += 32) {
-          uint32_t rawv[32];
-          tmem_ld32(taddr + (uint32_t)c0, rawv);
-          tmem_ld_wait();
-          if (c0 + 32 <= lim_all) {
+          for (int c = part; c < live; c += 4) {
+            const int c0 = c * 64;
+            if (c0 + 64 <= lim_all) {
+              uint32_t rawv[64];
+              tmem_ld32(taddr + (uint32_t)c0, rawv);
+              tmem_ld32(taddr + (uint32_t)c0 + 32u, rawv + 32);
+              tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rawv[j]));
-          } else {
+              for (int j = 0; j < 64; ++j) mx = fmaxf(mx, __uint_as_float(rawv[j]));
+            } else {
+#pragma unroll 1
+              for (int cc = c0; cc < c0 + 64 && cc < lim_warp; cc += 32) {
+                uint32_t rawv[32];
+                tmem_ld32(taddr + (uint32_t)cc, rawv);
+                tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c0 + j < lim) mx = fmaxf(mx, __uint_as_float(rawv[j]));
+                for (int j = 0; j < 32; ++j)
+                  if (cc + j < lim) mx = fmaxf(mx, __uint_as_float(rawv[j]));
+              }
+            }
           }
         }
-        mx = exchange(0, mx, true, seq) * sl2;
+        mx = exchange(0, mx, true) * sl2;
         // pass 2: exponentials (kept in tensor memory in place of the logits) and their sum
         float sum = 0.f;
+        if (ok) {
 #pragma unroll 1
-        for (int c0 = c_lo; c0 < min(c_hi, lim_warp); c0 += 32) {
-          uint32_t rawv[32];
-          tmem_ld32(taddr + (uint32_t)c0, rawv);
-          tmem_ld_wait();
-          if (c0 + 32 <= lim_all) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float e = ex2(fmaf(__uint_as_float(rawv[j]), sl2, -mx));
-              sum += e;
-              rawv[j] = __float_as_uint(e);
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float e = (c0 + j < lim) ? ex2(fmaf(__uint_as_float(rawv[j]), sl2, -mx)) : 0.f;
-              sum += e;
-              rawv[j] = __float_as_uint(e);
-            }
-          }
-          tmem_st32(taddr + (uint32_t)c0, rawv);
-        }
-        tmem_st_wait();
-        sum = exchange(1, sum, false, seq);
-        const float inv = 1.f / sum;
-        if (*abort_flag) { ok = false; }
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // pass 3: normalised weights, chunk by chunk of 64 keys, into the ring (live chunks: store + MMA operand)
-        // or straight from the zero box (chunks that lie wholly beyond the causal limit of the tile)
-        const int row0 = qt * 128 + q * 32;
-        for (int p = 0; p < nc && ok; ++p) {
-          const int c = chunk_at(p, nc);
-          const bool mine = (c >= nc / 2) == (my_half == 1);
-          if (c >= live) {
-            if (mine && lane == 0) tma_store_4d(&map_p, sZero, c * 64, row0, h, b);
-            continue;
-          }
-          const int buf = (int)(pseq % kPBufs);
-          const long long use = pseq / kPBufs;
-          ++pseq;
-          if (!mine) continue;
-          // the buffer is free when the MMAs that read its previous contents have retired (whoever stored from it waited for
-          // that store to have read the buffer before reporting the chunk, see below)
-          {
-            int w_ok = 1;
-            if (lane == 0) w_ok = mb_wait(bar(12 + buf), ((uint32_t)use & 1u) ^ 1u, 0x922, abort_flag) ? 1 : 0;
-            w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
-            if (!w_ok) { ok = false; break; }
-          }
-          const uint32_t box = sP + buf * kPBufBytes + (uint32_t)q * 4096u;        // this warp's 32 rows of the chunk
-          const uint32_t rowaddr = box + (uint32_t)lane * 128u;
-          const uint32_t swz = (uint32_t)(lane & 7);
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            const int c0 = c * 64 + hh * 32;
-            float v[32];
-            if (c0 < lim_warp) {
+          for (int c = part; c < live; c += 4) {
+#pragma unroll 1
+            for (int c0 = c * 64; c0 < c * 64 + 64 && c0 < lim_warp; c0 += 32) {
               uint32_t rawv[32];
               tmem_ld32(taddr + (uint32_t)c0, rawv);
               tmem_ld_wait();
+              if (c0 + 32 <= lim_all) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(rawv[j]) * inv;
-            } else {
+                for (int j = 0; j < 32; ++j) {
+                  const float e = ex2(fmaf(__uint_as_float(rawv[j]), sl2, -mx));
+                  sum += e;
+                  rawv[j] = __float_as_uint(e);
+                }
+              } else {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                for (int j = 0; j < 32; ++j) {
+                  const float e = (c0 + j < lim) ? ex2(fmaf(__uint_as_float(rawv[j]), sl2, -mx)) : 0.f;
+                  sum += e;
+                  rawv[j] = __float_as_uint(e);
+                }
+              }
+              tmem_st32(taddr + (uint32_t)c0, rawv);
             }
-#pragma unroll
-            for (int qq = 0; qq < 4; ++qq)
-              sts_v4(rowaddr + ((((uint32_t)(hh * 4 + qq)) ^ swz) << 4), pack2(v[qq * 8], v[qq * 8 + 1]), pack2(v[qq * 8 + 2], v[qq * 8 + 3]),
-                     pack2(v[qq * 8 + 4], v[qq * 8 + 5]), pack2(v[qq * 8 + 6], v[qq * 8 + 7]));
           }
+          tmem_st_wait();
+        }
+        sum = exchange(1, sum, false);
+        const float inv = 1.f / sum;
+        if (*abort_flag) ok = false;
+        ok = __all_sync(0xffffffffu, ok);
+        // pass 3: normalised weights of this warp's chunks: live ones into this part's chunk buffer (source of the store to
+        // HBM and A operand of O += P_c V_c), chunks wholly beyond the tile's causal limit straight from the zero box
+        const int row0 = qt * 128 + q * 32;
+        const uint32_t box = sP + (uint32_t)part * kPBufBytes + (uint32_t)q * 4096u;        // this warp's 32 rows of the buffer
+        const uint32_t rowaddr = box + (uint32_t)lane * 128u;
+        const uint32_t swz = (uint32_t)(lane & 7);
+        for (int c = part; c < nc && ok; c += 4) {
+          if (c >= live) {
+            if (lane == 0) tma_store_4d(&map_p, sZero, c * 64, row0, h, b);
+            continue;
+          }
+          // the values first (tensor-memory reads and arithmetic depend on nobody) ...
+          uint32_t pk[32];
+          if (c * 64 + 64 <= lim_warp) {
+            uint32_t rawv[64];
+            tmem_ld32(taddr + (uint32_t)(c * 64), rawv);
+            tmem_ld32(taddr + (uint32_t)(c * 64) + 32u, rawv + 32);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) pk[j] = pack2(__uint_as_float(rawv[2 * j]) * inv, __uint_as_float(rawv[2 * j + 1]) * inv);
+          } else {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const int c0 = c * 64 + hh * 32;
+              if (c0 < lim_warp) {
+                uint32_t rawv[32];
+                tmem_ld32(taddr + (uint32_t)c0, rawv);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[hh * 16 + j] = pack2(__uint_as_float(rawv[2 * j]) * inv, __uint_as_float(rawv[2 * j + 1]) * inv);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[hh * 16 + j] = 0u;
+              }
+            }
+          }
+          // ... then the box: free when this warp's previous store from it has read it and the MMAs that read the buffer's
+          // previous contents have retired
+          {
+            int w_ok = 1;
+            if (lane == 0) {
+              asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+              w_ok = mb_wait(bar(13 + part), (pu & 1u) ^ 1u, 0x922, abort_flag) ? 1 : 0;
+            }
+            w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
+            if (!w_ok) { ok = false; break; }
+          }
+#pragma unroll
+          for (int pc = 0; pc < 8; ++pc)
+            sts_v4(rowaddr + ((((uint32_t)pc) ^ swz) << 4), pk[pc * 4], pk[pc * 4 + 1], pk[pc * 4 + 2], pk[pc * 4 + 3]);
           fence_before();
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
           if (lane == 0) {
-            // store first and wait until the store has read the box: after that only the MMAs read it, and their
-            // completion (p_free) is all the next writer - possibly another warp - has to wait for
-            tma_store_4d(&map_p, box, c * 64, row0, h, b);
-            asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-            mb_arrive(bar(9 + buf));                                   // one of the four quarter boxes of the chunk is in place
+            mb_arrive(bar(9 + part));                                  // one of the four quarter boxes of the chunk is in place: the MMAs may read it
+            tma_store_4d(&map_p, box, c * 64, row0, h, b);             // ... and so does the store (both only read)
           }
+          ++pu;
         }
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // the first-half warps read O (64 columns, accumulated over the first chunk's columns) and write it out
-        if (my_half == 0) {
-          {
-            int w_ok = 1;
-            if (lane == 0) w_ok = mb_wait(bar(7), (uint32_t)tile_seq & 1u, 0x923, abort_flag) ? 1 : 0;
-            w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
-            if (!w_ok) { ok = false; break; }
-            if (lane != 0 && !mb_wait(bar(7), (uint32_t)tile_seq & 1u, 0x923, abort_flag)) ok = false;
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-          }
+        // the part-0 warps read O (64 columns, accumulated over the first chunk's columns) and write it out
+        if (part == 0 && ok) {
+          ok = wait_all(7, (uint32_t)tile_seq & 1u, 0x923);
           fence_after();
-          uint32_t r0[32], r1[32];
-          tmem_ld32(taddr, r0);
-          tmem_ld32(taddr + 32u, r1);
-          tmem_ld_wait();
-          uint4* dst = reinterpret_cast<uint4*>(a.o + (((long long)b * L + row) * a.H + h) * 64);
+          if (ok) {
+            uint32_t r0[32], r1[32];
+            tmem_ld32(taddr, r0);
+            tmem_ld32(taddr + 32u, r1);
+            tmem_ld_wait();
+            uint4* dst = reinterpret_cast<uint4*>(a.o + (((long long)b * L + row) * a.H + h) * 64);
 #pragma unroll
-          for (int qq = 0; qq < 4; ++qq)
-            dst[qq] = make_uint4(pack2(__uint_as_float(r0[qq * 8]), __uint_as_float(r0[qq * 8 + 1])), pack2(__uint_as_float(r0[qq * 8 + 2]), __uint_as_float(r0[qq * 8 + 3])),
-                                 pack2(__uint_as_float(r0[qq * 8 + 4]), __uint_as_float(r0[qq * 8 + 5])), pack2(__uint_as_float(r0[qq * 8 + 6]), __uint_as_float(r0[qq * 8 + 7])));
+            for (int qq = 0; qq < 4; ++qq)
+              dst[qq] = make_uint4(pack2(__uint_as_float(r0[qq * 8]), __uint_as_float(r0[qq * 8 + 1])), pack2(__uint_as_float(r0[qq * 8 + 2]), __uint_as_float(r0[qq * 8 + 3])),
+                                   pack2(__uint_as_float(r0[qq * 8 + 4]), __uint_as_float(r0[qq * 8 + 5])), pack2(__uint_as_float(r0[qq * 8 + 6]), __uint_as_float(r0[qq * 8 + 7])));
 #pragma unroll
-          for (int qq = 0; qq < 4; ++qq)
-            dst[4 + qq] = make_uint4(pack2(__uint_as_float(r1[qq * 8]), __uint_as_float(r1[qq * 8 + 1])), pack2(__uint_as_float(r1[qq * 8 + 2]), __uint_as_float(r1[qq * 8 + 3])),
-                                     pack2(__uint_as_float(r1[qq * 8 + 4]), __uint_as_float(r1[qq * 8 + 5])), pack2(__uint_as_float(r1[qq * 8 + 6]), __uint_as_float(r1[qq * 8 + 7])));
-          fence_before();
-          __syncwarp();
-          if (lane == 0) mb_arrive(bar(8));
+            for (int qq = 0; qq < 4; ++qq)
+              dst[4 + qq] = make_uint4(pack2(__uint_as_float(r1[qq * 8]), __uint_as_float(r1[qq * 8 + 1])), pack2(__uint_as_float(r1[qq * 8 + 2]), __uint_as_float(r1[qq * 8 + 3])),
+                                       pack2(__uint_as_float(r1[qq * 8 + 4]), __uint_as_float(r1[qq * 8 + 5])), pack2(__uint_as_float(r1[qq * 8 + 6]), __uint_as_float(r1[qq * 8 + 7])));
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mb_arrive(bar(8));
+          }
         }
       }
     }
@@ -502,14 +541,14 @@ mtf_status launch_attention_fwd_fused(const void* q, const void* kk, const void*
   a.B = (int)B; a.H = (int)H; a.L = (int)L; a.causal = causal ? 1 : 0; a.scale = scale;
   a.o = reinterpret_cast<__nv_bfloat16*>(o);
   a.units = B * H;
-  const size_t smem = 1024 + 2 * kQBytes + (size_t)L * 256 + kPBufs * kPBufBytes + 4096 + 2 * 8 * 32 * 8 + 16 * 8 + 64;
+  const size_t smem = 1024 + kQBytes + (size_t)L * 256 + kPBufs * kPBufBytes + 4096 + 2 * kSoftmaxWarps * 32 * 4 + 24 * 8 + 64;
   cudaError_t e = cudaFuncSetAttribute(attention_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
-  const long long grid = std::min<long long>(a.units, device_sm_count());
+  const long long grid = std::min<long long>(a.units * (L / 128), device_sm_count());
   cfg.gridDim = dim3((unsigned)grid, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1); cfg.dynamicSmemBytes = smem; cfg.stream = (cudaStream_t)stream;
   cfg.attrs = at; cfg.numAttrs = 1;
   e = cudaLaunchKernelEx(&cfg, attention_fwd_kernel, mq, mk, mv, mp, a);

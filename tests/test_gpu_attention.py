@@ -251,6 +251,32 @@ def test_attention_small_head_dims(mtf):
     end_to_end_report({k: from_torch(out[k]) for k in ref}, ref, "attention d_k=32")
 
 
+@pytest.mark.parametrize("length", [128, 256, 384, 512])
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_core_one_launch(mtf, length, causal):
+    # d_k = d_v = 64 and rows of whole 128-key blocks up to 512: logits, softmax, the stored weights and
+    # weights . v are one launch.  Every element of every stage against the exact oracle of that stage.
+    inp = attention_case(13, 2, length, 256, 4, 64)
+    lay = layout(mtf, [("rows", 2), ("cols", 2)], [("batch", "rows"), ("heads", "cols")])
+    n0 = mtf.mtf_launch_count()
+    run_attention_stagewise(mtf, lay, inp, causal, what=f"attention core L={length} causal={causal}")
+    # projections (1) + core (1) + output (1) forward; the backward's launches do not depend on the length
+    assert mtf.mtf_launch_count() - n0 <= 12
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_core_many_tiles_per_block(mtf, causal):
+    # more (pair, tile) items than the device has SMs: every thread block walks a range of query tiles that crosses
+    # from one (batch, head) pair into the next (keys and values reloaded in mid-range); sampled pairs and tokens
+    import seeded_inputs as si
+    B, L, D, H, K = 6, 384, 256, 12, 64                      # 72 pairs x 3 tiles = 216 items
+    inp = attention_case(17, B, L, D, H, K)
+    pairs = sorted({(0, 0), (B - 1, H - 1), (2, 5), (3, 7), (4, 1), (1, 11)})
+    tok = si.sample_indices(17, "core_tokens", B * L, 6, must_include=[0, B * L - 1, L - 1, L])
+    wcols = [(0, 0), (H - 1, K - 1), (5, 31)]
+    run_attention_stagewise(mtf, layout(mtf, [("all", 1)], []), inp, causal, tok=tok, pairs=pairs, wcols=wcols, what=f"attention core ranges causal={causal}")
+
+
 # ---- decoder layer -------------------------------------------------------------------------------------------
 
 def decoder_case(seed, B, L, D, H, K, F):
