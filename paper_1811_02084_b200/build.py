@@ -24,7 +24,7 @@ LIB_MC = os.path.join(HERE, "libmtf_b200_mc.so")
 MC_HEADER = os.path.join(CSRC, "tma_multicast.cuh")
 MC_SOURCE = "gemm_tcgen05.cu"
 SOURCES = ["planner.cpp", "api.cpp", "blocks.cpp", "ranks.cpp", "chooser.cpp", "ops.cpp", "einsum_simt.cu", "gemm_tcgen05.cu", "rowwise.cu",
-           "relayout.cu", "vocab.cu", "update.cu", "attention_fused.cu"]
+           "relayout.cu", "vocab.cu", "update.cu", "attention_fused.cu", "attention_bwd_fused.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
 
 

@@ -18,6 +18,7 @@ mtf_status read_bad_index(int* seen);
 mtf_status read_row_status(int* code);
 mtf_status debug_wait_test(long long limit_cycles, int skip_first_commit);
 mtf_status read_attention_status(int* code);
+mtf_status read_attention_bwd_status(int* code);
 }  // namespace mtf
 
 using mtf::Dim;
@@ -622,6 +623,7 @@ mtf_status mtf_device_status(int32_t* code) {
   if (st != MTF_OK) return st;
   int rc = 0;
   if ((st = mtf::read_attention_status(&rc)) != MTF_OK) return st;
+  if (!rc && (st = mtf::read_attention_bwd_status(&rc)) != MTF_OK) return st;
   if (!rc && (st = mtf::read_row_status(&rc)) != MTF_OK) return st;
   if (rc) {
     if (code) *code = rc;

@@ -19,6 +19,10 @@ mtf_status launch_layernorm_bwd(const void* dy, const void* x, const float* stat
                                 float* dgamma, float* dbeta, int64_t rows, int n, void* scratch, size_t scratch_bytes, void* stream);
 size_t layernorm_bwd_scratch_bytes(int n);
 bool attention_fused_supported(int64_t L, int64_t d_k, int64_t d_v);
+bool attention_bwd_fused_supported(int64_t L, int64_t d_k, int64_t d_v);
+mtf_status launch_attention_bwd_fused(const void* q, const void* kk, const void* vv, const void* weights, const void* dout, void* dq, void* dkk, void* dvv,
+                                      void* dlogits_dump, int64_t B, int64_t H, int64_t L, float scale, int causal, void* stream);
+bool tap_is_open();
 mtf_status launch_attention_fwd_fused(const void* q, const void* kk, const void* vv, void* weights, void* o, int64_t B, int64_t H, int64_t L, float scale,
                                       int causal, void* stream);
 mtf_status ffn_forward_impl(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* w, const mtf_tensor* bias, const mtf_tensor* v,
@@ -354,6 +358,31 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   if ((st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, *dy, *wo, &dob.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = mtf::tap("do", dob.t, stream)) != MTF_OK) return st;
+  // The whole core - dP, the softmax backward, dvv, dq, dkk - in one launch under the conditions of the forward core
+  // (d_k = d_v = 64, rows of at most 512, only batch and heads split, canonical dimension orders): the weights are read
+  // once and the gradient of the logits never leaves the chip.
+  bool core_done = false;
+  {
+    auto unsplit = [&](const mtf_dim& d) { const int j = layout->mesh_dim_of(d.name); return j < 0 || layout->mesh[j].size == 1; };
+    auto order = [](const mtf_tensor* t, std::initializer_list<mtf_dim> want) {
+      if (t->ndim != (int)want.size() || t->dtype != MTF_BF16 || !t->data) return false;
+      int i = 0;
+      for (auto& w : want) { if (strcmp(t->dims[i].name, w.name) != 0 || t->dims[i].size != w.size) return false; ++i; }
+      return true;
+    };
+    const bool canonical = order(q, {s.b, s.l, s.h, s.k}) && order(kk, {s.b, s.m, s.h, s.k}) && order(vv, {s.b, s.m, s.h, s.v}) &&
+                           order(weights, {s.b, s.h, s.l, s.m}) && order(o, {s.b, s.l, s.h, s.v});
+    if (canonical && mtf::attention_bwd_fused_supported(s.l.size, s.k.size, s.v.size) && unsplit(s.l) && unsplit(s.m) && unsplit(s.k) && unsplit(s.v)) {
+      // (with the stage tap open the gradient of the logits is written out as well, as the contractions consume it)
+      void* dump = mtf::tap_is_open() ? dlg.t.data : nullptr;
+      if ((st = mtf::launch_attention_bwd_fused(q->data, kk->data, vv->data, weights->data, dob.t.data, dq.t.data, dkk.t.data, dvv.t.data, dump, s.b.size, s.h.size,
+                                                s.l.size, (float)s.scale, 0 /* a causal P holds zeros right of the diagonal: nothing to be told */, stream)) != MTF_OK)
+        return st;
+      if (dump && (st = mtf::tap("dlogits", dlg.t, stream)) != MTF_OK) return st;
+      core_done = true;
+    }
+  }
+  if (!core_done) {
   // dP and the softmax backward in one launch where a row fits a tile (dP then stays in tensor
   // memory); otherwise dP goes through the workspace in fp32 and the row kernel follows
   st = mtf::einsum_row_softmax_bwd(layout, &dob.t, vv, weights, &dlg.t, 0 /* zeros of a causal P give zeros here without being told */, rest, rest_bytes, stream);
@@ -367,6 +396,9 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   es.scale = (float)s.scale;
   if ((st = ein(layout, dlg.t, *kk, &dq.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = ein(layout, dlg.t, *q, &dkk.t, &es, rest, rest_bytes, stream)) != MTF_OK) return st;
+  } else if ((st = mtf::tap("dvv", dvv.t, stream)) != MTF_OK) {
+    return st;
+  }
   if ((st = mtf::tap("dq", dq.t, stream)) != MTF_OK || (st = mtf::tap("dkk", dkk.t, stream)) != MTF_OK) return st;
   {
     // the three weight gradients are problems of one shape (few output tiles each): one grouped launch

@@ -160,6 +160,8 @@ struct TapState {
 thread_local TapState g_tap;
 }  // namespace
 
+bool tap_is_open() { return g_tap.active; }
+
 mtf_status tap_begin(void* device_buffer, size_t bytes) {
   if (!device_buffer || (reinterpret_cast<uintptr_t>(device_buffer) & 255)) return fail(MTF_ERR_INVALID_ARG, "stage tap: the buffer must be a 256-byte aligned device pointer");
   g_tap.base = reinterpret_cast<uint8_t*>(device_buffer);

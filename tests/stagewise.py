@@ -46,6 +46,9 @@ class Tap:
         self.entries = [self.mtf.mtf_stage_tap_entry(i) for i in range(n)]
         return self
 
+    def has(self, name):
+        return any(n == name for n, _, _ in self.entries)
+
     def get(self, name, shape, dtype, k=0):
         import torch
         tdt = {"bf16": torch.bfloat16, "f32": torch.float32}[dtype]
@@ -194,7 +197,7 @@ def attention_stage_checks(rep, T, causal, tok, pairs, wcols, prefix="", y_resid
     pos = np.arange(L) if causal else None
     for b, h in pairs:
         q, kk, vv = (_nt(["l", "k"], G(T["q"][b, :, h])), _nt(["m", "k"], G(T["kk"][b, :, h])), _nt(["m", "k"], G(T["vv"][b, :, h])))
-        P_g, do_g, dlg_g = G(T["P"][b, h]), G(T["do"][b, :, h]), G(T["dlogits"][b, h])
+        P_g, do_g = G(T["P"][b, h]), G(T["do"][b, :, h])
         lg, _ = stages.contraction(q, kk, ["l", "m"], scale=s)
         rep.add(prefix + "P", P_g, stages.softmax_last(lg, pos).a)
         if causal:
@@ -205,7 +208,15 @@ def attention_stage_checks(rep, T, causal, tok, pairs, wcols, prefix="", y_resid
         rep.add(prefix + "o", G(T["o"][b, :, h]), ref.a)
         don = _nt(["l", "k"], do_g)
         dP, _ = stages.contraction(don, vv, ["l", "m"])
-        rep.add(prefix + "dlogits", dlg_g, stages.softmax_last_backward(Pn, dP).a)
+        dlg_ref = stages.softmax_last_backward(Pn, dP).a
+        if T.get("dlogits") is not None:
+            # the gradient of the logits is a stored stage of its own: the two contractions after it are checked on what was stored
+            dlg_g = G(T["dlogits"][b, h])
+            rep.add(prefix + "dlogits", dlg_g, dlg_ref)
+        else:
+            # one launch for the whole backward core: the gradient of the logits never reaches memory, so dq and dkk
+            # are held against the exact chain from the launch's own inputs (P, do, vv, q, kk)
+            dlg_g = dlg_ref
         ref, _ = stages.contraction(Pn, don, ["m", "k"])
         rep.add(prefix + "dvv", G(T["dvv"][b, :, h]), ref.a)
         dlgn = _nt(["l", "m"], dlg_g)
@@ -264,7 +275,7 @@ def run_attention_stagewise(mtf, layout, inp, causal, tok=None, pairs=None, wcol
     T.update(out)
     for n in ("do", "dq", "dkk", "dvv"):
         T[n] = tap.get(n, [B, L, H, K], "bf16")
-    T["dlogits"] = tap.get("dlogits", [B, H, L, L], "bf16")
+    T["dlogits"] = tap.get("dlogits", [B, H, L, L], "bf16") if tap.has("dlogits") else None
     a_tok, a_pairs, a_wcols = all_samples(B, L, H, K)
     rep = StageReport(TOL["bf16"], what)
     attention_stage_checks(rep, T, causal, a_tok if tok is None else tok, a_pairs if pairs is None else pairs, a_wcols if wcols is None else wcols)
@@ -332,7 +343,7 @@ def run_decoder_stagewise(mtf, layout, inp, tok=None, pairs=None, wcols=None, hi
     # ---- forward: s1 = x + Attention(x); a = LN1(s1); s2 = a + FFN(a); out = LN2(s2) ----
     A = {"x": dev["x"], "dy": ds1, "wq": dev["wq"], "wk": dev["wk"], "wv": dev["wv"], "wo": dev["wo"], "q": saved_t["q"], "kk": saved_t["kk"],
          "vv": saved_t["vv"], "P": saved_t["weights"], "o": saved_t["o"], "y": saved_t["s1"], "dx": dx, "dwq": grads_t["wq"], "dwk": grads_t["wk"],
-         "dwv": grads_t["wv"], "dwo": grads_t["wo"], "dlogits": tap.get("dlogits", [B, H, L, L], "bf16")}
+         "dwv": grads_t["wv"], "dwo": grads_t["wo"], "dlogits": tap.get("dlogits", [B, H, L, L], "bf16") if tap.has("dlogits") else None}
     for n in ("do", "dq", "dkk", "dvv"):
         A[n] = tap.get(n, [B, L, H, K], "bf16")
     attention_stage_checks(rep, A, True, tok, pairs, wcols, prefix="att.", y_residual=dev["x"], dx_residual=ds1)
