@@ -7,8 +7,9 @@
 //     dvv[m, v]  = sum_l P[l, m] do[l, v]
 //     dq[l, k]   = scale * sum_m dS[l, m] kk[m, k]
 //     dkk[m, k]  = scale * sum_l dS[l, m] q[l, k]
-// dP and dS never leave the chip: dP lives in tensor memory, dS goes as bf16 through a shared-memory tile that
-// is the A operand of the two contractions that consume it.  The weights are read from HBM exactly once.
+// dP and dS never leave the chip: dP lives in tensor memory, dS is written as bf16 over the shared-memory tile
+// of P it was made from (once the dvv MMAs have read that tile) and is the A operand of the two contractions
+// that consume it.  The weights are read from HBM exactly once.
 // d_k = d_v = 64, length = memory_length in {128, 256, 384, 512}; other shapes take the launch-per-einsum path.
 // A causal P holds zeros right of the diagonal, so dS is zero there without being told; the blocks that lie
 // wholly right of it are skipped.
@@ -22,9 +23,9 @@
 //   [256, 320)  dkk of key block j, [320, 384) dvv of key block j, accumulated over i
 //   [384, 512)  dP of the current step
 // Warp roles (320 threads):
-//   warp 0     TMA producer: V_j and K_j per key block; q_i, do_i and the 128 x 128 tile of P per step (rings of two)
-//   warp 1     MMA issuer:   dP of the NEXT step as soon as this step's dP has been read out of tensor memory, then
-//                            this step's dvv += P^T do, dkk += dS^T q, dq_i += dS kk_j (tcgen05.mma kind::f16)
+//   warp 0     TMA producer: V_j and K_j per key block; q_i, do_i and the 128 x 128 tile of P per step (rings of three)
+//   warp 1     MMA issuer:   dP and dvv += P^T do of the NEXT step as soon as this step's dP has been read out of tensor
+//                            memory, then this step's dkk += dS^T q, dq_i += dS kk_j (tcgen05.mma kind::f16)
 //   warps 2-9  two per tensor-memory lane quarter (each owns 64 of the step's 128 key columns): dS from dP and P,
 //              and the read-out of finished accumulators to HBM
 // Every mbarrier wait is bounded; on expiry a code is recorded in the status word, a CTA-wide abort flag is
@@ -45,15 +46,16 @@ constexpr int kThreads = 64 + 32 * kCompWarps;
 constexpr uint32_t kBox = 128 * 64 * 2;           // one 128-row x 64-column bf16 box (128-byte rows, 128B swizzle)
 constexpr int kMaxL = 512;
 constexpr long long kWaitCycles = 4000000000LL;
-// shared memory (from a 1024-byte aligned base): K | V | q[2] | do[2] | P[2] (two boxes each) | dS[2] (two boxes each) | barriers
-constexpr uint32_t kOffK = 0, kOffV = kBox, kOffQ = 2 * kBox, kOffDO = 4 * kBox, kOffP = 6 * kBox, kOffDS = 10 * kBox, kOffBars = 14 * kBox;
-constexpr int kNumBars = 22;
+// shared memory (from a 1024-byte aligned base): K | V | q[3] | do[3] | P[3] (two boxes each; dS overwrites P in place) | barriers
+constexpr int kRing = 3;
+constexpr uint32_t kOffK = 0, kOffV = kBox, kOffQ = 2 * kBox, kOffDO = 5 * kBox, kOffP = 8 * kBox, kOffBars = 14 * kBox;
+constexpr int kNumBars = 32;
 constexpr size_t kSmemBytes = 1024 + kOffBars + kNumBars * 8 + 64;
 // tensor-memory columns
 constexpr uint32_t kColDK = 256, kColDV = 320, kColDP = 384;
 
-enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_QDO_FULL /*2*/, B_QDO_EMPTY = 6 /*2*/, B_P_FULL = 8 /*2*/, B_P_EMPTY = 10 /*2*/, B_DP_FULL = 12, B_DP_EMPTY,
-       B_DS_FULL = 14 /*2*/, B_DS_EMPTY = 16 /*2*/, B_DKV_FULL = 18, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY };
+enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_DP_FULL /*2*/, B_DP_EMPTY = 6 /*2*/, B_DKV_FULL = 8, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_D_SYNC,
+       B_QDO_FULL = 13 /*3*/, B_QDO_EMPTY = 16 /*3*/, B_P_FULL = 19 /*3*/, B_P_EMPTY = 22 /*3*/, B_PV_DONE = 25 /*3*/, B_DS_FULL = 28 /*3*/ };
 
 __device__ int g_attb_status = 0;
 
@@ -100,6 +102,9 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
   asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
                ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];" ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void umma(uint32_t tmem_c, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
@@ -119,6 +124,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // Shared-memory matrix descriptor of a 128B-swizzled tile whose rows are 128 bytes (64 bf16):
 //   K-major  (a row holds 64 k-elements of one m/n index; 8-row groups 1024 bytes apart)
@@ -155,19 +167,26 @@ struct StepIter {
   int nb, causal;
   int pass, j, i;
   long long step_seq, s1_seq, kv_seq, k_seq, unit_seq;      // counts of steps / steps of pass 1 / key blocks (both passes) / key blocks of pass 1 / pairs before this one
+  long long p0_seq;                  // steps of pass 0 before this one
+  long long dpu0, dpu1;              // uses of the two dP buffers before this step
+  __device__ long long dpu(int b) const { return b ? dpu1 : dpu0; }
   bool valid;
   __device__ void init(long long first, long long stride_, long long units_, int nb_, int causal_) {
     u = first; stride = stride_; units = units_; nb = nb_; causal = causal_;
-    pass = 0; j = 0; i = 0; step_seq = 0; s1_seq = 0; kv_seq = 0; k_seq = 0; unit_seq = 0;
+    pass = 0; j = 0; i = 0; step_seq = 0; s1_seq = 0; kv_seq = 0; k_seq = 0; unit_seq = 0; p0_seq = 0; dpu0 = dpu1 = 0;
     valid = u < units;
   }
+  // pass 0 alternates between two dP buffers (the second one stands where dkk, dvv accumulate in pass 1); pass 1 has one
+  __device__ int dp_buf() const { return pass == 0 ? (int)(p0_seq & 1) : 0; }
+  __device__ bool last_of_pass0() const { return pass == 0 && j == nb - 1 && i == nb - 1; }
   __device__ bool first_i() const { return i == (causal ? j : 0); }
   __device__ bool last_i() const { return i == nb - 1; }
   __device__ bool first_of_unit() const { return pass == 0 && j == 0 && first_i(); }
   __device__ bool last_of_unit() const { return pass == 1 && j == nb - 1 && i == nb - 1; }
   __device__ void advance() {
+    if (dp_buf()) ++dpu1; else ++dpu0;
     ++step_seq;
-    if (pass == 1) ++s1_seq;
+    if (pass == 1) ++s1_seq; else ++p0_seq;
     if (i + 1 < nb) { ++i; return; }
     ++kv_seq;
     if (pass == 1) ++k_seq;
@@ -189,7 +208,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const int L = a.L, nb = L / 128;
-  const uint32_t sK = base + kOffK, sV = base + kOffV, sQ = base + kOffQ, sDO = base + kOffDO, sP = base + kOffP, sDS = base + kOffDS;
+  const uint32_t sK = base + kOffK, sV = base + kOffV, sQ = base + kOffQ, sDO = base + kOffDO, sP = base + kOffP;
   const uint32_t bar0 = base + kOffBars;
   auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + kOffBars + kNumBars * 8);
@@ -198,8 +217,9 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kNumBars; ++i) mb_init(bar(i), 1);
-    mb_init(bar(B_DP_EMPTY), kCompWarps);
-    mb_init(bar(B_DS_FULL), kCompWarps); mb_init(bar(B_DS_FULL + 1), kCompWarps);
+    mb_init(bar(B_DP_EMPTY), kCompWarps); mb_init(bar(B_DP_EMPTY + 1), kCompWarps);
+    mb_init(bar(B_D_SYNC), kCompWarps);
+    for (int i = 0; i < kRing; ++i) mb_init(bar(B_DS_FULL + i), kCompWarps);
     mb_init(bar(B_DKV_EMPTY), kCompWarps);
     mb_init(bar(B_DQ_EMPTY), kCompWarps);
     *abort_flag = 0;
@@ -224,13 +244,24 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
   if (warp == 0) {
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
-      StepIter it;
+      StepIter it, pf;
       it.init(blockIdx.x, gridDim.x, a.units, nb, a.causal);
+      // the tiles of P are asked into L2 kPrefetch steps before their load into shared memory is issued: the rings hold
+      // two steps' worth of loads in flight, which alone does not cover the latency of HBM
+      constexpr int kPrefetch = 6;
+      pf = it;
+      auto prefetch_p = [&](const StepIter& t) {
+        const int pb = (int)(t.u / a.H), ph = (int)(t.u % a.H);
+        tma_prefetch_4d(&map_p, t.j * 128, t.i * 128, ph, pb);
+        tma_prefetch_4d(&map_p, t.j * 128 + 64, t.i * 128, ph, pb);
+      };
+      for (int n = 0; n < kPrefetch && pf.valid; ++n) { prefetch_p(pf); pf.advance(); }
       bool ok = true;
       while (ok && it.valid) {
         const int b = (int)(it.u / a.H), h = (int)(it.u % a.H);
-        const int slot = (int)(it.step_seq & 1);
-        const uint32_t par = (uint32_t)(it.step_seq >> 1) & 1u;
+        if (pf.valid) { prefetch_p(pf); pf.advance(); }
+        const int slot = (int)(it.step_seq % kRing);
+        const uint32_t par = (uint32_t)(it.step_seq / kRing) & 1u;
         const uint32_t kvpar = (uint32_t)it.kv_seq & 1u;
         if (it.first_i()) {      // a new key block: V first (the next step's dP wants it), K after this step's tiles
           if (!(ok = mb_wait(bar(B_V_EMPTY), kvpar ^ 1u, 0xA01, abort_flag))) break;
@@ -260,56 +291,82 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       cur.init(blockIdx.x, gridDim.x, a.units, nb, a.causal);
       nxt = cur;
       if (nxt.valid) nxt.advance();
-      long long n_dp = 0;                      // dP tiles issued so far
+      long long n_dp = 0;                      // dP tiles issued so far (one per step of either pass)
+      long long n_dv = 0;                      // dvv contributions issued so far (one per step of pass 1)
       bool ok = true;
       const uint32_t id_dp = idesc_of(0, 0, 128), id_kv = idesc_of(1, 1, 64), id_dq = idesc_of(0, 1, 64);
+      // dP of step t: wants do of the step, V of its key block and the dP columns read out by the warps
+      // pass 0: the warps say with one arrival that they have a step's dP and its tile of P in registers; the tile goes back
+      // to the producer when that arrival is seen, which is when the buffer's next dP is about to be issued
+      int rel_slot[2] = {-1, -1};
       auto issue_dp = [&](const StepIter& t) -> bool {
-        const int slot = (int)(t.step_seq & 1);
-        const uint32_t par = (uint32_t)(t.step_seq >> 1) & 1u;
+        const int slot = (int)(t.step_seq % kRing);
+        const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
+        const int buf = t.dp_buf();
         if (t.first_i() && !mb_wait(bar(B_V_FULL), (uint32_t)t.kv_seq & 1u, 0xB01, abort_flag)) return false;
         if (!mb_wait(bar(B_QDO_FULL + slot), par, 0xB02, abort_flag)) return false;
-        if (!mb_wait(bar(B_DP_EMPTY), ((uint32_t)n_dp & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // the previous dP has been read out
+        if (!mb_wait(bar(B_DP_EMPTY + buf), ((uint32_t)t.dpu(buf) & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // this buffer's previous dP has been read out
+        if (rel_slot[buf] >= 0) { mb_arrive(bar(B_P_EMPTY + rel_slot[buf])); rel_slot[buf] = -1; }   // (pass 0: ... and with it the tile of P of that step)
+        // (the second buffer stands on the accumulators of dkk, dvv: those of the previous pair have been read out)
+        if (buf == 1 && !mb_wait(bar(B_DKV_EMPTY), ((uint32_t)t.k_seq & 1u) ^ 1u, 0xB0A, abort_flag)) return false;
         fence_after();
         const uint64_t da = smem_desc(sDO + slot * kBox, 0, 0), db = smem_desc(sV, 0, 0);
+        const uint32_t col = buf ? kColDK : kColDP;
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) umma(tmem + kColDP, da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
-        umma_commit(bar(B_DP_FULL));
+        for (int ks = 0; ks < 4; ++ks) umma(tmem + col, da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
+        umma_commit(bar(B_DP_FULL + buf));
         if (t.pass == 0) umma_commit(bar(B_QDO_EMPTY + slot));      // pass 0: nothing else reads this do
         if (t.last_i()) umma_commit(bar(B_V_EMPTY));         // this key block's V is no longer read
+        if (t.pass == 0) rel_slot[buf] = slot;
         ++n_dp;
         return true;
       };
+      // dvv_j += P^T do_i of a step of pass 1 (M = keys, N = d_v, k = queries; both operands MN-major).  It needs nothing
+      // from the warps, and once it has run they may overwrite the tile of P with dS.
+      auto issue_dv = [&](const StepIter& t) -> bool {
+        const int slot = (int)(t.step_seq % kRing);
+        const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
+        if (!mb_wait(bar(B_P_FULL + slot), par, 0xB04, abort_flag)) return false;
+        if (t.first_i() && !mb_wait(bar(B_DKV_EMPTY), ((uint32_t)t.k_seq & 1u) ^ 1u, 0xB06, abort_flag)) return false;   // the previous key block's dkk, dvv have been read out
+        // (... and so has the last dP that pass 0 put in the same columns)
+        if (t.first_i() && t.j == 0 && t.dpu1 > 0) {
+          if (!mb_wait(bar(B_DP_EMPTY + 1), (uint32_t)(t.dpu1 - 1) & 1u, 0xB0B, abort_flag)) return false;
+          if (rel_slot[1] >= 0) { mb_arrive(bar(B_P_EMPTY + rel_slot[1])); rel_slot[1] = -1; }
+        }
+        fence_after();
+        const uint64_t da = smem_desc(sP + slot * 2 * kBox, 1, kBox), db = smem_desc(sDO + slot * kBox, 1, kBox);
+        const uint32_t acc = t.first_i() ? 0u : 1u;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) umma(tmem + kColDV, da + (uint64_t)(ks * (2048 >> 4)), db + (uint64_t)(ks * (2048 >> 4)), id_kv, acc | (uint32_t)ks);
+        umma_commit(bar(B_PV_DONE + (int)(t.s1_seq % kRing)));
+        ++n_dv;
+        return true;
+      };
       while (ok && cur.valid) {
+        const int slot = (int)(cur.step_seq % kRing);
         if (n_dp == cur.step_seq && !(ok = issue_dp(cur))) break;
-        if (nxt.valid && !(ok = issue_dp(nxt))) break;        // the next step's dP runs while this step's dS is made
-        const int slot = (int)(cur.step_seq & 1);
-        const uint32_t par = (uint32_t)(cur.step_seq >> 1) & 1u;
+        if (cur.pass == 1 && n_dv == cur.s1_seq && !(ok = issue_dv(cur))) break;
+        // ahead of this step's remaining MMAs: the next step's dP (pass 0: into the other buffer; pass 1: as soon as the
+        // warps have this step's dP in registers) and, inside a key block, its dvv contribution, so that the warps work
+        // on the next step while these run
+        if (nxt.valid) {
+          if (!(ok = issue_dp(nxt))) break;
+          if (nxt.pass == 1 && !nxt.first_i() && !(ok = issue_dv(nxt))) break;
+        }
         if (cur.pass == 0) {
-          // pass 0: the warps take the row sums of dP * P; once they have this step's dP and P in registers (they
-          // say so for both at once) the tile of P goes back to the producer
-          if (!nxt.valid && !(ok = mb_wait(bar(B_DP_EMPTY), (uint32_t)cur.step_seq & 1u, 0xB09, abort_flag))) break;
-          mb_arrive(bar(B_P_EMPTY + slot));
           cur = nxt;
           if (nxt.valid) nxt.advance();
           continue;
         }
-        const int dslot = (int)(cur.s1_seq & 1);                      // the dS ring is used by the steps of pass 1 alone
-        const uint32_t dpar = (uint32_t)(cur.s1_seq >> 1) & 1u;
-        if (!(ok = mb_wait(bar(B_P_FULL + slot), par, 0xB04, abort_flag))) break;
-        if (!(ok = mb_wait(bar(B_DS_FULL + dslot), dpar, 0xB05, abort_flag))) break;
+        const int s1slot = (int)(cur.s1_seq % kRing);
+        if (!(ok = mb_wait(bar(B_DS_FULL + s1slot), (uint32_t)(cur.s1_seq / kRing) & 1u, 0xB05, abort_flag))) break;      // dS stands where P stood
         if (cur.first_i()) {
-          if (!(ok = mb_wait(bar(B_DKV_EMPTY), ((uint32_t)cur.k_seq & 1u) ^ 1u, 0xB06, abort_flag))) break;      // the previous key block's dkk, dvv have been read out
           if (!(ok = mb_wait(bar(B_K_FULL), (uint32_t)cur.k_seq & 1u, 0xB07, abort_flag))) break;
           if (cur.j == 0 && !(ok = mb_wait(bar(B_DQ_EMPTY), ((uint32_t)cur.unit_seq & 1u) ^ 1u, 0xB08, abort_flag))) break;   // the previous pair's dq
         }
         fence_after();
         const uint32_t acc_kv = cur.first_i() ? 0u : 1u;
-        const uint32_t pS = sP + slot * 2 * kBox, dsS = sDS + dslot * 2 * kBox, qS = sQ + slot * kBox, doS = sDO + slot * kBox;
-        {   // dvv_j += P^T do_i   (M = keys, N = d_v, k = queries; both operands MN-major)
-          const uint64_t da = smem_desc(pS, 1, kBox), db = smem_desc(doS, 1, kBox);
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) umma(tmem + kColDV, da + (uint64_t)(ks * (2048 >> 4)), db + (uint64_t)(ks * (2048 >> 4)), id_kv, acc_kv | (uint32_t)ks);
-        }
+        const uint32_t dsS = sP + slot * 2 * kBox, qS = sQ + slot * kBox;
         {   // dkk_j += dS^T q_i
           const uint64_t da = smem_desc(dsS, 1, kBox), db = smem_desc(qS, 1, kBox);
 #pragma unroll
@@ -322,7 +379,6 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           for (int ks = 0; ks < 8; ++ks)
             umma(tmem + (uint32_t)cur.i * 64u, da + (uint64_t)((ks >> 2) * (kBox >> 4) + (ks & 3) * 2), db + (uint64_t)(ks * (2048 >> 4)), id_dq, acc_q | (uint32_t)ks);
         }
-        umma_commit(bar(B_DS_EMPTY + dslot));
         umma_commit(bar(B_P_EMPTY + slot));
         umma_commit(bar(B_QDO_EMPTY + slot));
         if (cur.last_i()) { umma_commit(bar(B_DKV_FULL)); umma_commit(bar(B_K_EMPTY)); }
@@ -359,27 +415,27 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     };
     StepIter it;
     it.init(blockIdx.x, gridDim.x, a.units, nb, a.causal);
-    long long dp_cnt = 0;
     float D0 = 0.f, D1 = 0.f, D2 = 0.f, D3 = 0.f;      // D of this thread's row in each of the pair's query blocks
     bool ok = true;
     while (ok && it.valid) {
       const int b = (int)(it.u / a.H), h = (int)(it.u % a.H);
-      const int slot = (int)(it.step_seq & 1);
-      const uint32_t par = (uint32_t)(it.step_seq >> 1) & 1u;
+      const int slot = (int)(it.step_seq % kRing);
+      const uint32_t par = (uint32_t)(it.step_seq / kRing) & 1u;
       if (it.first_of_unit()) { D0 = 0.f; D1 = 0.f; D2 = 0.f; D3 = 0.f; }
-      if (!(ok = wait_all(B_DP_FULL, (uint32_t)dp_cnt & 1u, 0xC01))) break;
+      const int buf = it.dp_buf();
+      if (!(ok = wait_all(B_DP_FULL + buf, (uint32_t)it.dpu(buf) & 1u, 0xC01))) break;
       fence_after();
       if (!(ok = wait_all(B_P_FULL + slot, par, 0xC02))) break;
       uint32_t r0[32], r1[32];
       if (it.pass == 0) {
-        // pass 0: D[l] += sum over the step's 128 keys of dP[l, m] P[l, m].  Both warps of a lane quarter take the whole
-        // row (64 keys at a time), so that each holds D of its rows without an exchange.
+        // pass 0: D[l] += sum over this warp's 64 of the step's 128 keys of dP[l, m] P[l, m]; the two warps of a lane
+        // quarter add their halves when the pass ends
         float d = 0.f;
-#pragma unroll
-        for (int hb = 0; hb < 2; ++hb) {
-          tmem_ld32(taddr + kColDP + (uint32_t)hb * 64u, r0);
-          tmem_ld32(taddr + kColDP + (uint32_t)hb * 64u + 32u, r1);
-          const uint32_t prow = sP + (uint32_t)slot * 2u * kBox + (uint32_t)hb * kBox + (uint32_t)row_l * 128u;
+        {
+          const uint32_t col = (buf ? kColDK : kColDP) + (uint32_t)half * 64u;
+          tmem_ld32(taddr + col, r0);
+          tmem_ld32(taddr + col + 32u, r1);
+          const uint32_t prow = sP + (uint32_t)slot * 2u * kBox + (uint32_t)half * kBox + (uint32_t)row_l * 128u;
           uint4 pv[8];
 #pragma unroll
           for (int pc = 0; pc < 8; ++pc) pv[pc] = lds_v4(prow + ((((uint32_t)pc) ^ sw) << 4));
@@ -395,9 +451,23 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         fence_before();
         __syncwarp();
-        if (lane == 0) mb_arrive(bar(B_DP_EMPTY));          // dP and P of this step are in registers
-        ++dp_cnt;
+        if (lane == 0) mb_arrive(bar(B_DP_EMPTY + buf));          // dP and P of this step are in registers
         if (it.i == 0) D0 += d; else if (it.i == 1) D1 += d; else if (it.i == 2) D2 += d; else D3 += d;
+        if (it.last_of_pass0()) {
+          // the two halves of every row sum meet through four tensor-memory columns of this warp's lanes (columns of dq,
+          // which nothing uses before the first dS of pass 1 exists)
+          uint32_t mine[4] = {__float_as_uint(D0), __float_as_uint(D1), __float_as_uint(D2), __float_as_uint(D3)}, other[4];
+          tmem_st4(taddr + (uint32_t)half * 4u, mine);
+          tmem_st_wait();
+          fence_before();
+          __syncwarp();
+          if (lane == 0) mb_arrive(bar(B_D_SYNC));
+          if (!(ok = wait_all(B_D_SYNC, (uint32_t)it.unit_seq & 1u, 0xC06))) break;
+          fence_after();
+          tmem_ld4(taddr + (uint32_t)(half ^ 1) * 4u, other);
+          tmem_ld_wait();
+          D0 += __uint_as_float(other[0]); D1 += __uint_as_float(other[1]); D2 += __uint_as_float(other[2]); D3 += __uint_as_float(other[3]);
+        }
         it.advance();
         continue;
       }
@@ -407,7 +477,6 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       fence_before();
       __syncwarp();
       if (lane == 0) mb_arrive(bar(B_DP_EMPTY));            // dP is in registers: the next step's dP may overwrite it
-      ++dp_cnt;
       const float Dr = it.i == 0 ? D0 : (it.i == 1 ? D1 : (it.i == 2 ? D2 : D3));
       const uint32_t prow = sP + (uint32_t)slot * 2u * kBox + (uint32_t)half * kBox + (uint32_t)row_l * 128u;
       uint4 out[8];
@@ -420,11 +489,10 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                              pack2(bf_lo(pv.z) * (__uint_as_float(rr[4]) - Dr), bf_hi(pv.z) * (__uint_as_float(rr[5]) - Dr)),
                              pack2(bf_lo(pv.w) * (__uint_as_float(rr[6]) - Dr), bf_hi(pv.w) * (__uint_as_float(rr[7]) - Dr)));
       }
-      const int dslot = (int)(it.s1_seq & 1);
-      const uint32_t dpar = (uint32_t)(it.s1_seq >> 1) & 1u;
-      {   // the dS tile of two steps ago has been read by its MMAs
+      const int s1slot = (int)(it.s1_seq % kRing);
+      {   // dS goes where this tile of P stands: its last reader, the dvv MMAs of this step, must have run
         int w_ok = 1;
-        if (lane == 0) w_ok = mb_wait(bar(B_DS_EMPTY + dslot), dpar ^ 1u, 0xC03, abort_flag) ? 1 : 0;
+        if (lane == 0) w_ok = mb_wait(bar(B_PV_DONE + s1slot), (uint32_t)(it.s1_seq / kRing) & 1u, 0xC03, abort_flag) ? 1 : 0;
         w_ok = __shfl_sync(0xffffffffu, w_ok, 0);
         if (!w_ok) { ok = false; break; }
       }
@@ -433,12 +501,12 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
         for (int pc = 0; pc < 8; ++pc) dd[pc] = out[pc];
       }
-      const uint32_t drow = sDS + (uint32_t)dslot * 2u * kBox + (uint32_t)half * kBox + (uint32_t)row_l * 128u;
+      const uint32_t drow = prow;
 #pragma unroll
       for (int pc = 0; pc < 8; ++pc) sts_v4(drow + ((((uint32_t)pc) ^ sw) << 4), out[pc].x, out[pc].y, out[pc].z, out[pc].w);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mb_arrive(bar(B_DS_FULL + dslot));
+      if (lane == 0) mb_arrive(bar(B_DS_FULL + s1slot));
       if (it.last_i()) {
         // key block j is complete: dkk (scaled) leaves through the warps of column half 0, dvv through those of half 1
         if (!(ok = wait_all(B_DKV_FULL, (uint32_t)it.k_seq & 1u, 0xC04))) break;
