@@ -106,9 +106,15 @@ __global__ void __launch_bounds__(256) permute_transpose_kernel(const T* __restr
 }
 
 // The same for 2-byte elements with whole 64 x 64 tiles and 16-byte aligned rows on both sides: 16-byte loads along
-// the source's contiguous dimension, 16-byte stores along the destination's (eight 2-byte reads of a tile column each).
+// the source's contiguous dimension, 16-byte stores along the destination's.  The tile is kept as 32-bit words (two
+// neighbouring source columns each) with a row stride of 33 words: the four word stores of a loaded piece and the
+// eight word reads of an output piece are both free of bank conflicts (a warp covers 4 pieces x 8 word columns), and
+// a thread turns its eight words into two output pieces (the low halves and the high halves) with byte permutes.
 __global__ void __launch_bounds__(256) permute_transpose16_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, const TileTranspose c) {
-  __shared__ __align__(16) uint16_t tile[64][64 + 8];
+  __shared__ uint32_t tile[64][33];
+  const int lp = threadIdx.x & 7, lr = threadIdx.x >> 3;                      // load: piece of 8 elements, row (and row + 32)
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int px = (warp & 1) * 4 + (lane & 3), rr = (warp >> 1) * 8 + (lane >> 2);      // store: piece of 8 output columns, pair of output rows
   for (long long t = blockIdx.x; t < c.total_tiles; t += gridDim.x) {
     uint32_t ta, tb, rem;
     uint32_t w = fd_divmod((uint32_t)t, c.tiles_a, &ta);
@@ -120,20 +126,24 @@ __global__ void __launch_bounds__(256) permute_transpose16_kernel(const uint16_t
       d_o += (long long)rem * c.bs_dst[d];
     }
     const int a0 = (int)ta * 64, b0 = (int)tb * 64;
-    const int px = threadIdx.x & 7, py = threadIdx.x >> 3;        // 8 pieces of 8 elements x 32 rows
+    uint4 in[2];
 #pragma unroll
-    for (int r = py; r < 64; r += 32)
-      *reinterpret_cast<uint4*>(&tile[r][px * 8]) = *reinterpret_cast<const uint4*>(src + so + (long long)(b0 + r) * c.sb_src + a0 + px * 8);
-    __syncthreads();
+    for (int k = 0; k < 2; ++k) in[k] = *reinterpret_cast<const uint4*>(src + so + (long long)(b0 + lr + 32 * k) * c.sb_src + a0 + lp * 8);
 #pragma unroll
-    for (int r = py; r < 64; r += 32) {                                // output row a0 + r, columns b0 + 8 px ... + 7
-      uint16_t v[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) v[e] = tile[px * 8 + e][r];
-      uint4 o;
-      o.x = v[0] | ((uint32_t)v[1] << 16); o.y = v[2] | ((uint32_t)v[3] << 16); o.z = v[4] | ((uint32_t)v[5] << 16); o.w = v[6] | ((uint32_t)v[7] << 16);
-      *reinterpret_cast<uint4*>(dst + d_o + (long long)(a0 + r) * c.sa_dst + b0 + px * 8) = o;
+    for (int k = 0; k < 2; ++k) {
+      uint32_t* row = &tile[lr + 32 * k][lp * 4];
+      row[0] = in[k].x; row[1] = in[k].y; row[2] = in[k].z; row[3] = in[k].w;
     }
+    __syncthreads();
+    uint32_t v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = tile[px * 8 + e][rr];
+    uint4 lo, hi;
+    lo.x = __byte_perm(v[0], v[1], 0x5410); lo.y = __byte_perm(v[2], v[3], 0x5410); lo.z = __byte_perm(v[4], v[5], 0x5410); lo.w = __byte_perm(v[6], v[7], 0x5410);
+    hi.x = __byte_perm(v[0], v[1], 0x7632); hi.y = __byte_perm(v[2], v[3], 0x7632); hi.z = __byte_perm(v[4], v[5], 0x7632); hi.w = __byte_perm(v[6], v[7], 0x7632);
+    uint16_t* out = dst + d_o + (long long)(a0 + 2 * rr) * c.sa_dst + b0 + px * 8;
+    *reinterpret_cast<uint4*>(out) = lo;
+    *reinterpret_cast<uint4*>(out + c.sa_dst) = hi;
     __syncthreads();
   }
 }
