@@ -694,11 +694,11 @@ def run_secondary(mtf, peaks, blocks=True, reps=None):
                              "frac": 2.0 * 8 * 64 * 256 / (ms * 1e-3) / (148 * 128 * 2 * 1.965e9),
                              "note": "fp32 FMA peak = 148 SMs x 128 lanes x 2 flop x 1.965 GHz; a 0.26 MFLOP problem measures launch latency only"}})
     gl = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 8)]), [("d_ff", "all")])
-    gsrc = torch.empty(8192, 8192, dtype=torch.bfloat16, device="cuda")
-    gdst = torch.empty(8192, 1024, dtype=torch.bfloat16, device="cuda")
+    gsrc = torch.empty(32768, 8192, dtype=torch.bfloat16, device="cuda")
+    gdst = torch.empty(32768, 1024, dtype=torch.bfloat16, device="cuda")
     ngs = Nn(gsrc, ["tokens", "d_ff"])
     ms = timer(lambda: mtf.mtf_slice_gather(gl, ngs, 3, gdst), 20, stream)
-    rows.append(("slice_gather_kernel", "processor 3's slice [8192, 1024] of a bf16 [8192, 8192] tensor (d_ff split 8 ways)", 2 * gdst.numel() * 2, ms))
+    rows.append(("mtf_slice_gather (permute_copy_kernel)", "processor 3's slice [32768, 1024] of a bf16 [32768, 8192] tensor (d_ff split 8 ways)", 2 * gdst.numel() * 2, ms))
     mtf.mtf_device_status()
     for kernel, shape, nbytes, ms in rows:
         gbs = nbytes / (ms * 1e-3) / 1e9

@@ -18,6 +18,7 @@ mtf_status read_bad_index(int* seen);
 mtf_status read_row_status(int* code);
 mtf_status debug_wait_test(long long limit_cycles, int skip_first_commit);
 mtf_status read_attention_status(int* code);
+mtf_status launch_permute_copy(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes, const int64_t* sstr, const int64_t* dstr, void* stream);
 mtf_status read_attention_bwd_status(int* code);
 }  // namespace mtf
 
@@ -276,7 +277,20 @@ mtf_status mtf_slice_gather(const mtf_layout_t* layout, const mtf_tensor* global
   int64_t offs[mtf::kMaxTensorDims], sizes[mtf::kMaxTensorDims];
   if ((st = mtf::slice_box(layout, d, processor, offs, sizes)) != MTF_OK) return st;
   auto gs = mtf::row_major_strides(d);
-  return mtf::launch_slice_gather(global->data, out_slice, elem_bytes(global->dtype), global->ndim, sizes, offs, gs.data(), stream);
+  const int eb = elem_bytes(global->dtype), nd = global->ndim;
+  // a box whose rows are whole 16-byte pieces on both sides goes through the vectorised row copy
+  if (nd >= 1) {
+    const int64_t vec = 16 / eb;
+    int64_t base = 0, total = 1, sstr[mtf::kMaxTensorDims], dstr[mtf::kMaxTensorDims];
+    for (int i = nd - 1; i >= 0; --i) { dstr[i] = total; total *= sizes[i]; }
+    bool ok = total > 0 && total < 0x7fffffffLL && sizes[nd - 1] % vec == 0;
+    for (int i = 0; i < nd; ++i) { sstr[i] = gs[i]; base += offs[i] * gs[i]; }
+    for (int i = 0; ok && i + 1 < nd; ++i) ok = sstr[i] % vec == 0 && dstr[i] % vec == 0;
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(global->data) + base * eb;
+    ok = ok && !(reinterpret_cast<uintptr_t>(src) & 15) && !(reinterpret_cast<uintptr_t>(out_slice) & 15);
+    if (ok) return mtf::launch_permute_copy(src, out_slice, eb, nd, sizes, sstr, dstr, stream);
+  }
+  return mtf::launch_slice_gather(global->data, out_slice, eb, nd, sizes, offs, gs.data(), stream);
 }
 
 mtf_status mtf_einsum_plan(const mtf_layout_t* layout, int32_t n_in, const mtf_tensor* in_desc, const mtf_tensor* out_desc,
