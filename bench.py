@@ -544,7 +544,7 @@ def block_step(mtf, dec, B=None):
 
         def step():
             mtf.mtf_decoder_layer_forward(lay, N["x"], P, True, 1e-6, S, mtf.named(out, act), ws)
-            mtf.mtf_decoder_layer_backward(lay, N["x"], P, S, N["dout"], mtf.named(dx, act), G, ws)
+            mtf.mtf_decoder_layer_backward(lay, N["x"], P, S, N["dout"], mtf.named(dx, act), G, ws, causal=True)
     else:
         ws = torch.empty(mtf.mtf_attention_workspace_bytes(lay, N["x"], N["wq"], N["wv"]), dtype=torch.uint8, device="cuda")
         flops = 3 * (8.0 * B * L * D * H * K + 4.0 * B * H * L * L * K)

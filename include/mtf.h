@@ -314,9 +314,14 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
                                  mtf_tensor* weights, mtf_tensor* o, mtf_tensor* y, void* workspace,
                                  size_t workspace_bytes, void* stream);
 /* Gradients of the above for upstream dy [batch, length, d_model]: dwq, dwk, dwv, dwo (reduce out the
- * token dims) and dx (reduces out heads; dx_residual, NULL or dx's dims, is added). */
+ * token dims) and dx (reduces out heads; dx_residual, NULL or dx's dims, is added).
+ * causal: a hint, never needed for the result (causal weights hold exact zeros where m > l and those
+ * zeros give zero gradients): non-zero promises that `weights` came from a causal forward call, and the
+ * one-launch backward core then skips the key blocks that lie wholly right of the diagonal.  A non-zero
+ * hint on weights that are not causal gives wrong gradients. */
 mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq,
-                                  const mtf_tensor* wk, const mtf_tensor* wv, const mtf_tensor* wo, const mtf_tensor* q,
+                                  const mtf_tensor* wk, const mtf_tensor* wv, const mtf_tensor* wo, int32_t causal,
+                                  const mtf_tensor* q,
                                   const mtf_tensor* kk, const mtf_tensor* vv, const mtf_tensor* weights,
                                   const mtf_tensor* o, const mtf_tensor* dy, const mtf_tensor* dx_residual,
                                   mtf_tensor* dx, mtf_tensor* dwq, mtf_tensor* dwk, mtf_tensor* dwv, mtf_tensor* dwo,
@@ -339,8 +344,9 @@ typedef struct {
 mtf_status mtf_decoder_layer_forward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* params,
                                      int32_t causal, float eps, const mtf_decoder_saved* saved, mtf_tensor* out,
                                      void* workspace, size_t workspace_bytes, void* stream);
+/* (causal: the hint of mtf_attention_backward; pass what the forward call was given, or 0) */
 mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* params,
-                                      const mtf_decoder_saved* saved, const mtf_tensor* dout, mtf_tensor* dx,
+                                      int32_t causal, const mtf_decoder_saved* saved, const mtf_tensor* dout, mtf_tensor* dx,
                                       const mtf_decoder_grads* grads, void* workspace, size_t workspace_bytes, void* stream);
 mtf_status mtf_decoder_layer_workspace_bytes(const mtf_layout_t* layout, const mtf_tensor* x,
                                              const mtf_decoder_params* params, size_t* bytes);

@@ -131,10 +131,10 @@ def _load():
         "mtf_layernorm_backward": [vp] + [POINTER(mtf_tensor)] * 8 + [vp, c_size_t, vp],
         "mtf_layernorm_workspace_bytes": [c_int64, POINTER(c_size_t)],
         "mtf_attention_forward": [vp] + [POINTER(mtf_tensor)] * 5 + [c_int32] + [POINTER(mtf_tensor)] * 7 + [vp, c_size_t, vp],
-        "mtf_attention_backward": [vp] + [POINTER(mtf_tensor)] * 17 + [vp, c_size_t, vp],
+        "mtf_attention_backward": [vp] + [POINTER(mtf_tensor)] * 5 + [c_int32] + [POINTER(mtf_tensor)] * 12 + [vp, c_size_t, vp],
         "mtf_attention_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
         "mtf_decoder_layer_forward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), c_int32, c_float, POINTER(mtf_decoder_saved), POINTER(mtf_tensor), vp, c_size_t, vp],
-        "mtf_decoder_layer_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(mtf_decoder_saved), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_decoder_grads), vp, c_size_t, vp],
+        "mtf_decoder_layer_backward": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), c_int32, POINTER(mtf_decoder_saved), POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_decoder_grads), vp, c_size_t, vp],
         "mtf_decoder_layer_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_decoder_params), POINTER(c_size_t)],
         "mtf_device_status": [POINTER(c_int32)],
         "mtf_layout_bind_ranks": [vp, c_char_p, c_int32, c_int32, RANK_ALLREDUCE_FN, RANK_WAIT_FN, vp, POINTER(vp)],
@@ -508,9 +508,10 @@ def mtf_attention_forward(layout, x, wq, wk, wv, wo, causal, residual, q, kk, vv
 
 
 def mtf_attention_backward(layout, x, wq, wk, wv, wo, q, kk, vv, weights, o, dy, dx_residual, dx, dwq, dwk, dwv, dwo, workspace=None,
-                           stream=None) -> None:
+                           stream=None, causal=False) -> None:
+    """causal: a hint (True promises that `weights` came from a causal forward call; False is always right)."""
     wp, wb = _ws(workspace)
-    _check(_lib.mtf_attention_backward(layout.handle, _p(x), _p(wq), _p(wk), _p(wv), _p(wo), _p(q), _p(kk), _p(vv), _p(weights), _p(o), _p(dy),
+    _check(_lib.mtf_attention_backward(layout.handle, _p(x), _p(wq), _p(wk), _p(wv), _p(wo), 1 if causal else 0, _p(q), _p(kk), _p(vv), _p(weights), _p(o), _p(dy),
                                        _p(dx_residual), _p(dx), _p(dwq), _p(dwk), _p(dwv), _p(dwo), wp, wb, _stream(stream)))
 
 
@@ -536,10 +537,10 @@ def mtf_decoder_layer_forward(layout, x, params: dict, causal, eps, saved: dict,
                                           _stream(stream)))
 
 
-def mtf_decoder_layer_backward(layout, x, params: dict, saved: dict, dout, dx, grads: dict, workspace=None, stream=None) -> None:
+def mtf_decoder_layer_backward(layout, x, params: dict, saved: dict, dout, dx, grads: dict, workspace=None, stream=None, causal=False) -> None:
     wp, wb = _ws(workspace)
     ps, sv, gs = _struct_of(mtf_decoder_params, params), _struct_of(mtf_decoder_saved, saved), _struct_of(mtf_decoder_grads, grads)
-    _check(_lib.mtf_decoder_layer_backward(layout.handle, _p(x), byref(ps), byref(sv), _p(dout), _p(dx), byref(gs), wp, wb, _stream(stream)))
+    _check(_lib.mtf_decoder_layer_backward(layout.handle, _p(x), byref(ps), 1 if causal else 0, byref(sv), _p(dout), _p(dx), byref(gs), wp, wb, _stream(stream)))
 
 
 def mtf_decoder_layer_workspace_bytes(layout, x, params: dict) -> int:

@@ -167,7 +167,7 @@ struct StepIter {
   int nb, causal;
   int pass, j, i;
   long long step_seq, s1_seq, kv_seq, k_seq, unit_seq;      // counts of steps / steps of pass 1 / key blocks (both passes) / key blocks of pass 1 / pairs before this one
-  long long p0_seq;                  // steps of pass 0 before this one
+  long long p0_seq;                  // steps of pass 0 of this pair before this one
   long long dpu0, dpu1;              // uses of the two dP buffers before this step
   __device__ long long dpu(int b) const { return b ? dpu1 : dpu0; }
   bool valid;
@@ -176,7 +176,9 @@ struct StepIter {
     pass = 0; j = 0; i = 0; step_seq = 0; s1_seq = 0; kv_seq = 0; k_seq = 0; unit_seq = 0; p0_seq = 0; dpu0 = dpu1 = 0;
     valid = u < units;
   }
-  // pass 0 alternates between two dP buffers (the second one stands where dkk, dvv accumulate in pass 1); pass 1 has one
+  // pass 0 alternates between two dP buffers (the second one stands where dkk, dvv accumulate in pass 1), starting with the
+  // first for every pair: the first dP of a pair is issued while the previous pair's last dkk, dvv are still being
+  // accumulated; pass 1 has one buffer
   __device__ int dp_buf() const { return pass == 0 ? (int)(p0_seq & 1) : 0; }
   __device__ bool last_of_pass0() const { return pass == 0 && j == nb - 1 && i == nb - 1; }
   __device__ bool first_i() const { return i == (causal ? j : 0); }
@@ -194,6 +196,7 @@ struct StepIter {
     j = 0; i = 0;
     if (pass == 0) { pass = 1; return; }
     pass = 0;
+    p0_seq = 0;
     ++unit_seq;
     u += stride;
     valid = u < units;

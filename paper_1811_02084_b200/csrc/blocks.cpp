@@ -334,7 +334,7 @@ mtf_status mtf_attention_forward(const mtf_layout_t* layout, const mtf_tensor* x
 // dq = s sum_m dlogits kk; dkk = s sum_l dlogits q; dwq = sum_{b,l} x dq; dwk = sum_{b,m} xm dkk;
 // dwv = sum_{b,m} xm dvv; dx = sum_{h,k} dq wq + sum_{h,k} dkk wk + sum_{h,v} dvv wv (+ dx_residual).
 mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_tensor* wq, const mtf_tensor* wk, const mtf_tensor* wv,
-                                  const mtf_tensor* wo, const mtf_tensor* q, const mtf_tensor* kk, const mtf_tensor* vv, const mtf_tensor* weights,
+                                  const mtf_tensor* wo, int32_t causal, const mtf_tensor* q, const mtf_tensor* kk, const mtf_tensor* vv, const mtf_tensor* weights,
                                   const mtf_tensor* o, const mtf_tensor* dy, const mtf_tensor* dx_residual, mtf_tensor* dx, mtf_tensor* dwq,
                                   mtf_tensor* dwk, mtf_tensor* dwv, mtf_tensor* dwo, void* workspace, size_t workspace_bytes, void* stream) {
   AttShapes s;
@@ -376,7 +376,7 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
       // (with the stage tap open the gradient of the logits is written out as well, as the contractions consume it)
       void* dump = mtf::tap_is_open() ? dlg.t.data : nullptr;
       if ((st = mtf::launch_attention_bwd_fused(q->data, kk->data, vv->data, weights->data, dob.t.data, dq.t.data, dkk.t.data, dvv.t.data, dump, s.b.size, s.h.size,
-                                                s.l.size, (float)s.scale, 0 /* a causal P holds zeros right of the diagonal: nothing to be told */, stream)) != MTF_OK)
+                                                s.l.size, (float)s.scale, causal ? 1 : 0 /* a hint: the zeros of a causal P give zero gradients anyway */, stream)) != MTF_OK)
         return st;
       if (dump && (st = mtf::tap("dlogits", dlg.t, stream)) != MTF_OK) return st;
       core_done = true;
@@ -467,8 +467,8 @@ mtf_status mtf_decoder_layer_forward(const mtf_layout_t* layout, const mtf_tenso
   return mtf_layernorm_forward(layout, sv->s2, p->ln2_gamma, p->ln2_beta, eps, out, sv->stats2, stream);
 }
 
-mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* p, const mtf_decoder_saved* sv,
-                                      const mtf_tensor* dout, mtf_tensor* dx, const mtf_decoder_grads* g, void* workspace, size_t workspace_bytes,
+mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tensor* x, const mtf_decoder_params* p, int32_t causal,
+                                      const mtf_decoder_saved* sv, const mtf_tensor* dout, mtf_tensor* dx, const mtf_decoder_grads* g, void* workspace, size_t workspace_bytes,
                                       void* stream) {
   if (!layout || !x || !p || !sv || !dout || !dx || !g) return fail(MTF_ERR_INVALID_ARG, "decoder_layer_backward: NULL argument");
   for (const mtf_tensor* t : {g->dwq, g->dwk, g->dwv, g->dwo, g->dln1_gamma, g->dln1_beta, g->dw, g->dv, g->dln2_gamma, g->dln2_beta})
@@ -494,7 +494,7 @@ mtf_status mtf_decoder_layer_backward(const mtf_layout_t* layout, const mtf_tens
   // ds1 (reusing ds2's buffer) = LN1 backward; dx = ds1 + dAttention/dx
   if ((st = mtf_layernorm_backward(layout, &da.t, sv->s1, sv->stats1, p->ln1_gamma, nullptr, &ds2.t, g->dln1_gamma, g->dln1_beta, rest, rest_bytes, stream)) != MTF_OK) return st;
   if ((st = mtf::tap("ds1", ds2.t, stream)) != MTF_OK) return st;
-  return mtf_attention_backward(layout, x, p->wq, p->wk, p->wv, p->wo, sv->q, sv->kk, sv->vv, sv->weights, sv->o, &ds2.t, &ds2.t, dx, g->dwq, g->dwk,
+  return mtf_attention_backward(layout, x, p->wq, p->wk, p->wv, p->wo, causal, sv->q, sv->kk, sv->vv, sv->weights, sv->o, &ds2.t, &ds2.t, dx, g->dwq, g->dwk,
                                 g->dwv, g->dwo, rest, rest_bytes, stream);
 }
 

@@ -248,7 +248,8 @@ def all_samples(B, L, H, K):
     return np.arange(B * L), [(b, h) for b in range(B) for h in range(H)], [(h, k) for h in range(H) for k in range(K)]
 
 
-def run_attention_stagewise(mtf, layout, inp, causal, tok=None, pairs=None, wcols=None, what="attention"):
+def run_attention_stagewise(mtf, layout, inp, causal, tok=None, pairs=None, wcols=None, what="attention", causal_hint=True):
+    """causal_hint: whether the backward call is told that the weights are causal (it is right either way)."""
     import torch
     dev = {k: to_torch(s) for k, (_, s) in inp.items()}
     N = {k: mtf.named(dev[k], [n for n, _ in d]) for k, (d, _) in inp.items()}
@@ -265,7 +266,7 @@ def run_attention_stagewise(mtf, layout, inp, causal, tok=None, pairs=None, wcol
     tap = Tap(mtf, 4 * B * L * H * K * 2 + B * H * L * L * 2 + 8192, guard)
     mtf.mtf_attention_forward(layout, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], causal, None, O["q"], O["kk"], O["vv"], O["P"], O["o"], O["y"], ws)
     mtf.mtf_attention_backward(layout, N["x"], N["wq"], N["wk"], N["wv"], N["wo"], O["q"], O["kk"], O["vv"], O["P"], O["o"], N["dy"], None,
-                               O["dx"], O["dwq"], O["dwk"], O["dwv"], O["dwo"], ws)
+                               O["dx"], O["dwq"], O["dwk"], O["dwv"], O["dwo"], ws, causal=causal and causal_hint)
     tap.close()
     mtf.mtf_device_status()
     guard.check()
@@ -291,7 +292,7 @@ GRAD_FIELD = {"wq": "dwq", "wk": "dwk", "wv": "dwv", "wo": "dwo", "ln1_gamma": "
               "v": "dv", "ln2_gamma": "dln2_gamma", "ln2_beta": "dln2_beta"}
 
 
-def run_decoder_stagewise(mtf, layout, inp, tok=None, pairs=None, wcols=None, hid=None, dcols=None, eps=1e-6, what="decoder"):
+def run_decoder_stagewise(mtf, layout, inp, tok=None, pairs=None, wcols=None, hid=None, dcols=None, eps=1e-6, what="decoder", causal_hint=True):
     """inp: test_gpu_attention.decoder_case(...).  Runs the decoder layer forward + backward with the
     stage tap open and checks every launch: the attention stages (residual x riding in the output
     projection), layer norm 1, the feed-forward stages on a (residual a), layer norm 2, and the
@@ -322,7 +323,7 @@ def run_decoder_stagewise(mtf, layout, inp, tok=None, pairs=None, wcols=None, hi
     ws = _alloc([mtf.mtf_decoder_layer_workspace_bytes(layout, N["x"], params)], "u8")
     tap = Tap(mtf, (7 * B * L * D + 2 * B * L * F + B * H * L * L) * 2 + 16384, guard)
     mtf.mtf_decoder_layer_forward(layout, N["x"], params, True, eps, saved, mtf.named(out, names), ws)
-    mtf.mtf_decoder_layer_backward(layout, N["x"], params, saved, N["dout"], mtf.named(dx, names), grads, ws)
+    mtf.mtf_decoder_layer_backward(layout, N["x"], params, saved, N["dout"], mtf.named(dx, names), grads, ws, causal=causal_hint)
     tap.close()
     mtf.mtf_device_status()
     guard.check()

@@ -252,14 +252,15 @@ def test_attention_small_head_dims(mtf):
 
 
 @pytest.mark.parametrize("length", [128, 256, 384, 512])
-@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("causal", [False, True, "unhinted"], ids=["full", "causal", "causal-unhinted"])
 def test_attention_core_one_launch(mtf, length, causal):
     # d_k = d_v = 64 and rows of whole 128-key blocks up to 512: logits, softmax, the stored weights and
     # weights . v are one launch.  Every element of every stage against the exact oracle of that stage.
     inp = attention_case(13, 2, length, 256, 4, 64)
     lay = layout(mtf, [("rows", 2), ("cols", 2)], [("batch", "rows"), ("heads", "cols")])
     n0 = mtf.mtf_launch_count()
-    run_attention_stagewise(mtf, lay, inp, causal, what=f"attention core L={length} causal={causal}")
+    # ("unhinted": causal weights, but the backward call is not told: it walks the all-zero blocks too)
+    run_attention_stagewise(mtf, lay, inp, bool(causal), what=f"attention core L={length} causal={causal}", causal_hint=causal is True)
     # projections (1) + core (1) + output (1) forward; the backward's launches do not depend on the length
     assert mtf.mtf_launch_count() - n0 <= 12
 
@@ -275,6 +276,19 @@ def test_attention_core_many_tiles_per_block(mtf, causal):
     tok = si.sample_indices(17, "core_tokens", B * L, 6, must_include=[0, B * L - 1, L - 1, L])
     wcols = [(0, 0), (H - 1, K - 1), (5, 31)]
     run_attention_stagewise(mtf, layout(mtf, [("all", 1)], []), inp, causal, tok=tok, pairs=pairs, wcols=wcols, what=f"attention core ranges causal={causal}")
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_attention_core_many_pairs_per_block(mtf, causal):
+    # more (batch, head) pairs than the device has SMs: a thread block of the backward core walks several pairs, with an
+    # odd number of steps per pass when the weights are causal (rows of 256: blocks (0,0), (0,1), (1,1))
+    import seeded_inputs as si
+    B, L, D, H, K = 20, 256, 128, 16, 64                      # 320 pairs
+    inp = attention_case(19, B, L, D, H, K)
+    pairs = sorted({(0, 0), (B - 1, H - 1), (9, 3), (9, 4), (10, 15), (17, 8)})      # first, last and pairs a block reaches second or third
+    tok = si.sample_indices(19, "pairs_tokens", B * L, 6, must_include=[0, B * L - 1, L - 1, L])
+    wcols = [(0, 0), (H - 1, K - 1), (7, 31)]
+    run_attention_stagewise(mtf, layout(mtf, [("all", 1)], []), inp, causal, tok=tok, pairs=pairs, wcols=wcols, what=f"attention core pairs causal={causal}")
 
 
 # ---- decoder layer -------------------------------------------------------------------------------------------

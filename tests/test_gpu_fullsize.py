@@ -141,7 +141,7 @@ def test_decoder_layer_config5_full_size_stagewise(mtf):
     base = None
     for tag, (mesh_dims, rules) in DECODER_SWEEP.items():
         errs, res = run_decoder_stagewise(mtf, layout(mtf, mesh_dims, rules), inp, tok=tok, pairs=pairs, wcols=wcols, hid=hid, dcols=dcols,
-                                          what=f"config5 {tag}")
+                                          what=f"config5 {tag}", causal_hint=tag != "model8")
         print("config5", tag, {k: f"{e:.2e}" for k, e in errs.items()})
         if base is None:
             base = {k: t.clone() for k, t in res.items()}
