@@ -582,9 +582,10 @@ def run_secondary(mtf, peaks, blocks=True, reps=None):
                                  "note": "whole block (contractions + row kernels) against the burst torch.matmul rate; timed region well under a second"}})
         del step, keep
         torch.cuda.empty_cache()
-    # memory-bound kernels at the shapes of config 5 (layer norm rows of 2048) and config 3 (softmax rows of 512)
+    # memory-bound kernels at the row lengths of config 5 (layer norm rows of 2048) and config 3 (softmax rows of 512);
+    # the layer norm runs on four times config 5's tokens so that its input (268 MB) is larger than L2
     lay = mtf.mtf_layout(mtf.mtf_mesh_create([("all", 8)]), [("batch", "all")])
-    B, L, D = 64, 256, 2048
+    B, L, D = 256, 256, 2048
     x, dy = to_device(si.normal(5, "x", [B, L, D], "bf16")), to_device(si.normal(5, "dy", [B, L, D], "bf16"))
     g, b = to_device(si.normal(5, "g", [D], "f32", 0.1, 1.0)), to_device(si.normal(5, "b", [D], "f32", 0.1))
     yb, dxb = torch.empty_like(x), torch.empty_like(x)
@@ -648,8 +649,14 @@ def run_secondary(mtf, peaks, blocks=True, reps=None):
                              "note": "whole step (3 contractions + 4 memory-bound kernels) against the burst torch.matmul rate"}})
     # the memory-bound kernels of that step, each alone
     nE, nxv, nlgt, nlse, nloss, ndls = Nn(E, ["vocab", "d_model"]), Nn(xv, av), Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), Nn(dls, tl)
-    ms = timer(lambda: mtf.mtf_embedding_forward(layv, ids, nE, nxv), 50, stream)
-    rows.append(("embedding_gather_kernel", f"{Tv} rows of {Dv} (bf16) from a table of {V} rows", 2 * Tv * Dv * 2, ms))
+    # (the lookup alone on 16 times the step's tokens, so that it moves more than L2 holds)
+    Tg = 16 * Tv
+    ids_g = torch.from_numpy(rng.randint(0, V, size=(16 * Bv, Lv)).astype(np.int32)).cuda()
+    xg = torch.empty(16 * Bv, Lv, Dv, dtype=torch.bfloat16, device="cuda")
+    nxg = Nn(xg, av)
+    ms = timer(lambda: mtf.mtf_embedding_forward(layv, ids_g, nE, nxg), 50, stream)
+    rows.append(("embedding_gather_kernel", f"{Tg} rows of {Dv} (bf16) from a table of {V} rows (the 67 MB table stays in L2: the reads are L2 hits)", 2 * Tg * Dv * 2, ms))
+    del xg, ids_g
     mtf.mtf_xent_forward(layv, Nn(xv, av), Nn(Wo, ["d_model", "vocab"]), tgt, Nn(lgt, lv), Nn(lse, tl), Nn(loss, tl), wsv)
     ms = timer(lambda: mtf.mtf_softmax_xent_forward(layv, nlgt, tgt, nlse, nloss), 20, stream)
     rows.append(("xent_rows_kernel", f"{Tv} rows of {V} (bf16 logits)", Tv * V * 2, ms))
