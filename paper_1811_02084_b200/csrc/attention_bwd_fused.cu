@@ -610,6 +610,10 @@ mtf_status launch_attention_bwd_fused(const void* q, const void* kk, const void*
   a.dk = reinterpret_cast<__nv_bfloat16*>(dkk);
   a.dv = reinterpret_cast<__nv_bfloat16*>(dvv);
   a.units = B * H;
+  if (dlogits_dump && causal) {      // the blocks the kernel skips under the hint hold zeros
+    cudaError_t ze = cudaMemsetAsync(dlogits_dump, 0, (size_t)B * H * L * L * 2, (cudaStream_t)stream);
+    if (ze != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(ze));
+  }
   cudaError_t e = cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   cudaLaunchConfig_t cfg = {};
