@@ -553,6 +553,22 @@ mtf_status mtf::einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor*
   return exec_plan(P, in, weights, &e, workspace, workspace_bytes, stream, 1, nullptr, causal ? 2 : 1);
 }
 
+// out = a . b (plain, bf16) with the per-row statistics of a log-sum-exp left at the head of the workspace by the
+// epilogue: float2 [rows][*parts] (maximum, sum of exp(value - maximum)) of the stored values of every column part.
+mtf_status mtf::einsum_row_lse(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* out, void* workspace, size_t workspace_bytes,
+                               void* stream, int* parts) {
+  if (!layout || !a || !b || !out || !parts) return fail(MTF_ERR_INVALID_ARG, "einsum_row_lse: NULL argument");
+  const mtf_tensor in[2] = {*a, *b};
+  const mtf_plan_t* P = nullptr;
+  mtf_status st = cached_plan(layout, 2, in, out, nullptr, &P);
+  if (st != MTF_OK) return st;
+  if (P->kernel_kind != MTF_KERNEL_TCGEN05 || P->tc.swapped || P->rank_sum || P->reduce_mode == MTF_REDUCE_WORKSPACE)
+    return fail(MTF_ERR_UNSUPPORTED, "einsum_row_lse: not on this plan");
+  const int64_t ns = P->tc.N / P->tc.sn;
+  *parts = (int)(P->tc.sn * ((ns + P->tc.block_n - 1) / P->tc.block_n) * 2);
+  return exec_plan(P, in, out, nullptr, workspace, workspace_bytes, stream, 1, nullptr, 5);
+}
+
 mtf_status mtf::einsum_row_softmax_bwd(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, const mtf_tensor* weights,
                                        mtf_tensor* dlogits, int causal, void* workspace, size_t workspace_bytes, void* stream) {
   if (!layout || !a || !b || !weights || !dlogits) return fail(MTF_ERR_INVALID_ARG, "einsum_row_softmax_bwd: NULL argument");

@@ -122,6 +122,8 @@ struct TcArgs {
   int resid_bf16;
   float scale;
   int relu;
+  float2* lse_partial;     // EPI_ROW_LSE_BF16: [row][lse_parts] (maximum, sum of exp(value - maximum)) of the row's stored values in every column part
+  int lse_parts;           // column parts per row: slices along N x tiles per slice x 2 warps
   float* rsum;             // fused reduce_sum over M of the epilogue value (fp32, pre-zeroed), indexed by n
   float* rsum_partial;     // not NULL: every 32-row group leaves its column sums here ([row group][N]) instead of adding them to rsum with
                            // atomics; a finishing launch adds the groups up in index order, so the sums repeat bit for bit
@@ -439,7 +441,8 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& m, float* f) {
 // Which component-wise stages a launch runs.  EPI_GENERIC reads them from the arguments; the other
 // kinds fix them at compile time, so that the common epilogues carry no branches on them and need
 // far fewer registers and instructions per chunk.
-enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_ROW_SOFTMAX_BWD = 6, EPI_KINDS = 7 };
+enum { EPI_GENERIC = 0, EPI_PLAIN_BF16 = 1, EPI_PLAIN_F32 = 2, EPI_BIAS_RELU_BF16 = 3, EPI_MASK_RSUM_BF16 = 4, EPI_ROW_SOFTMAX = 5, EPI_ROW_SOFTMAX_BWD = 6,
+       EPI_ROW_LSE_BF16 = 7 /* plain bf16 result + per row and column part the maximum and the sum of exponentials of what was stored */, EPI_KINDS = 8 };
 struct EpiFlags {
   bool scale, bias, bias_m, relu, relu_in_pack, mask, mask_bf16, mask_tma, resid, resid_tma, rsum, c_bf16, shared_tiles;
 };
@@ -1182,6 +1185,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const CUtensorMap* const pc = sg.group == 0 ? &map_c : &extra.c[sg.group - 1];       // (grouped launch: this problem's output)
         void* const c_base = sg.group == 0 ? a.C : a.C_group[sg.group - 1];
         float bias_cur = bias_at(tl.n0 + col_half * box_cols + lane);      // lane l keeps column l of the current chunk
+        float lse_m = -INFINITY, lse_s = 0.f;      // (EPI_ROW_LSE_BF16) running maximum and sum of exponentials of this row's stored values
 #pragma unroll 1
         for (int c0 = 0; c0 < a.block_n; c0 += 32) {
           if (((c0 / box_cols) & 1) != col_half) continue;    // the other warp of this lane quarter owns that box
@@ -1274,6 +1278,22 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           } else {
             epilogue_residual(a, f, v, row_off + n_first, live, n_valid);
           }
+          if (EPI == EPI_ROW_LSE_BF16 && live) {
+            // row statistics of the values as they are stored (rounded to bf16), so that they describe the tensor in memory
+            float cm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              v[j] = __bfloat162float(__float2bfloat16_rn(v[j]));
+              if (j < n_valid) cm = fmaxf(cm, v[j]);
+            }
+            const float nm = fmaxf(lse_m, cm);
+            float cs = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < n_valid) cs += exp2f((v[j] - nm) * 1.4426950408889634f);
+            lse_s = lse_s * exp2f((lse_m - nm) * 1.4426950408889634f) + cs;
+            lse_m = nm;
+          }
           if (staged) store_staged(f, v, box, lane, half);
           else if (live) store_direct(a, f, v, row_off + n_first, n_valid, c_base);
           if (staged && ((c0 + 32) & (box_cols - 1)) == 0) {     // box complete: hand it to the TMA
@@ -1293,6 +1313,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               else atomicAdd(a.rsum + n_first + lane, col);
             }
           }
+        }
+        if (EPI == EPI_ROW_LSE_BF16 && row_ok) {
+          const int slice_n = tl.n_end / a.Ns - 1, tile_n = (tl.n0 - slice_n * a.Ns) / a.block_n;
+          a.lse_partial[(long long)row * a.lse_parts + (slice_n * a.n_tiles + tile_n) * 2 + col_half] = make_float2(lse_m, lse_s);
         }
         tcgen05_fence_before();
         __syncwarp();
@@ -1502,6 +1526,9 @@ mtf_status launch_kind(int epi, const CUtensorMap& map_a, const CUtensorMap& map
     case EPI_PLAIN_BF16: return launch_variant<kPair, CM, CN, EPI_PLAIN_BF16>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     case EPI_PLAIN_F32: return launch_variant<kPair, CM, CN, EPI_PLAIN_F32>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     case EPI_BIAS_RELU_BF16: return launch_variant<kPair, CM, CN, EPI_BIAS_RELU_BF16>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    case EPI_ROW_LSE_BF16:
+      if (kAllKinds) return launch_variant<kPair, CM, CN, kAllKinds ? EPI_ROW_LSE_BF16 : EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+      return mtf::fail(MTF_ERR_UNSUPPORTED, "row log-sum-exp partials: no kernel for this cluster shape");
     case EPI_MASK_RSUM_BF16:
       if (kAllKinds) return launch_variant<kPair, CM, CN, kAllKinds ? EPI_MASK_RSUM_BF16 : EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
     default: return launch_variant<kPair, CM, CN, EPI_GENERIC>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
@@ -1576,7 +1603,13 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // the time of a 256 x 256 one (twice the MMAs at 3/4 of the L2 traffic each, epilogue exposed), so
   // they win when they halve the number of waves.
   bool wide = false;
+  // row_softmax == 5: a plain bf16 contraction that also leaves, per row and column part, the maximum and the sum of
+  // exponentials of the stored values at the head of the workspace (float2 [rows][parts]; the caller combines them)
+  const bool row_lse = row_softmax == 5;
+  if (row_lse) row_softmax = 0;
   const bool plain_epi = scale == 1.f && !resid && !bias && !relu && !mask && !rsum && !row_softmax;
+  if (row_lse && (!plain_epi || plan.dtC != MTF_BF16 || t.n_outer != 0 || t.ldc != t.N || t.reduce_mode == MTF_REDUCE_WORKSPACE || n_terms != 1 || n_groups != 1))
+    return fail(MTF_ERR_UNSUPPORTED, "row log-sum-exp partials need a plain bf16 contraction with dense rows and no workspace reduction");
   if (row_softmax) {
     // whole rows in one tile: the N slice is the whole dimension and fits a tile (256 columns, or 512 with a wide pair tile)
     const bool fits = a.sn == 1 && (a.Ns <= a.block_n || (a.Ns == 512 && t.cta_pair && t.block_n == 256));
@@ -1587,7 +1620,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
       return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a bf16 result whose rows fit one tile (N <= 256, or 512 with CTA pairs) and no other stage");
     wide = a.Ns == 512;
   }
-  const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && a.Ns % 512 == 0;
+  const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && !row_lse && a.Ns % 512 == 0;
   if (t.wide_pref == 1 && !wide_legal)
     return fail(MTF_ERR_UNSUPPORTED, "wide tiles need CTA pairs, a plain epilogue, no workspace reduction and an N slice that is a multiple of 512");
   if (wide_legal && t.wide_pref != 0) {
@@ -1601,7 +1634,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // optional single-GPU build: clusters of CTA pairs that share operand tiles
   int cm = 1, cn = 1;
 #if defined(MTF_CLUSTER_SHARE)
-  if (!wide && !row_softmax && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && n_terms == 1 && n_groups == 1 &&
+  if (!wide && !row_softmax && !row_lse && t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && n_terms == 1 && n_groups == 1 &&
       cluster_share_operands_local(A, B)) {      // both operands are allocations of the GPU this launch runs on
     // measured on the FFN shapes: sharing B between two pairs that are neighbours along M is worth
     // 5-10 % on the contractions whose epilogue is light; with a relu mask or a fused reduction in the
@@ -1638,6 +1671,14 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   a.scale = scale; a.relu = relu;
   a.rsum = rsum;
   a.rsum_partial = nullptr;
+  a.lse_partial = nullptr; a.lse_parts = 0;
+  if (row_lse) {
+    a.lse_parts = a.sn * a.n_tiles * 2;
+    const size_t need = (size_t)t.M * a.lse_parts * sizeof(float2);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 15) || workspace_bytes < need)
+      return fail(MTF_ERR_WORKSPACE_TOO_SMALL, "row log-sum-exp partials need %zu workspace bytes, got %zu", need, workspace_bytes);
+    a.lse_partial = reinterpret_cast<float2*>(workspace);
+  }
   a.ws_partials = nullptr; a.ws_counters = nullptr; a.ws_ncounters = 0;
   {
     const int b_cols = (t.cta_pair ? a.block_n / 2 : a.block_n);          // B columns staged by one CTA (wide: two runs of 128)
@@ -1661,7 +1702,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   if (a.total_work <= 0) return MTF_OK;
 
   cudaStream_t st = (cudaStream_t)stream;
-  if (t.balance && cn == 1 && !wide && n_terms == 1 && n_groups == 1 && !row_softmax && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+  if (t.balance && cn == 1 && !wide && n_terms == 1 && n_groups == 1 && !row_softmax && !row_lse && workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
     // Tail balancing: the tiles do not fill a whole number of waves, so the workers take equal ranges
     // of (tile, k-block) units; a tile cut by a range boundary is assembled from two fp32 fragments in
     // the workspace by whichever worker finishes last (arrive, never wait).
@@ -1751,6 +1792,7 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // launch that assembles tiles from fragments) takes the generic one
   int epi = EPI_GENERIC;
   if (row_softmax) epi = row_softmax >= 3 ? EPI_ROW_SOFTMAX_BWD : EPI_ROW_SOFTMAX;
+  else if (row_lse) epi = EPI_ROW_LSE_BF16;
   else if (!resid && !bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;
   else if (scale == 1.f && !resid) {
     if (!bias && !relu && !mask && !rsum) epi = a.c_bf16 ? EPI_PLAIN_BF16 : EPI_PLAIN_F32;

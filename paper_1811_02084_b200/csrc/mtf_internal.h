@@ -202,6 +202,10 @@ mtf_status einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_tenso
 // dlogits[.., l, m] = P (dP - sum_m dP P) with dP = sum_v a b, in one launch (same conditions, whole 32 x 64 boxes only).
 mtf_status einsum_row_softmax_bwd(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, const mtf_tensor* weights,
                                   mtf_tensor* dlogits, int causal, void* workspace, size_t workspace_bytes, void* stream);
+// a . b (plain, bf16) whose epilogue also leaves float2 [rows][*parts] row statistics (maximum, sum of exponentials of
+// the stored values per column part) at the head of the workspace
+mtf_status einsum_row_lse(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* out, void* workspace, size_t workspace_bytes,
+                          void* stream, int* parts);
 mtf_status einsum_row_softmax(const mtf_layout_t* layout, const mtf_tensor* a, const mtf_tensor* b, mtf_tensor* weights, float scale,
                               int causal, void* workspace, size_t workspace_bytes, void* stream);
 // Sum of n_terms (1..3) products of operand pairs with the dims of terms[0] (names may differ, sizes

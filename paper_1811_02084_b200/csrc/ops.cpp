@@ -9,6 +9,8 @@
 
 namespace mtf {
 mtf_status launch_sgd_update(float* master, void* param, const void* grad, int grad_bf16, float* mom, int64_t n, float lr, float mu, float wd, void* stream);
+mtf_status launch_xent_combine(const void* partial, int parts, const void* logits, const int32_t* targets, float* lse, float* loss, int64_t n_rows, int64_t vocab,
+                               void* stream);
 mtf_status launch_permute_copy(const void* src, void* dst, int elem_bytes, int ndim, const int64_t* sizes, const int64_t* sstr, const int64_t* dstr, void* stream);
 mtf_status launch_embedding_gather(const int32_t* ids, const void* table, void* x, int64_t n_tokens, int64_t d, int elem_bytes, int64_t vocab, void* stream);
 mtf_status launch_embedding_scatter_add(const int32_t* ids, const void* dx, int dx_bf16, float* dtable, int64_t n_tokens, int64_t d, int64_t vocab, void* stream);
@@ -209,6 +211,16 @@ mtf_status mtf_xent_forward(const mtf_layout_t* layout, const mtf_tensor* h, con
   mtf_status st = vocab_not_across_ranks(layout, wout->dims[1].name, "xent_forward");
   if (st != MTF_OK) return st;
   const mtf_tensor in[2] = {*h, *wout};
+  // With room in the workspace the logits contraction takes the local maximum and sum of exponentials of every column
+  // part of every row in its epilogue (Section 6 "Reduction": the local reduction), and a small launch combines the
+  // parts (the group combine): the logits are not read back for the log-sum-exp.
+  if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+    int parts = 0;
+    st = mtf::einsum_row_lse(layout, h, wout, logits, workspace, workspace_bytes, stream, &parts);
+    if (st == MTF_OK)
+      return mtf::launch_xent_combine(workspace, parts, logits->data, targets, reinterpret_cast<float*>(lse->data), reinterpret_cast<float*>(loss->data), rows, V, stream);
+    if (st != MTF_ERR_UNSUPPORTED && st != MTF_ERR_WORKSPACE_TOO_SMALL) return st;
+  }
   if ((st = mtf_einsum(layout, nullptr, 2, in, logits, nullptr, workspace, workspace_bytes, stream)) != MTF_OK) return st;
   return mtf_softmax_xent_forward(layout, logits, targets, lse, loss, stream);
 }

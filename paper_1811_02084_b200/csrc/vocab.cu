@@ -114,6 +114,34 @@ __global__ void __launch_bounds__(256) xent_rows_kernel(const __nv_bfloat16* __r
   }
 }
 
+// The group combine of Section 6's "Reduction" for row statistics that the logits contraction left per column part
+// (its epilogue took the local maximum and sum of exponentials of every part of every row while the tile was still
+// on the chip): one warp per row combines the parts in a fixed order, then lse and loss as above.
+__global__ void __launch_bounds__(256) xent_combine_kernel(const float2* __restrict__ partial, int parts, const __nv_bfloat16* __restrict__ logits,
+                                                           const int32_t* __restrict__ targets, float* __restrict__ lse, float* __restrict__ loss,
+                                                           long long n_rows, int vocab, int* __restrict__ bad) {
+  const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= n_rows) return;
+  const int lane = threadIdx.x & 31;
+  float m = -INFINITY, s = 0.f;
+  for (int p = lane; p < parts; p += 32) {
+    const float2 ps = partial[row * parts + p];
+    lse_combine(m, s, ps.x, ps.y);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    lse_combine(m, s, m2, s2);
+  }
+  if (lane == 0) {
+    const float l = m + logf(s);
+    lse[row] = l;
+    const int tg = targets[row];
+    if (tg < 0 || tg >= vocab) { atomicExch(bad, 1); loss[row] = 0.f; }
+    else loss[row] = l - __bfloat162float(logits[row * vocab + tg]);
+  }
+}
+
 // dlogits[t, v] = (exp(logits[t, v] - lse[t]) - [v == target[t]]) * dloss[t], written over the logits
 __global__ void __launch_bounds__(256) xent_backward_kernel(__nv_bfloat16* __restrict__ logits, const int32_t* __restrict__ targets, const float* __restrict__ lse,
                                                             const float* __restrict__ dloss, long long n_rows, int vocab) {
@@ -184,6 +212,16 @@ mtf_status launch_xent_rows(const void* logits, const int32_t* targets, float* l
   if (n_rows > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "cross-entropy: too many rows");
   xent_rows_kernel<<<(unsigned)n_rows, 256, 0, (cudaStream_t)stream>>>(reinterpret_cast<const __nv_bfloat16*>(logits), targets, lse, loss, (int)vocab, bad_flag());
   return after("xent_rows_kernel");
+}
+
+mtf_status launch_xent_combine(const void* partial, int parts, const void* logits, const int32_t* targets, float* lse, float* loss, int64_t n_rows, int64_t vocab,
+                               void* stream) {
+  if (n_rows <= 0) return MTF_OK;
+  if (parts <= 0 || n_rows > 0x7fffffffLL) return fail(MTF_ERR_UNSUPPORTED, "cross-entropy combine: bad sizes");
+  xent_combine_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, (cudaStream_t)stream>>>(reinterpret_cast<const float2*>(partial), parts,
+                                                                                   reinterpret_cast<const __nv_bfloat16*>(logits), targets, lse, loss, n_rows, (int)vocab,
+                                                                                   bad_flag());
+  return after("xent_combine_kernel");
 }
 
 mtf_status launch_xent_backward(void* logits, const int32_t* targets, const float* lse, const float* dloss, int64_t n_rows, int64_t vocab, void* stream) {
