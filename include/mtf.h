@@ -406,13 +406,16 @@ mtf_status mtf_layout_search(const mtf_mesh_t* mesh, int32_t n_einsums, const mt
  *       the call, fp32 atomics: order not fixed); summed across ranks when a token dim is split over them.
  *   mtf_xent_forward      : logits[t, v] = sum_d h[t, d] wout[d, v] (bf16, through mtf_einsum under the
  *       layout); per token lse = log sum_v exp(logits) - taken over the logits as stored, maximum
- *       subtracted, the local reduction of every vocab slice and the combine over the group in one pass
+ *       subtracted, the local reduction of every part of a row and the combine over the parts
  *       (Section 6 "Reduction") - and loss = lse - logits[t, target[t]].  lse, loss: f32, one per token.
+ *       With a 256-byte aligned workspace of at least tokens * 16 * ceil(vocab / 256) bytes per vocab
+ *       slice layout (tokens x column parts x 8 bytes) the contraction takes the local reductions in its
+ *       own epilogue and the logits are not read back; otherwise a second pass over the logits does both.
  *   mtf_xent_backward     : dlogits = (exp(logits - lse) - onehot(target)) * dloss[t], written over
  *       `logits`; dh = dlogits . wout^T (reduces vocab: the group sum of a vocab split);
  *       dwout = h^T . dlogits (reduces the token dims).  dloss f32, one per token.
  * A vocab dimension split across RANKS is refused (MTF_ERR_UNSUPPORTED): the row statistics would need
- * a max / sum combine across ranks.  workspace: as for mtf_einsum. */
+ * a max / sum combine across ranks.  workspace: as for mtf_einsum (plus the above for mtf_xent_forward). */
 mtf_status mtf_embedding_forward(const mtf_layout_t* layout, const int32_t* ids, const mtf_tensor* table, mtf_tensor* x, void* stream);
 mtf_status mtf_embedding_backward(const mtf_layout_t* layout, const int32_t* ids, const mtf_tensor* dx, mtf_tensor* dtable, void* stream);
 mtf_status mtf_xent_forward(const mtf_layout_t* layout, const mtf_tensor* h, const mtf_tensor* wout, const int32_t* targets, mtf_tensor* logits,
