@@ -1620,9 +1620,12 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
       return fail(MTF_ERR_UNSUPPORTED, "row softmax in the epilogue needs a bf16 result whose rows fit one tile (N <= 256, or 512 with CTA pairs) and no other stage");
     wide = a.Ns == 512;
   }
-  const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && plain_epi && !row_lse && a.Ns % 512 == 0;
+  // (wide tiles also with a residual as the only stage - the contractions whose result is added to a stream of the
+  //  decoder layer - through the generic epilogue kind)
+  const bool resid_only_epi = scale == 1.f && resid && !bias && !relu && !mask && !rsum && !row_softmax && n_terms == 1;
+  const bool wide_legal = t.cta_pair && t.block_n == 256 && t.reduce_mode != MTF_REDUCE_WORKSPACE && (plain_epi || resid_only_epi) && !row_lse && a.Ns % 512 == 0;
   if (t.wide_pref == 1 && !wide_legal)
-    return fail(MTF_ERR_UNSUPPORTED, "wide tiles need CTA pairs, a plain epilogue, no workspace reduction and an N slice that is a multiple of 512");
+    return fail(MTF_ERR_UNSUPPORTED, "wide tiles need CTA pairs, a plain or residual-only epilogue, no workspace reduction and an N slice that is a multiple of 512");
   if (wide_legal && t.wide_pref != 0) {
     long long tiles = (long long)((a.Ms + 2 * BM - 1) / (2 * BM)) * (a.Ns / 256) * a.sm * a.sn;
     for (int j = 0; j < t.n_outer; ++j) tiles *= t.outer_size[j];
@@ -1811,7 +1814,8 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
     else ls = launch_variant<false, 1, 1, EPI_ROW_SOFTMAX, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
   } else if (wide) {
     if (epi == EPI_PLAIN_BF16) ls = launch_variant<true, 1, 1, EPI_PLAIN_BF16, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
-    else ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else if (epi == EPI_PLAIN_F32) ls = launch_variant<true, 1, 1, EPI_PLAIN_F32, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+    else ls = launch_variant<true, 1, 1, EPI_GENERIC, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
   } else if (!t.cta_pair) ls = launch_kind<false, 1, 1, true>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
 #if defined(MTF_CLUSTER_SHARE)
   else if (cm == 1 && cn == 2) ls = launch_kind<true, 1, 2, false>(epi, map_a, map_b, map_c, map_m, map_w, extra, a, st);
