@@ -234,6 +234,19 @@ mtf_status mtf_einsum_builtin_scratch(const mtf_layout_t* layout, const char* eq
  * (tile, k-block) units and assemble cut tiles from fragments in the workspace).  A forced choice
  * the shape cannot run gives MTF_ERR_UNSUPPORTED. */
 mtf_status mtf_plan_force(int32_t kernel_kind, int32_t reduce_mode);
+/* A promise about the next contraction this thread launches (mtf_einsum, mtf_einsum_exec): it reads nothing
+ * that the launch before it on the same stream writes, and writes nothing that launch reads or writes.  A
+ * tensor-core contraction then does not wait for that launch before it starts: its tiles begin on the SMs the
+ * earlier launch's last round of tiles leaves idle, its workers take their tiles from a counter as they become
+ * free, and it waits for the earlier launch before it ends, so whatever follows on the stream still sees both
+ * complete.  Hinted launches that follow one another may all overlap each other and the launch before the first
+ * of them, so the promise must hold against all of those; everything launched before that launch is complete
+ * when they start.  The
+ * promise is used up by the next contraction whether or not it can honour it (launches with a workspace
+ * reduction or a fused reduce_sum, and the generic kernel, run in stream order as always; so does every
+ * fourth hinted launch in a row).  The Transformer blocks use it between their own independent launches
+ * (Algorithm 1 leaves the order of independent operations open).  Results do not depend on it. */
+mtf_status mtf_hint_independent(void);
 
 /* ---- feed-forward block (Section 8: y = Relu(x w + bias) v) ------------------------------------- */
 /* x [*tokens, d_in], w [d_in, hidden], bias [hidden] or NULL, v [hidden, d_in]; outputs h_saved

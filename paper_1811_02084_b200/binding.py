@@ -119,6 +119,7 @@ def _load():
         "mtf_einsum_builtin_scratch": [vp, c_char_p, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), vp],
         "mtf_einsum_workspace_bytes": [vp, c_int32, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(mtf_epilogue), POINTER(c_size_t)],
         "mtf_plan_force": [c_int32, c_int32],
+        "mtf_hint_independent": [],
         "mtf_ffn_forward": [vp] + [POINTER(mtf_tensor)] * 6 + [vp, c_size_t, vp],
         "mtf_ffn_backward": [vp] + [POINTER(mtf_tensor)] * 9 + [vp, c_size_t, vp],
         "mtf_ffn_workspace_bytes": [vp, POINTER(mtf_tensor), POINTER(mtf_tensor), POINTER(c_size_t)],
@@ -436,6 +437,11 @@ def mtf_einsum_workspace_bytes(layout: Layout, ins, out: Named, epilogue: Epilog
     b = c_size_t()
     _check(_lib.mtf_einsum_workspace_bytes(layout.handle, len(ins), _tensor_array(ins), byref(out.c), _epi(epilogue), byref(b)))
     return b.value
+
+
+def mtf_hint_independent() -> None:
+    """The next contraction of this thread is independent of the launch before it on its stream (see mtf.h)."""
+    _check(_lib.mtf_hint_independent())
 
 
 def mtf_plan_force(kernel_kind: int = -1, reduce_mode: int = -1) -> None:

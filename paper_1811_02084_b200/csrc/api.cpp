@@ -337,7 +337,11 @@ mtf_status mtf_plan_info(const mtf_plan_t* plan, int32_t* kernel_kind, int32_t* 
 
 mtf_status mtf_einsum_exec(const mtf_plan_t* plan, const mtf_tensor* in, mtf_tensor* out, const mtf_epilogue* epilogue,
                            void* workspace, size_t workspace_bytes, void* stream) {
-  return exec_plan(plan, in, out, epilogue, workspace, workspace_bytes, stream);
+  const bool independent = mtf::take_independent_hint();     // (cleared whatever happens below)
+  if (independent && plan && plan->kernel_kind == MTF_KERNEL_TCGEN05) mtf::hint_next_launch_independent();
+  const mtf_status st = exec_plan(plan, in, out, epilogue, workspace, workspace_bytes, stream);
+  (void)mtf::take_independent_hint();
+  return st;
 }
 
 mtf_status mtf_einsum(const mtf_layout_t* layout, const char* equation, int32_t n_in, const mtf_tensor* in, mtf_tensor* out,
@@ -379,6 +383,11 @@ mtf_status mtf_einsum_workspace_bytes(const mtf_layout_t* layout, int32_t n_in, 
   mtf_status st = cached_plan(layout, n_in, in, out, epilogue, &P);
   if (st != MTF_OK) return st;
   *bytes = P->workspace_bytes;
+  return MTF_OK;
+}
+
+mtf_status mtf_hint_independent(void) {
+  g_next_independent = true;
   return MTF_OK;
 }
 
@@ -509,6 +518,7 @@ mtf_status mtf::einsum_terms(const mtf_layout_t* layout, int n_terms, const mtf_
 }
 
 void mtf::hint_next_launch_independent() { g_next_independent = true; }
+int mtf::swap_force_reduce(int mode) { const int was = g_force_reduce; g_force_reduce = mode; return was; }
 bool mtf::take_independent_hint() {
   const bool v = g_next_independent;
   g_next_independent = false;

@@ -617,12 +617,17 @@ mtf_status launch_attention_bwd_fused(const void* q, const void* kk, const void*
   cudaError_t e = cudaFuncSetAttribute(attention_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
+  // Blocks 2k and 2k + 1 are launched as a cluster only so that they sit on the two SMs of one TPC: the blocks whose
+  // share of the pairs is one round shorter are the last ones, and when they leave, whole TPCs become free for the CTA
+  // pairs of an independent contraction launched behind this kernel.  The kernel itself uses nothing of the cluster.
+  at[1].id = cudaLaunchAttributeClusterDimension;
+  at[1].val.clusterDim.x = 2; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   const long long grid = std::min<long long>(a.units, device_sm_count());
   cfg.gridDim = dim3((unsigned)grid, 1, 1); cfg.blockDim = dim3(kThreads, 1, 1); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = (cudaStream_t)stream;
-  cfg.attrs = at; cfg.numAttrs = 1;
+  cfg.attrs = at; cfg.numAttrs = grid % 2 == 0 ? 2 : 1;
   e = cudaLaunchKernelEx(&cfg, attention_bwd_kernel, mq, mk, mv, md, mp, a);
   if (e != cudaSuccess) return fail(MTF_ERR_CUDA, "attention_bwd_kernel: %s", cudaGetErrorString(e));
   count_launch();

@@ -355,13 +355,10 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
   void* rest = ar.base + ar.used;
   const size_t rest_bytes = ar.size - ar.used;
   TD xm = renamed(*x, s.l.name, kMemory);
-  if ((st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = ein(layout, *dy, *wo, &dob.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
-  if ((st = mtf::tap("do", dob.t, stream)) != MTF_OK) return st;
   // The whole core - dP, the softmax backward, dvv, dq, dkk - in one launch under the conditions of the forward core
   // (d_k = d_v = 64, rows of at most 512, only batch and heads split, canonical dimension orders): the weights are read
   // once and the gradient of the logits never leaves the chip.
-  bool core_done = false;
+  bool core_ok = false;
   {
     auto unsplit = [&](const mtf_dim& d) { const int j = layout->mesh_dim_of(d.name); return j < 0 || layout->mesh[j].size == 1; };
     auto order = [](const mtf_tensor* t, std::initializer_list<mtf_dim> want) {
@@ -372,7 +369,18 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
     };
     const bool canonical = order(q, {s.b, s.l, s.h, s.k}) && order(kk, {s.b, s.m, s.h, s.k}) && order(vv, {s.b, s.m, s.h, s.v}) &&
                            order(weights, {s.b, s.h, s.l, s.m}) && order(o, {s.b, s.l, s.h, s.v});
-    if (canonical && mtf::attention_bwd_fused_supported(s.l.size, s.k.size, s.v.size) && unsplit(s.l) && unsplit(s.m) && unsplit(s.k) && unsplit(s.v)) {
+    core_ok = canonical && mtf::attention_bwd_fused_supported(s.l.size, s.k.size, s.v.size) && unsplit(s.l) && unsplit(s.m) && unsplit(s.k) && unsplit(s.v);
+  }
+  // dWo reads o and dy and nothing the core touches.  Behind the one-launch core it is issued as an independent launch
+  // with the group sum chained in its accumulators (no cleared counters in front of it), so its tiles start on the SMs
+  // that the core's last round of (batch, head) pairs leaves idle; otherwise it goes first.
+  const bool dwo_late = core_ok;
+  if (!dwo_late && (st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = ein(layout, *dy, *wo, &dob.t, nullptr, rest, rest_bytes, stream)) != MTF_OK) return st;
+  if ((st = mtf::tap("do", dob.t, stream)) != MTF_OK) return st;
+  bool core_done = false;
+  {
+    if (core_ok) {
       // (with the stage tap open the gradient of the logits is written out as well, as the contractions consume it)
       void* dump = mtf::tap_is_open() ? dlg.t.data : nullptr;
       if ((st = mtf::launch_attention_bwd_fused(q->data, kk->data, vv->data, weights->data, dob.t.data, dq.t.data, dkk.t.data, dvv.t.data, dump, s.b.size, s.h.size,
@@ -380,6 +388,13 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
         return st;
       if (dump && (st = mtf::tap("dlogits", dlg.t, stream)) != MTF_OK) return st;
       core_done = true;
+      if (dwo_late) {
+        const int was = mtf::swap_force_reduce(MTF_REDUCE_CHAINED);
+        mtf::hint_next_launch_independent();
+        st = ein(layout, *o, *dy, dwo, nullptr, rest, rest_bytes, stream);
+        mtf::swap_force_reduce(was);
+        if (st != MTF_OK) return st;
+      }
     }
   }
   if (!core_done) {
@@ -422,7 +437,11 @@ mtf_status mtf_attention_backward(const mtf_layout_t* layout, const mtf_tensor* 
     // one launch where the plan allows it: the k loop runs through dq.wq, then dkk.wk, then dvv.wv
     // into one accumulator (same shapes; the key / value side carries the memory_length name)
     const mtf_tensor terms[3][2] = {{dq.t, *wq}, {dkk.t, *wk}, {dvv.t, *wv}};
+    // (it reads what the weight-gradient launch before it only reads and writes dx: an independent launch, whose tiles
+    //  start on the SMs that launch's few tiles leave idle)
+    mtf::hint_next_launch_independent();
     st = mtf::einsum_terms(layout, 3, terms, dx, dx_residual ? &er : nullptr, rest, rest_bytes, stream);
+    (void)mtf::take_independent_hint();
     if (st == MTF_OK) return mtf::rank_wait(layout, stream);
     if (st != MTF_ERR_UNSUPPORTED) return st;
   }

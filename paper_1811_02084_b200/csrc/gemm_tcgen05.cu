@@ -46,7 +46,8 @@ constexpr int kBStageBytes = kMaxBN * BK * 2;    // 32 KB (a CTA of a pair stage
 constexpr int kRingBytes = 5 * (kAStageBytes + kBStageBytes / 2);   // pairs: 5 x (16 KB + 16 KB); single CTAs: 3 x 48 KB fit too
 constexpr int kStagingBytes = kEpilogueWarps * 2 * 4096;   // per epilogue warp: two 32-row x 128-byte boxes for TMA stores
 constexpr int kMaxStages = 8;                      // ring slots with barriers; a launch uses as many as fit its stage size
-constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 320 /*barriers*/;
+constexpr int kSchedSlots = 4;                      // ring of drawn tile numbers that a CTA's roles read in turn
+constexpr int kSmemBytes = kRingBytes + kStagingBytes + 1024 /*alignment slack*/ + 320 /*barriers*/ + 96 /*drawn tiles: 2 x 4 barriers, 4 numbers*/;
 constexpr int kThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kTmemCols = 512;
 constexpr long long kTimeoutCycles = 4000000000LL;
@@ -101,6 +102,8 @@ struct TcArgs {
   long long tiles_per_slice, total_tiles, total_work;
   int balanced;            // workers take equal contiguous ranges of (tile, k-block) units instead of whole tiles
   int late_wait;           // programmatic dependent launch: wait for the previous launch at the end instead of the start
+  unsigned* sched;         // not NULL: the workers draw their tiles from this counter pair (next ticket, workers done) instead of
+                           // taking every W-th one; zero before the launch, zero again when its last worker has finished
   int reverse;             // walk the tiles from the last to the first (see launch_tc)
   int n_stages, stage_bytes;   // operand ring: 16 KB of A plus this CTA's part of B per stage, as many stages as fit
   int kb_tile;             // k-blocks of one whole tile (all terms)
@@ -197,12 +200,32 @@ struct SegIter {
   const TcArgs& a;
   long long w, W, work, u, u_end, total_units;
   int kb_per_slice;
+  // drawn tiles (a.sched): the producer thread of a worker's first CTA draws tickets from the launch's counter and
+  // publishes each tile number in a small ring in the shared memory of the worker's CTAs; every other role reads the
+  // ring in order.  role 0: the drawing thread, 1: a single reading thread, 2: a reading warp (all lanes call next()).
+  uint32_t ring = 0;               // shared-memory address of the ring: full barriers, empty barriers, numbers
+  volatile int* abort_flag = nullptr;
+  uint32_t seq = 0;
+  unsigned pending = 0;
+  int role = 1, n_ctas = 1, lane = 0;
+  bool failed = false, have_pending = false;
   __device__ SegIter(const TcArgs& args, long long worker, long long workers) : a(args), w(worker), W(workers), work(worker) {
     kb_per_slice = a.Ks / BK;
     total_units = a.total_tiles * a.kb_tile;
     u = a.balanced ? (w * total_units) / W : 0;
     u_end = a.balanced ? ((w + 1) * total_units) / W : 0;
   }
+  __device__ void draw_from(uint32_t ring_addr, volatile int* abort, int role_, int ctas, int lane_) {
+    ring = ring_addr; abort_flag = abort; role = role_; n_ctas = ctas; lane = lane_;
+    if (role == 0) draw_ahead();
+  }
+  // The drawing thread asks for its next ticket a few k-blocks before it has issued the last loads of its tile: early
+  // enough to hide the round trip to the counter, late enough that a worker does not hold a tile it will only start
+  // much later while other workers run out of work.
+  __device__ __forceinline__ void draw_ahead() {
+    if (!have_pending) { pending = atomicAdd(a.sched, 1u); have_pending = true; }
+  }
+  __device__ __forceinline__ bool draw();
   __device__ long long owner(long long unit) const { return ((unit + 1) * W - 1) / total_units; }
   __device__ bool next(Seg& s) {
     s.group = 0;
@@ -219,6 +242,7 @@ struct SegIter {
       u = e;
       return true;
     }
+    if (ring != 0 && !draw()) return false;
     if (work >= a.total_work) return false;
     if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
       uint32_t frag;
@@ -236,7 +260,7 @@ struct SegIter {
       s.kb_begin = 0;
       s.kb_count = a.kb_tile;
     }
-    work += W;
+    if (ring == 0) work += W;
     return true;
   }
 };
@@ -337,6 +361,74 @@ __device__ __forceinline__ void mbar_arrive_pair(uint32_t bar, uint32_t leader_r
         ::"r"(bar), "r"(leader_rank) : "memory");
   else
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Ring of drawn tile numbers (see SegIter).  Slot s of kSchedSlots: full barrier at ring + 8 s (one arrival: the
+// drawing thread), empty barrier at ring + 32 + 8 s in the first CTA (one arrival per reading role of every CTA),
+// number at ring + 64 + 4 s.  A number >= total_work ends the sequence; the drawing thread then counts its worker as
+// done, and the last worker of the launch clears the counter pair for the next launch that is given it.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool SegIter::draw() {
+  const uint32_t slot = seq % kSchedSlots, phase = (seq / kSchedSlots) & 1u;
+  const uint32_t full = ring + 8u * slot, empty = ring + 32u + 8u * slot, num = ring + 64u + 4u * slot;
+  ++seq;
+  if (role == 0) {
+    draw_ahead();
+    const unsigned t = pending;
+    have_pending = false;
+    if (seq > (uint32_t)kSchedSlots) {
+      const long long t0 = clock64();
+      while (!mbar_try_wait_cluster(empty, phase ^ 1u)) {
+        if (*abort_flag) { failed = true; return false; }
+        if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, 0x900 + (int)slot); *abort_flag = 1; failed = true; return false; }
+      }
+    }
+    if (n_ctas == 1) {
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(num), "r"(t) : "memory");
+      asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(full) : "memory");
+    } else
+    for (int c = 0; c < n_ctas; ++c)
+      asm volatile(
+          "{\n\t.reg .b32 ra, rb;\n\t"
+          "mapa.shared::cluster.u32 ra, %0, %2;\n\t"
+          "mapa.shared::cluster.u32 rb, %1, %2;\n\t"
+          "st.shared::cluster.u32 [ra], %3;\n\t"
+          "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [rb];\n\t}"
+          ::"r"(num), "r"(full), "r"(c), "r"(t) : "memory");
+    if ((long long)t >= a.total_work) {
+      __threadfence();
+      if (atomicAdd(a.sched + 1, 1u) == (unsigned)W - 1u) {      // every worker has drawn its last ticket
+        a.sched[0] = 0u; a.sched[1] = 0u;
+        __threadfence();
+      }
+      return false;
+    }
+    work = (long long)t;
+    return true;
+  }
+  // readers: wait for the number, read it, hand the slot back to the drawing thread
+  const long long t0 = clock64();
+  while (!mbar_try_wait_cluster(full, phase)) {
+    if (*abort_flag) { failed = true; return false; }
+    if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, 0x910 + (int)slot); *abort_flag = 1; failed = true; return false; }
+  }
+  unsigned t;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t) : "r"(num) : "memory");
+  if (role == 2) __syncwarp();
+  if (role == 1 || lane == 0) {
+    if (n_ctas > 1) mbar_arrive_pair<true>(empty, 0u);
+    else mbar_arrive_pair<false>(empty, 0u);
+  }
+  work = (long long)t;
+  return (long long)t < a.total_work;
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -665,6 +757,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   // then [2S+4..2S+20): per epilogue warp two barriers for relu-mask boxes loaded into its staging buffers
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 4 + 2 * kEpilogueWarps);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // then the ring of drawn tile numbers (launches with a.sched): 4 full barriers, 4 empty barriers, 4 numbers
+  const uint32_t sched_ring = bar_base + 8u * (2 * kMaxStages + 4 + 2 * kEpilogueWarps) + 8u;
+  const bool drawn = a.sched != nullptr && !kCluster;
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -681,6 +776,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), CM + CN - 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(tfull_bar(i), 1); mbar_init(tempty_bar(i), (kPair ? 2 : 1) * kEpilogueWarps); }
     for (int i = 0; i < 2 * kEpilogueWarps; ++i) mbar_init(bar_base + 8u * (2 * kMaxStages + 4 + i), 1);
+    for (int i = 0; i < kSchedSlots; ++i) { mbar_init(sched_ring + 8u * i, 1); mbar_init(sched_ring + 32u + 8u * i, (kPair ? 2 : 1) * (1 + kEpilogueWarps)); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
@@ -724,6 +820,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t phase = 0;
       bool ok = true;
       SegIter it(a, work_first, work_step);
+      if (drawn) it.draw_from(sched_ring, abort_flag, leader ? 0 : 1, kPair ? 2 : 1, 0);
       Seg sg;
       while (ok && it.next(sg)) {
         const int kb_first = sg.kb_begin, kb_count = sg.kb_count;
@@ -732,6 +829,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int n0 = tl.n0 + pn * a.block_n + cta_rank * n_local;
         int term = kb_first / a.kb_term, kt = kb_first - term * a.kb_term;
         for (int kb = 0; kb < kb_count; ++kb) {
+          if (drawn && leader && kb == (kb_count > 4 ? kb_count - 4 : 0)) it.draw_ahead();
           // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
           // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor); a
           // multi-term launch then goes on with the next product's operands
@@ -801,6 +899,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int iter = 0;
       bool ok = true;
       SegIter it(a, work_first, work_step);
+      if (drawn) it.draw_from(sched_ring, abort_flag, 1, kPair ? 2 : 1, 0);
       Seg sg;
       for (; ok && it.next(sg); ++iter) {
         const int kb_count = sg.kb_count;
@@ -839,6 +938,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     int iter = 0;
     bool ok = true;
     SegIter it(a, work_first, work_step);
+    if (drawn) it.draw_from(sched_ring, abort_flag, 2, kPair ? 2 : 1, lane);
     Seg sg;
     for (; ok && it.next(sg); ++iter) {
       const long long t = sg.tile;
@@ -1448,6 +1548,55 @@ int sm_count() {
   return n;
 }
 
+// ---- counters for launches that draw their tiles ----------------------------------------------------------
+// A launch that starts while the launch before it still runs (late_wait) finds some SMs free at once and the
+// others later, so its workers draw tiles from a counter instead of owning every W-th one.  A counter pair must
+// be zero when its launch starts and is cleared by that launch's last worker, so two launches that may overlap
+// need different pairs: every stream has kSchedPerStream pairs, taken in turn by consecutive late launches, and
+// after that many in a row the next launch is made an ordinary one (it waits for everything before it, after
+// which all pairs are clear again).  Streams beyond kSchedStreams keep the fixed assignment.
+constexpr int kSchedStreams = 16, kSchedPerStream = 3;
+static __device__ unsigned g_sched_words[kSchedStreams * kSchedPerStream * 2];
+
+struct DeviceSched {
+  std::mutex mu;
+  unsigned* base = nullptr;
+  bool looked_up = false;
+  cudaStream_t stream[kSchedStreams];
+  int late_run[kSchedStreams];
+  int n = 0;
+};
+static DeviceSched g_dev_sched[kMaxDevices];
+
+// Called once per contraction launch: `late` is whether the launch may skip the wait at its start.  Returns the
+// counter pair the launch draws from (NULL: fixed assignment); clears *late when the chain of late launches on
+// this stream has used every pair.
+static unsigned* sched_for_launch(cudaStream_t st, bool drawable, int* late) {
+  DeviceSched& d = g_dev_sched[current_device()];
+  std::lock_guard<std::mutex> lock(d.mu);
+  if (!d.looked_up) {
+    d.looked_up = true;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_sched_words) == cudaSuccess) d.base = reinterpret_cast<unsigned*>(p);
+    else (void)cudaGetLastError();
+  }
+  int idx = -1;
+  for (int i = 0; i < d.n; ++i)
+    if (d.stream[i] == st) { idx = i; break; }
+  if (idx < 0 && d.n < kSchedStreams) { idx = d.n++; d.stream[idx] = st; d.late_run[idx] = 0; }
+  if (idx < 0 || !d.base) return nullptr;
+  if (!*late) { d.late_run[idx] = 0; return nullptr; }
+  if (d.late_run[idx] >= kSchedPerStream) { *late = 0; d.late_run[idx] = 0; return nullptr; }
+  const int slot = d.late_run[idx]++;
+  return drawable ? d.base + 2 * (idx * kSchedPerStream + slot) : nullptr;
+}
+
+static void sched_clear_all() {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_sched_words) == cudaSuccess) cudaMemset(p, 0, sizeof(unsigned) * kSchedStreams * kSchedPerStream * 2);
+  else (void)cudaGetLastError();
+}
+
 // Clears 32-bit words (the fused reduce_sum output, the arrival counters of shared tiles).  A kernel
 // rather than a memset so that it can sit in a chain of programmatically dependent launches: it
 // waits for the kernel before it, and the contraction after it overlaps its set-up with this one.
@@ -1696,6 +1845,8 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
   // the caller's word that this launch is independent of the one before it (consumed here); only honoured
   // for launches that clear nothing beforehand and use no workspace
   a.late_wait = (take_independent_hint() && !rsum && t.reduce_mode != MTF_REDUCE_WORKSPACE && !t.balance) ? 1 : 0;
+  // such a launch draws its tiles (plain pairs and single CTAs; see sched_for_launch)
+  a.sched = sched_for_launch((cudaStream_t)stream, cm * cn == 1, &a.late_wait);
   // Successive launches walk their tiles in opposite directions: a contraction that reads what the launch
   // before it wrote (h then y, the attention weights then P.v) starts with the part that is still in L2.
   static std::atomic<unsigned> launch_parity{0};
@@ -1881,6 +2032,7 @@ mtf_status read_device_status(int* code) {
   if (v != 0) {
     int zero = 0;
     cudaMemcpyToSymbol(g_status, &zero, sizeof(int));
+    sched_clear_all();      // a launch that gave up may have left its tile counter behind
   }
   if (code) *code = v;
   if (v != 0) return fail(MTF_ERR_TIMEOUT, "a bounded device-side wait gave up (code 0x%x)", v);

@@ -186,6 +186,8 @@ mtf_status launch_tc(const mtf_plan_t& plan, const void* A, const void* B, void*
 // Hint for the next tensor-core launch of this thread: it neither reads nor writes anything the launch
 // before it on the same stream touches (set by the block compositions, consumed by the launch).
 void hint_next_launch_independent();
+// Sets the reduce mode that plans made on this thread are forced to (-1: the planner's choice); returns the old one.
+int swap_force_reduce(int mode);
 bool take_independent_hint();
 // n_groups (1..3) independent einsums with the dims of group 0 (names may differ, sizes and types may
 // not) in one launch, so that contractions with few output tiles fill the GPU together.

@@ -358,3 +358,31 @@ def test_slice_gather_is_bit_exact(mtf):
             mtf.mtf_slice_gather(lay, mtf.named(payload, [d for d, _ in dims]), p, out)
             want = olay.global_flat_indices(dims, p).astype(np.float64)
             assert np.array_equal(from_torch(out).reshape(-1), want), (p, tdt)
+
+
+def test_independent_hint_gives_the_same_results(mtf):
+    """Contractions launched with mtf_hint_independent() may start while the launch before them still runs and
+    draw their tiles from a counter; the counters are handed out in turn and cleared by each launch.  A chain of
+    such launches (longer than the number of counters, so that the fall-back to an ordinary launch is taken
+    too), issued several times over, must give bit for bit what the same contractions give without the hint."""
+    import torch
+    lay = layout(mtf, [("all", 1)], [])
+    shapes = [(1024, 768, 4096), (4096, 2048, 512), (512, 512, 8192), (2304, 1280, 1024), (8192, 1024, 256), (768, 3072, 2048), (256, 256, 1024)]
+    probs = []
+    for i, (M, N, K) in enumerate(shapes):
+        a = to_torch(si.normal(40 + i, "ha", [M, K], "bf16"))
+        b = to_torch(si.normal(40 + i, "hb", [K, N], "bf16", K ** -0.5))
+        outs = [torch.zeros(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        probs.append((mtf.named(a, ["m%d" % i, "k%d" % i]), mtf.named(b, ["k%d" % i, "n%d" % i]), outs, ["m%d" % i, "n%d" % i], (a, b)))
+    for A, B, outs, names, _ in probs:
+        mtf.mtf_einsum(lay, None, [A, B], mtf.named(outs[0], names))
+    mtf.mtf_device_status()
+    for rep in range(3):
+        for _, _, outs, _, _ in probs:
+            outs[1].zero_()
+        for A, B, outs, names, _ in probs:
+            mtf.mtf_hint_independent()
+            mtf.mtf_einsum(lay, None, [A, B], mtf.named(outs[1], names))
+        mtf.mtf_device_status()
+        for i, (_, _, outs, _, _) in enumerate(probs):
+            assert torch.equal(outs[0], outs[1]), (rep, shapes[i])
