@@ -15,19 +15,22 @@
 // wholly right of it are skipped.
 //
 // A persistent CTA (one per SM) walks (batch, head) pairs.  For a pair the work is cut into steps (j, i): key
-// block j (128 keys, outer loop), query block i (128 queries), and the steps are walked twice: pass 0 computes dP of
-// every step and adds dP * P into the row terms D (which must be complete before any dS can be formed), pass 1
-// computes dP again (four MMAs) and everything else.  The second read of a tile of P comes from L2.
+// block j (128 keys, outer loop), query block i (128 queries), and the steps are walked twice.  Pass 0 forms the row
+// terms: D[l] = sum_m dP[l, m] P[l, m] = sum_v do[l, v] O[l, v] with O = P vv, so the MMA thread alone accumulates the
+// unrounded O_i = sum_j P_ij vv_j in fp32 in the tensor-memory columns that hold dq_i afterwards, and when the pass ends
+// every warp multiplies its rows of O with its rows of do (read from global memory).  Pass 1 computes dP (four MMAs per
+// step) and everything else.  The second read of a tile of P comes from L2 or HBM.
 // Tensor memory (512 columns):
-//   [0, 256)    dq of the (up to) four query blocks, accumulated over j
+//   [0, 256)    pass 0: O of the (up to) four query blocks; pass 1: dq of the same blocks, accumulated over j
 //   [256, 320)  dkk of key block j, [320, 384) dvv of key block j, accumulated over i
 //   [384, 512)  dP of the current step
 // Warp roles (320 threads):
-//   warp 0     TMA producer: V_j and K_j per key block; q_i, do_i and the 128 x 128 tile of P per step (rings of three)
-//   warp 1     MMA issuer:   dP and dvv += P^T do of the NEXT step as soon as this step's dP has been read out of tensor
-//                            memory, then this step's dkk += dS^T q, dq_i += dS kk_j (tcgen05.mma kind::f16)
-//   warps 2-9  two per tensor-memory lane quarter (each owns 64 of the step's 128 key columns): dS from dP and P,
-//              and the read-out of finished accumulators to HBM
+//   warp 0     TMA producer: V_j (both passes) and K_j (pass 1) per key block; the 128 x 128 tile of P per step, q_i and do_i
+//              per step of pass 1 (rings of three)
+//   warp 1     MMA issuer:   pass 0: O_i += P_ij vv_j; pass 1: dP and dvv += P^T do of the NEXT step as soon as this step's dP
+//                            has been read out of tensor memory, then this step's dkk += dS^T q, dq_i += dS kk_j
+//   warps 2-9  two per tensor-memory lane quarter (each owns 64 of the step's 128 key columns): the row terms, dS from dP
+//              and P, and the read-out of finished accumulators to HBM
 // Every mbarrier wait is bounded; on expiry a code is recorded in the status word, a CTA-wide abort flag is
 // raised, the remaining waits return at once and all roles leave through the teardown.
 #include <cuda.h>
@@ -54,7 +57,7 @@ constexpr size_t kSmemBytes = 1024 + kOffBars + kNumBars * 8 + 64;
 // tensor-memory columns
 constexpr uint32_t kColDK = 256, kColDV = 320, kColDP = 384;
 
-enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_DP_FULL /*2*/, B_DP_EMPTY = 6 /*2*/, B_DKV_FULL = 8, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_D_SYNC,
+enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_DP_FULL /*2: dP of a step; O of a pair complete*/, B_DP_EMPTY = 6, B_DKV_FULL = 8, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_D_SYNC,
        B_QDO_FULL = 13 /*3*/, B_QDO_EMPTY = 16 /*3*/, B_P_FULL = 19 /*3*/, B_P_EMPTY = 22 /*3*/, B_PV_DONE = 25 /*3*/, B_DS_FULL = 28 /*3*/ };
 
 __device__ int g_attb_status = 0;
@@ -63,6 +66,7 @@ struct BwdArgs {
   int B, H, L;
   int causal;
   float scale;
+  const __nv_bfloat16* dout;     // [B, L, H, 64]: read directly for the row terms
   __nv_bfloat16* ds_dump;        // [B, H, L, L] or NULL: where the gradient of the logits is written as well (testing)
   __nv_bfloat16* dq;             // [B, L, H, 64]
   __nv_bfloat16* dk;
@@ -167,28 +171,23 @@ struct StepIter {
   int nb, causal;
   int pass, j, i;
   long long step_seq, s1_seq, kv_seq, k_seq, unit_seq;      // counts of steps / steps of pass 1 / key blocks (both passes) / key blocks of pass 1 / pairs before this one
-  long long p0_seq;                  // steps of pass 0 of this pair before this one
-  long long dpu0, dpu1;              // uses of the two dP buffers before this step
-  __device__ long long dpu(int b) const { return b ? dpu1 : dpu0; }
+  long long dpu0;                    // dP tiles before this step (one per step of pass 1)
   bool valid;
   __device__ void init(long long first, long long stride_, long long units_, int nb_, int causal_) {
     u = first; stride = stride_; units = units_; nb = nb_; causal = causal_;
-    pass = 0; j = 0; i = 0; step_seq = 0; s1_seq = 0; kv_seq = 0; k_seq = 0; unit_seq = 0; p0_seq = 0; dpu0 = dpu1 = 0;
+    pass = 0; j = 0; i = 0; step_seq = 0; s1_seq = 0; kv_seq = 0; k_seq = 0; unit_seq = 0; dpu0 = 0;
     valid = u < units;
   }
-  // pass 0 alternates between two dP buffers (the second one stands where dkk, dvv accumulate in pass 1), starting with the
-  // first for every pair: the first dP of a pair is issued while the previous pair's last dkk, dvv are still being
-  // accumulated; pass 1 has one buffer
-  __device__ int dp_buf() const { return pass == 0 ? (int)(p0_seq & 1) : 0; }
+  // dP exists in pass 1 only, in one buffer
   __device__ bool last_of_pass0() const { return pass == 0 && j == nb - 1 && i == nb - 1; }
   __device__ bool first_i() const { return i == (causal ? j : 0); }
   __device__ bool last_i() const { return i == nb - 1; }
   __device__ bool first_of_unit() const { return pass == 0 && j == 0 && first_i(); }
   __device__ bool last_of_unit() const { return pass == 1 && j == nb - 1 && i == nb - 1; }
   __device__ void advance() {
-    if (dp_buf()) ++dpu1; else ++dpu0;
+    if (pass == 1) ++dpu0;
     ++step_seq;
-    if (pass == 1) ++s1_seq; else ++p0_seq;
+    if (pass == 1) ++s1_seq;
     if (i + 1 < nb) { ++i; return; }
     ++kv_seq;
     if (pass == 1) ++k_seq;
@@ -196,7 +195,6 @@ struct StepIter {
     j = 0; i = 0;
     if (pass == 0) { pass = 1; return; }
     pass = 0;
-    p0_seq = 0;
     ++unit_seq;
     u += stride;
     valid = u < units;
@@ -220,8 +218,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kNumBars; ++i) mb_init(bar(i), 1);
-    mb_init(bar(B_DP_EMPTY), kCompWarps); mb_init(bar(B_DP_EMPTY + 1), kCompWarps);
-    mb_init(bar(B_D_SYNC), kCompWarps);
+    mb_init(bar(B_DP_EMPTY), kCompWarps);
     for (int i = 0; i < kRing; ++i) mb_init(bar(B_DS_FULL + i), kCompWarps);
     mb_init(bar(B_DKV_EMPTY), kCompWarps);
     mb_init(bar(B_DQ_EMPTY), kCompWarps);
@@ -272,9 +269,11 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
           tma_load_4d(sV, &map_v, bar(B_V_FULL), 0, it.j * 128, h, b);
         }
         if (!(ok = mb_wait(bar(B_QDO_EMPTY + slot), par ^ 1u, 0xA02, abort_flag))) break;
-        mb_expect(bar(B_QDO_FULL + slot), it.pass == 0 ? kBox : 2 * kBox);       // (pass 0 needs do alone)
-        if (it.pass == 1) tma_load_4d(sQ + slot * kBox, &map_q, bar(B_QDO_FULL + slot), 0, it.i * 128, h, b);
-        tma_load_4d(sDO + slot * kBox, &map_do, bar(B_QDO_FULL + slot), 0, it.i * 128, h, b);
+        mb_expect(bar(B_QDO_FULL + slot), it.pass == 0 ? 0u : 2 * kBox);       // (pass 0 needs neither: the phase completes at once)
+        if (it.pass == 1) {
+          tma_load_4d(sQ + slot * kBox, &map_q, bar(B_QDO_FULL + slot), 0, it.i * 128, h, b);
+          tma_load_4d(sDO + slot * kBox, &map_do, bar(B_QDO_FULL + slot), 0, it.i * 128, h, b);
+        }
         if (!(ok = mb_wait(bar(B_P_EMPTY + slot), par ^ 1u, 0xA03, abort_flag))) break;
         mb_expect(bar(B_P_FULL + slot), 2 * kBox);
         tma_load_4d(sP + slot * 2 * kBox, &map_p, bar(B_P_FULL + slot), it.j * 128, it.i * 128, h, b);
@@ -294,33 +293,44 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       cur.init(blockIdx.x, gridDim.x, a.units, nb, a.causal);
       nxt = cur;
       if (nxt.valid) nxt.advance();
-      long long n_dp = 0;                      // dP tiles issued so far (one per step of either pass)
+      long long n_dp = 0;                      // dP tiles issued so far (one per step of pass 1)
       long long n_dv = 0;                      // dvv contributions issued so far (one per step of pass 1)
       bool ok = true;
       const uint32_t id_dp = idesc_of(0, 0, 128), id_kv = idesc_of(1, 1, 64), id_dq = idesc_of(0, 1, 64);
-      // dP of step t: wants do of the step, V of its key block and the dP columns read out by the warps
-      // pass 0: the warps say with one arrival that they have a step's dP and its tile of P in registers; the tile goes back
-      // to the producer when that arrival is seen, which is when the buffer's next dP is about to be issued
-      int rel_slot[2] = {-1, -1};
+      // pass 0, one step: O_i += P_ij vv_j (M = queries, N = d_v, k = keys; A K-major over two 64-key boxes, B MN-major) into the
+      // columns where dq_i will accumulate in pass 1.  Nothing of it concerns the warps until the pass ends.
+      auto issue_o = [&](const StepIter& t) -> bool {
+        const int slot = (int)(t.step_seq % kRing);
+        const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
+        if (t.first_of_unit() && !mb_wait(bar(B_DQ_EMPTY), ((uint32_t)t.unit_seq & 1u) ^ 1u, 0xB08, abort_flag)) return false;   // the previous pair's dq has been read out
+        if (t.first_i() && !mb_wait(bar(B_V_FULL), (uint32_t)t.kv_seq & 1u, 0xB01, abort_flag)) return false;
+        if (!mb_wait(bar(B_QDO_FULL + slot), par, 0xB02, abort_flag)) return false;      // (an empty phase in pass 0: keeps the ring's phases in step)
+        if (!mb_wait(bar(B_P_FULL + slot), par, 0xB04, abort_flag)) return false;
+        fence_after();
+        const uint64_t da = smem_desc(sP + slot * 2 * kBox, 0, 0), db = smem_desc(sV, 1, kBox);
+        const uint32_t acc = t.j != 0 ? 1u : 0u;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma(tmem + (uint32_t)t.i * 64u, da + (uint64_t)((ks >> 2) * (kBox >> 4) + (ks & 3) * 2), db + (uint64_t)(ks * (2048 >> 4)), id_dq, acc | (uint32_t)ks);
+        umma_commit(bar(B_P_EMPTY + slot));
+        umma_commit(bar(B_QDO_EMPTY + slot));
+        if (t.last_i()) umma_commit(bar(B_V_EMPTY));
+        if (t.last_of_pass0()) umma_commit(bar(B_DP_FULL + 1));      // every O_i of the pair is complete
+        return true;
+      };
+      // dP of a step of pass 1: wants do of the step, V of its key block and the dP columns read out by the warps
       auto issue_dp = [&](const StepIter& t) -> bool {
         const int slot = (int)(t.step_seq % kRing);
         const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
-        const int buf = t.dp_buf();
         if (t.first_i() && !mb_wait(bar(B_V_FULL), (uint32_t)t.kv_seq & 1u, 0xB01, abort_flag)) return false;
         if (!mb_wait(bar(B_QDO_FULL + slot), par, 0xB02, abort_flag)) return false;
-        if (!mb_wait(bar(B_DP_EMPTY + buf), ((uint32_t)t.dpu(buf) & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // this buffer's previous dP has been read out
-        if (rel_slot[buf] >= 0) { mb_arrive(bar(B_P_EMPTY + rel_slot[buf])); rel_slot[buf] = -1; }   // (pass 0: ... and with it the tile of P of that step)
-        // (the second buffer stands on the accumulators of dkk, dvv: those of the previous pair have been read out)
-        if (buf == 1 && !mb_wait(bar(B_DKV_EMPTY), ((uint32_t)t.k_seq & 1u) ^ 1u, 0xB0A, abort_flag)) return false;
+        if (!mb_wait(bar(B_DP_EMPTY), ((uint32_t)t.dpu0 & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // the previous dP has been read out
         fence_after();
         const uint64_t da = smem_desc(sDO + slot * kBox, 0, 0), db = smem_desc(sV, 0, 0);
-        const uint32_t col = buf ? kColDK : kColDP;
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) umma(tmem + col, da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
-        umma_commit(bar(B_DP_FULL + buf));
-        if (t.pass == 0) umma_commit(bar(B_QDO_EMPTY + slot));      // pass 0: nothing else reads this do
+        for (int ks = 0; ks < 4; ++ks) umma(tmem + kColDP, da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
+        umma_commit(bar(B_DP_FULL));
         if (t.last_i()) umma_commit(bar(B_V_EMPTY));         // this key block's V is no longer read
-        if (t.pass == 0) rel_slot[buf] = slot;
         ++n_dp;
         return true;
       };
@@ -331,11 +341,6 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
         if (!mb_wait(bar(B_P_FULL + slot), par, 0xB04, abort_flag)) return false;
         if (t.first_i() && !mb_wait(bar(B_DKV_EMPTY), ((uint32_t)t.k_seq & 1u) ^ 1u, 0xB06, abort_flag)) return false;   // the previous key block's dkk, dvv have been read out
-        // (... and so has the last dP that pass 0 put in the same columns)
-        if (t.first_i() && t.j == 0 && t.dpu1 > 0) {
-          if (!mb_wait(bar(B_DP_EMPTY + 1), (uint32_t)(t.dpu1 - 1) & 1u, 0xB0B, abort_flag)) return false;
-          if (rel_slot[1] >= 0) { mb_arrive(bar(B_P_EMPTY + rel_slot[1])); rel_slot[1] = -1; }
-        }
         fence_after();
         const uint64_t da = smem_desc(sP + slot * 2 * kBox, 1, kBox), db = smem_desc(sDO + slot * kBox, 1, kBox);
         const uint32_t acc = t.first_i() ? 0u : 1u;
@@ -346,27 +351,24 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         return true;
       };
       while (ok && cur.valid) {
-        const int slot = (int)(cur.step_seq % kRing);
-        if (n_dp == cur.step_seq && !(ok = issue_dp(cur))) break;
-        if (cur.pass == 1 && n_dv == cur.s1_seq && !(ok = issue_dv(cur))) break;
-        // ahead of this step's remaining MMAs: the next step's dP (pass 0: into the other buffer; pass 1: as soon as the
-        // warps have this step's dP in registers) and, inside a key block, its dvv contribution, so that the warps work
-        // on the next step while these run
-        if (nxt.valid) {
-          if (!(ok = issue_dp(nxt))) break;
-          if (nxt.pass == 1 && !nxt.first_i() && !(ok = issue_dv(nxt))) break;
-        }
         if (cur.pass == 0) {
+          if (!(ok = issue_o(cur))) break;
           cur = nxt;
           if (nxt.valid) nxt.advance();
           continue;
         }
+        const int slot = (int)(cur.step_seq % kRing);
+        if (n_dp == cur.s1_seq && !(ok = issue_dp(cur))) break;
+        if (n_dv == cur.s1_seq && !(ok = issue_dv(cur))) break;
+        // ahead of this step's remaining MMAs: the next step's dP (as soon as the warps have this step's dP in registers)
+        // and, inside a key block, its dvv contribution, so that the warps work on the next step while these run
+        if (nxt.valid && nxt.pass == 1) {
+          if (!(ok = issue_dp(nxt))) break;
+          if (!nxt.first_i() && !(ok = issue_dv(nxt))) break;
+        }
         const int s1slot = (int)(cur.s1_seq % kRing);
         if (!(ok = mb_wait(bar(B_DS_FULL + s1slot), (uint32_t)(cur.s1_seq / kRing) & 1u, 0xB05, abort_flag))) break;      // dS stands where P stood
-        if (cur.first_i()) {
-          if (!(ok = mb_wait(bar(B_K_FULL), (uint32_t)cur.k_seq & 1u, 0xB07, abort_flag))) break;
-          if (cur.j == 0 && !(ok = mb_wait(bar(B_DQ_EMPTY), ((uint32_t)cur.unit_seq & 1u) ^ 1u, 0xB08, abort_flag))) break;   // the previous pair's dq
-        }
+        if (cur.first_i() && !(ok = mb_wait(bar(B_K_FULL), (uint32_t)cur.k_seq & 1u, 0xB07, abort_flag))) break;
         fence_after();
         const uint32_t acc_kv = cur.first_i() ? 0u : 1u;
         const uint32_t dsS = sP + slot * 2 * kBox, qS = sQ + slot * kBox;
@@ -424,56 +426,41 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
       const int b = (int)(it.u / a.H), h = (int)(it.u % a.H);
       const int slot = (int)(it.step_seq % kRing);
       const uint32_t par = (uint32_t)(it.step_seq / kRing) & 1u;
-      if (it.first_of_unit()) { D0 = 0.f; D1 = 0.f; D2 = 0.f; D3 = 0.f; }
-      const int buf = it.dp_buf();
-      if (!(ok = wait_all(B_DP_FULL + buf, (uint32_t)it.dpu(buf) & 1u, 0xC01))) break;
-      fence_after();
-      if (!(ok = wait_all(B_P_FULL + slot, par, 0xC02))) break;
       uint32_t r0[32], r1[32];
       if (it.pass == 0) {
-        // pass 0: D[l] += sum over this warp's 64 of the step's 128 keys of dP[l, m] P[l, m]; the two warps of a lane
-        // quarter add their halves when the pass ends
-        float d = 0.f;
-        {
-          const uint32_t col = (buf ? kColDK : kColDP) + (uint32_t)half * 64u;
-          tmem_ld32(taddr + col, r0);
-          tmem_ld32(taddr + col + 32u, r1);
-          const uint32_t prow = sP + (uint32_t)slot * 2u * kBox + (uint32_t)half * kBox + (uint32_t)row_l * 128u;
-          uint4 pv[8];
-#pragma unroll
-          for (int pc = 0; pc < 8; ++pc) pv[pc] = lds_v4(prow + ((((uint32_t)pc) ^ sw) << 4));
-          tmem_ld_wait();
-#pragma unroll
-          for (int pc = 0; pc < 8; ++pc) {
-            const uint32_t* rr = pc < 4 ? r0 + pc * 8 : r1 + (pc - 4) * 8;
-            d = fmaf(bf_lo(pv[pc].x), __uint_as_float(rr[0]), d); d = fmaf(bf_hi(pv[pc].x), __uint_as_float(rr[1]), d);
-            d = fmaf(bf_lo(pv[pc].y), __uint_as_float(rr[2]), d); d = fmaf(bf_hi(pv[pc].y), __uint_as_float(rr[3]), d);
-            d = fmaf(bf_lo(pv[pc].z), __uint_as_float(rr[4]), d); d = fmaf(bf_hi(pv[pc].z), __uint_as_float(rr[5]), d);
-            d = fmaf(bf_lo(pv[pc].w), __uint_as_float(rr[6]), d); d = fmaf(bf_hi(pv[pc].w), __uint_as_float(rr[7]), d);
-          }
-        }
-        fence_before();
-        __syncwarp();
-        if (lane == 0) mb_arrive(bar(B_DP_EMPTY + buf));          // dP and P of this step are in registers
-        if (it.i == 0) D0 += d; else if (it.i == 1) D1 += d; else if (it.i == 2) D2 += d; else D3 += d;
+        // pass 0 belongs to the MMA thread (O_i = sum_j P_ij vv_j in fp32, in the columns of dq_i).  When it ends, every warp
+        // forms the row terms of its rows for all query blocks: D[l] = sum_v do[l, v] O[l, v], which equals sum_m dP[l, m] P[l, m]
+        // with the unrounded dP.  (Both warps of a lane quarter do this for the same rows: cheaper than an exchange.)
         if (it.last_of_pass0()) {
-          // the two halves of every row sum meet through four tensor-memory columns of this warp's lanes (columns of dq,
-          // which nothing uses before the first dS of pass 1 exists)
-          uint32_t mine[4] = {__float_as_uint(D0), __float_as_uint(D1), __float_as_uint(D2), __float_as_uint(D3)}, other[4];
-          tmem_st4(taddr + (uint32_t)half * 4u, mine);
-          tmem_st_wait();
-          fence_before();
-          __syncwarp();
-          if (lane == 0) mb_arrive(bar(B_D_SYNC));
-          if (!(ok = wait_all(B_D_SYNC, (uint32_t)it.unit_seq & 1u, 0xC06))) break;
+          if (!(ok = wait_all(B_DP_FULL + 1, (uint32_t)it.unit_seq & 1u, 0xC06))) break;
           fence_after();
-          tmem_ld4(taddr + (uint32_t)(half ^ 1) * 4u, other);
-          tmem_ld_wait();
-          D0 += __uint_as_float(other[0]); D1 += __uint_as_float(other[1]); D2 += __uint_as_float(other[2]); D3 += __uint_as_float(other[3]);
+          for (int i2 = 0; i2 < nb; ++i2) {
+            tmem_ld32(taddr + (uint32_t)i2 * 64u, r0);
+            tmem_ld32(taddr + (uint32_t)i2 * 64u + 32u, r1);
+            const uint4* drow = reinterpret_cast<const uint4*>(a.dout + (((long long)b * L + i2 * 128 + row_l) * a.H + h) * 64);
+            uint4 dv4[8];
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) dv4[pc] = __ldg(drow + pc);
+            tmem_ld_wait();
+            float d = 0.f;
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) {
+              const uint32_t* rr = pc < 4 ? r0 + pc * 8 : r1 + (pc - 4) * 8;
+              d = fmaf(bf_lo(dv4[pc].x), __uint_as_float(rr[0]), d); d = fmaf(bf_hi(dv4[pc].x), __uint_as_float(rr[1]), d);
+              d = fmaf(bf_lo(dv4[pc].y), __uint_as_float(rr[2]), d); d = fmaf(bf_hi(dv4[pc].y), __uint_as_float(rr[3]), d);
+              d = fmaf(bf_lo(dv4[pc].z), __uint_as_float(rr[4]), d); d = fmaf(bf_hi(dv4[pc].z), __uint_as_float(rr[5]), d);
+              d = fmaf(bf_lo(dv4[pc].w), __uint_as_float(rr[6]), d); d = fmaf(bf_hi(dv4[pc].w), __uint_as_float(rr[7]), d);
+            }
+            if (i2 == 0) D0 = d; else if (i2 == 1) D1 = d; else if (i2 == 2) D2 = d; else D3 = d;
+          }
+          fence_before();
         }
         it.advance();
         continue;
       }
+      if (!(ok = wait_all(B_DP_FULL, (uint32_t)it.dpu0 & 1u, 0xC01))) break;
+      fence_after();
+      if (!(ok = wait_all(B_P_FULL + slot, par, 0xC02))) break;
       tmem_ld32(taddr + kColDP + (uint32_t)half * 64u, r0);
       tmem_ld32(taddr + kColDP + (uint32_t)half * 64u + 32u, r1);
       tmem_ld_wait();
@@ -605,6 +592,7 @@ mtf_status launch_attention_bwd_fused(const void* q, const void* kk, const void*
     return st;
   BwdArgs a;
   a.B = (int)B; a.H = (int)H; a.L = (int)L; a.causal = causal ? 1 : 0; a.scale = scale;
+  a.dout = reinterpret_cast<const __nv_bfloat16*>(dout);
   a.ds_dump = reinterpret_cast<__nv_bfloat16*>(dlogits_dump);
   a.dq = reinterpret_cast<__nv_bfloat16*>(dq);
   a.dk = reinterpret_cast<__nv_bfloat16*>(dkk);
