@@ -200,32 +200,12 @@ struct SegIter {
   const TcArgs& a;
   long long w, W, work, u, u_end, total_units;
   int kb_per_slice;
-  // drawn tiles (a.sched): the producer thread of a worker's first CTA draws tickets from the launch's counter and
-  // publishes each tile number in a small ring in the shared memory of the worker's CTAs; every other role reads the
-  // ring in order.  role 0: the drawing thread, 1: a single reading thread, 2: a reading warp (all lanes call next()).
-  uint32_t ring = 0;               // shared-memory address of the ring: full barriers, empty barriers, numbers
-  volatile int* abort_flag = nullptr;
-  uint32_t seq = 0;
-  unsigned pending = 0;
-  int role = 1, n_ctas = 1, lane = 0;
-  bool failed = false, have_pending = false;
   __device__ SegIter(const TcArgs& args, long long worker, long long workers) : a(args), w(worker), W(workers), work(worker) {
     kb_per_slice = a.Ks / BK;
     total_units = a.total_tiles * a.kb_tile;
     u = a.balanced ? (w * total_units) / W : 0;
     u_end = a.balanced ? ((w + 1) * total_units) / W : 0;
   }
-  __device__ void draw_from(uint32_t ring_addr, volatile int* abort, int role_, int ctas, int lane_) {
-    ring = ring_addr; abort_flag = abort; role = role_; n_ctas = ctas; lane = lane_;
-    if (role == 0) draw_ahead();
-  }
-  // The drawing thread asks for its next ticket a few k-blocks before it has issued the last loads of its tile: early
-  // enough to hide the round trip to the counter, late enough that a worker does not hold a tile it will only start
-  // much later while other workers run out of work.
-  __device__ __forceinline__ void draw_ahead() {
-    if (!have_pending) { pending = atomicAdd(a.sched, 1u); have_pending = true; }
-  }
-  __device__ __forceinline__ bool draw();
   __device__ long long owner(long long unit) const { return ((unit + 1) * W - 1) / total_units; }
   __device__ bool next(Seg& s) {
     s.group = 0;
@@ -242,7 +222,6 @@ struct SegIter {
       u = e;
       return true;
     }
-    if (ring != 0 && !draw()) return false;
     if (work >= a.total_work) return false;
     if (a.reduce_mode == MTF_REDUCE_WORKSPACE) {
       uint32_t frag;
@@ -260,8 +239,13 @@ struct SegIter {
       s.kb_begin = 0;
       s.kb_count = a.kb_tile;
     }
-    if (ring == 0) work += W;
+    work += W;
     return true;
+  }
+  // the same for a tile number drawn from the launch's counter (whole tiles only)
+  __device__ bool take(Seg& s, long long drawn_work) {
+    work = drawn_work;
+    return next(s);
   }
 };
 
@@ -363,10 +347,12 @@ __device__ __forceinline__ void mbar_arrive_pair(uint32_t bar, uint32_t leader_r
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
-// Ring of drawn tile numbers (see SegIter).  Slot s of kSchedSlots: full barrier at ring + 8 s (one arrival: the
-// drawing thread), empty barrier at ring + 32 + 8 s in the first CTA (one arrival per reading role of every CTA),
-// number at ring + 64 + 4 s.  A number >= total_work ends the sequence; the drawing thread then counts its worker as
-// done, and the last worker of the launch clears the counter pair for the next launch that is given it.
+// Drawn tiles (TcArgs::sched): the producer thread of a worker's first CTA draws tickets from the launch's counter and
+// publishes each tile number in a small ring in the shared memory of the worker's CTAs; every other role reads the ring
+// in order (its n-th read is slot n mod kSchedSlots).  Slot s: full barrier at ring + 8 s (one arrival: the drawing
+// thread), empty barrier at ring + 32 + 8 s in the first CTA (one arrival per reading role of every CTA), number at
+// ring + 64 + 4 s.  A number >= total_work ends the sequence; the drawing thread then counts its worker as done, and
+// the last worker of the launch clears the counter pair for the next launch that is given it.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -376,25 +362,23 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool SegIter::draw() {
+__device__ __forceinline__ bool sched_wait(uint32_t bar, uint32_t parity, int code, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait_cluster(bar, parity)) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, code); *abort_flag = 1; return false; }
+  }
+  return true;
+}
+// The drawing thread: number `t` into slot seq mod kSchedSlots of every CTA of the worker.
+__device__ __forceinline__ bool sched_publish(uint32_t ring, uint32_t seq, unsigned t, int n_ctas, volatile int* abort_flag) {
   const uint32_t slot = seq % kSchedSlots, phase = (seq / kSchedSlots) & 1u;
   const uint32_t full = ring + 8u * slot, empty = ring + 32u + 8u * slot, num = ring + 64u + 4u * slot;
-  ++seq;
-  if (role == 0) {
-    draw_ahead();
-    const unsigned t = pending;
-    have_pending = false;
-    if (seq > (uint32_t)kSchedSlots) {
-      const long long t0 = clock64();
-      while (!mbar_try_wait_cluster(empty, phase ^ 1u)) {
-        if (*abort_flag) { failed = true; return false; }
-        if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, 0x900 + (int)slot); *abort_flag = 1; failed = true; return false; }
-      }
-    }
-    if (n_ctas == 1) {
-      asm volatile("st.shared.u32 [%0], %1;" ::"r"(num), "r"(t) : "memory");
-      asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(full) : "memory");
-    } else
+  if (seq >= (uint32_t)kSchedSlots && !sched_wait(empty, phase ^ 1u, 0x900 + (int)slot, abort_flag)) return false;
+  if (n_ctas == 1) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(num), "r"(t) : "memory");
+    asm volatile("mbarrier.arrive.release.cta.shared::cta.b64 _, [%0];" ::"r"(full) : "memory");
+  } else {
     for (int c = 0; c < n_ctas; ++c)
       asm volatile(
           "{\n\t.reg .b32 ra, rb;\n\t"
@@ -403,32 +387,27 @@ __device__ __forceinline__ bool SegIter::draw() {
           "st.shared::cluster.u32 [ra], %3;\n\t"
           "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [rb];\n\t}"
           ::"r"(num), "r"(full), "r"(c), "r"(t) : "memory");
-    if ((long long)t >= a.total_work) {
-      __threadfence();
-      if (atomicAdd(a.sched + 1, 1u) == (unsigned)W - 1u) {      // every worker has drawn its last ticket
-        a.sched[0] = 0u; a.sched[1] = 0u;
-        __threadfence();
-      }
-      return false;
-    }
-    work = (long long)t;
-    return true;
   }
-  // readers: wait for the number, read it, hand the slot back to the drawing thread
-  const long long t0 = clock64();
-  while (!mbar_try_wait_cluster(full, phase)) {
-    if (*abort_flag) { failed = true; return false; }
-    if (clock64() - t0 > g_wait_limit) { atomicCAS(&g_status, 0, 0x910 + (int)slot); *abort_flag = 1; failed = true; return false; }
+  return true;
+}
+// A reading role's seq-th number; `arrive`: this thread hands the slot back (one thread per role).
+template <bool kPair>
+__device__ __forceinline__ bool sched_read(uint32_t ring, uint32_t seq, bool warp_role, bool arrive, volatile int* abort_flag, unsigned* t) {
+  const uint32_t slot = seq % kSchedSlots, phase = (seq / kSchedSlots) & 1u;
+  const uint32_t full = ring + 8u * slot, empty = ring + 32u + 8u * slot, num = ring + 64u + 4u * slot;
+  if (!sched_wait(full, phase, 0x910 + (int)slot, abort_flag)) return false;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(*t) : "r"(num) : "memory");
+  if (warp_role) __syncwarp();
+  if (arrive) mbar_arrive_pair<kPair>(empty, 0u);
+  return true;
+}
+// The drawing thread has its worker's last ticket: count the worker as done; the last one clears the pair.
+__device__ __forceinline__ void sched_worker_done(unsigned* sched, unsigned workers) {
+  __threadfence();
+  if (atomicAdd(sched + 1, 1u) == workers - 1u) {
+    sched[0] = 0u; sched[1] = 0u;
+    __threadfence();
   }
-  unsigned t;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t) : "r"(num) : "memory");
-  if (role == 2) __syncwarp();
-  if (role == 1 || lane == 0) {
-    if (n_ctas > 1) mbar_arrive_pair<true>(empty, 0u);
-    else mbar_arrive_pair<false>(empty, 0u);
-  }
-  work = (long long)t;
-  return (long long)t < a.total_work;
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -721,7 +700,7 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t sr
 // 16 KB / CN + 16 KB / CM per k-block through L2 instead of 32 KB.  A stage may be refilled when
 // every pair that reads what this CTA writes has retired its MMAs: CM + CN - 1 pair leaders signal
 // each CTA's "empty" barrier.
-template <bool kPair, int CM, int CN, int EPI, bool kWide>
+template <bool kPair, int CM, int CN, int EPI, bool kWide, bool kDrawn = false>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_m,
@@ -759,7 +738,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // then the ring of drawn tile numbers (launches with a.sched): 4 full barriers, 4 empty barriers, 4 numbers
   const uint32_t sched_ring = bar_base + 8u * (2 * kMaxStages + 4 + 2 * kEpilogueWarps) + 8u;
-  const bool drawn = a.sched != nullptr && !kCluster;
+  constexpr bool drawn = kDrawn;       // a variant of its own: launches with the fixed tile assignment carry none of this
+  static_assert(!kDrawn || !kCluster, "drawn tiles: plain pairs and single CTAs only");
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -820,16 +800,37 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t phase = 0;
       bool ok = true;
       SegIter it(a, work_first, work_step);
-      if (drawn) it.draw_from(sched_ring, abort_flag, leader ? 0 : 1, kPair ? 2 : 1, 0);
       Seg sg;
-      while (ok && it.next(sg)) {
+      // drawn tiles: the first CTA's producer asks for its next ticket a few k-blocks before it has issued the last loads
+      // of its tile: early enough to hide the round trip to the counter, late enough that a worker does not hold a tile it
+      // will only start much later while other workers run out of work
+      uint32_t dseq = 0;
+      unsigned pending = 0;
+      bool have_pending = false;
+      if (drawn && leader) { pending = (unsigned)work_first; have_pending = true; }      // (the first tile needs no ticket: worker w starts with tile w, ticket n is tile W + n)
+      auto next_tile = [&]() -> bool {
+        if (!drawn) return it.next(sg);
+        unsigned t;
+        if (leader) {
+          if (!have_pending) pending = (unsigned)work_step + atomicAdd(a.sched, 1u);
+          have_pending = false;
+          t = pending;
+          if (!sched_publish(sched_ring, dseq, t, kPair ? 2 : 1, abort_flag)) { ok = false; return false; }
+          if ((long long)t >= a.total_work) { sched_worker_done(a.sched, (unsigned)work_step); return false; }
+        } else {
+          if (!sched_read<kPair>(sched_ring, dseq, false, true, abort_flag, &t)) { ok = false; return false; }
+        }
+        ++dseq;
+        return it.take(sg, (long long)t);
+      };
+      while (ok && next_tile()) {
         const int kb_first = sg.kb_begin, kb_count = sg.kb_count;
         const Tile tl = decode_tile(a, sg.tile, kTileRows, a.block_n * CN);
         const int m0 = tl.m0 + pm * kPairRows + cta_rank * BM;
         const int n0 = tl.n0 + pn * a.block_n + cta_rank * n_local;
         int term = kb_first / a.kb_term, kt = kb_first - term * a.kb_term;
         for (int kb = 0; kb < kb_count; ++kb) {
-          if (drawn && leader && kb == (kb_count > 4 ? kb_count - 4 : 0)) it.draw_ahead();
+          if (drawn && leader && !have_pending && kb == (kb_count > 4 ? kb_count - 4 : 0)) { pending = (unsigned)work_step + atomicAdd(a.sched, 1u); have_pending = true; }
           // slices of the reduce group are walked in ascending order: k0 runs through slice 0's
           // block of K, then slice 1's, ... (the blocks are contiguous in the global tensor); a
           // multi-term launch then goes on with the next product's operands
@@ -899,9 +900,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int iter = 0;
       bool ok = true;
       SegIter it(a, work_first, work_step);
-      if (drawn) it.draw_from(sched_ring, abort_flag, 1, kPair ? 2 : 1, 0);
       Seg sg;
-      for (; ok && it.next(sg); ++iter) {
+      auto next_tile = [&]() -> bool {
+        if (!drawn) return it.next(sg);
+        unsigned t;
+        if (!sched_read<kPair>(sched_ring, (uint32_t)iter, false, true, abort_flag, &t)) { ok = false; return false; }
+        return it.take(sg, (long long)t);
+      };
+      for (; ok && next_tile(); ++iter) {
         const int kb_count = sg.kb_count;
         const int acc = kWide ? 0 : (iter & 1);
         const uint32_t acc_phase = kWide ? ((uint32_t)iter & 1u) : ((uint32_t)(iter >> 1) & 1u);
@@ -938,9 +944,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     int iter = 0;
     bool ok = true;
     SegIter it(a, work_first, work_step);
-    if (drawn) it.draw_from(sched_ring, abort_flag, 2, kPair ? 2 : 1, lane);
     Seg sg;
-    for (; ok && it.next(sg); ++iter) {
+    auto next_tile = [&]() -> bool {
+      if (!drawn) return it.next(sg);
+      unsigned t;
+      if (!sched_read<kPair>(sched_ring, (uint32_t)iter, true, lane == 0, abort_flag, &t)) { ok = false; return false; }
+      return it.take(sg, (long long)t);
+    };
+    for (; ok && next_tile(); ++iter) {
       const long long t = sg.tile;
       const int ks = sg.frag;
       const bool ws_mode = f.shared_tiles && sg.nfrag > 1;       // this tile is assembled from fragments in the workspace
@@ -1622,9 +1633,9 @@ mtf_status zero_words(void* p, long long n, cudaStream_t st) {
 
 // One kernel variant: shared-memory opt-in and the number of clusters that can be resident at once
 // are looked up on first use; the grid is that many clusters (persistent) or fewer.
-template <bool kPair, int CM, int CN, int EPI, bool kWide = false>
-mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
-                          const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
+template <bool kPair, int CM, int CN, int EPI, bool kWide, bool kDrawn>
+mtf_status launch_variant_impl(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
+                               const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
   constexpr int kCtas = (kPair ? 2 : 1) * CM * CN;
   // the shared-memory opt-in and the number of resident clusters are properties of a device: one set-up per device
   struct PerDevice { std::once_flag once; cudaError_t attr_err = cudaSuccess; int max_clusters = 0; };
@@ -1633,9 +1644,9 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   std::call_once(pd.once, [&pd] {
     cudaError_t& attr_err = pd.attr_err;
     int& max_clusters = pd.max_clusters;
-    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide, kDrawn>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (attr_err != cudaSuccess) return;
-    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (kCtas > 8) attr_err = cudaFuncSetAttribute(gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide, kDrawn>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (attr_err != cudaSuccess) return;
     if (kCtas == 1) { max_clusters = sm_count(); return; }
     cudaLaunchConfig_t q = {};
@@ -1645,7 +1656,7 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
     q.gridDim = dim3(kCtas * sm_count(), 1, 1); q.blockDim = dim3(kThreads, 1, 1); q.dynamicSmemBytes = kSmemBytes;
     q.attrs = at; q.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, &q) == cudaSuccess && n > 0) max_clusters = n;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide, kDrawn>, &q) == cudaSuccess && n > 0) max_clusters = n;
     else { max_clusters = sm_count() / kCtas; (void)cudaGetLastError(); }
   });
   const cudaError_t attr_err = pd.attr_err;
@@ -1661,9 +1672,21 @@ mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, co
   at[1].val.clusterDim.x = kCtas; at[1].val.clusterDim.y = 1; at[1].val.clusterDim.z = 1;
   cfg.gridDim = dim3((unsigned)(kCtas * clusters), 1, 1); cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = st; cfg.attrs = at; cfg.numAttrs = kCtas > 1 ? 2 : 1;
-  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide>, map_a, map_b, map_c, map_m, map_w, extra, a);
+  cudaError_t le = cudaLaunchKernelEx(&cfg, gemm_tcgen05_kernel<kPair, CM, CN, EPI, kWide, kDrawn>, map_a, map_b, map_c, map_m, map_w, extra, a);
   if (le != cudaSuccess) return mtf::fail(MTF_ERR_CUDA, "gemm_tcgen05_kernel<%d,%d,%d,%d>: %s", (int)kPair, CM, CN, EPI, cudaGetErrorString(le));
   return MTF_OK;
+}
+
+// The variant whose workers draw their tiles exists for the kinds an independent launch can have (plain and generic
+// epilogues of plain pairs and single CTAs); every other launch ignores TcArgs::sched and leaves its counter untouched.
+template <bool kPair, int CM, int CN, int EPI, bool kWide = false>
+mtf_status launch_variant(const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_c, const CUtensorMap& map_m,
+                          const CUtensorMap& map_w, const ExtraMaps& extra, const TcArgs& a, cudaStream_t st) {
+  constexpr bool kCanDraw = CM * CN == 1 && (EPI == EPI_GENERIC || EPI == EPI_PLAIN_BF16 || EPI == EPI_PLAIN_F32);
+  if constexpr (kCanDraw) {
+    if (a.sched) return launch_variant_impl<kPair, CM, CN, EPI, kWide, true>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
+  }
+  return launch_variant_impl<kPair, CM, CN, EPI, kWide, false>(map_a, map_b, map_c, map_m, map_w, extra, a, st);
 }
 
 // Picks the epilogue kind of a launch.  kAllKinds = false leaves out the relu-mask kind (cluster
