@@ -37,7 +37,7 @@ LAYOUTS = {
 # dram__bytes_read.sum + dram__bytes_write.sum per contraction launch, averaged over the six launches of a
 # step of this workload (one ncu capture; the summary under profiles/ names the command and the commit)
 NCU_DRAM_BYTES_PER_LAUNCH = 167.9e6
-NCU_TRAFFIC_COMMIT = "80f3c6c"
+NCU_TRAFFIC_COMMIT = "abd89d6"
 METRIC = "transformer_ffn_fwd_bwd_tflops"
 UNIT = "TFLOP/s"
 
