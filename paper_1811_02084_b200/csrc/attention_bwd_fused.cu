@@ -57,7 +57,7 @@ constexpr size_t kSmemBytes = 1024 + kOffBars + kNumBars * 8 + 64;
 // tensor-memory columns
 constexpr uint32_t kColDK = 256, kColDV = 320, kColDP = 384;
 
-enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_DP_FULL /*2: dP of a step; O of a pair complete*/, B_DP_EMPTY = 6, B_DKV_FULL = 8, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_D_SYNC,
+enum { B_K_FULL = 0, B_K_EMPTY, B_V_FULL, B_V_EMPTY, B_DP_FULL /*2*/, B_DP_EMPTY = 6 /*2*/, B_DKV_FULL = 8, B_DKV_EMPTY, B_DQ_FULL, B_DQ_EMPTY, B_D_SYNC /*O of a pair complete*/,
        B_QDO_FULL = 13 /*3*/, B_QDO_EMPTY = 16 /*3*/, B_P_FULL = 19 /*3*/, B_P_EMPTY = 22 /*3*/, B_PV_DONE = 25 /*3*/, B_DS_FULL = 28 /*3*/ };
 
 __device__ int g_attb_status = 0;
@@ -172,6 +172,11 @@ struct StepIter {
   int pass, j, i;
   long long step_seq, s1_seq, kv_seq, k_seq, unit_seq;      // counts of steps / steps of pass 1 / key blocks (both passes) / key blocks of pass 1 / pairs before this one
   long long dpu0;                    // dP tiles before this step (one per step of pass 1)
+  // Rows of at most 256 leave tensor-memory columns [128, 256) free (dq takes 64 per query block): dP then alternates
+  // between two buffers, so the next step's dP is computed while the warps still read this one.
+  __device__ int dp_buf() const { return nb <= 2 ? (int)(dpu0 & 1) : 0; }
+  __device__ long long dp_use() const { return nb <= 2 ? (dpu0 >> 1) : dpu0; }      // earlier uses of this step's buffer
+  __device__ uint32_t dp_col() const { return dp_buf() ? 128u : 384u; }
   bool valid;
   __device__ void init(long long first, long long stride_, long long units_, int nb_, int causal_) {
     u = first; stride = stride_; units = units_; nb = nb_; causal = causal_;
@@ -218,7 +223,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kNumBars; ++i) mb_init(bar(i), 1);
-    mb_init(bar(B_DP_EMPTY), kCompWarps);
+    mb_init(bar(B_DP_EMPTY), kCompWarps); mb_init(bar(B_DP_EMPTY + 1), kCompWarps);
     for (int i = 0; i < kRing; ++i) mb_init(bar(B_DS_FULL + i), kCompWarps);
     mb_init(bar(B_DKV_EMPTY), kCompWarps);
     mb_init(bar(B_DQ_EMPTY), kCompWarps);
@@ -315,7 +320,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         umma_commit(bar(B_P_EMPTY + slot));
         umma_commit(bar(B_QDO_EMPTY + slot));
         if (t.last_i()) umma_commit(bar(B_V_EMPTY));
-        if (t.last_of_pass0()) umma_commit(bar(B_DP_FULL + 1));      // every O_i of the pair is complete
+        if (t.last_of_pass0()) umma_commit(bar(B_D_SYNC));      // every O_i of the pair is complete
         return true;
       };
       // dP of a step of pass 1: wants do of the step, V of its key block and the dP columns read out by the warps
@@ -324,12 +329,12 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const uint32_t par = (uint32_t)(t.step_seq / kRing) & 1u;
         if (t.first_i() && !mb_wait(bar(B_V_FULL), (uint32_t)t.kv_seq & 1u, 0xB01, abort_flag)) return false;
         if (!mb_wait(bar(B_QDO_FULL + slot), par, 0xB02, abort_flag)) return false;
-        if (!mb_wait(bar(B_DP_EMPTY), ((uint32_t)t.dpu0 & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // the previous dP has been read out
+        if (!mb_wait(bar(B_DP_EMPTY + t.dp_buf()), ((uint32_t)t.dp_use() & 1u) ^ 1u, 0xB03, abort_flag)) return false;      // the buffer's previous dP has been read out
         fence_after();
         const uint64_t da = smem_desc(sDO + slot * kBox, 0, 0), db = smem_desc(sV, 0, 0);
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) umma(tmem + kColDP, da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
-        umma_commit(bar(B_DP_FULL));
+        for (int ks = 0; ks < 4; ++ks) umma(tmem + t.dp_col(), da + 2u * ks, db + 2u * ks, id_dp, ks != 0);
+        umma_commit(bar(B_DP_FULL + t.dp_buf()));
         if (t.last_i()) umma_commit(bar(B_V_EMPTY));         // this key block's V is no longer read
         ++n_dp;
         return true;
@@ -432,7 +437,7 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         // forms the row terms of its rows for all query blocks: D[l] = sum_v do[l, v] O[l, v], which equals sum_m dP[l, m] P[l, m]
         // with the unrounded dP.  (Both warps of a lane quarter do this for the same rows: cheaper than an exchange.)
         if (it.last_of_pass0()) {
-          if (!(ok = wait_all(B_DP_FULL + 1, (uint32_t)it.unit_seq & 1u, 0xC06))) break;
+          if (!(ok = wait_all(B_D_SYNC, (uint32_t)it.unit_seq & 1u, 0xC06))) break;
           fence_after();
           for (int i2 = 0; i2 < nb; ++i2) {
             tmem_ld32(taddr + (uint32_t)i2 * 64u, r0);
@@ -458,15 +463,15 @@ attention_bwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         it.advance();
         continue;
       }
-      if (!(ok = wait_all(B_DP_FULL, (uint32_t)it.dpu0 & 1u, 0xC01))) break;
+      if (!(ok = wait_all(B_DP_FULL + it.dp_buf(), (uint32_t)it.dp_use() & 1u, 0xC01))) break;
       fence_after();
       if (!(ok = wait_all(B_P_FULL + slot, par, 0xC02))) break;
-      tmem_ld32(taddr + kColDP + (uint32_t)half * 64u, r0);
-      tmem_ld32(taddr + kColDP + (uint32_t)half * 64u + 32u, r1);
+      tmem_ld32(taddr + it.dp_col() + (uint32_t)half * 64u, r0);
+      tmem_ld32(taddr + it.dp_col() + (uint32_t)half * 64u + 32u, r1);
       tmem_ld_wait();
       fence_before();
       __syncwarp();
-      if (lane == 0) mb_arrive(bar(B_DP_EMPTY));            // dP is in registers: the next step's dP may overwrite it
+      if (lane == 0) mb_arrive(bar(B_DP_EMPTY + it.dp_buf()));            // dP is in registers: the buffer's next dP may overwrite it
       const float Dr = it.i == 0 ? D0 : (it.i == 1 ? D1 : (it.i == 2 ? D2 : D3));
       const uint32_t prow = sP + (uint32_t)slot * 2u * kBox + (uint32_t)half * kBox + (uint32_t)row_l * 128u;
       uint4 out[8];
