@@ -23,7 +23,7 @@
 // Tensor memory (512 columns):
 //   [0, 256)    pass 0: O of the (up to) four query blocks; pass 1: dq of the same blocks, accumulated over j
 //   [256, 320)  dkk of key block j, [320, 384) dvv of key block j, accumulated over i
-//   [384, 512)  dP of the current step
+//   [384, 512)  dP of the current step (rows of at most 256: dq ends at column 128 and [128, 256) is a second dP buffer)
 // Warp roles (320 threads):
 //   warp 0     TMA producer: V_j (both passes) and K_j (pass 1) per key block; the 128 x 128 tile of P per step, q_i and do_i
 //              per step of pass 1 (rings of three)
