@@ -386,3 +386,28 @@ def test_independent_hint_gives_the_same_results(mtf):
         mtf.mtf_device_status()
         for i, (_, _, outs, _, _) in enumerate(probs):
             assert torch.equal(outs[0], outs[1]), (rep, shapes[i])
+
+
+def test_independent_hint_is_used_up_by_the_next_einsum_whatever_runs_it(mtf):
+    """The promise belongs to the next contraction only: an fp32 einsum on the generic kernel cannot honour it and must
+    not pass it on to the launch after it, which here reads what the launch before it writes."""
+    import torch
+    lay = layout(mtf, [("all", 1)], [])
+    a32 = to_torch(si.normal(61, "a32", [24, 40], "f32")); b32 = to_torch(si.normal(61, "b32", [40, 16], "f32"))
+    c32 = torch.zeros(24, 16, dtype=torch.float32, device="cuda")
+    M, N, K = 2048, 2048, 2048
+    a = to_torch(si.normal(62, "a", [M, K], "bf16")); b = to_torch(si.normal(62, "b", [K, N], "bf16", K ** -0.5))
+    mid = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda"); out = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+    w2 = to_torch(si.normal(63, "w2", [N, N], "bf16", N ** -0.5))
+    def chain(hint):
+        mtf.mtf_einsum(lay, None, [mtf.named(a, ["m", "k"]), mtf.named(b, ["k", "n"])], mtf.named(mid, ["m", "n"]))
+        if hint:
+            mtf.mtf_hint_independent()
+        mtf.mtf_einsum(lay, None, [mtf.named(a32, ["i", "j"]), mtf.named(b32, ["j", "l"])], mtf.named(c32, ["i", "l"]))      # generic kernel: uses the hint up
+        mtf.mtf_einsum(lay, None, [mtf.named(mid, ["m", "n"]), mtf.named(w2, ["n", "p"])], mtf.named(out, ["m", "p"]))       # depends on the first launch
+        mtf.mtf_device_status()
+        return out.clone()
+    want = chain(False)
+    for _ in range(3):
+        mid.zero_(); out.zero_()
+        assert torch.equal(chain(True), want)
